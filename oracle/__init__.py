@@ -1,0 +1,39 @@
+"""CPU checker for the fused operators.  TEST INFRASTRUCTURE, NOT A PRODUCT PATH.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It shares no code with the CUDA library or its Python binding and
+imports neither.
+
+What it computes.  The paper's premise (Section 1, "Fusion Opportunities";
+Section 2.2) is that a fused operator returns exactly what the chain of basic
+operators it replaces returns.  So every function here evaluates its expression
+*unfused*: one basic operator at a time over whole arrays, every intermediate
+materialised as a full numpy array, all in float64, sums accumulated pairwise
+in extended precision (numpy ``longdouble``) and rounded once at the end.
+Library primitives used as single steps: elementwise numpy ufuncs, ``@``
+(matrix product), ``np.bincount`` (segmented sum), fancy-index gathers.
+
+Pins (see tests/test_oracle_pins.py): closed forms with exactly representable
+values, brute-force pure-Python loops on tiny inputs with exact rational
+arithmetic, algebraic identities, and the dense-vs-masked agreement of the
+Outer template.  Every function below is covered by at least one of them.
+
+Chains.  A scalar operator chain is a list of steps ``(op, dst, a[, b[, c]])``:
+``dst`` is a temporary name ``"t0".."t7"``; operands are ``"a"`` (main-input
+value), ``"d"`` (Row: the row's dot product; Outer: U_i . V_j), ``"sideK"``,
+``"sK"`` (K-th scalar), ``"tK"`` or a Python float.  Outputs are operand names.
+"""
+from .ops import (
+    OPS, eval_chain, full_sum, row_sums, col_sums,
+    cell, magg, row, outer,
+    sum_xyz, magg_xy_xz_xx, row_chain_dense, row_chain_csr,
+    outer_wsloss_dense, outer_wsloss_masked,
+    csr_row_ids,
+)
+
+__all__ = [
+    "OPS", "eval_chain", "full_sum", "row_sums", "col_sums",
+    "cell", "magg", "row", "outer",
+    "sum_xyz", "magg_xy_xz_xx", "row_chain_dense", "row_chain_csr",
+    "outer_wsloss_dense", "outer_wsloss_masked", "csr_row_ids",
+]
