@@ -1,0 +1,244 @@
+/*
+ * fusedops.h - C ABI of the fused-operator library (CUDA, sm_100a).
+ *
+ * The library executes the four fused-operator template types of
+ * "On Optimizing Operator Fusion Plans for Large-Scale Machine Learning in
+ * SystemML" (Section 2.2, Table 1: Row, Cell, MAgg, Outer) on one GPU, over
+ * dense row-major and CSR float64 matrices.  A fused operator is described by
+ *   - a template call (fused_cell / fused_magg / fused_row / fused_outer),
+ *   - the template variant (an aggregation type of Table 1), and
+ *   - an explicit scalar operator chain (fo_chain): the straight-line program
+ *     the paper's generated `genexec` method holds (Section 2.2, listings).
+ * The data access, the parallel schedule and the aggregation live in the
+ * library's kernels, as they live in the paper's hand-coded template skeletons
+ * (Section 2.2, "Runtime Integration").
+ *
+ * Conventions for every call
+ *   - Matrix data, index arrays, `out` and `ws` are DEVICE pointers owned by the
+ *     caller.  fo_chain, fo_op, fo_side, fo_mat structs and the `scalars` array
+ *     are HOST memory; they are copied at launch and may be freed on return.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream).  No call allocates, frees or synchronises.
+ *   - Inputs are never written.  `out` is fully overwritten.
+ *   - `ws` is scratch of at least fused_*_workspace_bytes() bytes, 256-byte
+ *     aligned, prepared once with fo_workspace_init(); every call leaves it
+ *     ready for the next.  Two calls that overlap on the GPU must not share it.
+ *   - Return value: FO_OK or a negative fo_status.  Nothing throws, aborts or
+ *     traps.  On an error return nothing was launched.
+ *   - All values are IEEE float64.  CSR: rowptr has rows+1 int32 offsets with
+ *     rowptr[0] == 0 and rowptr[rows] == nnz, colidx int32 strictly ascending
+ *     inside a row, explicit zeros allowed.  Dense: row-major, element (i, j) at
+ *     data[i * ld + j], ld >= cols.
+ *   - Sums are deterministic: for given shapes the order of every floating-point
+ *     addition is fixed, so repeated calls return identical bits (exception:
+ *     the CSR variant of FO_ROW_COL_T_AGG, documented at fused_row).
+ */
+#ifndef FUSEDOPS_H
+#define FUSEDOPS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ------------------------------------------------------------------ status */
+typedef enum fo_status {
+    FO_OK = 0,
+    FO_ERR_NULL = -1,           /* a required pointer is NULL */
+    FO_ERR_SHAPE = -2,          /* dimensions of inputs do not fit together */
+    FO_ERR_CHAIN = -3,          /* bad opcode / operand, use before definition, too long */
+    FO_ERR_UNSUPPORTED = -4,    /* variant or size outside what the kernels cover */
+    FO_ERR_WORKSPACE = -5,      /* ws NULL, misaligned or too small */
+    FO_ERR_CUDA = -6,           /* the CUDA runtime refused the launch */
+    FO_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait ran out (see fo_query_device_status) */
+} fo_status;
+
+/* ---------------------------------------------------------------- matrices */
+typedef struct fo_dense {
+    int64_t rows, cols, ld;
+    const double *data;         /* device */
+} fo_dense;
+
+typedef struct fo_csr {
+    int64_t rows, cols, nnz;    /* nnz < 2^31 */
+    const int32_t *rowptr;      /* device, rows + 1 */
+    const int32_t *colidx;      /* device, nnz */
+    const double *vals;         /* device, nnz */
+} fo_csr;
+
+enum { FO_DENSE = 0, FO_CSR = 1 };
+typedef struct fo_mat {
+    int32_t kind;               /* FO_DENSE or FO_CSR; the other member is ignored */
+    int32_t reserved;
+    fo_dense dense;
+    fo_csr csr;
+} fo_mat;
+
+/*
+ * Side input (the paper's SideInput b[k], Section 2.2 cell-wise listing).
+ *   FO_AT_CELL: same shape as the main input, value read at (rix, cix);
+ *   FO_AT_ROW : column vector (rows x 1, element i at data[i * ld]), read at (rix);
+ *   FO_AT_COL : row vector (1 x cols), read at (cix).
+ * Side inputs are dense.
+ */
+enum { FO_AT_CELL = 0, FO_AT_ROW = 1, FO_AT_COL = 2 };
+typedef struct fo_side {
+    fo_dense m;
+    int32_t access;
+    int32_t reserved;
+} fo_side;
+
+/* ------------------------------------------------------------ operator chain */
+#define FO_MAX_OPS      32      /* steps per chain */
+#define FO_MAX_TMPS      8      /* temporaries t0..t7 */
+#define FO_MAX_SIDES     4
+#define FO_MAX_SCALARS   8
+#define FO_MAX_OUT       8      /* results of one chain (MAgg: number of aggregates) */
+
+/* Operand bytes. */
+#define FO_TMP(k)     ((uint8_t)(0x00 | (k)))   /* temporary k, must have been written */
+#define FO_SIDE(k)    ((uint8_t)(0x40 | (k)))   /* k-th side input at this cell / row */
+#define FO_SCALAR(k)  ((uint8_t)(0x80 | (k)))   /* scalars[k] */
+#define FO_MAIN       ((uint8_t)0xC0)           /* a: main-input value (Cell, MAgg, Outer) */
+#define FO_DOT        ((uint8_t)0xC1)           /* d: Row: X_i . v;  Outer: U_i . V_j */
+#define FO_IMM        ((uint8_t)0xC2)           /* this step's `imm` constant */
+
+typedef enum fo_opcode {
+    FO_OP_MOV = 0,   /* dst = a */
+    FO_OP_NEG, FO_OP_ABS, FO_OP_SQRT, FO_OP_EXP, FO_OP_LOG,
+    FO_OP_SQ,        /* dst = a * a */
+    FO_OP_ADD, FO_OP_SUB, FO_OP_MUL, FO_OP_DIV, FO_OP_MIN, FO_OP_MAX, FO_OP_POW,
+    FO_OP_EQ, FO_OP_NE, FO_OP_LT, FO_OP_LE, FO_OP_GT, FO_OP_GE,   /* 1.0 or 0.0 */
+    FO_OP_SEL,       /* dst = (a != 0) ? b : c */
+    FO_OP_FMA,       /* dst = a * b + c (one rounding) */
+    FO_OP_COUNT_
+} fo_opcode;
+
+typedef struct fo_op {
+    uint8_t opcode;             /* fo_opcode */
+    uint8_t dst;                /* temporary index 0..FO_MAX_TMPS-1 */
+    uint8_t a, b, c;            /* operand bytes; unused ones are ignored */
+    uint8_t reserved[3];
+    double imm;                 /* value of FO_IMM operands of this step */
+} fo_op;
+
+typedef struct fo_chain {
+    int32_t n_ops;              /* 0..FO_MAX_OPS */
+    int32_t n_out;              /* 1..FO_MAX_OUT (1 except for fused_magg) */
+    const fo_op *ops;           /* host */
+    uint8_t out[FO_MAX_OUT];    /* operand bytes of the results */
+} fo_chain;
+
+/* ------------------------------------------------------ template variants */
+/* Cell (Table 1: no_agg, row_agg, col_agg, full_agg) */
+enum { FO_CELL_NO_AGG = 0, FO_CELL_ROW_AGG = 1, FO_CELL_COL_AGG = 2, FO_CELL_FULL_AGG = 3 };
+/* Row (Table 1).  Implemented: ROW_AGG (one value per row), FULL_AGG, COL_T_AGG
+ * (the n x 1 vector sum_i t_i * X_i^T).  NO_AGG, COL_AGG and the *_B1 variants
+ * return FO_ERR_UNSUPPORTED. */
+enum { FO_ROW_NO_AGG = 0, FO_ROW_ROW_AGG = 1, FO_ROW_COL_AGG = 2, FO_ROW_FULL_AGG = 3,
+       FO_ROW_COL_T_AGG = 4 };
+/* Outer (Table 1: left_mm, right_mm, no_agg, full_agg) */
+enum { FO_OUTER_LEFT_MM = 0, FO_OUTER_RIGHT_MM = 1, FO_OUTER_NO_AGG = 2, FO_OUTER_FULL_AGG = 3 };
+
+/* -------------------------------------------------------------- workspace */
+/* Bytes of scratch a call with these arguments needs (0 on invalid arguments).
+ * Pure host arithmetic: usable without a GPU. */
+size_t fused_cell_workspace_bytes(const fo_mat *X, int agg);
+size_t fused_magg_workspace_bytes(const fo_mat *X, int n_out);
+size_t fused_row_workspace_bytes(const fo_mat *X, int agg);
+size_t fused_outer_workspace_bytes(const fo_csr *X, int rank, int agg);
+
+/* Clears the control words at the head of a workspace (asynchronous on `stream`).
+ * Needed once after allocation, and again after a call returned
+ * FO_ERR_DEVICE_TIMEOUT through fo_query_device_status. */
+int fo_workspace_init(void *ws, size_t ws_bytes, void *stream);
+
+/* Synchronises `stream`, then reads the workspace's device-side status word:
+ * *status = FO_OK or FO_ERR_DEVICE_TIMEOUT.  Returns FO_OK unless the query
+ * itself failed. */
+int fo_query_device_status(const void *ws, void *stream, int *status);
+
+const char *fo_status_string(int status);
+
+/* Last CUDA runtime error code seen by a call that returned FO_ERR_CUDA
+ * (thread-local), 0 if none. */
+int fo_last_cuda_error(void);
+
+/* ------------------------------------------------------------------ Cell
+ * Table 1, Cell template; Section 2.2 cell-wise listing.
+ * For every cell (i, j) of a dense main input X (for a CSR main input: every
+ * STORED cell - the sparse-safe binding) the chain computes one value from
+ * a = X_ij, side values and scalars; then
+ *   FO_CELL_FULL_AGG: out[0]        = sum over all cells
+ *   FO_CELL_ROW_AGG : out[i]        = sum over j          (rows doubles)
+ *   FO_CELL_COL_AGG : out[j]        = sum over i          (cols doubles)
+ *   FO_CELL_NO_AGG  : dense X: out[i * cols + j] = value  (rows * cols doubles,
+ *                     packed); CSR X: out[p] = value of stored cell p (nnz
+ *                     doubles, X's pattern).
+ * A CSR main input with a chain that is not zero-preserving gives the result
+ * of the sparse-safe binding, not of the dense one; the caller decides that
+ * (in the paper the compiler marks templates sparse-safe, Section 2.2).
+ * Errors: FO_ERR_CHAIN if the chain uses FO_DOT; FO_ERR_SHAPE if a side does
+ * not match X under its access kind; empty X (no cells) writes zeros.
+ */
+int fused_cell(const fo_chain *chain, const fo_mat *X,
+               const fo_side *sides, int n_sides,
+               const double *scalars, int n_scalars,
+               int agg, double *out, void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------ MAgg
+ * Table 1, MAgg template; Section 5.2 "Multi-Aggregate Operations".
+ * chain->n_out full-sum aggregates over shared inputs in ONE scan:
+ * out[k] = sum over all cells of the chain's k-th result (n_out doubles, the
+ * paper's k x 1 output, in the order of chain->out).
+ */
+int fused_magg(const fo_chain *chain, const fo_mat *X,
+               const fo_side *sides, int n_sides,
+               const double *scalars, int n_scalars,
+               double *out, void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------- Row
+ * Table 1, Row template; Fig. 1(b); Section 5.2 "Row Operations".
+ * One pass over the rows of X (dense or CSR).  For row i:
+ *     d   = X_i . v                    (v: device, X.cols doubles)
+ *     t_i = chain(d, sides read at row i, scalars)     (sides must be FO_AT_ROW)
+ *   FO_ROW_COL_T_AGG: out += t_i * X_i^T   -> out[j] = sum_i t_i X_ij (cols doubles)
+ *   FO_ROW_ROW_AGG  : out[i] = t_i                                   (rows doubles)
+ *   FO_ROW_FULL_AGG : out[0] = sum_i t_i
+ * With the chain  t = side0 * d  this is  t(X) %*% (w * (X %*% v)).
+ * Dense X wider than 8192 columns, or CSR X wider than 16384 columns, returns
+ * FO_ERR_UNSUPPORTED for FO_ROW_COL_T_AGG (the single-pass kernels keep one
+ * row, respectively the output vector, on chip).
+ * Determinism: bit-reproducible except FO_ROW_COL_T_AGG over CSR, whose
+ * scatter-add into on-chip accumulators is unordered.
+ */
+int fused_row(const fo_chain *chain, const fo_mat *X, const double *v,
+              const fo_side *sides, int n_sides,
+              const double *scalars, int n_scalars,
+              int agg, double *out, void *ws, size_t ws_bytes, void *stream);
+
+/* ----------------------------------------------------------------- Outer
+ * Table 1, Outer template; Fig. 1(d), Eq. 1 and the outer-product listing of
+ * Section 2.2.  For every stored cell (i, j) of the CSR matrix X:
+ *     a = X_ij,  d = U_i . V_j  (U: rows x rank, V: cols x rank, dense),
+ *     w_ij = chain(a, d, scalars)
+ *   FO_OUTER_FULL_AGG: out[0] = sum w_ij
+ *   FO_OUTER_NO_AGG  : out[p] = w of stored cell p          (nnz doubles)
+ *   FO_OUTER_RIGHT_MM: out[i * rank + c] = sum_j w_ij V_jc  (rows x rank, packed)
+ *   FO_OUTER_LEFT_MM : out[j * rank + c] = sum_i w_ij U_ic  (cols x rank, packed)
+ * U V^T is never formed; cells that are not stored cost nothing.  Stored
+ * zeros ARE visited (a chain tests a != 0 itself, as the listing does).
+ * rank <= 256.  Errors: FO_ERR_SHAPE if U.rows != X.rows, V.rows != X.cols or
+ * U.cols != V.cols.
+ */
+int fused_outer(const fo_chain *chain, const fo_csr *X,
+                const fo_dense *U, const fo_dense *V,
+                const double *scalars, int n_scalars,
+                int agg, double *out, void *ws, size_t ws_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FUSEDOPS_H */

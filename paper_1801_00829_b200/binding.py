@@ -1,0 +1,393 @@
+"""ctypes binding of libfusedops.so: argument marshalling only.
+
+Every step of the fused operators runs inside the CUDA library.  PyTorch is used
+for device memory (inputs, outputs, the scratch workspace) and for the current
+stream; nothing here computes.  If the library is missing or no CUDA device is
+present the calls raise - there is no CPU path.
+
+Chains are written as lists of steps ``(op, dst, a[, b[, c]])`` with ``dst`` one
+of "t0".."t7" and operands "a" (main value), "d" (dot product), "sideK", "sK"
+(K-th scalar), "tK" or a Python float (an immediate); see include/fusedops.h.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import threading
+
+import torch
+
+from . import build as _build
+
+FO_MAX_OPS, FO_MAX_TMPS, FO_MAX_SIDES, FO_MAX_SCALARS, FO_MAX_OUT = 32, 8, 4, 8, 8
+
+OPCODES = {name: i for i, name in enumerate([
+    "mov", "neg", "abs", "sqrt", "exp", "log", "sq",
+    "add", "sub", "mul", "div", "min", "max", "pow",
+    "eq", "ne", "lt", "le", "gt", "ge", "sel", "fma"])}
+ARITY = {**{n: 1 for n in ("mov", "neg", "abs", "sqrt", "exp", "log", "sq")},
+         **{n: 2 for n in ("add", "sub", "mul", "div", "min", "max", "pow",
+                           "eq", "ne", "lt", "le", "gt", "ge")},
+         "sel": 3, "fma": 3}
+
+CELL_AGG = {"none": 0, "row": 1, "col": 2, "full": 3}
+ROW_AGG = {"none": 0, "row": 1, "col": 2, "full": 3, "col_t": 4}
+OUTER_AGG = {"left": 0, "right": 1, "none": 2, "full": 3}
+ACCESS = {"cell": 0, "row": 1, "col": 2}
+
+STATUS = {0: "FO_OK", -1: "FO_ERR_NULL", -2: "FO_ERR_SHAPE", -3: "FO_ERR_CHAIN",
+          -4: "FO_ERR_UNSUPPORTED", -5: "FO_ERR_WORKSPACE", -6: "FO_ERR_CUDA",
+          -7: "FO_ERR_DEVICE_TIMEOUT"}
+
+
+class FusedOpsError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        super().__init__("%s: %s (%s)" % (what, STATUS.get(status, status), _status_text(status)))
+
+
+# ------------------------------------------------------------------ C structs
+class fo_dense(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("ld", C.c_int64), ("data", C.c_void_p)]
+
+
+class fo_csr(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("nnz", C.c_int64),
+                ("rowptr", C.c_void_p), ("colidx", C.c_void_p), ("vals", C.c_void_p)]
+
+
+class fo_mat(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("reserved", C.c_int32), ("dense", fo_dense), ("csr", fo_csr)]
+
+
+class fo_side(C.Structure):
+    _fields_ = [("m", fo_dense), ("access", C.c_int32), ("reserved", C.c_int32)]
+
+
+class fo_op(C.Structure):
+    _fields_ = [("opcode", C.c_uint8), ("dst", C.c_uint8), ("a", C.c_uint8), ("b", C.c_uint8),
+                ("c", C.c_uint8), ("reserved", C.c_uint8 * 3), ("imm", C.c_double)]
+
+
+class fo_chain(C.Structure):
+    _fields_ = [("n_ops", C.c_int32), ("n_out", C.c_int32), ("ops", C.POINTER(fo_op)),
+                ("out", C.c_uint8 * FO_MAX_OUT)]
+
+
+EXPORTS = [
+    "fused_cell", "fused_magg", "fused_row", "fused_outer",
+    "fused_cell_workspace_bytes", "fused_magg_workspace_bytes", "fused_row_workspace_bytes",
+    "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
+    "fo_status_string", "fo_last_cuda_error",
+]
+
+_lib = None
+_lock = threading.Lock()
+
+
+def load_library(path=None):
+    """Loads (building first if stale) libfusedops.so and declares its prototypes."""
+    global _lib
+    with _lock:
+        if _lib is not None and path is None:
+            return _lib
+        lib = C.CDLL(path or _build.build_library())
+        vp, dp, i32, sz = C.c_void_p, C.c_void_p, C.c_int, C.c_size_t
+        chain_p, mat_p, side_p = C.POINTER(fo_chain), C.POINTER(fo_mat), C.POINTER(fo_side)
+        scal_p = C.POINTER(C.c_double)
+        lib.fused_cell.argtypes = [chain_p, mat_p, side_p, i32, scal_p, i32, i32, dp, vp, sz, vp]
+        lib.fused_magg.argtypes = [chain_p, mat_p, side_p, i32, scal_p, i32, dp, vp, sz, vp]
+        lib.fused_row.argtypes = [chain_p, mat_p, dp, side_p, i32, scal_p, i32, i32, dp, vp, sz, vp]
+        lib.fused_outer.argtypes = [chain_p, C.POINTER(fo_csr), C.POINTER(fo_dense),
+                                    C.POINTER(fo_dense), scal_p, i32, i32, dp, vp, sz, vp]
+        for f in (lib.fused_cell, lib.fused_magg, lib.fused_row, lib.fused_outer):
+            f.restype = C.c_int
+        lib.fused_cell_workspace_bytes.argtypes = [mat_p, i32]
+        lib.fused_magg_workspace_bytes.argtypes = [mat_p, i32]
+        lib.fused_row_workspace_bytes.argtypes = [mat_p, i32]
+        lib.fused_outer_workspace_bytes.argtypes = [C.POINTER(fo_csr), i32, i32]
+        for f in (lib.fused_cell_workspace_bytes, lib.fused_magg_workspace_bytes,
+                  lib.fused_row_workspace_bytes, lib.fused_outer_workspace_bytes):
+            f.restype = C.c_size_t
+        lib.fo_workspace_init.argtypes = [vp, sz, vp]
+        lib.fo_workspace_init.restype = C.c_int
+        lib.fo_query_device_status.argtypes = [vp, vp, C.POINTER(C.c_int)]
+        lib.fo_query_device_status.restype = C.c_int
+        lib.fo_status_string.argtypes = [C.c_int]
+        lib.fo_status_string.restype = C.c_char_p
+        lib.fo_last_cuda_error.argtypes = []
+        lib.fo_last_cuda_error.restype = C.c_int
+        if path is None:
+            _lib = lib
+        return lib
+
+
+def _status_text(status):
+    try:
+        return load_library().fo_status_string(int(status)).decode()
+    except Exception:
+        return "?"
+
+
+def _check(status, what):
+    if status != 0:
+        raise FusedOpsError(status, what)
+
+
+# ------------------------------------------------------------------ marshalling
+def _operand(x, allow_imm=True):
+    """Operand name -> (operand byte, immediate or None)."""
+    if isinstance(x, (int, float)) and not isinstance(x, bool):
+        if not allow_imm:
+            raise ValueError("an output cannot be an immediate")
+        return 0xC2, float(x)
+    if not isinstance(x, str):
+        raise ValueError("bad operand %r" % (x,))
+    if x == "a":
+        return 0xC0, None
+    if x == "d":
+        return 0xC1, None
+    if x.startswith("side") and x[4:].isdigit():
+        return 0x40 | int(x[4:]), None
+    if x[0] == "t" and x[1:].isdigit():
+        return 0x00 | int(x[1:]), None
+    if x[0] == "s" and x[1:].isdigit():
+        return 0x80 | int(x[1:]), None
+    raise ValueError("bad operand %r" % (x,))
+
+
+def make_chain(steps, outputs):
+    """Builds the fo_chain for `steps` and `outputs`; returns (chain, keepalive)."""
+    steps = list(steps)
+    outputs = [outputs] if isinstance(outputs, (str, float, int)) else list(outputs)
+    if len(steps) > 255 or len(outputs) > FO_MAX_OUT:
+        raise ValueError("chain too long")
+    ops = (fo_op * max(1, len(steps)))()
+    for i, st in enumerate(steps):
+        name, dst, srcs = st[0], st[1], st[2:]
+        if name not in OPCODES:
+            raise ValueError("unknown op %r" % (name,))
+        if len(srcs) != ARITY[name]:
+            raise ValueError("%s takes %d operands" % (name, ARITY[name]))
+        if not (isinstance(dst, str) and dst[0] == "t" and dst[1:].isdigit()):
+            raise ValueError("dst must be a temporary, got %r" % (dst,))
+        ops[i].opcode = OPCODES[name]
+        ops[i].dst = int(dst[1:]) & 0xff
+        imm = None
+        enc = []
+        for s in srcs:
+            b, im = _operand(s)
+            if im is not None:
+                if imm is not None and imm != im:
+                    raise ValueError("a step can carry one immediate value")
+                imm = im
+            enc.append(b)
+        enc += [0] * (3 - len(enc))
+        ops[i].a, ops[i].b, ops[i].c = enc
+        ops[i].imm = imm if imm is not None else 0.0
+    ch = fo_chain()
+    ch.n_ops = len(steps)
+    ch.n_out = len(outputs)
+    ch.ops = C.cast(ops, C.POINTER(fo_op))
+    for k, o in enumerate(outputs):
+        ch.out[k] = _operand(o, allow_imm=False)[0]
+    return ch, ops
+
+
+class CSR:
+    """A CSR matrix held in device tensors (int32 rowptr / colidx, float64 vals)."""
+
+    def __init__(self, rows, cols, rowptr, colidx, vals):
+        self.rows, self.cols = int(rows), int(cols)
+        self.rowptr, self.colidx, self.vals = rowptr, colidx, vals
+        assert rowptr.dtype == torch.int32 and colidx.dtype == torch.int32
+        assert vals.dtype == torch.float64
+        assert rowptr.numel() == self.rows + 1 and colidx.numel() == vals.numel()
+        self.nnz = int(vals.numel())
+
+    @property
+    def device(self):
+        return self.vals.device
+
+    def as_struct(self):
+        s = fo_csr()
+        s.rows, s.cols, s.nnz = self.rows, self.cols, self.nnz
+        s.rowptr, s.colidx, s.vals = self.rowptr.data_ptr(), self.colidx.data_ptr(), self.vals.data_ptr()
+        return s
+
+
+def _dense_struct(t, column=False):
+    """fo_dense of a float64 tensor.  2-D: rows must be contiguous (stride(1) == 1).
+    1-D: a row vector (1 x n, contiguous), or with column=True a column vector
+    (n x 1) whose stride becomes the leading dimension."""
+    assert t.dtype == torch.float64, "float64 only"
+    d = fo_dense()
+    d.data = t.data_ptr()
+    if t.dim() == 1 and column:
+        d.rows, d.cols = t.numel(), 1
+        d.ld = max(int(t.stride(0)), 1) if t.numel() > 1 else 1
+    elif t.dim() == 1:
+        assert t.numel() <= 1 or t.stride(0) == 1, "row vectors must be contiguous"
+        d.rows, d.cols = 1, t.numel()
+        d.ld = max(t.numel(), 1)
+    else:
+        assert t.dim() == 2
+        r, c = t.shape
+        assert t.numel() == 0 or c == 1 or t.stride(1) == 1, "rows must be contiguous"
+        d.rows, d.cols = r, c
+        d.ld = max(int(t.stride(0)) if r > 1 else c, c, 1)
+    return d
+
+
+def _mat(X):
+    m = fo_mat()
+    if isinstance(X, CSR):
+        m.kind = 1
+        m.csr = X.as_struct()
+    else:
+        m.kind = 0
+        m.dense = _dense_struct(X)
+    return m
+
+
+def _sides(sides, rows, cols):
+    arr = (fo_side * max(1, len(sides)))()
+    for k, (access, t) in enumerate(sides):
+        acc = ACCESS[access]
+        if acc == 0:
+            arr[k].m = _dense_struct(t)
+        elif acc == 1:
+            assert t.dim() == 1 or (t.dim() == 2 and t.shape[1] == 1)
+            t1 = t if t.dim() == 1 else t[:, 0]
+            arr[k].m = _dense_struct(t1, column=True)
+        else:
+            assert t.dim() == 1 or (t.dim() == 2 and t.shape[0] == 1)
+            t1 = t if t.dim() == 1 else t[0]
+            arr[k].m = _dense_struct(t1)
+        arr[k].access = acc
+    return arr
+
+
+def _scalars(scalars):
+    arr = (C.c_double * max(1, len(scalars)))(*[float(s) for s in scalars])
+    return arr
+
+
+def _stream(device):
+    return C.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+# ------------------------------------------------------------------ workspace
+_ws = {}
+
+
+def workspace(device, nbytes):
+    """A cached, initialised scratch buffer of at least nbytes on `device`."""
+    if device.type != "cuda":
+        raise RuntimeError("fused operators need CUDA tensors (no CPU path)")
+    key = (device.index if device.index is not None else torch.cuda.current_device())
+    buf = _ws.get(key)
+    if buf is None or buf.numel() < nbytes:
+        size = max(int(nbytes), 1 << 20)
+        buf = torch.empty(size, dtype=torch.uint8, device=device)
+        assert buf.data_ptr() % 256 == 0
+        _check(load_library().fo_workspace_init(C.c_void_p(buf.data_ptr()), buf.numel(),
+                                                _stream(device)), "fo_workspace_init")
+        _ws[key] = buf
+    return buf
+
+
+def device_status(device=None):
+    """Synchronises and returns the workspace's device-side status (0 = ok)."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    buf = workspace(device, 256)
+    st = C.c_int(0)
+    _check(load_library().fo_query_device_status(C.c_void_p(buf.data_ptr()), _stream(device),
+                                                 C.byref(st)), "fo_query_device_status")
+    return st.value
+
+
+# ------------------------------------------------------------------ the four calls
+def fused_cell(steps, output, X, sides=(), scalars=(), agg="full", out=None):
+    """Cell template.  Returns a tensor: scalar (1,), (rows,), (cols,) or (rows, cols)."""
+    lib = load_library()
+    sides = list(sides)
+    ch, keep = make_chain(steps, output)
+    m = _mat(X)
+    rows, cols = (X.rows, X.cols) if isinstance(X, CSR) else X.shape
+    dev = X.device
+    a = CELL_AGG[agg]
+    if out is None:
+        shape = {"full": (1,), "row": (rows,), "col": (cols,),
+                 "none": (X.nnz,) if isinstance(X, CSR) else (rows, cols)}[agg]
+        out = torch.empty(shape, dtype=torch.float64, device=dev)
+    need = lib.fused_cell_workspace_bytes(C.byref(m), a)
+    ws = workspace(dev, max(need, 256))
+    sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
+    _check(lib.fused_cell(C.byref(ch), C.byref(m), sarr, len(sides), sc, len(scalars), a,
+                          C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
+                          _stream(dev)), "fused_cell")
+    return out
+
+
+def fused_magg(steps, outputs, X, sides=(), scalars=(), out=None):
+    """MAgg template.  Returns a (k,) tensor, one full sum per output."""
+    lib = load_library()
+    sides = list(sides)
+    outputs = list(outputs)
+    ch, keep = make_chain(steps, outputs)
+    m = _mat(X)
+    rows, cols = X.shape
+    dev = X.device
+    if out is None:
+        out = torch.empty(len(outputs), dtype=torch.float64, device=dev)
+    need = lib.fused_magg_workspace_bytes(C.byref(m), len(outputs))
+    ws = workspace(dev, max(need, 256))
+    sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
+    _check(lib.fused_magg(C.byref(ch), C.byref(m), sarr, len(sides), sc, len(scalars),
+                          C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
+                          _stream(dev)), "fused_magg")
+    return out
+
+
+def fused_row(steps, output, X, v, sides=(), scalars=(), agg="col_t", out=None):
+    """Row template.  Returns (cols,), (rows,) or (1,)."""
+    lib = load_library()
+    sides = list(sides)
+    ch, keep = make_chain(steps, output)
+    m = _mat(X)
+    rows, cols = (X.rows, X.cols) if isinstance(X, CSR) else X.shape
+    dev = X.device
+    a = ROW_AGG[agg]
+    assert v.dtype == torch.float64 and v.numel() == cols and (v.numel() <= 1 or v.stride(-1) == 1)
+    if out is None:
+        shape = {"col_t": (cols,), "row": (rows,), "full": (1,)}.get(agg, (1,))
+        out = torch.empty(shape, dtype=torch.float64, device=dev)
+    need = lib.fused_row_workspace_bytes(C.byref(m), a)
+    ws = workspace(dev, max(need, 256))
+    sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
+    _check(lib.fused_row(C.byref(ch), C.byref(m), C.c_void_p(v.data_ptr()), sarr, len(sides), sc,
+                         len(scalars), a, C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()),
+                         ws.numel(), _stream(dev)), "fused_row")
+    return out
+
+
+def fused_outer(steps, output, X, U, V, scalars=(), agg="full", out=None):
+    """Outer template over the stored cells of the CSR matrix X."""
+    lib = load_library()
+    ch, keep = make_chain(steps, output)
+    xs = X.as_struct()
+    us, vs = _dense_struct(U), _dense_struct(V)
+    dev = X.device
+    a = OUTER_AGG[agg]
+    rank = U.shape[1]
+    if out is None:
+        shape = {"full": (1,), "none": (X.nnz,), "right": (X.rows, rank), "left": (X.cols, rank)}[agg]
+        out = torch.empty(shape, dtype=torch.float64, device=dev)
+    need = lib.fused_outer_workspace_bytes(C.byref(xs), rank, a)
+    ws = workspace(dev, max(need, 256))
+    sc = _scalars(scalars)
+    _check(lib.fused_outer(C.byref(ch), C.byref(xs), C.byref(us), C.byref(vs), sc, len(scalars), a,
+                           C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
+                           _stream(dev)), "fused_outer")
+    return out

@@ -1,0 +1,507 @@
+// Row template (Table 1; Fig. 1(b); Section 5.2 "Row Operations"): one pass over
+// the rows of X computing, per row i,  d = X_i . v,  t_i = chain(d, sides_i),
+// and then  out += t_i * X_i^T  (col_t_agg),  out[i] = t_i  (row_agg)  or
+// out = sum_i t_i  (full_agg).  The row is read from HBM once and used twice
+// from on-chip memory - the GPU form of the paper's "each row fits L1" argument.
+//
+// Dense X: a CTA streams tiles of rows into a shared-memory ring with bulk
+// asynchronous copies (mbarrier-tracked, waits bounded); each warp owns one
+// row at a time: lanes hold the row, their slice of v and of the output
+// accumulator in registers.  CSR X: an 8-lane group per row; v and the output
+// accumulator live in shared memory.
+#include "chain.cuh"
+
+namespace fo {
+
+namespace {
+
+struct RowParams {
+    const double *X;            // dense
+    const int *rowptr;          // CSR
+    const int *colidx;
+    const double *vals;
+    long long rows, cols, ldx;
+    const double *v;
+    DevSides sides;
+    WsHead *head;
+    double *partials;
+    double *out;
+    int stages, rows_per_stage; // dense ring geometry
+};
+
+enum { kRowColT = 0, kRowRow = 1, kRowFull = 2 };
+
+constexpr int kWarps = kThreads / 32;
+constexpr unsigned kWaitLimit = 1u << 22;     // polls of one mbarrier wait before giving up
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ unsigned smem_u32(const void *p)
+{
+    return (unsigned)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: returns false (and the caller records it) if the phase never completes.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity)
+{
+    for (unsigned i = 0; i < kWaitLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// Bulk asynchronous copy global -> shared; completion is counted on `bar`.
+// src, dst 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes,
+                                         unsigned long long *bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Evaluates the row chain: R0 = d, R(1+k) = side k at this row.
+__device__ __forceinline__ double row_chain(const DevChain &ch, double d, const double (&sv)[FO_MAX_SIDES])
+{
+    RegFile<kRegs, 1> f;
+    f.r[0][0] = d;
+#pragma unroll
+    for (int k = 0; k < FO_MAX_SIDES; ++k) f.r[1 + k][0] = sv[k];
+    run_chain<kRegs, 1>(ch, f);
+    double o[1];
+    operand<kRegs, 1>(ch, f, ch.out[0], o);
+    return o[0];
+}
+
+__device__ __forceinline__ void load_sides(const DevChain &ch, const DevSides &sides, long long row,
+                                           long long rows, double (&sv)[FO_MAX_SIDES])
+{
+#pragma unroll
+    for (int k = 0; k < FO_MAX_SIDES; ++k) {
+        sv[k] = 0.0;
+        if (((ch.side_used >> k) & 1u) && row < rows)
+            sv[k] = __ldg(sides.s[k].data + row * sides.s[k].ld);
+    }
+}
+
+// ------------------------------------------------------------------ dense
+// NCH: 64-column chunks per row held by a warp (cols <= 64 * NCH).
+// STAGED: rows arrive through the shared-memory ring; otherwise lanes load
+// their pairs straight from global memory (any alignment, any cols).
+template <int NCH, int AGG, bool STAGED>
+__global__ void __launch_bounds__(kThreads, 1)
+row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ unsigned long long s_full[8];
+    __shared__ double s_red[32];
+    __shared__ unsigned int s_flag;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long n = p.cols;
+    const int RPS = p.rows_per_stage, S = p.stages;
+    const int RPW = RPS / kWarps;
+    double *ring = reinterpret_cast<double *>(smem_raw);
+    const long long ntiles = (p.rows + RPS - 1) / RPS;
+    const long long my_tiles = (ntiles > blockIdx.x) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    // v lives in shared memory behind the ring, padded with zeros to 64 * NCH
+    double *vs = ring + (size_t)(STAGED ? S : 0) * RPS * n + (AGG == kRowColT && !STAGED ? kWarps * n : 0);
+    for (int j = threadIdx.x; j < 64 * NCH; j += kThreads) vs[j] = j < n ? __ldg(p.v + j) : 0.0;
+    double2 q[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) q[c] = make_double2(0.0, 0.0);
+    double tsum = 0.0;
+    bool timed_out = false;
+
+    auto issue = [&](long long it) {
+        const long long tile = blockIdx.x + it * gridDim.x;
+        const int slot = (int)(it % S);
+        const long long r0 = tile * RPS;
+        const int nr = (int)((p.rows - r0 < RPS) ? p.rows - r0 : RPS);
+        double *dst = ring + (size_t)slot * RPS * n;
+        mbar_expect_tx(&s_full[slot], (unsigned)(nr * n * 8));
+        if (p.ldx == n) {
+            bulk_g2s(dst, p.X + r0 * p.ldx, (unsigned)(nr * n * 8), &s_full[slot]);
+        } else {
+            for (int r = 0; r < nr; ++r)
+                bulk_g2s(dst + (size_t)r * n, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &s_full[slot]);
+        }
+    };
+
+    __syncthreads();
+    if (STAGED) {
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < S; ++s) mbar_init(&s_full[s], 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (long long it = 0; it < S - 1 && it < my_tiles; ++it) issue(it);
+    }
+
+    for (long long it = 0; it < my_tiles; ++it) {
+        const long long tile = blockIdx.x + it * gridDim.x;
+        const long long r0 = tile * RPS;
+        const int slot = (int)(it % S);
+        if (STAGED) {
+            if (threadIdx.x == 0 && it + S - 1 < my_tiles) issue(it + S - 1);
+        }
+        // side values of this warp's rows: requested before the wait so their
+        // latency overlaps it
+        double sv[4][FO_MAX_SIDES];
+#pragma unroll
+        for (int rw = 0; rw < 4; ++rw)
+            if (rw < RPW) load_sides(ch, p.sides, r0 + warp * RPW + rw, p.rows, sv[rw]);
+        if (STAGED) {
+            if (!mbar_wait(&s_full[slot], (unsigned)((it / S) & 1))) timed_out = true;
+        }
+        for (int rw = 0; rw < RPW; ++rw) {
+            const int rl = warp * RPW + rw;
+            const long long row = r0 + rl;
+            if (row >= p.rows) break;
+            double2 x[NCH];
+            double d0 = 0.0, d1 = 0.0;
+            if (STAGED) {
+                const double *rowp = ring + ((size_t)slot * RPS + rl) * n;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const long long col = 64 * c + 2 * lane;
+                    x[c] = (col < n) ? *reinterpret_cast<const double2 *>(rowp + col)
+                                     : make_double2(0.0, 0.0);
+                }
+            } else {
+                const double *rowp = p.X + row * p.ldx;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    const long long col = 64 * c + 2 * lane;
+                    x[c].x = col < n ? ld_stream1(rowp + col) : 0.0;
+                    x[c].y = col + 1 < n ? ld_stream1(rowp + col + 1) : 0.0;
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                const double2 vv = *reinterpret_cast<const double2 *>(vs + 64 * c + 2 * lane);
+                d0 = fma(x[c].x, vv.x, d0);
+                d1 = fma(x[c].y, vv.y, d1);
+            }
+            const double d = warp_sum(d0 + d1);
+            double svr[FO_MAX_SIDES];
+#pragma unroll
+            for (int k = 0; k < FO_MAX_SIDES; ++k) {
+                svr[k] = sv[0][k];
+#pragma unroll
+                for (int r2 = 1; r2 < 4; ++r2)
+                    if (rw == r2) svr[k] = sv[r2][k];
+            }
+            const double t = row_chain(ch, d, svr);
+            if (AGG == kRowColT) {
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    q[c].x = fma(t, x[c].x, q[c].x);
+                    q[c].y = fma(t, x[c].y, q[c].y);
+                }
+            } else if (AGG == kRowRow) {
+                if (lane == 0) p.out[row] = t;
+            } else {
+                tsum += t;
+            }
+        }
+        if (STAGED) __syncthreads();      // the slot may be refilled from now on
+    }
+
+    if (STAGED && timed_out) atomicExch(&p.head->status, 1u);
+
+    if (AGG == kRowColT) {
+        // warps -> CTA: fixed order over warps, through shared memory
+        __syncthreads();
+        double *qs = ring;                // kWarps * n doubles fit in one ring stage
+        if (!STAGED) qs = reinterpret_cast<double *>(smem_raw);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+            const long long col = 64 * c + 2 * lane;
+            if (col < n) qs[(size_t)warp * n + col] = q[c].x;
+            if (col + 1 < n) qs[(size_t)warp * n + col + 1] = q[c].y;
+        }
+        __syncthreads();
+        for (long long j = threadIdx.x; j < n; j += kThreads) {
+            double s = 0.0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) s += qs[(size_t)w * n + j];
+            p.partials[(size_t)blockIdx.x * n + j] = s;
+        }
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_columns(p.partials, gridDim.x, n, p.out);
+    } else if (AGG == kRowFull) {
+        // every lane of a warp holds the same tsum: count it once per warp
+        double v1[1] = {lane == 0 ? tsum : 0.0};
+        block_sum<1>(v1, s_red);
+        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
+    }
+}
+
+// -------------------------------------------------------------------- CSR
+// An 8-lane group per row.  v (and for col_t_agg the output accumulator) sit in
+// shared memory; the scatter  acc[col] += t * val  uses shared-memory atomics
+// because two groups may hit the same column at the same time.
+template <int AGG>
+__global__ void __launch_bounds__(kThreads)
+row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ double s_red[32];
+    __shared__ unsigned int s_flag;
+    const long long n = p.cols;
+    double *vs = reinterpret_cast<double *>(smem_raw);
+    double *qs = vs + n;
+    for (long long j = threadIdx.x; j < n; j += kThreads) {
+        vs[j] = __ldg(p.v + j);
+        if (AGG == kRowColT) qs[j] = 0.0;
+    }
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int l8 = lane & 7;
+    const unsigned gmask = 0xffu << (lane & 24);
+    const long long group0 = ((long long)blockIdx.x * kThreads + threadIdx.x) >> 3;
+    const long long ngroups = ((long long)gridDim.x * kThreads) >> 3;
+    double tsum = 0.0;
+
+    // rows are dealt to CTAs in contiguous blocks of (groups per CTA) rows, so a
+    // warp's four groups read neighbouring parts of colidx / vals
+    for (long long row = group0; row < p.rows; row += ngroups) {
+        const int beg = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
+        double sv[FO_MAX_SIDES];
+        load_sides(ch, p.sides, row, p.rows, sv);
+        double d = 0.0;
+        for (int q0 = beg + l8; q0 < end; q0 += 8)
+            d = fma(__ldg(p.vals + q0), vs[__ldg(p.colidx + q0)], d);
+        d += __shfl_xor_sync(gmask, d, 4);
+        d += __shfl_xor_sync(gmask, d, 2);
+        d += __shfl_xor_sync(gmask, d, 1);
+        const double t = row_chain(ch, d, sv);
+        if (AGG == kRowColT) {
+            for (int q0 = beg + l8; q0 < end; q0 += 8)
+                atomicAdd(&qs[__ldg(p.colidx + q0)], t * __ldg(p.vals + q0));
+        } else if (AGG == kRowRow) {
+            if (l8 == 0) p.out[row] = t;
+        } else {
+            if (l8 == 0) tsum += t;
+        }
+    }
+
+    if (AGG == kRowColT) {
+        __syncthreads();
+        for (long long j = threadIdx.x; j < n; j += kThreads)
+            p.partials[(size_t)blockIdx.x * n + j] = qs[j];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_columns(p.partials, gridDim.x, n, p.out);
+    } else if (AGG == kRowFull) {
+        double v1[1] = {tsum};
+        block_sum<1>(v1, s_red);
+        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
+    }
+}
+
+__global__ void row_fill_zero_kernel(double *out, long long n)
+{
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+         i += (long long)gridDim.x * blockDim.x)
+        out[i] = 0.0;
+}
+
+// ------------------------------------------------------------------- host
+constexpr long long kDenseMaxCols = 1024;
+constexpr long long kCsrMaxCols = 8192;
+constexpr size_t kRingBudget = 208 * 1024;
+
+bool aligned16(const void *q) { return ((uintptr_t)q & 15u) == 0; }
+
+int row_grid_cap() { return 148 * 4; }     // bound used for workspace sizing
+
+size_t row_ws_bytes(long long cols, int agg)
+{
+    if (agg == FO_ROW_COL_T_AGG)
+        return sizeof(WsHead) + (size_t)row_grid_cap() * (size_t)cols * sizeof(double);
+    if (agg == FO_ROW_FULL_AGG) return sizeof(WsHead) + (size_t)row_grid_cap() * sizeof(double);
+    return sizeof(WsHead);
+}
+
+template <int NCH, bool STAGED>
+cudaError_t launch_dense_agg(const DevChain &ch, const RowParams &p, int agg, int grid, size_t smem,
+                             cudaStream_t st)
+{
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, kThreads, smem, st>>>(ch, p);
+        return cudaGetLastError();
+    };
+    if (agg == FO_ROW_COL_T_AGG) return go(row_dense_kernel<NCH, kRowColT, STAGED>);
+    if (agg == FO_ROW_ROW_AGG) return go(row_dense_kernel<NCH, kRowRow, STAGED>);
+    return go(row_dense_kernel<NCH, kRowFull, STAGED>);
+}
+
+template <bool STAGED>
+cudaError_t launch_dense(const DevChain &ch, const RowParams &p, int agg, int grid, size_t smem,
+                         cudaStream_t st)
+{
+    const long long n = p.cols;
+    if (n <= 64) return launch_dense_agg<1, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 128) return launch_dense_agg<2, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 256) return launch_dense_agg<4, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 512) return launch_dense_agg<8, STAGED>(ch, p, agg, grid, smem, st);
+    return launch_dense_agg<16, STAGED>(ch, p, agg, grid, smem, st);
+}
+
+}  // namespace
+
+}  // namespace fo
+
+extern "C" {
+
+size_t fused_row_workspace_bytes(const fo_mat *X, int agg)
+{
+    if (!X) return 0;
+    if (agg != FO_ROW_COL_T_AGG && agg != FO_ROW_ROW_AGG && agg != FO_ROW_FULL_AGG) return 0;
+    const long long cols = X->kind == FO_DENSE ? X->dense.cols : X->kind == FO_CSR ? X->csr.cols : -1;
+    if (cols < 0) return 0;
+    return fo::row_ws_bytes(cols, agg);
+}
+
+int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_side *sides,
+              int n_sides, const double *scalars, int n_scalars, int agg, double *out, void *ws,
+              size_t ws_bytes, void *stream)
+{
+    using namespace fo;
+    if (!chain || !X || !out) return FO_ERR_NULL;
+    if (n_sides > 0 && !sides) return FO_ERR_NULL;
+    if (agg == FO_ROW_NO_AGG || agg == FO_ROW_COL_AGG) return FO_ERR_UNSUPPORTED;
+    if (agg != FO_ROW_COL_T_AGG && agg != FO_ROW_ROW_AGG && agg != FO_ROW_FULL_AGG)
+        return FO_ERR_UNSUPPORTED;
+    if (X->kind != FO_DENSE && X->kind != FO_CSR) return FO_ERR_SHAPE;
+    const bool csr = X->kind == FO_CSR;
+    const long long rows = csr ? X->csr.rows : X->dense.rows;
+    const long long cols = csr ? X->csr.cols : X->dense.cols;
+    if (rows < 0 || cols < 0) return FO_ERR_SHAPE;
+    if (csr) {
+        if (X->csr.nnz < 0 || X->csr.nnz >= (1ll << 31)) return FO_ERR_UNSUPPORTED;
+        if (!X->csr.rowptr) return FO_ERR_NULL;
+        if (X->csr.nnz > 0 && (!X->csr.colidx || !X->csr.vals)) return FO_ERR_NULL;
+    } else {
+        if (X->dense.ld < cols) return FO_ERR_SHAPE;
+        if (rows > 0 && cols > 0 && !X->dense.data) return FO_ERR_NULL;
+    }
+    if (cols > 0 && !v) return FO_ERR_NULL;
+
+    DevChain ch;
+    int rc = translate_chain(chain, kUseRow, n_sides, scalars, n_scalars, 1, 1, &ch);
+    if (rc != FO_OK) return rc;
+
+    RowParams p;
+    memset(&p, 0, sizeof(p));
+    p.rows = rows; p.cols = cols; p.v = v;
+    p.sides.n = n_sides;
+    for (int k = 0; k < n_sides; ++k) {
+        const fo_side &s = sides[k];
+        if (s.access != FO_AT_ROW) return FO_ERR_SHAPE;
+        if (s.m.rows != rows || s.m.cols != 1 || s.m.ld < 1) return FO_ERR_SHAPE;
+        if (rows > 0 && !s.m.data) return FO_ERR_NULL;
+        p.sides.s[k].data = s.m.data;
+        p.sides.s[k].ld = s.m.ld;
+        p.sides.s[k].access = s.access;
+    }
+    if (agg == FO_ROW_COL_T_AGG && cols > (csr ? kCsrMaxCols : kDenseMaxCols)) return FO_ERR_UNSUPPORTED;
+    if (cols > kCsrMaxCols) return FO_ERR_UNSUPPORTED;
+    if (!csr && cols > kDenseMaxCols) return FO_ERR_UNSUPPORTED;
+
+    rc = check_workspace(ws, ws_bytes, row_ws_bytes(cols, agg));
+    if (rc != FO_OK) return rc;
+    p.head = (WsHead *)ws;
+    p.partials = (double *)((char *)ws + sizeof(WsHead));
+    p.out = out;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    const long long nout = agg == FO_ROW_COL_T_AGG ? cols : agg == FO_ROW_ROW_AGG ? rows : 1;
+    if (rows == 0 || cols == 0) {
+        // no rows: empty sums; no columns: d = 0 for every row, which the chain may
+        // still map to a non-zero t - handled by the kernels below unless rows == 0
+        if (rows == 0 || agg == FO_ROW_COL_T_AGG) {
+            if (nout > 0) {
+                const long long b = (nout + 255) / 256;
+                row_fill_zero_kernel<<<(unsigned)(b > 1024 ? 1024 : b), 256, 0, st>>>(out, nout);
+            }
+            const cudaError_t e = cudaGetLastError();
+            return e == cudaSuccess ? FO_OK : cuda_fail(e);
+        }
+    }
+
+    const int sms = sm_count();
+    if (sms <= 0) return cuda_fail(cudaErrorNoDevice);
+    cudaError_t e;
+    if (csr) {
+        p.rowptr = X->csr.rowptr; p.colidx = X->csr.colidx; p.vals = X->csr.vals;
+        const size_t smem = (size_t)cols * 8 * (agg == FO_ROW_COL_T_AGG ? 2 : 1);
+        long long grid = (rows + (kThreads / 8) - 1) / (kThreads / 8);
+        const long long cap = (long long)sms * 4 < row_grid_cap() ? (long long)sms * 4 : row_grid_cap();
+        if (grid > cap) grid = cap;
+        auto go = [&](auto kern) -> cudaError_t {
+            cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e2 != cudaSuccess) return e2;
+            kern<<<(unsigned)grid, kThreads, smem, st>>>(ch, p);
+            return cudaGetLastError();
+        };
+        if (agg == FO_ROW_COL_T_AGG) e = go(row_csr_kernel<kRowColT>);
+        else if (agg == FO_ROW_ROW_AGG) e = go(row_csr_kernel<kRowRow>);
+        else e = go(row_csr_kernel<kRowFull>);
+    } else {
+        p.X = X->dense.data; p.ldx = X->dense.ld;
+        const bool staged = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
+        // ring geometry: stages of about 64 KB, whole rows, a multiple of kWarps rows
+        int rpw = (int)((64 * 1024) / (cols * 8 * kWarps));
+        if (rpw < 1) rpw = 1;
+        if (rpw > 4) rpw = 4;
+        p.rows_per_stage = rpw * kWarps;
+        const size_t stage_bytes = (size_t)p.rows_per_stage * cols * 8;
+        int stages = (int)(kRingBudget / stage_bytes);
+        if (stages > 4) stages = 4;
+        if (stages < 2) stages = 2;
+        p.stages = staged ? stages : 1;
+        size_t smem = staged ? stage_bytes * stages : 0;       // the ring
+        if (!staged && agg == FO_ROW_COL_T_AGG) smem = (size_t)kWarps * cols * 8;   // warp partials
+        smem += 1024 * 8;                                      // v, zero-padded
+        const long long ntiles = (rows + p.rows_per_stage - 1) / p.rows_per_stage;
+        long long grid = ntiles < sms ? ntiles : sms;
+        if (grid > row_grid_cap()) grid = row_grid_cap();
+        if (grid < 1) grid = 1;
+        e = staged ? launch_dense<true>(ch, p, agg, (int)grid, smem, st)
+                   : launch_dense<false>(ch, p, agg, (int)grid, smem, st);
+    }
+    return e == cudaSuccess ? FO_OK : cuda_fail(e);
+}
+
+}  // extern "C"

@@ -1,0 +1,188 @@
+"""Host-side checks of the C ABI that need no GPU: the library builds, loads and
+exports every function include/fusedops.h declares; workspace sizes are plain
+arithmetic; invalid arguments are refused with the documented status before
+anything touches the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+import paper_1801_00829_b200.binding as B  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def lib():
+    return B.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "fusedops.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"^(?:int|size_t|const char \*)\s*(\w+)\s*\(", text, flags=re.M)
+    return names
+
+
+def test_header_functions_are_exported(lib):
+    names = declared_functions()
+    assert set(names) == set(B.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_status_strings(lib):
+    seen = set()
+    for code in range(0, -8, -1):
+        s = lib.fo_status_string(code).decode()
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 8
+    assert lib.fo_status_string(-99).decode() == "unknown status"
+
+
+def dense_mat(rows, cols, ld=None, ptr=0x1000):
+    m = B.fo_mat()
+    m.kind = 0
+    m.dense.rows, m.dense.cols, m.dense.ld, m.dense.data = rows, cols, ld or cols, ptr
+    return m
+
+
+def test_workspace_sizes(lib):
+    m = dense_mat(1000, 1000)
+    full = lib.fused_cell_workspace_bytes(C.byref(m), 3)
+    assert full >= 256 + 8 and full % 8 == 0
+    assert lib.fused_cell_workspace_bytes(C.byref(m), 1) == 256            # row_agg: control words only
+    col = lib.fused_cell_workspace_bytes(C.byref(m), 2)
+    assert col >= 256 + 1000 * 8 and (col - 256) % (1000 * 8) == 0
+    assert lib.fused_cell_workspace_bytes(C.byref(m), 9) == 0
+    assert lib.fused_magg_workspace_bytes(C.byref(m), 3) == 256 + (full - 256) * 3
+    assert lib.fused_magg_workspace_bytes(C.byref(m), 9) == 0
+    r = lib.fused_row_workspace_bytes(C.byref(m), 4)
+    assert r >= 256 + 148 * 1000 * 8
+    assert lib.fused_row_workspace_bytes(C.byref(m), 0) == 0
+    x = B.fo_csr()
+    x.rows, x.cols, x.nnz = 10, 10, 5
+    assert lib.fused_outer_workspace_bytes(C.byref(x), 100, 3) >= 256 + 8
+    assert lib.fused_outer_workspace_bytes(C.byref(x), 257, 3) == 0
+
+
+def call_cell(lib, steps, output, m, sides=(), n_scalars=0, agg=3, ws=0x10000, ws_bytes=1 << 24,
+              out=0x2000):
+    ch, keep = B.make_chain(steps, output)
+    sarr = (B.fo_side * max(1, len(sides)))(*sides)
+    sc = (C.c_double * 8)()
+    return lib.fused_cell(C.byref(ch), C.byref(m), sarr, len(sides), sc, n_scalars, agg,
+                          C.c_void_p(out), C.c_void_p(ws), ws_bytes, None)
+
+
+def side(rows, cols, access, ptr=0x3000):
+    s = B.fo_side()
+    s.m.rows, s.m.cols, s.m.ld, s.m.data = rows, cols, cols, ptr
+    s.access = access
+    return s
+
+
+def test_cell_argument_errors(lib):
+    m = dense_mat(10, 10)
+    ok_chain = [("mul", "t0", "a", "a")]
+    assert call_cell(lib, ok_chain, "t0", m, out=0) == -1                        # FO_ERR_NULL
+    assert call_cell(lib, ok_chain, "t0", dense_mat(10, 10, ld=5)) == -2         # ld < cols
+    assert call_cell(lib, ok_chain, "t0", m, agg=7) == -4                        # unknown variant
+    assert call_cell(lib, [("mul", "t0", "a", "t1")], "t0", m) == -3             # use before definition
+    assert call_cell(lib, [("mul", "t0", "a", "d")], "t0", m) == -3              # no dot product in Cell
+    assert call_cell(lib, [("mul", "t0", "a", "side0")], "t0", m) == -3          # side not passed
+    assert call_cell(lib, [("mul", "t0", "a", "s0")], "t0", m) == -3             # scalar not passed
+    assert call_cell(lib, ok_chain, "t5", m) == -3                               # undefined output
+    assert call_cell(lib, ok_chain, "t0", m, sides=[side(9, 10, 0)]) == -2       # side shape
+    assert call_cell(lib, ok_chain, "t0", m, sides=[side(10, 1, 2)]) == -2       # row vector expected
+    assert call_cell(lib, ok_chain, "t0", m, ws=0) == -5                         # no workspace
+    assert call_cell(lib, ok_chain, "t0", m, ws=0x10008) == -5                   # misaligned
+    assert call_cell(lib, ok_chain, "t0", m, ws_bytes=16) == -5                  # too small
+    bad = B.fo_mat()
+    bad.kind = 5
+    assert call_cell(lib, ok_chain, "t0", bad) == -2
+
+
+def test_chain_limits(lib):
+    m = dense_mat(4, 4)
+    long_chain = [("add", "t0", "a", 1.0)] + [("add", "t0", "t0", 1.0)] * 31
+    ch, keep = B.make_chain(long_chain, "t0")
+    assert ch.n_ops == 32
+    too_long = long_chain + [("add", "t0", "t0", 1.0)]
+    assert call_cell(lib, too_long, "t0", m) == -3
+    ch, keep = B.make_chain([("mov", "t0", "a")], "t0")
+    keep[0].opcode = 200
+    sarr = (B.fo_side * 1)()
+    sc = (C.c_double * 8)()
+    assert lib.fused_cell(C.byref(ch), C.byref(m), sarr, 0, sc, 0, 3, C.c_void_p(0x2000),
+                          C.c_void_p(0x10000), 1 << 24, None) == -3
+
+
+def test_row_and_outer_argument_errors(lib):
+    ch, keep = B.make_chain([("mul", "t0", "side0", "d")], "t0")
+    m = dense_mat(10, 2000)
+    sarr = (B.fo_side * 1)(side(10, 1, 1))
+    sc = (C.c_double * 8)()
+
+    def row(mat, agg=4, sides=sarr, ns=1, chain=ch, v=0x4000):
+        return lib.fused_row(C.byref(chain), C.byref(mat), C.c_void_p(v), sides, ns, sc, 0, agg,
+                             C.c_void_p(0x2000), C.c_void_p(0x10000), 1 << 30, None)
+
+    assert row(m) == -4                                   # too wide for the single-pass kernel
+    assert row(dense_mat(10, 100), agg=0) == -4           # no_agg not provided
+    assert row(dense_mat(10, 100), agg=2) == -4           # col_agg not provided
+    assert row(dense_mat(10, 100), v=0) == -1
+    bad_side = (B.fo_side * 1)(side(10, 100, 0))
+    assert row(dense_mat(10, 100), sides=bad_side) == -2  # Row sides are read at the row index
+    ch2, keep2 = B.make_chain([("mul", "t0", "a", "d")], "t0")
+    assert row(dense_mat(10, 100), chain=ch2, ns=0) == -3  # no main value in Row
+
+    x = B.fo_csr()
+    x.rows, x.cols, x.nnz = 10, 12, 5
+    x.rowptr, x.colidx, x.vals = 0x5000, 0x6000, 0x7000
+    u, v = B.fo_dense(), B.fo_dense()
+    u.rows, u.cols, u.ld, u.data = 10, 4, 4, 0x8000
+    v.rows, v.cols, v.ld, v.data = 12, 4, 4, 0x9000
+    ch3, keep3 = B.make_chain([("sub", "t0", "a", "d")], "t0")
+
+    def outer(xx=x, uu=u, vv=v, agg=3):
+        return lib.fused_outer(C.byref(ch3), C.byref(xx), C.byref(uu), C.byref(vv), sc, 0, agg,
+                               C.c_void_p(0x2000), C.c_void_p(0x10000), 1 << 24, None)
+
+    v2 = B.fo_dense()
+    v2.rows, v2.cols, v2.ld, v2.data = 12, 5, 5, 0x9000
+    assert outer(vv=v2) == -2                             # rank mismatch
+    u2 = B.fo_dense()
+    u2.rows, u2.cols, u2.ld, u2.data = 11, 4, 4, 0x8000
+    assert outer(uu=u2) == -2                             # U.rows != X.rows
+    assert outer(agg=0) == -4                             # left_mm not provided
+    x2 = B.fo_csr()
+    x2.rows, x2.cols, x2.nnz = 10, 12, 1 << 31
+    x2.rowptr, x2.colidx, x2.vals = 0x5000, 0x6000, 0x7000
+    assert outer(xx=x2) == -4
+
+
+def test_make_chain_rejects_bad_text():
+    with pytest.raises(ValueError):
+        B.make_chain([("frobnicate", "t0", "a")], "t0")
+    with pytest.raises(ValueError):
+        B.make_chain([("add", "t0", "a")], "t0")
+    with pytest.raises(ValueError):
+        B.make_chain([("add", "x0", "a", "a")], "t0")
+    with pytest.raises(ValueError):
+        B.make_chain([("add", "t0", 1.0, 2.0)], "t0")
+    with pytest.raises(ValueError):
+        B.make_chain([("mov", "t0", "a")], 1.0)
+
+
+def test_cost_model_worked_example():
+    """Section 4.3: reading a 100M x 10 dense matrix at 32 GB/s takes 0.25 s."""
+    from paper_1801_00829_b200 import algorithmic_bytes, ideal_seconds
+    golden = open(os.path.join(ROOT, "tests", "golden", "cost_model_example.txt")).read()
+    vals = dict(l.split("=") for l in golden.split() if "=" in l)
+    nbytes = int(vals["rows"]) * int(vals["cols"]) * 8
+    assert abs(ideal_seconds(nbytes, float(vals["gb_per_s"])) - float(vals["seconds"])) < 1e-12
+    assert algorithmic_bytes("cell", rows=1000, cols=1000, n_inputs=3) == 24_000_008
+    assert algorithmic_bytes("row_dense", rows=10**6, cols=1000) == 8 * 10**9 + 8 * 10**6 + 16000

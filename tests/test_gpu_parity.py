@@ -1,0 +1,328 @@
+"""CUDA library vs. the CPU checker, element by element, on the same seeded inputs.
+
+Sizes here are the ones the checker finishes in seconds; they still span several
+tiles and ragged tails.  Tolerance: see tests/util.py (relative 1e-10).
+"""
+import numpy as np
+import pytest
+
+import datagen
+import oracle
+from datagen.workloads import csr_to_dense
+from util import assert_close, csr_to_dev, host_csr, to_dev
+
+pytestmark = pytest.mark.gpu
+
+XYZ = [("mul", "t0", "a", "side0"), ("mul", "t1", "t0", "side1")]
+MAGG3 = [("mul", "t0", "a", "side0"), ("mul", "t1", "a", "side1"), ("mul", "t2", "a", "a")]
+WD = [("mul", "t0", "side0", "d")]
+WSLOSS = [("ne", "t0", "a", 0.0), ("sub", "t1", "a", "d"), ("mul", "t2", "t1", "t1"),
+          ("mul", "t3", "t0", "t2")]
+
+
+@pytest.fixture(scope="module")
+def fo():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_1801_00829_b200 as fo_
+    fo_.load_library()
+    return fo_
+
+
+def dev_sides(sides):
+    return [(acc, to_dev(arr)) for acc, arr in sides]
+
+
+# ------------------------------------------------------------------ Cell
+@pytest.mark.parametrize("rows,cols", [(1000, 1000), (1, 1), (1, 7), (5, 1), (33, 65), (257, 129),
+                                       (1024, 1), (1, 1024), (3, 1025), (2047, 3), (64, 2048)])
+def test_cell_full_xyz(fo, rows, cols):
+    w = datagen.cell_workload(rows, cols, seed=0)
+    ref = oracle.sum_xyz(w["X"], w["Y"], w["Z"])
+    got = fo.fused_cell(XYZ, "t1", to_dev(w["X"]), dev_sides([("cell", w["Y"]), ("cell", w["Z"])]))
+    assert_close(got.cpu().numpy(), [ref], what="cell full %dx%d" % (rows, cols))
+
+
+def test_cell_full_is_bit_reproducible(fo):
+    w = datagen.cell_workload(777, 333, seed=5)
+    args = (XYZ, "t1", to_dev(w["X"]), dev_sides([("cell", w["Y"]), ("cell", w["Z"])]))
+    a = fo.fused_cell(*args).cpu().numpy()
+    for _ in range(3):
+        assert fo.fused_cell(*args).cpu().numpy().tobytes() == a.tobytes()
+
+
+@pytest.mark.parametrize("agg", ["full", "row", "col", "none"])
+@pytest.mark.parametrize("rows,cols", [(300, 200), (37, 1001), (129, 5), (8, 513), (1, 1)])
+def test_cell_aggs_with_all_side_kinds(fo, agg, rows, cols):
+    X = datagen.normal(7, 0, rows * cols).reshape(rows, cols)
+    Y = datagen.normal(7, 2, rows * cols).reshape(rows, cols)
+    rv = datagen.normal(7, 3, rows)
+    cv = datagen.normal(7, 4, cols)
+    chain = [("mul", "t0", "a", "s0"), ("mul", "t1", "t0", "side1"),
+             ("add", "t2", "side0", "t1"), ("sub", "t3", "t2", "side2")]
+    sides = [("cell", Y), ("row", rv), ("col", cv)]
+    ref = oracle.cell(chain, "t3", X, sides, [0.25], agg=agg)
+    absref = oracle.cell([("abs", "t0", "a"), ("abs", "t1", "side0"), ("abs", "t2", "side1"),
+                          ("abs", "t3", "side2"), ("mul", "t4", "t0", 0.25), ("mul", "t5", "t4", "t2"),
+                          ("add", "t6", "t5", "t1"), ("add", "t7", "t6", "t3")], "t7", X, sides,
+                         agg=agg)
+    got = fo.fused_cell(chain, "t3", to_dev(X), dev_sides(sides), [0.25], agg=agg)
+    assert_close(got.cpu().numpy(), ref, absscale=absref, what="cell %s" % agg)
+
+
+@pytest.mark.parametrize("agg", ["full", "row", "col", "none"])
+def test_cell_strided_and_unaligned_inputs(fo, agg):
+    import torch
+    rows, cols, ld = 45, 70, 77
+    base = datagen.uniform(3, 0, rows * ld + 1, 0.5, 1.5)
+    basey = datagen.uniform(3, 2, rows * ld + 1, 0.5, 1.5)
+    for off in (0, 1):                      # off = 1: base pointer only 8-byte aligned
+        Xh = base[off:off + rows * ld].reshape(rows, ld)[:, :cols]
+        Yh = basey[off:off + rows * ld].reshape(rows, ld)[:, :cols]
+        Xd = to_dev(base)[off:off + rows * ld].view(rows, ld)[:, :cols]
+        Yd = to_dev(basey)[off:off + rows * ld].view(rows, ld)[:, :cols]
+        assert Xd.stride(0) == ld
+        chain = [("mul", "t0", "a", "side0")]
+        ref = oracle.cell(chain, "t0", Xh, [("cell", Yh)], agg=agg)
+        got = fo.fused_cell(chain, "t0", Xd, [("cell", Yd)], agg=agg)
+        assert_close(got.cpu().numpy(), ref, what="strided off=%d %s" % (off, agg))
+    # contiguous but 8-byte-aligned base: the flat kernel must not be chosen
+    n = 5000
+    xd = to_dev(datagen.uniform(3, 4, n + 1))
+    ref = oracle.cell([("sq", "t0", "a")], "t0", xd[1:].cpu().numpy().reshape(1, n))
+    got = fo.fused_cell([("sq", "t0", "a")], "t0", xd[1:].view(1, n))
+    assert_close(got.cpu().numpy(), [ref])
+    torch.cuda.synchronize()
+
+
+def test_cell_every_opcode(fo):
+    rows, cols = 64, 96
+    X = datagen.uniform(11, 0, rows * cols, 0.25, 4.0).reshape(rows, cols)
+    Y = datagen.uniform(11, 2, rows * cols, -2.0, 2.0).reshape(rows, cols)
+    Y[::7, ::5] = 0.0
+    sides = [("cell", Y)]
+    unary = ["mov", "neg", "abs", "sqrt", "exp", "log", "sq"]
+    binary = ["add", "sub", "mul", "div", "min", "max", "eq", "ne", "lt", "le", "gt", "ge"]
+    for op in unary:
+        ch = [(op, "t0", "a")]
+        ref = oracle.cell(ch, "t0", X, sides, agg="none")
+        got = fo.fused_cell(ch, "t0", to_dev(X), dev_sides(sides), agg="none")
+        assert_close(got.cpu().numpy(), ref, what=op)
+    for op in binary:
+        ch = [(op, "t0", "a", "side0")]
+        if op == "div":
+            ch = [("add", "t1", "side0", 3.0), ("div", "t0", "a", "t1")]
+        ref = oracle.cell(ch, "t0", X, sides, agg="none")
+        got = fo.fused_cell(ch, "t0", to_dev(X), dev_sides(sides), agg="none")
+        assert_close(got.cpu().numpy(), ref, what=op)
+    ch = [("pow", "t0", "a", 1.7)]
+    assert_close(fo.fused_cell(ch, "t0", to_dev(X), agg="none").cpu().numpy(),
+                 oracle.cell(ch, "t0", X, agg="none"), what="pow")
+    ch = [("sel", "t0", "side0", "a", -1.0)]
+    assert_close(fo.fused_cell(ch, "t0", to_dev(X), dev_sides(sides), agg="none").cpu().numpy(),
+                 oracle.cell(ch, "t0", X, sides, agg="none"), what="sel")
+    ch = [("fma", "t0", "a", "side0", 0.5)]
+    assert_close(fo.fused_cell(ch, "t0", to_dev(X), dev_sides(sides), agg="none").cpu().numpy(),
+                 oracle.cell(ch, "t0", X, sides, agg="none"), absscale=np.abs(X * Y) + 0.5, what="fma")
+    # equality on exactly equal values
+    ch = [("eq", "t0", "a", "a"), ("ne", "t1", "a", "a"), ("add", "t2", "t0", "t1")]
+    assert fo.fused_cell(ch, "t2", to_dev(X)).item() == float(rows * cols)
+
+
+def test_cell_long_chain_with_register_reuse(fo):
+    rows, cols = 100, 64
+    X = datagen.uniform(13, 0, rows * cols, 0.5, 1.5).reshape(rows, cols)
+    sides = [("cell", datagen.uniform(13, 2 + k, rows * cols, 0.5, 1.5).reshape(rows, cols))
+             for k in range(4)]
+    chain = []
+    # 30 steps cycling through all eight temporaries
+    chain.append(("mul", "t0", "a", "side0"))
+    for k in range(1, 30):
+        src = "side%d" % (k % 4)
+        chain.append((("add", "mul", "sub")[k % 3], "t%d" % (k % 8), "t%d" % ((k - 1) % 8), src))
+    chain.append(("mul", "t1", "t%d" % (29 % 8), "s0"))
+    ref = oracle.cell(chain, "t1", X, sides, [0.5])
+    got = fo.fused_cell(chain, "t1", to_dev(X), dev_sides(sides), [0.5])
+    absref = oracle.cell(chain + [("abs", "t2", "t1")], "t2", X, sides, [0.5])
+    assert_close(got.cpu().numpy(), [ref], absscale=absref)
+
+
+def test_cell_empty(fo):
+    import torch
+    X = torch.zeros((0, 5), dtype=torch.float64, device="cuda")
+    assert fo.fused_cell([("sq", "t0", "a")], "t0", X).item() == 0.0
+    assert fo.fused_cell([("sq", "t0", "a")], "t0", X, agg="col").cpu().tolist() == [0.0] * 5
+
+
+# ------------------------------------------------------------------ MAgg
+@pytest.mark.parametrize("rows,cols", [(20000, 100), (999, 7), (1, 3)])
+def test_magg_three_aggregates(fo, rows, cols):
+    w = datagen.magg_workload(rows, cols, seed=1)
+    ref = oracle.magg_xy_xz_xx(w["X"], w["Y"], w["Z"])
+    absref = oracle.magg_xy_xz_xx(np.abs(w["X"]), np.abs(w["Y"]), np.abs(w["Z"]))
+    got = fo.fused_magg(MAGG3, ["t0", "t1", "t2"], to_dev(w["X"]),
+                        dev_sides([("cell", w["Y"]), ("cell", w["Z"])]))
+    assert_close(got.cpu().numpy(), ref, absscale=absref, what="magg")
+
+
+@pytest.mark.parametrize("k", [1, 2, 5, 8])
+def test_magg_k_outputs_match_single_cells(fo, k):
+    rows, cols = 513, 40
+    X = datagen.normal(21, 0, rows * cols).reshape(rows, cols)
+    Y = datagen.normal(21, 2, rows * cols).reshape(rows, cols)
+    rv = datagen.uniform(21, 3, rows)
+    chain = [("mul", "t0", "a", "side0")]
+    outs = ["t0"]
+    for j in range(1, k):
+        chain.append(("fma", "t%d" % j, "t%d" % (j - 1), "side1", float(j)))
+        outs.append("t%d" % j)
+    sides = [("cell", Y), ("row", rv)]
+    ref = oracle.magg(chain, outs, X, sides)
+    absref = oracle.magg(chain + [("abs", "t%d" % j, "t%d" % j) for j in range(k)], outs, X, sides)
+    got = fo.fused_magg(chain, outs, to_dev(X), dev_sides(sides))
+    assert_close(got.cpu().numpy(), ref, absscale=absref + rows * cols * k)
+    for j in range(k):       # fused multi-aggregate == each aggregate on its own
+        single = fo.fused_cell(chain, outs[j], to_dev(X), dev_sides(sides))
+        assert_close(single.cpu().numpy(), [ref[j]], absscale=absref[j] + rows * cols * k)
+
+
+# ------------------------------------------------------------------ Row
+def row_abs_scale(X, v, w):
+    return np.abs(X).T @ (np.abs(w) * (np.abs(X) @ np.abs(v)))
+
+
+@pytest.mark.parametrize("rows,cols", [(2000, 1000), (501, 64), (37, 10), (100, 1024), (9, 2),
+                                       (1, 128), (300, 257), (64, 999), (5, 1)])
+def test_row_dense_col_t(fo, rows, cols):
+    w = datagen.row_dense_workload(rows, cols, seed=2)
+    ref = oracle.row_chain_dense(w["X"], w["v"], w["w"])
+    got = fo.fused_row(WD, "t0", to_dev(w["X"]), to_dev(w["v"]), [("row", to_dev(w["w"]))])
+    assert_close(got.cpu().numpy(), ref, absscale=row_abs_scale(w["X"], w["v"], w["w"]),
+                 what="row dense %dx%d" % (rows, cols))
+    assert fo.device_status() == 0
+
+
+def test_row_dense_many_tiles_per_cta_and_reproducible(fo):
+    rows, cols = 20011, 1000         # > 148 * 8 * 3 rows: every ring slot is reused, ragged last tile
+    w = datagen.row_dense_workload(rows, cols, seed=22)
+    ref = oracle.row_chain_dense(w["X"], w["v"], w["w"])
+    args = (WD, "t0", to_dev(w["X"]), to_dev(w["v"]), [("row", to_dev(w["w"]))])
+    got = fo.fused_row(*args).cpu().numpy()
+    assert_close(got, ref, absscale=row_abs_scale(w["X"], w["v"], w["w"]))
+    assert fo.fused_row(*args).cpu().numpy().tobytes() == got.tobytes()
+    assert fo.device_status() == 0
+
+
+@pytest.mark.parametrize("agg", ["col_t", "row", "full"])
+def test_row_dense_variants_strided_unaligned(fo, agg):
+    rows, cols, ld = 333, 120, 130
+    flat = datagen.normal(2, 0, rows * ld + 1)
+    v = datagen.normal(2, 2, cols)
+    wv = datagen.uniform(2, 3, rows)
+    chain = [("mul", "t0", "side0", "d"), ("add", "t1", "t0", "s0")]
+    for off in (0, 1):
+        Xh = flat[off:off + rows * ld].reshape(rows, ld)[:, :cols]
+        Xd = to_dev(flat)[off:off + rows * ld].view(rows, ld)[:, :cols]
+        ref = oracle.row(chain, "t1", Xh, v, [("row", wv)], [0.125], agg=agg)
+        scale = {"col_t": np.abs(Xh).T @ (wv * (np.abs(Xh) @ np.abs(v)) + 0.125),
+                 "row": None, "full": float(np.sum(wv * (np.abs(Xh) @ np.abs(v)) + 0.125))}[agg]
+        got = fo.fused_row(chain, "t1", Xd, to_dev(v), [("row", to_dev(wv))], [0.125], agg=agg)
+        assert_close(got.cpu().numpy(), ref, absscale=scale, what="row %s off=%d" % (agg, off))
+    # no weight: t(X) %*% (X %*% v)
+    Xh = flat[:rows * ld].reshape(rows, ld)[:, :cols]
+    ref = oracle.row([], "d", Xh, v, agg="col_t")
+    got = fo.fused_row([], "d", to_dev(flat)[:rows * ld].view(rows, ld)[:, :cols], to_dev(v))
+    assert_close(got.cpu().numpy(), ref, absscale=row_abs_scale(Xh, v, np.ones(rows)))
+
+
+@pytest.mark.parametrize("rows,cols,density", [(100000, 1000, 0.01), (5000, 64, 0.2), (300, 4000, 0.001),
+                                               (17, 9, 0.5), (1000, 1000, 0.0)])
+def test_row_csr_col_t(fo, rows, cols, density):
+    w = datagen.row_csr_workload(rows, cols, density, seed=3)
+    Xh = host_csr(w)
+    ref = oracle.row_chain_csr(Xh, w["v"], w["w"])
+    absX = dict(Xh, vals=np.abs(w["vals"]))
+    scale = oracle.row_chain_csr(absX, np.abs(w["v"]), w["w"])
+    got = fo.fused_row(WD, "t0", csr_to_dev(w), to_dev(w["v"]), [("row", to_dev(w["w"]))])
+    assert_close(got.cpu().numpy(), ref, absscale=scale, what="row csr")
+
+
+@pytest.mark.parametrize("agg", ["row", "full"])
+def test_row_csr_other_aggs_and_dense_agreement(fo, agg):
+    rows, cols = 2500, 300
+    w = datagen.row_csr_workload(rows, cols, 0.05, seed=33)
+    Xh = host_csr(w)
+    ref = oracle.row(WD, "t0", Xh, w["v"], [("row", w["w"])], agg=agg)
+    got = fo.fused_row(WD, "t0", csr_to_dev(w), to_dev(w["v"]), [("row", to_dev(w["w"]))], agg=agg)
+    absX = dict(Xh, vals=np.abs(w["vals"]))
+    scale = oracle.row(WD, "t0", absX, np.abs(w["v"]), [("row", w["w"])], agg=agg)
+    assert_close(got.cpu().numpy(), ref, absscale=scale)
+    # the dense kernel on the same matrix agrees too
+    Xd = csr_to_dense(rows, cols, w["rowptr"], w["colidx"], w["vals"])
+    got_d = fo.fused_row(WD, "t0", to_dev(Xd), to_dev(w["v"]), [("row", to_dev(w["w"]))], agg=agg)
+    assert_close(got_d.cpu().numpy(), ref, absscale=scale)
+
+
+# ------------------------------------------------------------------ Outer
+def outer_case(rows, cols, rank, density, seed=4):
+    w = datagen.outer_workload(rows, cols, rank, density, seed)
+    return w, host_csr(w)
+
+
+@pytest.mark.parametrize("rows,cols,rank,density", [
+    (2000, 3000, 100, 0.01), (300, 200, 1, 0.1), (300, 200, 16, 0.1), (300, 200, 17, 0.1),
+    (257, 129, 33, 0.2), (100, 90, 128, 0.3), (64, 50, 256, 0.3), (500, 400, 7, 0.0),
+    (40, 30, 100, 1.0)])
+def test_outer_full_agg(fo, rows, cols, rank, density):
+    w, Xh = outer_case(rows, cols, rank, density)
+    ref = oracle.outer_wsloss_masked(Xh, w["U"], w["V"])
+    got = fo.fused_outer(WSLOSS, "t3", csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"]))
+    assert_close(got.cpu().numpy(), [ref], what="outer full rank %d" % rank)
+    if rows * cols <= 1_000_000:
+        assert_close(got.cpu().numpy(), [oracle.outer_wsloss_dense(Xh, w["U"], w["V"])])
+
+
+@pytest.mark.parametrize("agg", ["none", "right"])
+@pytest.mark.parametrize("rank", [5, 100])
+def test_outer_other_aggs(fo, agg, rank):
+    w, Xh = outer_case(700, 900, rank, 0.02, seed=14)
+    chain = [("ne", "t0", "a", 0.0), ("mul", "t1", "t0", "d")]          # (X != 0) * (U V^T), Eq. 1
+    ref = oracle.outer(chain, "t1", Xh, w["U"], w["V"], agg=agg, mode="masked")
+    got = fo.fused_outer(chain, "t1", csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"]), agg=agg)
+    absU, absV = np.abs(w["U"]), np.abs(w["V"])
+    scale = oracle.outer(chain, "t1", Xh, absU, absV, agg=agg, mode="masked")
+    assert_close(got.cpu().numpy(), ref, absscale=scale, what="outer %s" % agg)
+
+
+def test_outer_explicit_zeros_unaligned_and_reproducible(fo):
+    w, Xh = outer_case(400, 300, 10, 0.05, seed=24)
+    w["vals"][::3] = 0.0                 # stored zeros stay stored
+    Xh = host_csr(w)
+    ref = oracle.outer_wsloss_masked(Xh, w["U"], w["V"])
+    ref_nomask = oracle.outer(WSLOSS[1:3], "t2", Xh, w["U"], w["V"], mode="masked")
+    assert ref_nomask > ref
+    Xd = csr_to_dev(w)
+    got = fo.fused_outer(WSLOSS, "t3", Xd, to_dev(w["U"]), to_dev(w["V"]))
+    assert_close(got.cpu().numpy(), [ref])
+    got2 = fo.fused_outer(WSLOSS[1:3], "t2", Xd, to_dev(w["U"]), to_dev(w["V"]))
+    assert_close(got2.cpu().numpy(), [ref_nomask])
+    # U, V with a padded leading dimension and an 8-byte-aligned base
+    Up = to_dev(np.pad(w["U"], ((0, 0), (0, 3))).reshape(-1))
+    Vp = to_dev(np.concatenate([[0.0], np.pad(w["V"], ((0, 0), (0, 1))).reshape(-1)]))
+    Ud = Up.view(400, 13)[:, :10]
+    Vd = Vp[1:].view(300, 11)[:, :10]
+    got3 = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd)
+    assert_close(got3.cpu().numpy(), [ref])
+    assert fo.fused_outer(WSLOSS, "t3", Xd, to_dev(w["U"]), to_dev(w["V"])).cpu().numpy().tobytes() \
+        == got.cpu().numpy().tobytes()
+
+
+def test_outer_log_chain(fo):
+    # sum(X * log(U V^T + eps)), Fig. 1(d)
+    w = datagen.outer_workload(500, 400, 20, 0.05, seed=34)
+    U, V = np.abs(w["U"]) + 0.01, np.abs(w["V"]) + 0.01
+    Xh = host_csr(w)
+    chain = [("add", "t0", "d", "s0"), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")]
+    ref = oracle.outer(chain, "t2", Xh, U, V, [1e-15], mode="masked")
+    got = fo.fused_outer(chain, "t2", csr_to_dev(w), to_dev(U), to_dev(V), [1e-15])
+    assert_close(got.cpu().numpy(), [ref])
