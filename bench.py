@@ -1,0 +1,516 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-operator hot path.
+
+A step is one pass of the whole path: the five fused operators (Cell, MAgg,
+Row dense, Row CSR, Outer) each run once on their full-size seeded workload.
+The reported value is effective input bandwidth: the bytes the five operators
+must read once, divided by the time of a step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+`--impl reference` times the CPU checker (oracle/) on bounded samples of the same
+workloads; it runs on host cores only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "effective_hbm_bandwidth_all_fused_ops"
+UNIT = "GB/s"
+
+XYZ = [("mul", "t0", "a", "side0"), ("mul", "t1", "t0", "side1")]
+MAGG3 = [("mul", "t0", "a", "side0"), ("mul", "t1", "a", "side1"), ("mul", "t2", "a", "a")]
+WD = [("mul", "t0", "side0", "d")]
+WSLOSS = [("ne", "t0", "a", 0.0), ("sub", "t1", "a", "d"), ("mul", "t2", "t1", "t1"),
+          ("mul", "t3", "t0", "t2")]
+
+FULL = {
+    "cell": dict(rows=1000, cols=1000),
+    "magg": dict(rows=1_000_000, cols=100),
+    "row_dense": dict(rows=1_000_000, cols=1000),
+    "row_csr": dict(rows=10_000_000, cols=1000, density=0.01),
+    "outer": dict(rows=100_000, cols=100_000, rank=100, density=0.001),
+}
+OPS = ["cell", "magg", "row_dense", "row_csr", "outer"]
+
+
+def scaled(shapes, frac):
+    """The same workloads with the row counts scaled by `frac` (columns, rank, density kept)."""
+    out = {}
+    for k, s in shapes.items():
+        s = dict(s)
+        if k != "cell":
+            s["rows"] = max(8, int(round(s["rows"] * frac)))
+        out[k] = s
+    return out
+
+
+# ---------------------------------------------------------------------- inputs
+def make_host_inputs(shapes, pinned):
+    """Seeded inputs of all five workloads as torch CPU tensors (pinned if asked)."""
+    import torch
+    import datagen
+
+    def buf(n, dtype=torch.float64):
+        return torch.empty(n, dtype=dtype, pin_memory=pinned)
+
+    h = {}
+    s = shapes["cell"]
+    n = s["rows"] * s["cols"]
+    for name, stream in (("X", 0), ("Y", 2), ("Z", 3)):
+        t = buf(n)
+        datagen.uniform(0, stream, n, out=t.numpy())
+        h["cell." + name] = t.view(s["rows"], s["cols"])
+    s = shapes["magg"]
+    n = s["rows"] * s["cols"]
+    for name, stream in (("X", 0), ("Y", 2), ("Z", 3)):
+        t = buf(n)
+        datagen.normal(1, stream, n, out=t.numpy())
+        h["magg." + name] = t.view(s["rows"], s["cols"])
+    s = shapes["row_dense"]
+    t = buf(s["rows"] * s["cols"])
+    datagen.normal(2, 0, s["rows"] * s["cols"], out=t.numpy())
+    h["row_dense.X"] = t.view(s["rows"], s["cols"])
+    h["row_dense.v"] = buf(s["cols"])
+    datagen.normal(2, 2, s["cols"], out=h["row_dense.v"].numpy())
+    h["row_dense.w"] = buf(s["rows"])
+    datagen.uniform(2, 3, s["rows"], out=h["row_dense.w"].numpy())
+    s = shapes["row_csr"]
+    rp, ci, va = datagen.csr_bernoulli(3, 0, s["rows"], s["cols"], s["density"], 0.0, 1.0)
+    for name, arr, dt in (("rowptr", rp, torch.int32), ("colidx", ci, torch.int32), ("vals", va, torch.float64)):
+        t = buf(arr.size, dt)
+        t.numpy()[:] = arr
+        h["row_csr." + name] = t
+    h["row_csr.v"] = buf(s["cols"])
+    datagen.normal(3, 2, s["cols"], out=h["row_csr.v"].numpy())
+    h["row_csr.w"] = buf(s["rows"])
+    datagen.uniform(3, 3, s["rows"], out=h["row_csr.w"].numpy())
+    s = shapes["outer"]
+    rp, ci, va = datagen.csr_bernoulli(4, 0, s["rows"], s["cols"], s["density"], 1.0, 5.0)
+    for name, arr, dt in (("rowptr", rp, torch.int32), ("colidx", ci, torch.int32), ("vals", va, torch.float64)):
+        t = buf(arr.size, dt)
+        t.numpy()[:] = arr
+        h["outer." + name] = t
+    t = buf(s["rows"] * s["rank"])
+    datagen.normal(4, 2, s["rows"] * s["rank"], 0.0, 0.1, out=t.numpy())
+    h["outer.U"] = t.view(s["rows"], s["rank"])
+    t = buf(s["cols"] * s["rank"])
+    datagen.normal(4, 3, s["cols"] * s["rank"], 0.0, 0.1, out=t.numpy())
+    h["outer.V"] = t.view(s["cols"], s["rank"])
+    return h
+
+
+def algorithmic_bytes(shapes, host):
+    from paper_1801_00829_b200 import algorithmic_bytes as ab
+    s = shapes
+    return {
+        "cell": ab("cell", rows=s["cell"]["rows"], cols=s["cell"]["cols"], n_inputs=3),
+        "magg": ab("magg", rows=s["magg"]["rows"], cols=s["magg"]["cols"], n_inputs=3, n_out=3),
+        "row_dense": ab("row_dense", rows=s["row_dense"]["rows"], cols=s["row_dense"]["cols"]),
+        "row_csr": ab("row_csr", rows=s["row_csr"]["rows"], cols=s["row_csr"]["cols"],
+                      nnz=int(host["row_csr.vals"].numel())),
+        "outer": ab("outer", rows=s["outer"]["rows"], cols=s["outer"]["cols"],
+                    nnz=int(host["outer.vals"].numel()), rank=s["outer"]["rank"]),
+    }
+
+
+def upload(host, dev_bufs, stream_sync=False):
+    """Copies every host tensor into its preallocated device tensor (async on the current stream)."""
+    for k, t in host.items():
+        dev_bufs[k].copy_(t, non_blocking=True)
+
+
+def alloc_device(host, device):
+    import torch
+    return {k: torch.empty(t.shape, dtype=t.dtype, device=device) for k, t in host.items()}
+
+
+class Step:
+    """The five fused-operator calls on device-resident inputs."""
+
+    def __init__(self, fo, shapes, d):
+        import torch
+        self.fo, self.d = fo, d
+        dev = d["cell.X"].device
+        s = shapes
+        self.csr4 = fo.CSR(s["row_csr"]["rows"], s["row_csr"]["cols"], d["row_csr.rowptr"],
+                           d["row_csr.colidx"], d["row_csr.vals"])
+        self.csr5 = fo.CSR(s["outer"]["rows"], s["outer"]["cols"], d["outer.rowptr"],
+                           d["outer.colidx"], d["outer.vals"])
+        self.out = {
+            "cell": torch.empty(1, dtype=torch.float64, device=dev),
+            "magg": torch.empty(3, dtype=torch.float64, device=dev),
+            "row_dense": torch.empty(s["row_dense"]["cols"], dtype=torch.float64, device=dev),
+            "row_csr": torch.empty(s["row_csr"]["cols"], dtype=torch.float64, device=dev),
+            "outer": torch.empty(1, dtype=torch.float64, device=dev),
+        }
+        self.launches = 0
+
+    def run(self, name):
+        fo, d, o = self.fo, self.d, self.out
+        if name == "cell":
+            fo.fused_cell(XYZ, "t1", d["cell.X"], [("cell", d["cell.Y"]), ("cell", d["cell.Z"])],
+                          out=o["cell"])
+        elif name == "magg":
+            fo.fused_magg(MAGG3, ["t0", "t1", "t2"], d["magg.X"],
+                          [("cell", d["magg.Y"]), ("cell", d["magg.Z"])], out=o["magg"])
+        elif name == "row_dense":
+            fo.fused_row(WD, "t0", d["row_dense.X"], d["row_dense.v"], [("row", d["row_dense.w"])],
+                         out=o["row_dense"])
+        elif name == "row_csr":
+            fo.fused_row(WD, "t0", self.csr4, d["row_csr.v"], [("row", d["row_csr.w"])],
+                         out=o["row_csr"])
+        elif name == "outer":
+            fo.fused_outer(WSLOSS, "t3", self.csr5, d["outer.U"], d["outer.V"], out=o["outer"])
+        self.launches += 1
+
+    def all(self, events=None):
+        import torch
+        for i, name in enumerate(OPS):
+            if events is not None:
+                events[i][0].record()
+            self.run(name)
+            if events is not None:
+                events[i][1].record()
+
+
+# ---------------------------------------------------------------------- clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        return {
+            "sm_mhz": statistics.median(self.samples) if self.samples else None,
+            "sm_max_mhz": self.max_mhz,
+            "reasons": sorted(self.reasons),
+            "samples": len(self.samples),
+        }
+
+
+def physical_gpu_index(local_index):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+# ---------------------------------------------------------------------- oracle legs
+def oracle_step(np_inputs, shapes):
+    """One pass of the CPU checker over (a sample of) the five workloads; returns per-op seconds."""
+    import oracle
+    h = np_inputs
+    t = {}
+    t0 = time.perf_counter()
+    r = {"cell": oracle.sum_xyz(h["cell.X"], h["cell.Y"], h["cell.Z"])}
+    t["cell"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    r["magg"] = oracle.magg_xy_xz_xx(h["magg.X"], h["magg.Y"], h["magg.Z"])
+    t["magg"] = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    r["row_dense"] = oracle.row_chain_dense(h["row_dense.X"], h["row_dense.v"], h["row_dense.w"])
+    t["row_dense"] = time.perf_counter() - t0
+    s = shapes["row_csr"]
+    X4 = dict(rows=s["rows"], cols=s["cols"], rowptr=h["row_csr.rowptr"], colidx=h["row_csr.colidx"],
+              vals=h["row_csr.vals"])
+    t0 = time.perf_counter()
+    r["row_csr"] = oracle.row_chain_csr(X4, h["row_csr.v"], h["row_csr.w"])
+    t["row_csr"] = time.perf_counter() - t0
+    s = shapes["outer"]
+    X5 = dict(rows=s["rows"], cols=s["cols"], rowptr=h["outer.rowptr"], colidx=h["outer.colidx"],
+              vals=h["outer.vals"])
+    t0 = time.perf_counter()
+    r["outer"] = oracle.outer_wsloss_masked(X5, h["outer.U"], h["outer.V"])
+    t["outer"] = time.perf_counter() - t0
+    return t, r
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def sample_description(shapes):
+    return ("rows scaled: magg %dx%d, row_dense %dx%d, row_csr %dx%d@%.3g, outer %dx%d rank %d@%.3g "
+            "(row panel, all of V); cell full size" % (
+                shapes["magg"]["rows"], shapes["magg"]["cols"], shapes["row_dense"]["rows"],
+                shapes["row_dense"]["cols"], shapes["row_csr"]["rows"], shapes["row_csr"]["cols"],
+                shapes["row_csr"]["density"], shapes["outer"]["rows"], shapes["outer"]["cols"],
+                shapes["outer"]["rank"], shapes["outer"]["density"]))
+
+
+def numpy_inputs(host):
+    return {k: t.numpy() for k, t in host.items()}
+
+
+def run_reference(args):
+    """The CPU checker, as it stands, on bounded samples; host cores only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    shapes = scaled(FULL, args.ref_frac)
+    # the Outer sample is a panel of rows against all of V
+    shapes["outer"]["cols"] = FULL["outer"]["cols"]
+    host = make_host_inputs(shapes, pinned=False)
+    nbytes = algorithmic_bytes(shapes, host)
+    total = sum(nbytes.values())
+    h = numpy_inputs(host)
+    for _ in range(args.warmup):
+        oracle_step(h, shapes)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(h, shapes)
+    dt = time.perf_counter() - t0
+    value = total * args.steps / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic (seeded, in-repo generator)",
+        "config": {"workload": "all five fused operators, bounded sample of the full-size configs",
+                   "sample": sample_description(shapes)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                         "sample": sample_description(shapes)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------- main arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the fused operators have no CPU path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    import paper_1801_00829_b200 as fo
+    fo.load_library()
+
+    shapes = scaled(FULL, args.frac) if args.frac != 1.0 else {k: dict(v) for k, v in FULL.items()}
+    if args.frac != 1.0:
+        shapes["outer"]["cols"] = max(8, int(round(FULL["outer"]["cols"] * args.frac)))
+    t_gen = time.perf_counter()
+    host = make_host_inputs(shapes, pinned=True)
+    t_gen = time.perf_counter() - t_gen
+    nbytes = algorithmic_bytes(shapes, host)
+    total_bytes = sum(nbytes.values())
+    dev = alloc_device(host, device)
+    upload(host, dev)
+    torch.cuda.synchronize()
+    step = Step(fo, shapes, dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: K steps between two events
+    for _ in range(args.warmup):
+        step.all()
+    barrier()
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in OPS]
+          for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    launches0 = step.launches
+    barrier()
+    e0.record()
+    for k in range(args.steps):
+        step.all(ev[k])
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = e0.elapsed_time(e1)
+    gpu_launches = step.launches - launches0
+    per_op_ms = {name: [ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)]
+                 for i, name in enumerate(OPS)}
+    results = {k: v.cpu().numpy().copy() for k, v in step.out.items()}
+    status = fo.device_status(device)
+
+    # ---- end to end: host buffers -> device -> five calls -> results back on the host
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in step.out.items()}
+    d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+    def e2e_once():
+        upload(host, dev)
+        step.all()
+        for k2, v2 in step.out.items():
+            host_out[k2].copy_(v2, non_blocking=True)
+
+    e2e_once()
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(e2e_steps):
+        e2e_once()
+    f1.record()
+    barrier()
+    ms_e2e = f0.elapsed_time(f1)
+
+    # ---- max over ranks
+    if world > 1:
+        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = float(t[0]), float(t[1])
+
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak_gbs = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
+
+    ms_step = ms_total / args.steps
+    value = world * total_bytes / (ms_step * 1e-3) / 1e9
+    e2e_value = world * total_bytes / (ms_e2e / e2e_steps * 1e-3) / 1e9
+    per_op = {}
+    for name in OPS:
+        ms = statistics.mean(per_op_ms[name])
+        gbs = nbytes[name] / (ms * 1e-3) / 1e9
+        per_op[name] = {"ms": ms, "ms_min": min(per_op_ms[name]), "bytes": nbytes[name], "gbs": gbs,
+                        "frac_of_" + peak_kind: gbs / peak_gbs}
+    nnz4, nnz5 = int(host["row_csr.vals"].numel()), int(host["outer.vals"].numel())
+    per_op["row_csr"]["nnz_per_s"] = nnz4 / (per_op["row_csr"]["ms"] * 1e-3)
+    per_op["outer"]["nnz_per_s"] = nnz5 / (per_op["outer"]["ms"] * 1e-3)
+    dominant = max(OPS, key=lambda n: per_op[n]["ms"])
+    traffic = None
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": per_op[dominant]["gbs"], "peak": peak_gbs,
+                "peak_kind": peak_kind, "unit": "GB/s", "frac": per_op[dominant]["gbs"] / peak_gbs,
+                "traffic": traffic}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded, in-repo generator)",
+        "config": {"workload": "all five fused operators at full size: cell 1000x1000x3, magg 1e6x100x3, "
+                               "row dense 1e6x1000, row csr 1e7x1000@0.01, outer 1e5x1e5@0.001 rank 100"
+                               if args.frac == 1.0 else "five fused operators, rows scaled by %g" % args.frac,
+                   "shapes": shapes, "nnz": {"row_csr": nnz4, "outer": nnz5},
+                   "l2": "inputs larger than L2: 12 GB stream through between two uses of any array",
+                   "multi_gpu": "replicas only"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
+        "gpu_launches": gpu_launches,
+        "roofline": roofline,
+        "per_op": per_op,
+        "device_status": status,
+        "results": {k: [float(x) for x in v.reshape(-1)[:3]] for k, v in results.items()},
+        "input_generation_s": t_gen,
+    }
+
+    # ---- CPU baseline: the checker on a bounded sample, rank 0 at N = 1 only
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cshapes = scaled(FULL, args.cpu_frac)
+        cshapes["outer"]["cols"] = FULL["outer"]["cols"]
+        chost = make_host_inputs(cshapes, pinned=False)
+        cbytes = algorithmic_bytes(cshapes, chost)
+        t0 = time.perf_counter()
+        ct, _ = oracle_step(numpy_inputs(chost), cshapes)
+        cdt = time.perf_counter() - t0
+        line["cpu_baseline"] = {
+            "value": sum(cbytes.values()) / cdt / 1e9, "unit": UNIT, "cores": host_threads(),
+            "kind": "oracle", "sample": sample_description(cshapes), "seconds": cdt,
+            "per_op_gbs": {k: cbytes[k] / ct[k] / 1e9 for k in OPS},
+        }
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--frac", type=float, default=1.0, help="scale the row counts (debugging)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-frac", type=float, default=0.05, help="sample of the workloads the CPU baseline runs")
+    ap.add_argument("--ref-frac", type=float, default=0.01, help="sample per step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
