@@ -157,6 +157,7 @@ class Step:
             "outer": torch.empty(1, dtype=torch.float64, device=dev),
         }
         self.launches = 0
+        self.enabled = set(OPS)
 
     def run(self, name):
         fo, d, o = self.fo, self.d, self.out
@@ -177,8 +178,9 @@ class Step:
         self.launches += 1
 
     def all(self, events=None):
-        import torch
         for i, name in enumerate(OPS):
+            if name not in self.enabled:
+                continue
             if events is not None:
                 events[i][0].record()
             self.run(name)
@@ -369,6 +371,11 @@ def run_ours(args):
     upload(host, dev)
     torch.cuda.synchronize()
     step = Step(fo, shapes, dev)
+    if args.ops:
+        step.enabled = set(args.ops.split(","))
+        assert step.enabled <= set(OPS), "unknown op in --ops"
+    if args.interp:
+        fo.force_interpreter(True)
 
     def barrier():
         if world > 1:
@@ -394,7 +401,8 @@ def run_ours(args):
     clocks = sampler.stop()
     ms_total = e0.elapsed_time(e1)
     gpu_launches = step.launches - launches0
-    per_op_ms = {name: [ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)]
+    per_op_ms = {name: ([ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)]
+                        if name in step.enabled else [float("nan")])
                  for i, name in enumerate(OPS)}
     results = {k: v.cpu().numpy().copy() for k, v in step.out.items()}
     status = fo.device_status(device)
@@ -435,6 +443,7 @@ def run_ours(args):
     peak_gbs = float(peaks.get("hbm_gbs", 6650.0))
     peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
 
+    total_bytes = sum(nbytes[n] for n in step.enabled)
     ms_step = ms_total / args.steps
     value = world * total_bytes / (ms_step * 1e-3) / 1e9
     e2e_value = world * total_bytes / (ms_e2e / e2e_steps * 1e-3) / 1e9
@@ -447,7 +456,7 @@ def run_ours(args):
     nnz4, nnz5 = int(host["row_csr.vals"].numel()), int(host["outer.vals"].numel())
     per_op["row_csr"]["nnz_per_s"] = nnz4 / (per_op["row_csr"]["ms"] * 1e-3)
     per_op["outer"]["nnz_per_s"] = nnz5 / (per_op["outer"]["ms"] * 1e-3)
-    dominant = max(OPS, key=lambda n: per_op[n]["ms"])
+    dominant = max(sorted(step.enabled), key=lambda n: per_op[n]["ms"])
     traffic = None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": per_op[dominant]["gbs"], "peak": peak_gbs,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": per_op[dominant]["gbs"] / peak_gbs,
@@ -506,6 +515,8 @@ def main():
     ap.add_argument("--cpu-frac", type=float, default=0.05, help="sample of the workloads the CPU baseline runs")
     ap.add_argument("--ref-frac", type=float, default=0.01, help="sample per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ops", default="", help="comma-separated subset of the five operators (profiling)")
+    ap.add_argument("--interp", action="store_true", help="run Cell / MAgg chains through the interpreter")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -166,6 +166,13 @@ const char *fo_status_string(int status);
  * (thread-local), 0 if none. */
 int fo_last_cuda_error(void);
 
+/* Chains that match one of the library's compile-time specialisations (the
+ * products and multi-aggregates of Fig. 1(a), (c)) normally run as straight-line
+ * code; every other chain runs through the general interpreter.  Both give the
+ * same bits.  on != 0 sends every Cell / MAgg chain through the interpreter
+ * (process-wide; for tests and measurements).  Returns the previous setting. */
+int fo_set_force_interpreter(int on);
+
 /* ------------------------------------------------------------------ Cell
  * Table 1, Cell template; Section 2.2 cell-wise listing.
  * For every cell (i, j) of a dense main input X (for a CSR main input: every

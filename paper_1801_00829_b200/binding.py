@@ -78,7 +78,7 @@ EXPORTS = [
     "fused_cell", "fused_magg", "fused_row", "fused_outer",
     "fused_cell_workspace_bytes", "fused_magg_workspace_bytes", "fused_row_workspace_bytes",
     "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
-    "fo_status_string", "fo_last_cuda_error",
+    "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
 ]
 
 _lib = None
@@ -117,6 +117,8 @@ def load_library(path=None):
         lib.fo_status_string.restype = C.c_char_p
         lib.fo_last_cuda_error.argtypes = []
         lib.fo_last_cuda_error.restype = C.c_int
+        lib.fo_set_force_interpreter.argtypes = [C.c_int]
+        lib.fo_set_force_interpreter.restype = C.c_int
         if path is None:
             _lib = lib
         return lib
@@ -295,6 +297,12 @@ def workspace(device, nbytes):
                                                 _stream(device)), "fo_workspace_init")
         _ws[key] = buf
     return buf
+
+
+def force_interpreter(on):
+    """Route every Cell / MAgg chain through the interpreter (True) or let known
+    chains use their compile-time specialisation (False).  Returns the old setting."""
+    return bool(load_library().fo_set_force_interpreter(1 if on else 0))
 
 
 def device_status(device=None):

@@ -11,7 +11,7 @@
 //   cell_rows_kernel  general case (leading dimensions, row / column vector
 //                     sides): a warp per row (no_agg, row_agg, full_agg, MAgg);
 //   cell_cols_kernel  col_agg: a thread per column pair, a CTA per panel of rows.
-#include "chain.cuh"
+#include "spec.cuh"
 
 namespace fo {
 
@@ -32,24 +32,27 @@ constexpr int kV = 4;     // cells per thread per chain evaluation
 
 enum { kAggNone = 0, kAggRow = 1, kAggFull = 3 };
 
-template <int NR>
-__device__ __forceinline__ void add_outputs(const DevChain &ch, const RegFile<NR, kV> &f,
-                                            const bool (&valid)[kV], double *acc, int nout_max)
+// Adds the chain's results for four cells to the running sums (invalid cells count 0).
+template <int NOUT>
+__device__ __forceinline__ void add_outputs(const double (&o)[NOUT][kV], const bool (&valid)[kV],
+                                            double (&acc)[NOUT])
 {
-    for (int k = 0; k < nout_max; ++k) {
-        if (k < ch.n_out) {
-            double o[kV];
-            operand<NR, kV>(ch, f, ch.out[k], o);
-            double s = 0.0;
 #pragma unroll
-            for (int i = 0; i < kV; ++i) s += valid[i] ? o[i] : 0.0;
-            acc[k] += s;
-        }
+    for (int k = 0; k < NOUT; ++k) {
+        double s = 0.0;
+#pragma unroll
+        for (int i = 0; i < kV; ++i) s += valid[i] ? o[k][i] : 0.0;
+        acc[k] += s;
     }
 }
 
+__device__ __forceinline__ void put4(double (&dst)[kV], double2 m0, double2 m1)
+{
+    dst[0] = m0.x; dst[1] = m0.y; dst[2] = m1.x; dst[3] = m1.y;
+}
+
 // ------------------------------------------------------------------ flat
-template <int NR, int NOUT, bool STORE>
+template <class EVAL, int NOUT, bool STORE>
 __global__ void __launch_bounds__(kThreads)
 cell_flat_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ CellParams p)
 {
@@ -65,68 +68,61 @@ cell_flat_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
 
     for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const long long o0 = (tile << 10) + 2 * t, o1 = o0 + 512;
-        RegFile<NR, kV> f;
-        {
-            const double2 m0 = ld_stream2(p.X + o0), m1 = ld_stream2(p.X + o1);
-            f.r[0][0] = m0.x; f.r[0][1] = m0.y; f.r[0][2] = m1.x; f.r[0][3] = m1.y;
-        }
+        double in[kIn][kV];
+        put4(in[0], ld_stream2(p.X + o0), ld_stream2(p.X + o1));
 #pragma unroll
         for (int k = 0; k < FO_MAX_SIDES; ++k) {
-            if (1 + k < NR && (ch.side_used >> k) & 1u) {
+            if (EVAL::uses_side(ch, k)) {
                 const double *sp = p.sides.s[k].data;
-                const double2 m0 = ld_stream2(sp + o0), m1 = ld_stream2(sp + o1);
-                const int R = (1 + k < NR) ? 1 + k : 0;
-                f.r[R][0] = m0.x; f.r[R][1] = m0.y; f.r[R][2] = m1.x; f.r[R][3] = m1.y;
+                put4(in[1 + k], ld_stream2(sp + o0), ld_stream2(sp + o1));
             }
         }
-        run_chain<NR, kV>(ch, f);
+        double o[NOUT][kV];
+        EVAL::template run<kV, NOUT>(ch, in, o);
         if (STORE) {
-            double o[kV];
-            operand<NR, kV>(ch, f, ch.out[0], o);
-            *reinterpret_cast<double2 *>(p.out + o0) = make_double2(o[0], o[1]);
-            *reinterpret_cast<double2 *>(p.out + o1) = make_double2(o[2], o[3]);
+            *reinterpret_cast<double2 *>(p.out + o0) = make_double2(o[0][0], o[0][1]);
+            *reinterpret_cast<double2 *>(p.out + o1) = make_double2(o[0][2], o[0][3]);
         } else {
             const bool valid[kV] = {true, true, true, true};
-            add_outputs<NR>(ch, f, valid, acc, NOUT);
+            add_outputs<NOUT>(o, valid, acc);
         }
     }
 
     // ragged tail (< 1024 cells): one CTA, scalar loads
     const long long tail0 = ntiles << 10;
     if (tail0 < ncells && blockIdx.x == (unsigned)(ntiles % gridDim.x)) {
-        RegFile<NR, kV> f;
+        double in[kIn][kV];
         bool valid[kV];
         long long idx[kV];
 #pragma unroll
         for (int i = 0; i < kV; ++i) {
             idx[i] = tail0 + t + i * kThreads;
             valid[i] = idx[i] < ncells;
-            f.r[0][i] = valid[i] ? ld_stream1(p.X + idx[i]) : 0.0;
+            in[0][i] = valid[i] ? ld_stream1(p.X + idx[i]) : 0.0;
         }
 #pragma unroll
         for (int k = 0; k < FO_MAX_SIDES; ++k) {
-            if (1 + k < NR && (ch.side_used >> k) & 1u) {
-                const int R = (1 + k < NR) ? 1 + k : 0;
+            if (EVAL::uses_side(ch, k)) {
 #pragma unroll
                 for (int i = 0; i < kV; ++i)
-                    f.r[R][i] = valid[i] ? ld_stream1(p.sides.s[k].data + idx[i]) : 0.0;
+                    in[1 + k][i] = valid[i] ? ld_stream1(p.sides.s[k].data + idx[i]) : 0.0;
             }
         }
-        run_chain<NR, kV>(ch, f);
+        double o[NOUT][kV];
+        EVAL::template run<kV, NOUT>(ch, in, o);
         if (STORE) {
-            double o[kV];
-            operand<NR, kV>(ch, f, ch.out[0], o);
 #pragma unroll
             for (int i = 0; i < kV; ++i)
-                if (valid[i]) p.out[idx[i]] = o[i];
+                if (valid[i]) p.out[idx[i]] = o[0][i];
         } else {
-            add_outputs<NR>(ch, f, valid, acc, NOUT);
+            add_outputs<NOUT>(o, valid, acc);
         }
     }
 
     if (!STORE) {
         block_sum<NOUT>(acc, s_red);
         if (t == 0) {
+#pragma unroll
             for (int k = 0; k < NOUT; ++k)
                 if (k < ch.n_out) p.partials[(size_t)blockIdx.x * ch.n_out + k] = acc[k];
         }
@@ -148,43 +144,40 @@ __device__ __forceinline__ double2 load_pair(const double *row, long long col, l
     return make_double2(0.0, 0.0);
 }
 
-template <int NR, bool ALIGNED>
-__device__ __forceinline__ void load_row_inputs(const DevChain &ch, const CellParams &p,
-                                                long long row, long long ca, long long cb,
-                                                RegFile<NR, kV> &f)
+__device__ __forceinline__ double2 load_pair_cached(const double *row, long long col, long long cols)
 {
-    {
-        const double *xr = p.X + row * p.ldx;
-        const double2 m0 = load_pair<ALIGNED>(xr, ca, p.cols), m1 = load_pair<ALIGNED>(xr, cb, p.cols);
-        f.r[0][0] = m0.x; f.r[0][1] = m0.y; f.r[0][2] = m1.x; f.r[0][3] = m1.y;
-    }
+    return make_double2(col < cols ? __ldg(row + col) : 0.0, col + 1 < cols ? __ldg(row + col + 1) : 0.0);
+}
+
+// Inputs of the cells (rowa, ca), (rowa, ca+1), (rowb, cb), (rowb, cb+1).
+template <class EVAL, bool ALIGNED>
+__device__ __forceinline__ void load_inputs_2d(const DevChain &ch, const CellParams &p,
+                                               long long rowa, long long ca, long long rowb,
+                                               long long cb, bool have_b, double (&in)[kIn][kV])
+{
+    put4(in[0], load_pair<ALIGNED>(p.X + rowa * p.ldx, ca, p.cols),
+         have_b ? load_pair<ALIGNED>(p.X + rowb * p.ldx, cb, p.cols) : make_double2(0.0, 0.0));
 #pragma unroll
     for (int k = 0; k < FO_MAX_SIDES; ++k) {
-        if (1 + k < NR && (ch.side_used >> k) & 1u) {
-            const int R = (1 + k < NR) ? 1 + k : 0;
+        if (EVAL::uses_side(ch, k)) {
             const DevSide sd = p.sides.s[k];
             if (sd.access == FO_AT_ROW) {
-                const double v = __ldg(sd.data + row * sd.ld);
-                f.r[R][0] = v; f.r[R][1] = v; f.r[R][2] = v; f.r[R][3] = v;
-            } else {
-                const double *sr = sd.data + (sd.access == FO_AT_CELL ? row * sd.ld : 0);
-                double2 m0, m1;
-                if (sd.access == FO_AT_CELL) {
-                    m0 = load_pair<ALIGNED>(sr, ca, p.cols);
-                    m1 = load_pair<ALIGNED>(sr, cb, p.cols);
-                } else {          // row vector, reused by every row: keep it cached
-                    m0 = make_double2(ca < p.cols ? __ldg(sr + ca) : 0.0,
-                                      ca + 1 < p.cols ? __ldg(sr + ca + 1) : 0.0);
-                    m1 = make_double2(cb < p.cols ? __ldg(sr + cb) : 0.0,
-                                      cb + 1 < p.cols ? __ldg(sr + cb + 1) : 0.0);
-                }
-                f.r[R][0] = m0.x; f.r[R][1] = m0.y; f.r[R][2] = m1.x; f.r[R][3] = m1.y;
+                const double va = __ldg(sd.data + rowa * sd.ld);
+                const double vb = have_b ? __ldg(sd.data + rowb * sd.ld) : 0.0;
+                put4(in[1 + k], make_double2(va, va), make_double2(vb, vb));
+            } else if (sd.access == FO_AT_CELL) {
+                put4(in[1 + k], load_pair<ALIGNED>(sd.data + rowa * sd.ld, ca, p.cols),
+                     have_b ? load_pair<ALIGNED>(sd.data + rowb * sd.ld, cb, p.cols)
+                            : make_double2(0.0, 0.0));
+            } else {              // row vector, reused by every row: keep it cached
+                put4(in[1 + k], load_pair_cached(sd.data, ca, p.cols),
+                     have_b ? load_pair_cached(sd.data, cb, p.cols) : make_double2(0.0, 0.0));
             }
         }
     }
 }
 
-template <int NR, int NOUT, int AGG, bool ALIGNED>
+template <class EVAL, int NOUT, int AGG, bool ALIGNED>
 __global__ void __launch_bounds__(kThreads)
 cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ CellParams p)
 {
@@ -199,25 +192,26 @@ cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
     const long long nwarps = (long long)gridDim.x * (kThreads / 32);
 
     for (long long row = warp0; row < p.rows; row += nwarps) {
-        double rowacc[1] = {0.0};
+        double rowacc[NOUT];
+#pragma unroll
+        for (int k = 0; k < NOUT; ++k) rowacc[k] = 0.0;
         for (long long c0 = 0; c0 < p.cols; c0 += 128) {
             const long long ca = c0 + 2 * lane, cb = ca + 64;
-            RegFile<NR, kV> f;
-            load_row_inputs<NR, ALIGNED>(ch, p, row, ca, cb, f);
-            run_chain<NR, kV>(ch, f);
+            double in[kIn][kV];
+            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, ca, row, cb, true, in);
+            double o[NOUT][kV];
+            EVAL::template run<kV, NOUT>(ch, in, o);
             const bool valid[kV] = {ca < p.cols, ca + 1 < p.cols, cb < p.cols, cb + 1 < p.cols};
             if (AGG == kAggNone) {
-                double o[kV];
-                operand<NR, kV>(ch, f, ch.out[0], o);
                 double *orow = p.out + row * p.cols;
-                if (valid[0]) orow[ca] = o[0];
-                if (valid[1]) orow[ca + 1] = o[1];
-                if (valid[2]) orow[cb] = o[2];
-                if (valid[3]) orow[cb + 1] = o[3];
+                if (valid[0]) orow[ca] = o[0][0];
+                if (valid[1]) orow[ca + 1] = o[0][1];
+                if (valid[2]) orow[cb] = o[0][2];
+                if (valid[3]) orow[cb + 1] = o[0][3];
             } else if (AGG == kAggRow) {
-                add_outputs<NR>(ch, f, valid, rowacc, 1);
+                add_outputs<NOUT>(o, valid, rowacc);
             } else {
-                add_outputs<NR>(ch, f, valid, acc, NOUT);
+                add_outputs<NOUT>(o, valid, acc);
             }
         }
         if (AGG == kAggRow) {
@@ -229,6 +223,7 @@ cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
     if (AGG == kAggFull) {
         block_sum<NOUT>(acc, s_red);
         if (threadIdx.x == 0) {
+#pragma unroll
             for (int k = 0; k < NOUT; ++k)
                 if (k < ch.n_out) p.partials[(size_t)blockIdx.x * ch.n_out + k] = acc[k];
         }
@@ -240,7 +235,7 @@ cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
 // ------------------------------------------------------------------ cols
 // grid.x: tiles of 512 columns; grid.y: row panels.  A thread owns a column pair
 // and walks its panel two rows at a time.
-template <int NR, bool ALIGNED>
+template <class EVAL, bool ALIGNED>
 __global__ void __launch_bounds__(kThreads)
 cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ CellParams p)
 {
@@ -254,44 +249,15 @@ cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
     if (col < p.cols) {
         for (long long row = r0; row < r1; row += 2) {
             const bool two = row + 1 < r1;
-            RegFile<NR, kV> f;
-            {
-                const double2 m0 = load_pair<ALIGNED>(p.X + row * p.ldx, col, p.cols);
-                const double2 m1 = two ? load_pair<ALIGNED>(p.X + (row + 1) * p.ldx, col, p.cols)
-                                       : make_double2(0.0, 0.0);
-                f.r[0][0] = m0.x; f.r[0][1] = m0.y; f.r[0][2] = m1.x; f.r[0][3] = m1.y;
-            }
-#pragma unroll
-            for (int k = 0; k < FO_MAX_SIDES; ++k) {
-                if (1 + k < NR && (ch.side_used >> k) & 1u) {
-                    const int R = (1 + k < NR) ? 1 + k : 0;
-                    const DevSide sd = p.sides.s[k];
-                    double2 m0, m1;
-                    if (sd.access == FO_AT_ROW) {
-                        const double v0 = __ldg(sd.data + row * sd.ld);
-                        const double v1 = two ? __ldg(sd.data + (row + 1) * sd.ld) : 0.0;
-                        m0 = make_double2(v0, v0);
-                        m1 = make_double2(v1, v1);
-                    } else if (sd.access == FO_AT_CELL) {
-                        m0 = load_pair<ALIGNED>(sd.data + row * sd.ld, col, p.cols);
-                        m1 = two ? load_pair<ALIGNED>(sd.data + (row + 1) * sd.ld, col, p.cols)
-                                 : make_double2(0.0, 0.0);
-                    } else {
-                        m0 = make_double2(__ldg(sd.data + col),
-                                          col + 1 < p.cols ? __ldg(sd.data + col + 1) : 0.0);
-                        m1 = m0;
-                    }
-                    f.r[R][0] = m0.x; f.r[R][1] = m0.y; f.r[R][2] = m1.x; f.r[R][3] = m1.y;
-                }
-            }
-            run_chain<NR, kV>(ch, f);
-            double o[kV];
-            operand<NR, kV>(ch, f, ch.out[0], o);
-            a0 += o[0];
-            a1 += o[1];
+            double in[kIn][kV];
+            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, col, row + 1, col, two, in);
+            double o[1][kV];
+            EVAL::template run<kV, 1>(ch, in, o);
+            a0 += o[0][0];
+            a1 += o[0][1];
             if (two) {
-                a0 += o[2];
-                a1 += o[3];
+                a0 += o[0][2];
+                a1 += o[0][3];
             }
         }
         double *pp = p.partials + (size_t)blockIdx.y * p.cols;
@@ -311,14 +277,6 @@ __global__ void fill_zero_kernel(double *out, long long n)
 
 // ------------------------------------------------------------------ host
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
-
-struct CellPlan {
-    bool flat;          // flat streaming kernel applies
-    bool aligned;       // 128-bit loads are legal in the row / column kernels
-    int grid;           // CTAs (flat / rows) or column tiles (cols)
-    int panels;         // cols kernel
-    size_t ws_need;
-};
 
 // Grid of a streaming kernel: every CTA gets work, at most `cap` CTAs.
 int stream_grid(long long units, int sms)
@@ -358,45 +316,55 @@ int check_dense(const fo_dense &d)
     return FO_OK;
 }
 
-template <int NR, int NOUT>
+template <class EVAL, int NOUT>
 cudaError_t launch_cell(const DevChain &ch, const CellParams &p, int agg, bool flat, bool aligned,
                         int grid, cudaStream_t st)
 {
     if (agg == FO_CELL_COL_AGG) {
         if constexpr (NOUT == 1) {
             const dim3 g((unsigned)((p.cols + 511) / 512), (unsigned)p.panels);
-            if (aligned) cell_cols_kernel<NR, true><<<g, kThreads, 0, st>>>(ch, p);
-            else cell_cols_kernel<NR, false><<<g, kThreads, 0, st>>>(ch, p);
+            if (aligned) cell_cols_kernel<EVAL, true><<<g, kThreads, 0, st>>>(ch, p);
+            else cell_cols_kernel<EVAL, false><<<g, kThreads, 0, st>>>(ch, p);
         }
     } else if (flat) {
         if (agg == FO_CELL_NO_AGG) {
-            if constexpr (NOUT == 1) cell_flat_kernel<NR, 1, true><<<grid, kThreads, 0, st>>>(ch, p);
+            if constexpr (NOUT == 1) cell_flat_kernel<EVAL, 1, true><<<grid, kThreads, 0, st>>>(ch, p);
         } else {
-            cell_flat_kernel<NR, NOUT, false><<<grid, kThreads, 0, st>>>(ch, p);
+            cell_flat_kernel<EVAL, NOUT, false><<<grid, kThreads, 0, st>>>(ch, p);
         }
     } else if (agg == FO_CELL_FULL_AGG) {
-        if (aligned) cell_rows_kernel<NR, NOUT, kAggFull, true><<<grid, kThreads, 0, st>>>(ch, p);
-        else cell_rows_kernel<NR, NOUT, kAggFull, false><<<grid, kThreads, 0, st>>>(ch, p);
+        if (aligned) cell_rows_kernel<EVAL, NOUT, kAggFull, true><<<grid, kThreads, 0, st>>>(ch, p);
+        else cell_rows_kernel<EVAL, NOUT, kAggFull, false><<<grid, kThreads, 0, st>>>(ch, p);
     } else if constexpr (NOUT == 1) {
         if (agg == FO_CELL_ROW_AGG) {
-            if (aligned) cell_rows_kernel<NR, 1, kAggRow, true><<<grid, kThreads, 0, st>>>(ch, p);
-            else cell_rows_kernel<NR, 1, kAggRow, false><<<grid, kThreads, 0, st>>>(ch, p);
+            if (aligned) cell_rows_kernel<EVAL, 1, kAggRow, true><<<grid, kThreads, 0, st>>>(ch, p);
+            else cell_rows_kernel<EVAL, 1, kAggRow, false><<<grid, kThreads, 0, st>>>(ch, p);
         } else {
-            if (aligned) cell_rows_kernel<NR, 1, kAggNone, true><<<grid, kThreads, 0, st>>>(ch, p);
-            else cell_rows_kernel<NR, 1, kAggNone, false><<<grid, kThreads, 0, st>>>(ch, p);
+            if (aligned) cell_rows_kernel<EVAL, 1, kAggNone, true><<<grid, kThreads, 0, st>>>(ch, p);
+            else cell_rows_kernel<EVAL, 1, kAggNone, false><<<grid, kThreads, 0, st>>>(ch, p);
         }
     }
     return cudaGetLastError();
 }
 
 template <int NR>
-cudaError_t launch_cell_nr(const DevChain &ch, const CellParams &p, int agg, bool flat,
-                           bool aligned, int grid, cudaStream_t st)
+cudaError_t launch_cell_interp(const DevChain &ch, const CellParams &p, int agg, bool flat,
+                               bool aligned, int grid, cudaStream_t st)
 {
-    if (ch.n_out == 1) return launch_cell<NR, 1>(ch, p, agg, flat, aligned, grid, st);
-    if (ch.n_out <= 4) return launch_cell<NR, 4>(ch, p, agg, flat, aligned, grid, st);
-    return launch_cell<NR, 8>(ch, p, agg, flat, aligned, grid, st);
+    if (ch.n_out == 1) return launch_cell<EvalInterp<NR>, 1>(ch, p, agg, flat, aligned, grid, st);
+    if (ch.n_out <= 4) return launch_cell<EvalInterp<NR>, 4>(ch, p, agg, flat, aligned, grid, st);
+    return launch_cell<EvalInterp<NR>, 8>(ch, p, agg, flat, aligned, grid, st);
 }
+
+template <int ID>
+cudaError_t launch_cell_spec(const DevChain &ch, const CellParams &p, int agg, bool flat,
+                             bool aligned, int grid, cudaStream_t st)
+{
+    return launch_cell<EvalSpec<ID>, SpecFn<ID>::kOut>(ch, p, agg, flat, aligned, grid, st);
+}
+
+// Test / benchmark switch: run every chain through the interpreter.
+bool g_force_interpreter = false;
 
 // Common body of fused_cell and fused_magg.
 int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
@@ -482,9 +450,17 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     }
 
     cudaError_t e;
-    if (ch.n_regs <= 4) e = launch_cell_nr<4>(ch, p, agg, flat, aligned, grid, st);
-    else if (ch.n_regs <= 8) e = launch_cell_nr<8>(ch, p, agg, flat, aligned, grid, st);
-    else e = launch_cell_nr<kRegs>(ch, p, agg, flat, aligned, grid, st);
+    switch (g_force_interpreter ? kSpecNone : match_cell_spec(ch)) {
+        case kSpecMul2: e = launch_cell_spec<kSpecMul2>(ch, p, agg, flat, aligned, grid, st); break;
+        case kSpecMul3: e = launch_cell_spec<kSpecMul3>(ch, p, agg, flat, aligned, grid, st); break;
+        case kSpecSq: e = launch_cell_spec<kSpecSq>(ch, p, agg, flat, aligned, grid, st); break;
+        case kSpecMagg2: e = launch_cell_spec<kSpecMagg2>(ch, p, agg, flat, aligned, grid, st); break;
+        case kSpecMagg3: e = launch_cell_spec<kSpecMagg3>(ch, p, agg, flat, aligned, grid, st); break;
+        default:
+            if (ch.n_regs <= 4) e = launch_cell_interp<4>(ch, p, agg, flat, aligned, grid, st);
+            else if (ch.n_regs <= 8) e = launch_cell_interp<8>(ch, p, agg, flat, aligned, grid, st);
+            else e = launch_cell_interp<kRegs>(ch, p, agg, flat, aligned, grid, st);
+    }
     return e == cudaSuccess ? FO_OK : cuda_fail(e);
 }
 
@@ -493,6 +469,13 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
 }  // namespace fo
 
 extern "C" {
+
+int fo_set_force_interpreter(int on)
+{
+    const int prev = fo::g_force_interpreter ? 1 : 0;
+    fo::g_force_interpreter = on != 0;
+    return prev;
+}
 
 size_t fused_cell_workspace_bytes(const fo_mat *X, int agg)
 {

@@ -164,6 +164,7 @@ int translate_chain(const fo_chain *chain, ChainUse use, int n_sides,
     out->n_out = chain->n_out;
     out->n_regs = al.high;
     out->side_used = al.side_used;
+    out->tmp_base = al.base;
     return FO_OK;
 }
 

@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "../../include/fusedops.h"
 
@@ -42,6 +43,8 @@ struct DevChain {
     int32_t n_out;
     int32_t n_regs;                  // registers in use (upper bound on every index)
     uint32_t side_used;              // bit k: the chain reads side k
+    int32_t tmp_base;                // first temporary register (inputs sit below it)
+    int32_t pad0;
     uint8_t out[FO_MAX_OUT];         // operand bytes (register or constant)
     DevOp ops[FO_MAX_OPS];
     double consts[kConsts];

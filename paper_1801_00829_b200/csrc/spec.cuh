@@ -1,0 +1,129 @@
+// Two ways to evaluate an operator chain inside a kernel, behind one interface:
+//
+//   EvalInterp<NR>  the general register-machine interpreter of chain.cuh;
+//   EvalSpec<ID>    the same arithmetic, in the same order, written out at
+//                   compile time for a few chains that the paper's fusion
+//                   examples keep producing (Fig. 1; Section 5.2).
+//
+// The host recognises a specialised chain by comparing the translated program
+// with the specialisation's reference program (spec_host.cu); any other chain
+// runs through the interpreter.  Both give bit-identical results.
+#pragma once
+
+#include "chain.cuh"
+
+namespace fo {
+
+enum SpecId {
+    kSpecNone = 0,
+    kSpecMul2,      // a * side0                         sum(X * Y)
+    kSpecMul3,      // (a * side0) * side1               sum(X * Y * Z), Fig. 1(a)
+    kSpecSq,        // a * a                             sum(X^2)
+    kSpecMagg2,     // (a * side0, a * side1)            Section 5.2 multi-aggregate
+    kSpecMagg3,     // (a * side0, a * side1, a * a)     Fig. 1(c)-style
+    kSpecCount
+};
+
+// Host: specialisation matching a translated Cell / MAgg chain, or kSpecNone.
+int match_cell_spec(const DevChain &ch);
+
+constexpr int kIn = 1 + FO_MAX_SIDES;      // input slots: a, side0..side3
+
+template <int NR>
+struct EvalInterp {
+    static constexpr bool kInterp = true;
+    static constexpr int kOutMax = FO_MAX_OUT;
+    __device__ __forceinline__ static bool uses_side(const DevChain &ch, int k)
+    {
+        return 1 + k < NR && ((ch.side_used >> k) & 1u);
+    }
+    template <int V, int NOUT>
+    __device__ __forceinline__ static void run(const DevChain &ch, const double (&in)[kIn][V],
+                                               double (&o)[NOUT][V])
+    {
+        RegFile<NR, V> f;
+#pragma unroll
+        for (int k = 0; k < kIn; ++k) {
+            if (k < NR) {
+#pragma unroll
+                for (int i = 0; i < V; ++i) f.r[k < NR ? k : 0][i] = in[k][i];
+            }
+        }
+        run_chain<NR, V>(ch, f);
+#pragma unroll
+        for (int k = 0; k < NOUT; ++k) {
+            if (k < ch.n_out) {
+                operand<NR, V>(ch, f, ch.out[k], o[k]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < V; ++i) o[k][i] = 0.0;
+            }
+        }
+    }
+};
+
+template <int ID>
+struct SpecFn;
+
+template <>
+struct SpecFn<kSpecMul2> {
+    static constexpr int kSides = 1, kOut = 1;
+    __device__ __forceinline__ static void eval(const double *in, double *o) { o[0] = in[0] * in[1]; }
+};
+template <>
+struct SpecFn<kSpecMul3> {
+    static constexpr int kSides = 2, kOut = 1;
+    __device__ __forceinline__ static void eval(const double *in, double *o)
+    {
+        o[0] = (in[0] * in[1]) * in[2];
+    }
+};
+template <>
+struct SpecFn<kSpecSq> {
+    static constexpr int kSides = 0, kOut = 1;
+    __device__ __forceinline__ static void eval(const double *in, double *o) { o[0] = in[0] * in[0]; }
+};
+template <>
+struct SpecFn<kSpecMagg2> {
+    static constexpr int kSides = 2, kOut = 2;
+    __device__ __forceinline__ static void eval(const double *in, double *o)
+    {
+        o[0] = in[0] * in[1];
+        o[1] = in[0] * in[2];
+    }
+};
+template <>
+struct SpecFn<kSpecMagg3> {
+    static constexpr int kSides = 2, kOut = 3;
+    __device__ __forceinline__ static void eval(const double *in, double *o)
+    {
+        o[0] = in[0] * in[1];
+        o[1] = in[0] * in[2];
+        o[2] = in[0] * in[0];
+    }
+};
+
+template <int ID>
+struct EvalSpec {
+    using Fn = SpecFn<ID>;
+    static constexpr bool kInterp = false;
+    static constexpr int kOutMax = Fn::kOut;
+    __device__ __forceinline__ static bool uses_side(const DevChain &, int k) { return k < Fn::kSides; }
+    template <int V, int NOUT>
+    __device__ __forceinline__ static void run(const DevChain &, const double (&in)[kIn][V],
+                                               double (&o)[NOUT][V])
+    {
+        static_assert(NOUT >= Fn::kOut, "accumulator count");
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            double x[kIn], y[Fn::kOut];
+#pragma unroll
+            for (int k = 0; k < kIn; ++k) x[k] = (k <= Fn::kSides) ? in[k][i] : 0.0;
+            Fn::eval(x, y);
+#pragma unroll
+            for (int k = 0; k < NOUT; ++k) o[k][i] = (k < Fn::kOut) ? y[k < Fn::kOut ? k : 0] : 0.0;
+        }
+    }
+};
+
+}  // namespace fo

@@ -326,3 +326,44 @@ def test_outer_log_chain(fo):
     ref = oracle.outer(chain, "t2", Xh, U, V, [1e-15], mode="masked")
     got = fo.fused_outer(chain, "t2", csr_to_dev(w), to_dev(U), to_dev(V), [1e-15])
     assert_close(got.cpu().numpy(), [ref])
+
+
+# ------------------------------------------------------------------ specialised vs interpreted chains
+@pytest.mark.parametrize("name,chain,outs,nsides", [
+    ("mul2", [("mul", "t0", "a", "side0")], ["t0"], 1),
+    ("mul3", XYZ, ["t1"], 2),
+    ("mul3-renamed", [("mul", "t5", "a", "side0"), ("mul", "t2", "t5", "side1")], ["t2"], 2),
+    ("sq", [("mul", "t0", "a", "a")], ["t0"], 0),
+    ("sq-op", [("sq", "t3", "a")], ["t3"], 2),
+    ("magg2", [("mul", "t0", "a", "side0"), ("mul", "t1", "a", "side1")], ["t0", "t1"], 2),
+    ("magg3", MAGG3, ["t0", "t1", "t2"], 2),
+])
+def test_specialised_chains_equal_interpreter_bitwise(fo, name, chain, outs, nsides):
+    rows, cols = 700, 300
+    w = datagen.magg_workload(rows, cols, seed=41)
+    sides_h = [("cell", w["Y"]), ("cell", w["Z"])][:nsides]
+    X, sides = to_dev(w["X"]), dev_sides(sides_h)
+    ref = oracle.magg(chain, outs, w["X"], sides_h)
+    absref = oracle.magg(chain + [("abs", o, o) for o in outs], outs, w["X"], sides_h)
+    try:
+        fo.force_interpreter(False)
+        fast = fo.fused_magg(chain, outs, X, sides).cpu().numpy()
+        fo.force_interpreter(True)
+        slow = fo.fused_magg(chain, outs, X, sides).cpu().numpy()
+    finally:
+        fo.force_interpreter(False)
+    assert fast.tobytes() == slow.tobytes(), name
+    assert_close(fast, ref, absscale=absref, what=name)
+    if len(outs) == 1:
+        for agg in ("row", "col", "none"):
+            r = oracle.cell(chain, outs[0], w["X"], sides_h, agg=agg)
+            a = oracle.cell(chain + [("abs", outs[0], outs[0])], outs[0], w["X"], sides_h, agg=agg)
+            try:
+                fo.force_interpreter(False)
+                f1 = fo.fused_cell(chain, outs[0], X, sides, agg=agg).cpu().numpy()
+                fo.force_interpreter(True)
+                f2 = fo.fused_cell(chain, outs[0], X, sides, agg=agg).cpu().numpy()
+            finally:
+                fo.force_interpreter(False)
+            assert f1.tobytes() == f2.tobytes(), (name, agg)
+            assert_close(f1, r, absscale=a, what="%s %s" % (name, agg))
