@@ -22,6 +22,10 @@ LIB_PATH = os.path.join(HERE, "libfusedops.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",
+    # no implicit multiply-add contraction: every chain step rounds on its own, so
+    # specialised and interpreted chains agree bit for bit; fused multiply-adds
+    # are written explicitly (fma) where a kernel wants them
+    "-fmad=false",
 ]
 
 

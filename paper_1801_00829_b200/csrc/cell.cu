@@ -260,12 +260,27 @@ cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
                 a1 += o[0][3];
             }
         }
-        double *pp = p.partials + (size_t)blockIdx.y * p.cols;
-        pp[col] = a0;
-        if (col + 1 < p.cols) pp[col + 1] = a1;
+        if (p.panels == 1) {
+            p.out[col] = a0;
+            if (col + 1 < p.cols) p.out[col + 1] = a1;
+        } else {
+            double *pp = p.partials + (size_t)blockIdx.y * p.cols;
+            pp[col] = a0;
+            if (col + 1 < p.cols) pp[col + 1] = a1;
+        }
     }
-    if (publish_and_is_last(p.head, &s_flag))
-        final_sum_columns(p.partials, p.panels, p.cols, p.out);
+    if (p.panels == 1) return;
+    // the last panel of this column tile to finish adds the tile's partials, panel 0 first
+    if (take_ticket(&p.head->group[blockIdx.x], (unsigned)p.panels, &s_flag) && col < p.cols) {
+        double s0 = 0.0, s1 = 0.0;
+        const bool two = col + 1 < p.cols;
+        for (int g = 0; g < p.panels; ++g) {
+            s0 += __ldcg(p.partials + (size_t)g * p.cols + col);
+            if (two) s1 += __ldcg(p.partials + (size_t)g * p.cols + col + 1);
+        }
+        p.out[col] = s0;
+        if (two) p.out[col + 1] = s1;
+    }
 }
 
 __global__ void fill_zero_kernel(double *out, long long n)
@@ -288,11 +303,14 @@ int stream_grid(long long units, int sms)
     return (int)g;
 }
 
+// Row panels of the column-aggregation kernel: enough CTAs to fill the GPU, at
+// least 32 rows per panel, one ticket per column tile.
 int col_panels(long long rows, long long cols)
 {
     const long long tiles = (cols + 511) / 512;
+    if (tiles > kMaxGroups) return 1;
     long long p = (148 * 8 + tiles - 1) / tiles;
-    const long long maxp = (rows + 7) / 8;          // at least 8 rows per panel
+    const long long maxp = (rows + 31) / 32;
     if (p > maxp) p = maxp;
     if (p > kMaxPartials) p = kMaxPartials;
     if (p < 1) p = 1;

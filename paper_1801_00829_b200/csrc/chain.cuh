@@ -125,4 +125,55 @@ __device__ __forceinline__ void run_chain(const DevChain &ch, RegFile<NR, V> &f)
     }
 }
 
+// One scalar evaluation of the chain by a whole warp.  The register file is
+// spread over the lanes: lane k holds register k (`mine`), operands are fetched
+// with a shuffle from the lane named by the operand byte, and the lane named by
+// `dst` keeps the result.  No register is indexed at run time and no lane
+// diverges; the cost is a few shuffles per step.  All 32 lanes must call it with
+// the same chain; the result is returned in every lane.
+__device__ __forceinline__ double warp_operand(const DevChain &ch, double mine, int opnd)
+{
+    if (opnd & 0x80) return ch.consts[opnd & 0x7f];
+    return __shfl_sync(0xffffffffu, mine, opnd & 31);
+}
+
+__device__ __forceinline__ double warp_chain(const DevChain &ch, double mine, int lane)
+{
+    const int n = ch.n_ops;
+    for (int s = 0; s < n; ++s) {
+        const DevOp op = ch.ops[s];
+        const double a = warp_operand(ch, mine, op.a);
+        double b = 0.0, c = 0.0, r;
+        if (op.opcode >= FO_OP_ADD) b = warp_operand(ch, mine, op.b);
+        if (op.opcode >= FO_OP_SEL) c = warp_operand(ch, mine, op.c);
+        switch (op.opcode) {
+            case FO_OP_MOV: r = a; break;
+            case FO_OP_NEG: r = -a; break;
+            case FO_OP_ABS: r = fabs(a); break;
+            case FO_OP_SQRT: r = slow_sqrt(a); break;
+            case FO_OP_EXP: r = slow_exp(a); break;
+            case FO_OP_LOG: r = slow_log(a); break;
+            case FO_OP_SQ: r = a * a; break;
+            case FO_OP_ADD: r = a + b; break;
+            case FO_OP_SUB: r = a - b; break;
+            case FO_OP_MUL: r = a * b; break;
+            case FO_OP_DIV: r = slow_div(a, b); break;
+            case FO_OP_MIN: r = fmin(a, b); break;
+            case FO_OP_MAX: r = fmax(a, b); break;
+            case FO_OP_POW: r = slow_pow(a, b); break;
+            case FO_OP_EQ: r = a == b ? 1.0 : 0.0; break;
+            case FO_OP_NE: r = a != b ? 1.0 : 0.0; break;
+            case FO_OP_LT: r = a < b ? 1.0 : 0.0; break;
+            case FO_OP_LE: r = a <= b ? 1.0 : 0.0; break;
+            case FO_OP_GT: r = a > b ? 1.0 : 0.0; break;
+            case FO_OP_GE: r = a >= b ? 1.0 : 0.0; break;
+            case FO_OP_SEL: r = a != 0.0 ? b : c; break;
+            case FO_OP_FMA: r = fma(a, b, c); break;
+            default: r = 0.0; break;
+        }
+        if (lane == op.dst) mine = r;
+    }
+    return warp_operand(ch, mine, ch.out[0]);
+}
+
 }  // namespace fo

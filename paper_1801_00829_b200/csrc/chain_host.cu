@@ -229,12 +229,12 @@ int fo_workspace_init(void *ws, size_t ws_bytes, void *stream)
 int fo_query_device_status(const void *ws, void *stream, int *status)
 {
     if (!ws || !status) return FO_ERR_NULL;
-    fo::WsHead head;
-    cudaError_t e = cudaMemcpyAsync(&head, ws, sizeof(head), cudaMemcpyDeviceToHost,
+    unsigned int words[2] = {0u, 0u};      // ticket, status
+    cudaError_t e = cudaMemcpyAsync(words, ws, sizeof(words), cudaMemcpyDeviceToHost,
                                     (cudaStream_t)stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return fo::cuda_fail(e);
-    *status = head.status ? FO_ERR_DEVICE_TIMEOUT : FO_OK;
+    *status = words[1] ? FO_ERR_DEVICE_TIMEOUT : FO_OK;
     return FO_OK;
 }
 

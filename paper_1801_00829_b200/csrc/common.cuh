@@ -10,13 +10,17 @@
 namespace fo {
 
 // ---------------------------------------------------------------- workspace
-// Head of every workspace: control words, then the per-CTA partials.
+// Head of every workspace: control words, then the per-CTA partials.  All
+// counters are zero between calls: whoever takes the last ticket resets it.
 struct WsHead {
-    unsigned int ticket;     // CTAs that have published their partial; reset by the last one
-    unsigned int status;     // 0, or 1 once a bounded device-side wait ran out
+    unsigned int ticket;        // CTAs (or groups) that have published; reset by the last one
+    unsigned int status;        // 0, or 1 once a bounded device-side wait ran out
     unsigned int pad[62];
+    unsigned int group[4032];   // tickets of CTA groups / column tiles
 };
-static_assert(sizeof(WsHead) == 256, "workspace head is 256 bytes");
+static_assert(sizeof(WsHead) == 16384, "workspace head is 16 KB");
+constexpr int kMaxGroups = 4032;
+constexpr int kGroup = 16;      // CTAs per group in the two-level column reduction
 
 constexpr int kMaxPartials = 2048;   // upper bound on CTAs that publish partials
 constexpr int kThreads = 256;        // CTA size of the reduction kernels
@@ -122,23 +126,28 @@ __device__ __forceinline__ void block_sum(double (&v)[NV], double *smem /* NV * 
     }
 }
 
-// Publishes this CTA's partial vector (`width` doubles already written to
-// partials[blockIdx.x * width ..]) and tells whether this CTA is the last one.
-// The last CTA sees every other CTA's partial.  Nobody waits.
-__device__ __forceinline__ bool publish_and_is_last(WsHead *head, unsigned int *s_flag)
+// Takes a ticket; true for the CTA that took the last of `count`.  Every CTA's
+// global writes made before the call are visible to that last CTA.
+__device__ __forceinline__ bool take_ticket(unsigned int *counter, unsigned int count,
+                                            unsigned int *s_flag)
 {
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
-        __threadfence();
-        const unsigned int prev = atomicAdd(&head->ticket, 1u);
-        const bool last = (prev == gridDim.x * gridDim.y - 1);
-        if (last) head->ticket = 0u;     // ready for the next call
+        const unsigned int prev = atomicAdd(counter, 1u);
+        const bool last = (prev == count - 1);
+        if (last) *counter = 0u;         // ready for the next call
         *s_flag = last ? 1u : 0u;
         __threadfence();
     }
     __syncthreads();
     return *s_flag != 0u;
+}
+
+// Tells whether this CTA is the last of the grid to arrive (see take_ticket).
+__device__ __forceinline__ bool publish_and_is_last(WsHead *head, unsigned int *s_flag)
+{
+    return take_ticket(&head->ticket, gridDim.x * gridDim.y, s_flag);
 }
 
 // Final stage of a scalar (or k-vector) sum: the last CTA adds the G partials
@@ -157,9 +166,9 @@ __device__ __forceinline__ void final_sum_small(const double *partials, int G, i
     }
 }
 
-// Final stage of a vector sum: out[j] = sum_g partials[g * width + j], g ascending.
-__device__ __forceinline__ void final_sum_columns(const double *partials, int G, long long width,
-                                                  double *out)
+// out[j] = sum_g src[g * width + j], g ascending, for the columns this CTA's
+// threads cover.  128-bit loads when `width` is even and src is 16-byte aligned.
+__device__ __forceinline__ void sum_columns(const double *src, int G, long long width, double *out)
 {
     for (long long j = threadIdx.x; j < width; j += blockDim.x) {
         double s = 0.0;
@@ -167,13 +176,35 @@ __device__ __forceinline__ void final_sum_columns(const double *partials, int G,
         for (; g + 8 <= G; g += 8) {
             double t[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) t[u] = __ldcg(partials + (size_t)(g + u) * width + j);
+            for (int u = 0; u < 8; ++u) t[u] = __ldcg(src + (size_t)(g + u) * width + j);
 #pragma unroll
             for (int u = 0; u < 8; ++u) s += t[u];
         }
-        for (; g < G; ++g) s += __ldcg(partials + (size_t)g * width + j);
+        for (; g < G; ++g) s += __ldcg(src + (size_t)g * width + j);
         out[j] = s;
     }
+}
+
+// Two-level, fixed-order sum of the G per-CTA vectors in `partials` (G x width,
+// CTA-major; G <= kGroup * kMaxGroups): the last CTA of each group of kGroup
+// CTAs adds that group's vectors into `gpart` (groups x width), the last group
+// to finish adds the group vectors into `out`.  Nobody waits.
+__device__ __forceinline__ void reduce_columns_two_level(WsHead *head, const double *partials,
+                                                         double *gpart, long long width,
+                                                         double *out, unsigned int *s_flag)
+{
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int ngroups = (G + kGroup - 1) / kGroup;
+    const int gid = cta / kGroup;
+    const int gsize = (G - gid * kGroup < kGroup) ? G - gid * kGroup : kGroup;
+    if (!take_ticket(&head->group[gid], (unsigned)gsize, s_flag)) return;
+    if (ngroups == 1) {
+        sum_columns(partials, gsize, width, out);
+        return;
+    }
+    sum_columns(partials + (size_t)gid * kGroup * width, gsize, width, gpart + (size_t)gid * width);
+    if (!take_ticket(&head->ticket, (unsigned)ngroups, s_flag)) return;
+    sum_columns(gpart, ngroups, width, out);
 }
 #endif  // __CUDACC__
 

@@ -5,8 +5,8 @@
 // Schedule: CTAs own contiguous row ranges holding equal shares of the stored
 // cells (binary search on rowptr); inside a CTA a warp owns a row at a time.
 // The row U_i sits in registers, spread over the 8 lanes of a group; the four
-// groups of a warp take stored cells p, p+1, p+2, p+3 of the row and gather
-// their V_j rows with 128-bit loads (V is read many times and stays in L2).
+// groups of a warp take different stored cells of the row and gather their V_j
+// rows with 128-bit loads (V is read many times and stays in L2).
 #include "chain.cuh"
 
 namespace fo {
@@ -52,14 +52,6 @@ __device__ __forceinline__ double outer_chain(const DevChain &ch, double a, doub
     return o[0];
 }
 
-__device__ __forceinline__ double group_sum(double v, unsigned gmask)
-{
-    v += __shfl_xor_sync(gmask, v, 4);
-    v += __shfl_xor_sync(gmask, v, 2);
-    v += __shfl_xor_sync(gmask, v, 1);
-    return v;
-}
-
 // First row r in [0, rows] with rowptr[r] >= target.
 __device__ __forceinline__ long long lower_row(const int *rowptr, long long rows, long long target)
 {
@@ -72,8 +64,15 @@ __device__ __forceinline__ long long lower_row(const int *rowptr, long long rows
 }
 
 // NK2: double2 chunks per lane (rank <= 16 * NK2).
+//
+// A warp walks its row in chunks of 32 stored cells.  Column indices and values
+// of a chunk are loaded one per lane (coalesced); the four 8-lane groups then
+// take cells 0-3, 4-7, ... of the chunk, two cells per group and trip, gather
+// the V rows and reduce their dot products; each dot product is routed back to
+// the lane that holds its cell, so the operator chain runs once per chunk with
+// one cell per lane.
 template <int NK2, int AGG, bool ALIGNED>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, (NK2 > 8 ? 1 : 2))
 outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
 {
     __shared__ double s_red[32];
@@ -90,69 +89,81 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int l8 = lane & 7, grp = lane >> 3;
-    const unsigned gmask = 0xffu << (lane & 24);
+    const unsigned full = 0xffffffffu;
     const int rank = p.rank;
     double acc = 0.0;
 
     for (long long row = row_lo + warp; row < row_hi; row += kThreads / 32) {
         const int beg = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
-        if (beg == end) {
-            if (AGG == kOutRight) {
-                for (int c = lane; c < rank; c += 32) p.out[row * rank + c] = 0.0;
-            }
-            continue;
-        }
         double2 u[NK2], racc[NK2];
         const double *urow = p.U + row * p.ldu;
 #pragma unroll
         for (int c = 0; c < NK2; ++c) {
-            u[c] = ld_pair_cached<ALIGNED>(urow, 16 * c + 2 * l8, rank);
+            u[c] = (beg < end) ? ld_pair_cached<ALIGNED>(urow, 16 * c + 2 * l8, rank)
+                               : make_double2(0.0, 0.0);
             racc[c] = make_double2(0.0, 0.0);
         }
-        for (int q0 = beg + grp; q0 < end; q0 += 8) {
-            // two stored cells per group and trip: q0 and q0 + 4
-            const int q1 = q0 + 4;
-            const bool two = q1 < end;
-            const int j0 = __ldg(p.colidx + q0);
-            const int j1 = two ? __ldg(p.colidx + q1) : j0;
-            const double a0 = __ldg(p.vals + q0);
-            const double a1 = two ? __ldg(p.vals + q1) : 0.0;
-            const double *v0 = p.V + (long long)j0 * p.ldv;
-            const double *v1 = p.V + (long long)j1 * p.ldv;
-            double2 x0[NK2], x1[NK2];
-#pragma unroll
-            for (int c = 0; c < NK2; ++c) {
-                x0[c] = ld_pair_cached<ALIGNED>(v0, 16 * c + 2 * l8, rank);
-                x1[c] = ld_pair_cached<ALIGNED>(v1, 16 * c + 2 * l8, rank);
-            }
-            double d0 = 0.0, d1 = 0.0;
-#pragma unroll
-            for (int c = 0; c < NK2; ++c) {
-                d0 = fma(u[c].x, x0[c].x, d0);
-                d0 = fma(u[c].y, x0[c].y, d0);
-                d1 = fma(u[c].x, x1[c].x, d1);
-                d1 = fma(u[c].y, x1[c].y, d1);
-            }
-            d0 = group_sum(d0, gmask);
-            d1 = group_sum(d1, gmask);
-            // lane 0 of the group evaluates cell q0, lane 1 cell q1 (one pass of the chain)
-            const double a = (l8 == 1) ? a1 : a0;
-            const double d = (l8 == 1) ? d1 : d0;
-            const double w = outer_chain(ch, a, d);
-            if (AGG == kOutFull) {
-                if (l8 == 0 || (l8 == 1 && two)) acc += w;
-            } else if (AGG == kOutNone) {
-                if (l8 == 0) p.out[q0] = w;
-                if (l8 == 1 && two) p.out[q1] = w;
-            } else {
-                const double w0 = __shfl_sync(gmask, w, (lane & 24) + 0);
-                const double w1 = two ? __shfl_sync(gmask, w, (lane & 24) + 1) : 0.0;
+        for (int c0 = beg; c0 < end; c0 += 32) {
+            const int cnt = (end - c0 < 32) ? end - c0 : 32;
+            const bool valid = lane < cnt;
+            const int jmine = valid ? __ldg(p.colidx + c0 + lane) : 0;
+            const double amine = valid ? __ldg(p.vals + c0 + lane) : 0.0;
+            double dmine = 0.0;
+            const int nit = (cnt + 3) >> 2;
+            for (int it = 0; it < nit; it += 2) {
+                const int srcA = it * 4 + grp, srcB = srcA + 4;
+                const bool actA = srcA < cnt, actB = srcB < cnt;
+                const int jA = __shfl_sync(full, jmine, srcA & 31);
+                const int jB = __shfl_sync(full, jmine, srcB & 31);
+                const double *vA = p.V + (long long)jA * p.ldv;
+                const double *vB = p.V + (long long)jB * p.ldv;
+                double2 xA[NK2], xB[NK2];
 #pragma unroll
                 for (int c = 0; c < NK2; ++c) {
-                    racc[c].x = fma(w0, x0[c].x, racc[c].x);
-                    racc[c].y = fma(w0, x0[c].y, racc[c].y);
-                    racc[c].x = fma(w1, x1[c].x, racc[c].x);
-                    racc[c].y = fma(w1, x1[c].y, racc[c].y);
+                    xA[c] = actA ? ld_pair_cached<ALIGNED>(vA, 16 * c + 2 * l8, rank) : make_double2(0.0, 0.0);
+                    xB[c] = actB ? ld_pair_cached<ALIGNED>(vB, 16 * c + 2 * l8, rank) : make_double2(0.0, 0.0);
+                }
+                double dA = 0.0, dB = 0.0;
+#pragma unroll
+                for (int c = 0; c < NK2; ++c) {
+                    dA = fma(u[c].x, xA[c].x, dA);
+                    dA = fma(u[c].y, xA[c].y, dA);
+                    dB = fma(u[c].x, xB[c].x, dB);
+                    dB = fma(u[c].y, xB[c].y, dB);
+                }
+                dA += __shfl_xor_sync(full, dA, 4);
+                dB += __shfl_xor_sync(full, dB, 4);
+                dA += __shfl_xor_sync(full, dA, 2);
+                dB += __shfl_xor_sync(full, dB, 2);
+                dA += __shfl_xor_sync(full, dA, 1);
+                dB += __shfl_xor_sync(full, dB, 1);
+                // cell s of the chunk was handled by group (s & 3) in trip (s >> 2)
+                const double allA = __shfl_sync(full, dA, (lane & 3) * 8);
+                const double allB = __shfl_sync(full, dB, (lane & 3) * 8);
+                if ((lane >> 2) == it) dmine = allA;
+                if ((lane >> 2) == it + 1) dmine = allB;
+            }
+            const double w = outer_chain(ch, amine, dmine);
+            if (AGG == kOutFull) {
+                if (valid) acc += w;
+            } else if (AGG == kOutNone) {
+                if (valid) p.out[c0 + lane] = w;
+            } else {
+                // second walk over the chunk: O_i += w_ij * V_j (rows of V come from cache)
+                for (int it = 0; it < nit; ++it) {
+                    const int src = it * 4 + grp;
+                    const bool act = src < cnt;
+                    const int j = __shfl_sync(full, jmine, src & 31);
+                    const double ww = __shfl_sync(full, w, src & 31);
+                    const double *vj = p.V + (long long)j * p.ldv;
+                    if (act) {
+#pragma unroll
+                        for (int c = 0; c < NK2; ++c) {
+                            const double2 x = ld_pair_cached<ALIGNED>(vj, 16 * c + 2 * l8, rank);
+                            racc[c].x = fma(ww, x.x, racc[c].x);
+                            racc[c].y = fma(ww, x.y, racc[c].y);
+                        }
+                    }
                 }
             }
         }
@@ -160,10 +171,10 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
             // the four groups hold partial rows: add them in a fixed order
 #pragma unroll
             for (int c = 0; c < NK2; ++c) {
-                racc[c].x += __shfl_xor_sync(0xffffffffu, racc[c].x, 8);
-                racc[c].y += __shfl_xor_sync(0xffffffffu, racc[c].y, 8);
-                racc[c].x += __shfl_xor_sync(0xffffffffu, racc[c].x, 16);
-                racc[c].y += __shfl_xor_sync(0xffffffffu, racc[c].y, 16);
+                racc[c].x += __shfl_xor_sync(full, racc[c].x, 8);
+                racc[c].y += __shfl_xor_sync(full, racc[c].y, 8);
+                racc[c].x += __shfl_xor_sync(full, racc[c].x, 16);
+                racc[c].y += __shfl_xor_sync(full, racc[c].y, 16);
                 const int col = 16 * c + 2 * l8;
                 if (grp == 0) {
                     if (col < rank) p.out[row * rank + col] = racc[c].x;

@@ -79,8 +79,21 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
         : "memory");
 }
 
-// Evaluates the row chain: R0 = d, R(1+k) = side k at this row.
-__device__ __forceinline__ double row_chain(const DevChain &ch, double d, const double (&sv)[FO_MAX_SIDES])
+// Side values of one row, spread over the lanes the way warp_chain wants its
+// register file: lane 1 + k holds side k (lane 0 is reserved for d).
+__device__ __forceinline__ double load_sides_lanes(const DevChain &ch, const DevSides &sides,
+                                                   long long row, long long rows, int lane)
+{
+    double v = 0.0;
+#pragma unroll
+    for (int k = 0; k < FO_MAX_SIDES; ++k)
+        if (lane == 1 + k && ((ch.side_used >> k) & 1u) && row < rows)
+            v = __ldg(sides.s[k].data + row * sides.s[k].ld);
+    return v;
+}
+
+// The chain for one row per lane: R0 = d, R(1+k) = side k of that lane's row.
+__device__ __forceinline__ double lane_chain(const DevChain &ch, double d, const double (&sv)[FO_MAX_SIDES])
 {
     RegFile<kRegs, 1> f;
     f.r[0][0] = d;
@@ -90,17 +103,6 @@ __device__ __forceinline__ double row_chain(const DevChain &ch, double d, const 
     double o[1];
     operand<kRegs, 1>(ch, f, ch.out[0], o);
     return o[0];
-}
-
-__device__ __forceinline__ void load_sides(const DevChain &ch, const DevSides &sides, long long row,
-                                           long long rows, double (&sv)[FO_MAX_SIDES])
-{
-#pragma unroll
-    for (int k = 0; k < FO_MAX_SIDES; ++k) {
-        sv[k] = 0.0;
-        if (((ch.side_used >> k) & 1u) && row < rows)
-            sv[k] = __ldg(sides.s[k].data + row * sides.s[k].ld);
-    }
 }
 
 // ------------------------------------------------------------------ dense
@@ -167,12 +169,12 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
         if (STAGED) {
             if (threadIdx.x == 0 && it + S - 1 < my_tiles) issue(it + S - 1);
         }
-        // side values of this warp's rows: requested before the wait so their
-        // latency overlaps it
-        double sv[4][FO_MAX_SIDES];
+        // side values of this warp's rows (lane 1 + k holds side k): requested
+        // before the wait so their latency overlaps it
+        double sv[4];
 #pragma unroll
         for (int rw = 0; rw < 4; ++rw)
-            if (rw < RPW) load_sides(ch, p.sides, r0 + warp * RPW + rw, p.rows, sv[rw]);
+            sv[rw] = rw < RPW ? load_sides_lanes(ch, p.sides, r0 + warp * RPW + rw, p.rows, lane) : 0.0;
         if (STAGED) {
             if (!mbar_wait(&s_full[slot], (unsigned)((it / S) & 1))) timed_out = true;
         }
@@ -206,15 +208,12 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
                 d1 = fma(x[c].y, vv.y, d1);
             }
             const double d = warp_sum(d0 + d1);
-            double svr[FO_MAX_SIDES];
+            double mine = sv[0];
 #pragma unroll
-            for (int k = 0; k < FO_MAX_SIDES; ++k) {
-                svr[k] = sv[0][k];
-#pragma unroll
-                for (int r2 = 1; r2 < 4; ++r2)
-                    if (rw == r2) svr[k] = sv[r2][k];
-            }
-            const double t = row_chain(ch, d, svr);
+            for (int r2 = 1; r2 < 4; ++r2)
+                if (rw == r2) mine = sv[r2];
+            if (lane == 0) mine = d;
+            const double t = warp_chain(ch, mine, lane);
             if (AGG == kRowColT) {
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
@@ -250,8 +249,8 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
             for (int w = 0; w < kWarps; ++w) s += qs[(size_t)w * n + j];
             p.partials[(size_t)blockIdx.x * n + j] = s;
         }
-        if (publish_and_is_last(p.head, &s_flag))
-            final_sum_columns(p.partials, gridDim.x, n, p.out);
+        reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * n, n, p.out,
+                                 &s_flag);
     } else if (AGG == kRowFull) {
         // every lane of a warp holds the same tsum: count it once per warp
         double v1[1] = {lane == 0 ? tsum : 0.0};
@@ -263,9 +262,16 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
 }
 
 // -------------------------------------------------------------------- CSR
-// An 8-lane group per row.  v (and for col_t_agg the output accumulator) sit in
-// shared memory; the scatter  acc[col] += t * val  uses shared-memory atomics
-// because two groups may hit the same column at the same time.
+// A warp takes blocks of 32 consecutive rows.  Row offsets, side values and the
+// chain are handled one row per lane (coalesced loads, one chain evaluation for
+// 32 rows); the block's stored cells - one contiguous piece of colidx / vals -
+// are first copied into the warp's slice of shared memory with coalesced loads,
+// then an 8-lane group walks each row: dot product against v (shared memory),
+// and for col_t_agg the scatter  acc[col] += t * val  into the CTA's shared
+// accumulator.  Two groups may hit the same column at the same time, so the
+// scatter uses shared-memory atomics (their order is not fixed).
+constexpr int kCsrStage = 512;            // stored cells a warp can stage per block of rows
+
 template <int AGG>
 __global__ void __launch_bounds__(kThreads)
 row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
@@ -274,50 +280,98 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
     __shared__ double s_red[32];
     __shared__ unsigned int s_flag;
     const long long n = p.cols;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int l8 = lane & 7, grp = lane >> 3;
+
     double *vs = reinterpret_cast<double *>(smem_raw);
-    double *qs = vs + n;
+    double *qs = vs + n;                                       // col_t_agg only
+    double *sx = vs + (AGG == kRowColT ? 2 : 1) * n + (size_t)warp * kCsrStage;
+    int *sc = reinterpret_cast<int *>(vs + (AGG == kRowColT ? 2 : 1) * n + (size_t)kWarps * kCsrStage)
+              + (size_t)warp * kCsrStage;
     for (long long j = threadIdx.x; j < n; j += kThreads) {
         vs[j] = __ldg(p.v + j);
         if (AGG == kRowColT) qs[j] = 0.0;
     }
     __syncthreads();
 
-    const int lane = threadIdx.x & 31;
-    const int l8 = lane & 7;
-    const unsigned gmask = 0xffu << (lane & 24);
-    const long long group0 = ((long long)blockIdx.x * kThreads + threadIdx.x) >> 3;
-    const long long ngroups = ((long long)gridDim.x * kThreads) >> 3;
+    const long long nblocks = (p.rows + 31) >> 5;
+    const long long warp0 = (long long)blockIdx.x * kWarps + warp;
+    const long long nwarps = (long long)gridDim.x * kWarps;
     double tsum = 0.0;
 
-    // rows are dealt to CTAs in contiguous blocks of (groups per CTA) rows, so a
-    // warp's four groups read neighbouring parts of colidx / vals
-    for (long long row = group0; row < p.rows; row += ngroups) {
-        const int beg = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
+    for (long long blk = warp0; blk < nblocks; blk += nwarps) {
+        const long long myrow = (blk << 5) + lane;
+        const bool have = myrow < p.rows;
+        const int beg_l = have ? __ldg(p.rowptr + myrow) : 0;
+        const int end_l = have ? __ldg(p.rowptr + myrow + 1) : beg_l;
         double sv[FO_MAX_SIDES];
-        load_sides(ch, p.sides, row, p.rows, sv);
-        double d = 0.0;
-        for (int q0 = beg + l8; q0 < end; q0 += 8)
-            d = fma(__ldg(p.vals + q0), vs[__ldg(p.colidx + q0)], d);
-        d += __shfl_xor_sync(gmask, d, 4);
-        d += __shfl_xor_sync(gmask, d, 2);
-        d += __shfl_xor_sync(gmask, d, 1);
-        const double t = row_chain(ch, d, sv);
-        if (AGG == kRowColT) {
-            for (int q0 = beg + l8; q0 < end; q0 += 8)
-                atomicAdd(&qs[__ldg(p.colidx + q0)], t * __ldg(p.vals + q0));
-        } else if (AGG == kRowRow) {
-            if (l8 == 0) p.out[row] = t;
-        } else {
-            if (l8 == 0) tsum += t;
+#pragma unroll
+        for (int k = 0; k < FO_MAX_SIDES; ++k)
+            sv[k] = (have && ((ch.side_used >> k) & 1u))
+                        ? __ldg(p.sides.s[k].data + myrow * p.sides.s[k].ld) : 0.0;
+
+        // stage the block's stored cells (skipped, and read from global memory
+        // below, when the block holds more than the slice can take)
+        const int base = __shfl_sync(0xffffffffu, beg_l, 0);
+        const int last_end = __shfl_sync(0xffffffffu, end_l, (int)((p.rows - (blk << 5) < 32) ? p.rows - (blk << 5) - 1 : 31));
+        const int total = last_end - base;
+        const bool staged = total <= kCsrStage;
+        if (staged) {
+            for (int e = lane; e < total; e += 32) {
+                sc[e] = __ldg(p.colidx + base + e);
+                sx[e] = __ldg(p.vals + base + e);
+            }
         }
+        __syncwarp();
+
+        double dmine = 0.0;
+        for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + grp;
+            const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
+            const int end = __shfl_sync(0xffffffffu, end_l, rr);
+            double d = 0.0;
+            if (staged) {
+                for (int q0 = beg - base + l8; q0 < end - base; q0 += 8) d = fma(sx[q0], vs[sc[q0]], d);
+            } else {
+                for (int q0 = beg + l8; q0 < end; q0 += 8)
+                    d = fma(__ldg(p.vals + q0), vs[__ldg(p.colidx + q0)], d);
+            }
+            d += __shfl_xor_sync(0xffffffffu, d, 4);
+            d += __shfl_xor_sync(0xffffffffu, d, 2);
+            d += __shfl_xor_sync(0xffffffffu, d, 1);
+            // row rr's dot product sits in group (rr & 3); lane rr keeps it
+            const double dall = __shfl_sync(0xffffffffu, d, (lane & 3) * 8);
+            if ((lane >> 2) == it) dmine = dall;
+        }
+        const double t = lane_chain(ch, dmine, sv);
+        if (AGG == kRowRow) {
+            if (have) p.out[myrow] = t;
+        } else if (AGG == kRowFull) {
+            if (have) tsum += t;
+        } else {
+            for (int it = 0; it < 8; ++it) {
+                const int rr = it * 4 + grp;
+                const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
+                const int end = __shfl_sync(0xffffffffu, end_l, rr);
+                const double tt = __shfl_sync(0xffffffffu, t, rr);
+                if (staged) {
+                    for (int q0 = beg - base + l8; q0 < end - base; q0 += 8)
+                        atomicAdd(&qs[sc[q0]], tt * sx[q0]);
+                } else {
+                    for (int q0 = beg + l8; q0 < end; q0 += 8)
+                        atomicAdd(&qs[__ldg(p.colidx + q0)], tt * __ldg(p.vals + q0));
+                }
+            }
+        }
+        __syncwarp();          // the slice is reused by the next block
     }
 
     if (AGG == kRowColT) {
         __syncthreads();
         for (long long j = threadIdx.x; j < n; j += kThreads)
             p.partials[(size_t)blockIdx.x * n + j] = qs[j];
-        if (publish_and_is_last(p.head, &s_flag))
-            final_sum_columns(p.partials, gridDim.x, n, p.out);
+        reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * n, n, p.out,
+                                 &s_flag);
     } else if (AGG == kRowFull) {
         double v1[1] = {tsum};
         block_sum<1>(v1, s_red);
@@ -345,8 +399,8 @@ int row_grid_cap() { return 148 * 4; }     // bound used for workspace sizing
 
 size_t row_ws_bytes(long long cols, int agg)
 {
-    if (agg == FO_ROW_COL_T_AGG)
-        return sizeof(WsHead) + (size_t)row_grid_cap() * (size_t)cols * sizeof(double);
+    if (agg == FO_ROW_COL_T_AGG)      // per-CTA vectors plus one vector per group of CTAs
+        return sizeof(WsHead) + (size_t)(row_grid_cap() + row_grid_cap() / kGroup + 1) * (size_t)cols * sizeof(double);
     if (agg == FO_ROW_FULL_AGG) return sizeof(WsHead) + (size_t)row_grid_cap() * sizeof(double);
     return sizeof(WsHead);
 }
@@ -465,9 +519,10 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     cudaError_t e;
     if (csr) {
         p.rowptr = X->csr.rowptr; p.colidx = X->csr.colidx; p.vals = X->csr.vals;
-        const size_t smem = (size_t)cols * 8 * (agg == FO_ROW_COL_T_AGG ? 2 : 1);
-        long long grid = (rows + (kThreads / 8) - 1) / (kThreads / 8);
-        const long long cap = (long long)sms * 4 < row_grid_cap() ? (long long)sms * 4 : row_grid_cap();
+        const size_t smem = (size_t)cols * 8 * (agg == FO_ROW_COL_T_AGG ? 2 : 1)
+                            + (size_t)kWarps * kCsrStage * 12;
+        long long grid = (rows + kThreads - 1) / kThreads;
+        const long long cap = (long long)sms * 3 < row_grid_cap() ? (long long)sms * 3 : row_grid_cap();
         if (grid > cap) grid = cap;
         auto go = [&](auto kern) -> cudaError_t {
             cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
