@@ -362,6 +362,8 @@ def run_ours(args):
     shapes = scaled(FULL, args.frac) if args.frac != 1.0 else {k: dict(v) for k, v in FULL.items()}
     if args.frac != 1.0:
         shapes["outer"]["cols"] = max(8, int(round(FULL["outer"]["cols"] * args.frac)))
+        if args.full_outer:
+            shapes["outer"] = dict(FULL["outer"])
     t_gen = time.perf_counter()
     host = make_host_inputs(shapes, pinned=True)
     t_gen = time.perf_counter() - t_gen
@@ -515,6 +517,7 @@ def main():
     ap.add_argument("--cpu-frac", type=float, default=0.05, help="sample of the workloads the CPU baseline runs")
     ap.add_argument("--ref-frac", type=float, default=0.01, help="sample per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--full-outer", action="store_true", help="keep the Outer workload at full size under --frac")
     ap.add_argument("--ops", default="", help="comma-separated subset of the five operators (profiling)")
     ap.add_argument("--interp", action="store_true", help="run Cell / MAgg chains through the interpreter")
     args = ap.parse_args()

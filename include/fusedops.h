@@ -215,9 +215,8 @@ int fused_magg(const fo_chain *chain, const fo_mat *X,
  *   FO_ROW_ROW_AGG  : out[i] = t_i                                   (rows doubles)
  *   FO_ROW_FULL_AGG : out[0] = sum_i t_i
  * With the chain  t = side0 * d  this is  t(X) %*% (w * (X %*% v)).
- * Dense X wider than 8192 columns, or CSR X wider than 16384 columns, returns
- * FO_ERR_UNSUPPORTED for FO_ROW_COL_T_AGG (the single-pass kernels keep one
- * row, respectively the output vector, on chip).
+ * X wider than 8192 columns returns FO_ERR_UNSUPPORTED (the single-pass
+ * kernels keep a row, respectively v and the output vector, on chip).
  * Determinism: bit-reproducible except FO_ROW_COL_T_AGG over CSR, whose
  * scatter-add into on-chip accumulators is unordered.
  */

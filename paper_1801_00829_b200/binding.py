@@ -308,7 +308,7 @@ def force_interpreter(on):
 def device_status(device=None):
     """Synchronises and returns the workspace's device-side status (0 = ok)."""
     device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
-    buf = workspace(device, 256)
+    buf = workspace(device, 16384)
     st = C.c_int(0)
     _check(load_library().fo_query_device_status(C.c_void_p(buf.data_ptr()), _stream(device),
                                                  C.byref(st)), "fo_query_device_status")
@@ -330,7 +330,7 @@ def fused_cell(steps, output, X, sides=(), scalars=(), agg="full", out=None):
                  "none": (X.nnz,) if isinstance(X, CSR) else (rows, cols)}[agg]
         out = torch.empty(shape, dtype=torch.float64, device=dev)
     need = lib.fused_cell_workspace_bytes(C.byref(m), a)
-    ws = workspace(dev, max(need, 256))
+    ws = workspace(dev, max(need, 16384))
     sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
     _check(lib.fused_cell(C.byref(ch), C.byref(m), sarr, len(sides), sc, len(scalars), a,
                           C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
@@ -350,7 +350,7 @@ def fused_magg(steps, outputs, X, sides=(), scalars=(), out=None):
     if out is None:
         out = torch.empty(len(outputs), dtype=torch.float64, device=dev)
     need = lib.fused_magg_workspace_bytes(C.byref(m), len(outputs))
-    ws = workspace(dev, max(need, 256))
+    ws = workspace(dev, max(need, 16384))
     sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
     _check(lib.fused_magg(C.byref(ch), C.byref(m), sarr, len(sides), sc, len(scalars),
                           C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
@@ -372,7 +372,7 @@ def fused_row(steps, output, X, v, sides=(), scalars=(), agg="col_t", out=None):
         shape = {"col_t": (cols,), "row": (rows,), "full": (1,)}.get(agg, (1,))
         out = torch.empty(shape, dtype=torch.float64, device=dev)
     need = lib.fused_row_workspace_bytes(C.byref(m), a)
-    ws = workspace(dev, max(need, 256))
+    ws = workspace(dev, max(need, 16384))
     sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
     _check(lib.fused_row(C.byref(ch), C.byref(m), C.c_void_p(v.data_ptr()), sarr, len(sides), sc,
                          len(scalars), a, C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()),
@@ -393,7 +393,7 @@ def fused_outer(steps, output, X, U, V, scalars=(), agg="full", out=None):
         shape = {"full": (1,), "none": (X.nnz,), "right": (X.rows, rank), "left": (X.cols, rank)}[agg]
         out = torch.empty(shape, dtype=torch.float64, device=dev)
     need = lib.fused_outer_workspace_bytes(C.byref(xs), rank, a)
-    ws = workspace(dev, max(need, 256))
+    ws = workspace(dev, max(need, 16384))
     sc = _scalars(scalars)
     _check(lib.fused_outer(C.byref(ch), C.byref(xs), C.byref(us), C.byref(vs), sc, len(scalars), a,
                            C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),

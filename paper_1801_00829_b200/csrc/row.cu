@@ -106,34 +106,46 @@ __device__ __forceinline__ double lane_chain(const DevChain &ch, double d, const
 }
 
 // ------------------------------------------------------------------ dense
-// NCH: 64-column chunks per row held by a warp (cols <= 64 * NCH).
+// 512 threads.  TEAM warps share a row: warp h of a team holds the 64-column
+// chunks c * TEAM + h (c < NCH) of the row and of the output accumulator in
+// registers, so cols <= 64 * NCH * TEAM; v sits in shared memory.  Per row a
+// warp forms its part of X_i . v, the team adds the parts in a fixed order
+// through shared memory (one named barrier per row), every warp evaluates the
+// chain, and each adds t * X_i into its accumulator columns.
 // STAGED: rows arrive through the shared-memory ring; otherwise lanes load
 // their pairs straight from global memory (any alignment, any cols).
-template <int NCH, int AGG, bool STAGED>
-__global__ void __launch_bounds__(kThreads, 1)
+constexpr int kDenseThreads = 512;
+constexpr int kDenseWarps = kDenseThreads / 32;
+
+template <int NCH, int TEAM, int AGG, bool STAGED>
+__global__ void __launch_bounds__(kDenseThreads, 1)
 row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ unsigned long long s_full[8];
+    __shared__ double s_part[2 * kDenseWarps];
     __shared__ double s_red[32];
     __shared__ unsigned int s_flag;
 
+    constexpr int TEAMS = kDenseWarps / TEAM;       // rows in flight per CTA
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long n = p.cols;
+    const int team = warp / TEAM, h = warp % TEAM;
+    const int n = (int)p.cols;
     const int RPS = p.rows_per_stage, S = p.stages;
-    const int RPW = RPS / kWarps;
+    const int RPT = RPS / TEAMS;                    // rows per team and stage (<= 4)
     double *ring = reinterpret_cast<double *>(smem_raw);
     const long long ntiles = (p.rows + RPS - 1) / RPS;
     const long long my_tiles = (ntiles > blockIdx.x) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
-    // v lives in shared memory behind the ring, padded with zeros to 64 * NCH
-    double *vs = ring + (size_t)(STAGED ? S : 0) * RPS * n + (AGG == kRowColT && !STAGED ? kWarps * n : 0);
-    for (int j = threadIdx.x; j < 64 * NCH; j += kThreads) vs[j] = j < n ? __ldg(p.v + j) : 0.0;
+    // v lives in shared memory behind the ring, padded with zeros to 64 * NCH * TEAM
+    double *vs = ring + (size_t)(STAGED ? S : 0) * RPS * n + (AGG == kRowColT && !STAGED ? TEAMS * n : 0);
+    for (int j = threadIdx.x; j < 64 * NCH * TEAM; j += kDenseThreads) vs[j] = j < n ? __ldg(p.v + j) : 0.0;
     double2 q[NCH];
 #pragma unroll
     for (int c = 0; c < NCH; ++c) q[c] = make_double2(0.0, 0.0);
     double tsum = 0.0;
     bool timed_out = false;
+    unsigned parity = 0;
 
     auto issue = [&](long long it) {
         const long long tile = blockIdx.x + it * gridDim.x;
@@ -149,6 +161,14 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
                 bulk_g2s(dst + (size_t)r * n, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &s_full[slot]);
         }
     };
+    // side values of this team's rows in a tile: lane 1 + k holds side k
+    auto load_tile_sides = [&](long long it, double (&sv)[4]) {
+        const long long r0 = (blockIdx.x + it * gridDim.x) * RPS;
+#pragma unroll
+        for (int rt = 0; rt < 4; ++rt)
+            sv[rt] = (rt < RPT && it < my_tiles)
+                         ? load_sides_lanes(ch, p.sides, r0 + team * RPT + rt, p.rows, lane) : 0.0;
+    };
 
     __syncthreads();
     if (STAGED) {
@@ -162,6 +182,8 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
             for (long long it = 0; it < S - 1 && it < my_tiles; ++it) issue(it);
     }
 
+    double sv_next[4];
+    load_tile_sides(0, sv_next);
     for (long long it = 0; it < my_tiles; ++it) {
         const long long tile = blockIdx.x + it * gridDim.x;
         const long long r0 = tile * RPS;
@@ -169,26 +191,24 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
         if (STAGED) {
             if (threadIdx.x == 0 && it + S - 1 < my_tiles) issue(it + S - 1);
         }
-        // side values of this warp's rows (lane 1 + k holds side k): requested
-        // before the wait so their latency overlaps it
         double sv[4];
 #pragma unroll
-        for (int rw = 0; rw < 4; ++rw)
-            sv[rw] = rw < RPW ? load_sides_lanes(ch, p.sides, r0 + warp * RPW + rw, p.rows, lane) : 0.0;
+        for (int rt = 0; rt < 4; ++rt) sv[rt] = sv_next[rt];
+        load_tile_sides(it + 1, sv_next);       // one tile ahead: hidden behind this tile's work
         if (STAGED) {
             if (!mbar_wait(&s_full[slot], (unsigned)((it / S) & 1))) timed_out = true;
         }
-        for (int rw = 0; rw < RPW; ++rw) {
-            const int rl = warp * RPW + rw;
+        for (int rt = 0; rt < RPT; ++rt) {
+            const int rl = team * RPT + rt;
             const long long row = r0 + rl;
+            // all warps of a team see the same row, so they leave together
             if (row >= p.rows) break;
             double2 x[NCH];
-            double d0 = 0.0, d1 = 0.0;
             if (STAGED) {
                 const double *rowp = ring + ((size_t)slot * RPS + rl) * n;
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
-                    const long long col = 64 * c + 2 * lane;
+                    const int col = 64 * (c * TEAM + h) + 2 * lane;
                     x[c] = (col < n) ? *reinterpret_cast<const double2 *>(rowp + col)
                                      : make_double2(0.0, 0.0);
                 }
@@ -196,22 +216,32 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
                 const double *rowp = p.X + row * p.ldx;
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
-                    const long long col = 64 * c + 2 * lane;
+                    const int col = 64 * (c * TEAM + h) + 2 * lane;
                     x[c].x = col < n ? ld_stream1(rowp + col) : 0.0;
                     x[c].y = col + 1 < n ? ld_stream1(rowp + col + 1) : 0.0;
                 }
             }
+            double d0 = 0.0, d1 = 0.0;
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-                const double2 vv = *reinterpret_cast<const double2 *>(vs + 64 * c + 2 * lane);
+                const double2 vv = *reinterpret_cast<const double2 *>(vs + 64 * (c * TEAM + h) + 2 * lane);
                 d0 = fma(x[c].x, vv.x, d0);
                 d1 = fma(x[c].y, vv.y, d1);
             }
-            const double d = warp_sum(d0 + d1);
+            double d = warp_sum(d0 + d1);
+            if (TEAM > 1) {
+                double *part = s_part + parity * kDenseWarps + team * TEAM;
+                if (lane == 0) part[h] = d;
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(TEAM * 32) : "memory");
+                d = 0.0;
+#pragma unroll
+                for (int k = 0; k < TEAM; ++k) d += part[k];
+                parity ^= 1u;
+            }
             double mine = sv[0];
 #pragma unroll
             for (int r2 = 1; r2 < 4; ++r2)
-                if (rw == r2) mine = sv[r2];
+                if (rt == r2) mine = sv[r2];
             if (lane == 0) mine = d;
             const double t = warp_chain(ch, mine, lane);
             if (AGG == kRowColT) {
@@ -221,9 +251,9 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
                     q[c].y = fma(t, x[c].y, q[c].y);
                 }
             } else if (AGG == kRowRow) {
-                if (lane == 0) p.out[row] = t;
+                if (lane == 0 && h == 0) p.out[row] = t;
             } else {
-                tsum += t;
+                if (h == 0) tsum += t;
             }
         }
         if (STAGED) __syncthreads();      // the slot may be refilled from now on
@@ -232,27 +262,26 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
     if (STAGED && timed_out) atomicExch(&p.head->status, 1u);
 
     if (AGG == kRowColT) {
-        // warps -> CTA: fixed order over warps, through shared memory
+        // teams -> CTA: fixed order over teams, through shared memory
         __syncthreads();
-        double *qs = ring;                // kWarps * n doubles fit in one ring stage
-        if (!STAGED) qs = reinterpret_cast<double *>(smem_raw);
+        double *qs = reinterpret_cast<double *>(smem_raw);      // TEAMS * n doubles fit in one ring stage
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
-            const long long col = 64 * c + 2 * lane;
-            if (col < n) qs[(size_t)warp * n + col] = q[c].x;
-            if (col + 1 < n) qs[(size_t)warp * n + col + 1] = q[c].y;
+            const int col = 64 * (c * TEAM + h) + 2 * lane;
+            if (col < n) qs[(size_t)team * n + col] = q[c].x;
+            if (col + 1 < n) qs[(size_t)team * n + col + 1] = q[c].y;
         }
         __syncthreads();
-        for (long long j = threadIdx.x; j < n; j += kThreads) {
+        for (int j = threadIdx.x; j < n; j += kDenseThreads) {
             double s = 0.0;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) s += qs[(size_t)w * n + j];
+            for (int w = 0; w < TEAMS; ++w) s += qs[(size_t)w * n + j];
             p.partials[(size_t)blockIdx.x * n + j] = s;
         }
         reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * n, n, p.out,
                                  &s_flag);
     } else if (AGG == kRowFull) {
-        // every lane of a warp holds the same tsum: count it once per warp
+        // every lane of a warp holds the same tsum: count it once per team
         double v1[1] = {lane == 0 ? tsum : 0.0};
         block_sum<1>(v1, s_red);
         if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
@@ -389,9 +418,9 @@ __global__ void row_fill_zero_kernel(double *out, long long n)
 }
 
 // ------------------------------------------------------------------- host
-constexpr long long kDenseMaxCols = 1024;
+constexpr long long kDenseMaxCols = 8192;
 constexpr long long kCsrMaxCols = 8192;
-constexpr size_t kRingBudget = 208 * 1024;
+constexpr size_t kSmemBudget = 208 * 1024;   // dynamic shared memory of the dense kernel
 
 bool aligned16(const void *q) { return ((uintptr_t)q & 15u) == 0; }
 
@@ -405,19 +434,28 @@ size_t row_ws_bytes(long long cols, int agg)
     return sizeof(WsHead);
 }
 
-template <int NCH, bool STAGED>
+template <int NCH, int TEAM, bool STAGED>
 cudaError_t launch_dense_agg(const DevChain &ch, const RowParams &p, int agg, int grid, size_t smem,
                              cudaStream_t st)
 {
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kern<<<grid, kThreads, smem, st>>>(ch, p);
+        kern<<<grid, kDenseThreads, smem, st>>>(ch, p);
         return cudaGetLastError();
     };
-    if (agg == FO_ROW_COL_T_AGG) return go(row_dense_kernel<NCH, kRowColT, STAGED>);
-    if (agg == FO_ROW_ROW_AGG) return go(row_dense_kernel<NCH, kRowRow, STAGED>);
-    return go(row_dense_kernel<NCH, kRowFull, STAGED>);
+    if (agg == FO_ROW_COL_T_AGG) return go(row_dense_kernel<NCH, TEAM, kRowColT, STAGED>);
+    if (agg == FO_ROW_ROW_AGG) return go(row_dense_kernel<NCH, TEAM, kRowRow, STAGED>);
+    return go(row_dense_kernel<NCH, TEAM, kRowFull, STAGED>);
+}
+
+// Team size and chunks per warp for a row of n columns: at most 8 chunks (16
+// registers of row data and 16 of accumulator) per lane.
+int dense_team(long long n)
+{
+    int team = 1;
+    while ((long long)64 * 8 * team < n) team *= 2;
+    return team;
 }
 
 template <bool STAGED>
@@ -425,11 +463,17 @@ cudaError_t launch_dense(const DevChain &ch, const RowParams &p, int agg, int gr
                          cudaStream_t st)
 {
     const long long n = p.cols;
-    if (n <= 64) return launch_dense_agg<1, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 128) return launch_dense_agg<2, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 256) return launch_dense_agg<4, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 512) return launch_dense_agg<8, STAGED>(ch, p, agg, grid, smem, st);
-    return launch_dense_agg<16, STAGED>(ch, p, agg, grid, smem, st);
+    switch (dense_team(n)) {
+        case 1:
+            if (n <= 64) return launch_dense_agg<1, 1, STAGED>(ch, p, agg, grid, smem, st);
+            if (n <= 128) return launch_dense_agg<2, 1, STAGED>(ch, p, agg, grid, smem, st);
+            if (n <= 256) return launch_dense_agg<4, 1, STAGED>(ch, p, agg, grid, smem, st);
+            return launch_dense_agg<8, 1, STAGED>(ch, p, agg, grid, smem, st);
+        case 2: return launch_dense_agg<8, 2, STAGED>(ch, p, agg, grid, smem, st);
+        case 4: return launch_dense_agg<8, 4, STAGED>(ch, p, agg, grid, smem, st);
+        case 8: return launch_dense_agg<8, 8, STAGED>(ch, p, agg, grid, smem, st);
+        default: return launch_dense_agg<8, 16, STAGED>(ch, p, agg, grid, smem, st);
+    }
 }
 
 }  // namespace
@@ -536,19 +580,21 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     } else {
         p.X = X->dense.data; p.ldx = X->dense.ld;
         const bool staged = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
-        // ring geometry: stages of about 64 KB, whole rows, a multiple of kWarps rows
-        int rpw = (int)((64 * 1024) / (cols * 8 * kWarps));
-        if (rpw < 1) rpw = 1;
-        if (rpw > 4) rpw = 4;
-        p.rows_per_stage = rpw * kWarps;
+        // ring geometry: stages of about 64 KB, whole rows, one to four rows per team
+        const int teams = kDenseWarps / dense_team(cols);
+        int rpt = (int)((64 * 1024) / (cols * 8 * teams));
+        if (rpt < 1) rpt = 1;
+        if (rpt > 4) rpt = 4;
+        p.rows_per_stage = rpt * teams;
         const size_t stage_bytes = (size_t)p.rows_per_stage * cols * 8;
-        int stages = (int)(kRingBudget / stage_bytes);
+        const size_t v_bytes = (size_t)64 * 8 * dense_team(cols) * 8;      // v, zero-padded
+        int stages = (int)((kSmemBudget - v_bytes) / stage_bytes);
         if (stages > 4) stages = 4;
         if (stages < 2) stages = 2;
         p.stages = staged ? stages : 1;
         size_t smem = staged ? stage_bytes * stages : 0;       // the ring
-        if (!staged && agg == FO_ROW_COL_T_AGG) smem = (size_t)kWarps * cols * 8;   // warp partials
-        smem += 1024 * 8;                                      // v, zero-padded
+        if (!staged && agg == FO_ROW_COL_T_AGG) smem = (size_t)teams * cols * 8;   // team partials
+        smem += v_bytes;
         const long long ntiles = (rows + p.rows_per_stage - 1) / p.rows_per_stage;
         long long grid = ntiles < sms ? ntiles : sms;
         if (grid > row_grid_cap()) grid = row_grid_cap();

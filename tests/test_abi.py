@@ -49,22 +49,25 @@ def dense_mat(rows, cols, ld=None, ptr=0x1000):
     return m
 
 
+HEAD = 16384        # control words at the head of every workspace
+
+
 def test_workspace_sizes(lib):
     m = dense_mat(1000, 1000)
     full = lib.fused_cell_workspace_bytes(C.byref(m), 3)
-    assert full >= 256 + 8 and full % 8 == 0
-    assert lib.fused_cell_workspace_bytes(C.byref(m), 1) == 256            # row_agg: control words only
+    assert full >= HEAD + 8 and full % 8 == 0
+    assert lib.fused_cell_workspace_bytes(C.byref(m), 1) == HEAD           # row_agg: control words only
     col = lib.fused_cell_workspace_bytes(C.byref(m), 2)
-    assert col >= 256 + 1000 * 8 and (col - 256) % (1000 * 8) == 0
+    assert col >= HEAD + 1000 * 8 and (col - HEAD) % (1000 * 8) == 0
     assert lib.fused_cell_workspace_bytes(C.byref(m), 9) == 0
-    assert lib.fused_magg_workspace_bytes(C.byref(m), 3) == 256 + (full - 256) * 3
+    assert lib.fused_magg_workspace_bytes(C.byref(m), 3) == HEAD + (full - HEAD) * 3
     assert lib.fused_magg_workspace_bytes(C.byref(m), 9) == 0
     r = lib.fused_row_workspace_bytes(C.byref(m), 4)
-    assert r >= 256 + 148 * 1000 * 8
+    assert r >= HEAD + 148 * 1000 * 8
     assert lib.fused_row_workspace_bytes(C.byref(m), 0) == 0
     x = B.fo_csr()
     x.rows, x.cols, x.nnz = 10, 10, 5
-    assert lib.fused_outer_workspace_bytes(C.byref(x), 100, 3) >= 256 + 8
+    assert lib.fused_outer_workspace_bytes(C.byref(x), 100, 3) >= HEAD + 8
     assert lib.fused_outer_workspace_bytes(C.byref(x), 257, 3) == 0
 
 
@@ -122,7 +125,7 @@ def test_chain_limits(lib):
 
 def test_row_and_outer_argument_errors(lib):
     ch, keep = B.make_chain([("mul", "t0", "side0", "d")], "t0")
-    m = dense_mat(10, 2000)
+    m = dense_mat(10, 10000)
     sarr = (B.fo_side * 1)(side(10, 1, 1))
     sc = (C.c_double * 8)()
 

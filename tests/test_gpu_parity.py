@@ -192,7 +192,8 @@ def row_abs_scale(X, v, w):
 
 
 @pytest.mark.parametrize("rows,cols", [(2000, 1000), (501, 64), (37, 10), (100, 1024), (9, 2),
-                                       (1, 128), (300, 257), (64, 999), (5, 1)])
+                                       (1, 128), (300, 257), (64, 999), (5, 1), (333, 512), (200, 1026),
+                                       (77, 2048), (50, 3000), (21, 4100), (19, 8192), (18, 8191)])
 def test_row_dense_col_t(fo, rows, cols):
     w = datagen.row_dense_workload(rows, cols, seed=2)
     ref = oracle.row_chain_dense(w["X"], w["v"], w["w"])
