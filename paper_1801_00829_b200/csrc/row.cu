@@ -138,7 +138,9 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
     const long long my_tiles = (ntiles > blockIdx.x) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
     // v lives in shared memory behind the ring, padded with zeros to 64 * NCH * TEAM
-    double *vs = ring + (size_t)(STAGED ? S : 0) * RPS * n + (AGG == kRowColT && !STAGED ? TEAMS * n : 0);
+    // (the offset is kept even so that 128-bit reads of v stay aligned when cols is odd)
+    double *vs = ring + (size_t)(STAGED ? S : 0) * RPS * n
+                 + (AGG == kRowColT && !STAGED ? ((TEAMS * n + 1) & ~1) : 0);
     for (int j = threadIdx.x; j < 64 * NCH * TEAM; j += kDenseThreads) vs[j] = j < n ? __ldg(p.v + j) : 0.0;
     double2 q[NCH];
 #pragma unroll
@@ -593,7 +595,7 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
         if (stages < 2) stages = 2;
         p.stages = staged ? stages : 1;
         size_t smem = staged ? stage_bytes * stages : 0;       // the ring
-        if (!staged && agg == FO_ROW_COL_T_AGG) smem = (size_t)teams * cols * 8;   // team partials
+        if (!staged && agg == FO_ROW_COL_T_AGG) smem = (((size_t)teams * cols + 1) & ~(size_t)1) * 8;   // team partials
         smem += v_bytes;
         const long long ntiles = (rows + p.rows_per_stage - 1) / p.rows_per_stage;
         long long grid = ntiles < sms ? ntiles : sms;
