@@ -5,9 +5,9 @@
 // from on-chip memory - the GPU form of the paper's "each row fits L1" argument.
 //
 // Dense X: a CTA streams tiles of rows into a shared-memory ring with bulk
-// asynchronous copies (mbarrier-tracked, waits bounded); each warp owns one
-// row at a time: lanes hold the row, their slice of v and of the output
-// accumulator in registers.  CSR X: an 8-lane group per row; v and the output
+// asynchronous copies (mbarrier-tracked, waits bounded); warps own column slices
+// of the rows, of v and of the output accumulator, all in registers.  CSR X: a
+// warp per block of 32 rows, an 8-lane group per row; v and the output
 // accumulator live in shared memory.
 #include "chain.cuh"
 
@@ -79,19 +79,6 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
         : "memory");
 }
 
-// Side values of one row, spread over the lanes the way warp_chain wants its
-// register file: lane 1 + k holds side k (lane 0 is reserved for d).
-__device__ __forceinline__ double load_sides_lanes(const DevChain &ch, const DevSides &sides,
-                                                   long long row, long long rows, int lane)
-{
-    double v = 0.0;
-#pragma unroll
-    for (int k = 0; k < FO_MAX_SIDES; ++k)
-        if (lane == 1 + k && ((ch.side_used >> k) & 1u) && row < rows)
-            v = __ldg(sides.s[k].data + row * sides.s[k].ld);
-    return v;
-}
-
 // The chain for one row per lane: R0 = d, R(1+k) = side k of that lane's row.
 __device__ __forceinline__ double lane_chain(const DevChain &ch, double d, const double (&sv)[FO_MAX_SIDES])
 {
@@ -106,48 +93,81 @@ __device__ __forceinline__ double lane_chain(const DevChain &ch, double d, const
 }
 
 // ------------------------------------------------------------------ dense
-// 512 threads.  TEAM warps share a row: warp h of a team holds the 64-column
-// chunks c * TEAM + h (c < NCH) of the row and of the output accumulator in
-// registers, so cols <= 64 * NCH * TEAM; v sits in shared memory.  Per row a
-// warp forms its part of X_i . v, the team adds the parts in a fixed order
-// through shared memory (one named barrier per row), every warp evaluates the
-// chain, and each adds t * X_i into its accumulator columns.
+// 512 threads = 16 warps.  W warps form a group that works on R rows at a time;
+// warp w of a group owns the 64-column chunks c * W + w (c < NCH) of those rows,
+// of v and of the output accumulator - all in registers - so cols <= 64*NCH*W.
+// Per stage of the ring: every warp reads its pieces of the R rows, forms R
+// partial dot products, reduces them over its lanes (R values in one butterfly)
+// and leaves them in shared memory; after ONE CTA barrier - at which point the
+// ring slot is free again, the rows being held in registers - lane r of every
+// warp adds the W partials of row r in a fixed order, evaluates the chain for
+// that row, and the warp adds t_r * X_r into its accumulator columns.
 // STAGED: rows arrive through the shared-memory ring; otherwise lanes load
 // their pairs straight from global memory (any alignment, any cols).
 constexpr int kDenseThreads = 512;
 constexpr int kDenseWarps = kDenseThreads / 32;
 
-template <int NCH, int TEAM, int AGG, bool STAGED>
+// Sums R values per lane over the 32 lanes of a warp in a fixed order.  On
+// return v[0] holds, in every lane l, the total of value number (l >> (5 - log2 R)).
+template <int R>
+__device__ __forceinline__ void warp_sum_multi(double (&v)[R], int lane)
+{
+    int mask = 16;
+#pragma unroll
+    for (int half = R / 2; half >= 1; half /= 2) {
+        const bool up = (lane & mask) != 0;
+#pragma unroll
+        for (int i = 0; i < half; ++i) {
+            const double send = up ? v[i] : v[i + half];
+            const double keep = up ? v[i + half] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
+        }
+        mask >>= 1;
+    }
+    for (; mask >= 1; mask >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], mask);
+}
+
+template <int R>
+struct Log2 {
+    static constexpr int value = 1 + Log2<R / 2>::value;
+};
+template <>
+struct Log2<1> {
+    static constexpr int value = 0;
+};
+
+template <int NCH, int W, int R, int AGG, bool STAGED>
 __global__ void __launch_bounds__(kDenseThreads, 1)
 row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ unsigned long long s_full[8];
-    __shared__ double s_part[2 * kDenseWarps];
+    __shared__ double s_part[2][kDenseWarps][8];     // [parity][warp][row of the group]
     __shared__ double s_red[32];
     __shared__ unsigned int s_flag;
 
-    constexpr int TEAMS = kDenseWarps / TEAM;       // rows in flight per CTA
+    constexpr int GROUPS = kDenseWarps / W;
+    constexpr int RPS = GROUPS * R;                  // rows per stage
+    constexpr int SH = 5 - Log2<R>::value;           // lane l holds row (l >> SH) after the butterfly
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int team = warp / TEAM, h = warp % TEAM;
+    const int grp = warp / W, w = warp % W;
     const int n = (int)p.cols;
-    const int RPS = p.rows_per_stage, S = p.stages;
-    const int RPT = RPS / TEAMS;                    // rows per team and stage (<= 4)
+    const int S = p.stages;
     double *ring = reinterpret_cast<double *>(smem_raw);
     const long long ntiles = (p.rows + RPS - 1) / RPS;
     const long long my_tiles = (ntiles > blockIdx.x) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
-    // v lives in shared memory behind the ring, padded with zeros to 64 * NCH * TEAM
-    // (the offset is kept even so that 128-bit reads of v stay aligned when cols is odd)
-    double *vs = ring + (size_t)(STAGED ? S : 0) * RPS * n
-                 + (AGG == kRowColT && !STAGED ? ((TEAMS * n + 1) & ~1) : 0);
-    for (int j = threadIdx.x; j < 64 * NCH * TEAM; j += kDenseThreads) vs[j] = j < n ? __ldg(p.v + j) : 0.0;
-    double2 q[NCH];
+    // this lane's columns: pair (col, col + 1) of chunk c
+    double2 vreg[NCH], q[NCH];
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) q[c] = make_double2(0.0, 0.0);
+    for (int c = 0; c < NCH; ++c) {
+        const int col = 64 * (c * W + w) + 2 * lane;
+        vreg[c].x = col < n ? __ldg(p.v + col) : 0.0;
+        vreg[c].y = col + 1 < n ? __ldg(p.v + col + 1) : 0.0;
+        q[c] = make_double2(0.0, 0.0);
+    }
     double tsum = 0.0;
     bool timed_out = false;
-    unsigned parity = 0;
 
     auto issue = [&](long long it) {
         const long long tile = blockIdx.x + it * gridDim.x;
@@ -163,16 +183,15 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
                 bulk_g2s(dst + (size_t)r * n, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &s_full[slot]);
         }
     };
-    // side values of this team's rows in a tile: lane 1 + k holds side k
-    auto load_tile_sides = [&](long long it, double (&sv)[4]) {
-        const long long r0 = (blockIdx.x + it * gridDim.x) * RPS;
+    // side values of the row this lane evaluates the chain for (lanes 0..R-1)
+    auto load_tile_sides = [&](long long it, double (&sv)[FO_MAX_SIDES]) {
+        const long long row = (blockIdx.x + it * gridDim.x) * RPS + grp * R + lane;
 #pragma unroll
-        for (int rt = 0; rt < 4; ++rt)
-            sv[rt] = (rt < RPT && it < my_tiles)
-                         ? load_sides_lanes(ch, p.sides, r0 + team * RPT + rt, p.rows, lane) : 0.0;
+        for (int k = 0; k < FO_MAX_SIDES; ++k)
+            sv[k] = (lane < R && it < my_tiles && row < p.rows && ((ch.side_used >> k) & 1u))
+                        ? __ldg(p.sides.s[k].data + row * p.sides.s[k].ld) : 0.0;
     };
 
-    __syncthreads();
     if (STAGED) {
         if (threadIdx.x == 0) {
             for (int s = 0; s < S; ++s) mbar_init(&s_full[s], 1);
@@ -181,110 +200,103 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
         }
         __syncthreads();
         if (threadIdx.x == 0)
-            for (long long it = 0; it < S - 1 && it < my_tiles; ++it) issue(it);
+            for (long long it = 0; it < S && it < my_tiles; ++it) issue(it);
     }
 
-    double sv_next[4];
+    double sv_next[FO_MAX_SIDES];
     load_tile_sides(0, sv_next);
     for (long long it = 0; it < my_tiles; ++it) {
-        const long long tile = blockIdx.x + it * gridDim.x;
-        const long long r0 = tile * RPS;
+        const long long r0 = (blockIdx.x + it * gridDim.x) * RPS;
         const int slot = (int)(it % S);
-        if (STAGED) {
-            if (threadIdx.x == 0 && it + S - 1 < my_tiles) issue(it + S - 1);
-        }
-        double sv[4];
+        const int par = (int)(it & 1);
+        double sv[FO_MAX_SIDES];
 #pragma unroll
-        for (int rt = 0; rt < 4; ++rt) sv[rt] = sv_next[rt];
+        for (int k = 0; k < FO_MAX_SIDES; ++k) sv[k] = sv_next[k];
         load_tile_sides(it + 1, sv_next);       // one tile ahead: hidden behind this tile's work
         if (STAGED) {
             if (!mbar_wait(&s_full[slot], (unsigned)((it / S) & 1))) timed_out = true;
         }
-        for (int rt = 0; rt < RPT; ++rt) {
-            const int rl = team * RPT + rt;
-            const long long row = r0 + rl;
-            // all warps of a team see the same row, so they leave together
-            if (row >= p.rows) break;
-            double2 x[NCH];
-            if (STAGED) {
-                const double *rowp = ring + ((size_t)slot * RPS + rl) * n;
+        // rows of this group into registers, partial dot products
+        double2 x[R][NCH];
+        double part[R];
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int col = 64 * (c * TEAM + h) + 2 * lane;
-                    x[c] = (col < n) ? *reinterpret_cast<const double2 *>(rowp + col)
-                                     : make_double2(0.0, 0.0);
-                }
-            } else {
-                const double *rowp = p.X + row * p.ldx;
-#pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    const int col = 64 * (c * TEAM + h) + 2 * lane;
-                    x[c].x = col < n ? ld_stream1(rowp + col) : 0.0;
-                    x[c].y = col + 1 < n ? ld_stream1(rowp + col + 1) : 0.0;
-                }
-            }
+        for (int r = 0; r < R; ++r) {
+            const int rl = grp * R + r;
+            const bool have = r0 + rl < p.rows;
             double d0 = 0.0, d1 = 0.0;
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
-                const double2 vv = *reinterpret_cast<const double2 *>(vs + 64 * (c * TEAM + h) + 2 * lane);
-                d0 = fma(x[c].x, vv.x, d0);
-                d1 = fma(x[c].y, vv.y, d1);
+                const int col = 64 * (c * W + w) + 2 * lane;
+                if (STAGED) {
+                    const double *rowp = ring + ((size_t)slot * RPS + rl) * n;
+                    x[r][c] = (have && col < n) ? *reinterpret_cast<const double2 *>(rowp + col)
+                                                : make_double2(0.0, 0.0);
+                } else {
+                    const double *rowp = p.X + (r0 + rl) * p.ldx;
+                    x[r][c].x = (have && col < n) ? ld_stream1(rowp + col) : 0.0;
+                    x[r][c].y = (have && col + 1 < n) ? ld_stream1(rowp + col + 1) : 0.0;
+                }
+                d0 = fma(x[r][c].x, vreg[c].x, d0);
+                d1 = fma(x[r][c].y, vreg[c].y, d1);
             }
-            double d = warp_sum(d0 + d1);
-            if (TEAM > 1) {
-                double *part = s_part + parity * kDenseWarps + team * TEAM;
-                if (lane == 0) part[h] = d;
-                asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(TEAM * 32) : "memory");
-                d = 0.0;
+            part[r] = d0 + d1;
+        }
+        warp_sum_multi<R>(part, lane);
+        if ((lane & ((1 << SH) - 1)) == 0) s_part[par][warp][lane >> SH] = part[0];
+        __syncthreads();
+        // every thread holds its pieces in registers: the slot can be refilled
+        if (STAGED) {
+            if (threadIdx.x == 0 && it + S < my_tiles) issue(it + S);
+        }
+        // lane r: dot product of row r (warps of the group in order), then the chain
+        double d = 0.0;
+        if (lane < R) {
 #pragma unroll
-                for (int k = 0; k < TEAM; ++k) d += part[k];
-                parity ^= 1u;
-            }
-            double mine = sv[0];
+            for (int k = 0; k < W; ++k) d += s_part[par][grp * W + k][lane];
+        }
+        const double t = lane_chain(ch, d, sv);
+        if (AGG == kRowColT) {
 #pragma unroll
-            for (int r2 = 1; r2 < 4; ++r2)
-                if (rt == r2) mine = sv[r2];
-            if (lane == 0) mine = d;
-            const double t = warp_chain(ch, mine, lane);
-            if (AGG == kRowColT) {
+            for (int r = 0; r < R; ++r) {
+                const double tr = __shfl_sync(0xffffffffu, t, r);
 #pragma unroll
                 for (int c = 0; c < NCH; ++c) {
-                    q[c].x = fma(t, x[c].x, q[c].x);
-                    q[c].y = fma(t, x[c].y, q[c].y);
+                    q[c].x = fma(tr, x[r][c].x, q[c].x);
+                    q[c].y = fma(tr, x[r][c].y, q[c].y);
                 }
-            } else if (AGG == kRowRow) {
-                if (lane == 0 && h == 0) p.out[row] = t;
-            } else {
-                if (h == 0) tsum += t;
+            }
+        } else {
+            const long long row = r0 + grp * R + lane;
+            if (w == 0 && lane < R && row < p.rows) {
+                if (AGG == kRowRow) p.out[row] = t;
+                else tsum += t;
             }
         }
-        if (STAGED) __syncthreads();      // the slot may be refilled from now on
     }
 
     if (STAGED && timed_out) atomicExch(&p.head->status, 1u);
 
     if (AGG == kRowColT) {
-        // teams -> CTA: fixed order over teams, through shared memory
+        // groups -> CTA: fixed order over groups, through shared memory
         __syncthreads();
-        double *qs = reinterpret_cast<double *>(smem_raw);      // TEAMS * n doubles fit in one ring stage
+        double *qs = reinterpret_cast<double *>(smem_raw);      // GROUPS * n doubles
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
-            const int col = 64 * (c * TEAM + h) + 2 * lane;
-            if (col < n) qs[(size_t)team * n + col] = q[c].x;
-            if (col + 1 < n) qs[(size_t)team * n + col + 1] = q[c].y;
+            const int col = 64 * (c * W + w) + 2 * lane;
+            if (col < n) qs[(size_t)grp * n + col] = q[c].x;
+            if (col + 1 < n) qs[(size_t)grp * n + col + 1] = q[c].y;
         }
         __syncthreads();
         for (int j = threadIdx.x; j < n; j += kDenseThreads) {
             double s = 0.0;
 #pragma unroll
-            for (int w = 0; w < TEAMS; ++w) s += qs[(size_t)w * n + j];
+            for (int g = 0; g < GROUPS; ++g) s += qs[(size_t)g * n + j];
             p.partials[(size_t)blockIdx.x * n + j] = s;
         }
         reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * n, n, p.out,
                                  &s_flag);
     } else if (AGG == kRowFull) {
-        // every lane of a warp holds the same tsum: count it once per team
-        double v1[1] = {lane == 0 ? tsum : 0.0};
+        double v1[1] = {tsum};
         block_sum<1>(v1, s_red);
         if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
         if (publish_and_is_last(p.head, &s_flag))
@@ -436,7 +448,7 @@ size_t row_ws_bytes(long long cols, int agg)
     return sizeof(WsHead);
 }
 
-template <int NCH, int TEAM, bool STAGED>
+template <int NCH, int W, int R, bool STAGED>
 cudaError_t launch_dense_agg(const DevChain &ch, const RowParams &p, int agg, int grid, size_t smem,
                              cudaStream_t st)
 {
@@ -446,18 +458,28 @@ cudaError_t launch_dense_agg(const DevChain &ch, const RowParams &p, int agg, in
         kern<<<grid, kDenseThreads, smem, st>>>(ch, p);
         return cudaGetLastError();
     };
-    if (agg == FO_ROW_COL_T_AGG) return go(row_dense_kernel<NCH, TEAM, kRowColT, STAGED>);
-    if (agg == FO_ROW_ROW_AGG) return go(row_dense_kernel<NCH, TEAM, kRowRow, STAGED>);
-    return go(row_dense_kernel<NCH, TEAM, kRowFull, STAGED>);
+    if (agg == FO_ROW_COL_T_AGG) return go(row_dense_kernel<NCH, W, R, kRowColT, STAGED>);
+    if (agg == FO_ROW_ROW_AGG) return go(row_dense_kernel<NCH, W, R, kRowRow, STAGED>);
+    return go(row_dense_kernel<NCH, W, R, kRowFull, STAGED>);
 }
 
-// Team size and chunks per warp for a row of n columns: at most 8 chunks (16
-// registers of row data and 16 of accumulator) per lane.
-int dense_team(long long n)
+// Shape of the dense kernel for rows of n columns: chunks per lane, warps per
+// group, rows per group and stage.  cols <= 64 * nch * w; nch * r <= 8 keeps a
+// stage's rows in 32 registers per lane.
+struct DenseShape {
+    int nch, w, r;
+};
+
+DenseShape dense_shape(long long n)
 {
-    int team = 1;
-    while ((long long)64 * 8 * team < n) team *= 2;
-    return team;
+    if (n <= 64) return {1, 1, 4};
+    if (n <= 128) return {1, 2, 4};
+    if (n <= 256) return {1, 4, 8};
+    if (n <= 512) return {1, 8, 8};
+    if (n <= 1024) return {1, 16, 8};
+    if (n <= 2048) return {2, 16, 4};
+    if (n <= 4096) return {4, 16, 2};
+    return {8, 16, 1};
 }
 
 template <bool STAGED>
@@ -465,17 +487,14 @@ cudaError_t launch_dense(const DevChain &ch, const RowParams &p, int agg, int gr
                          cudaStream_t st)
 {
     const long long n = p.cols;
-    switch (dense_team(n)) {
-        case 1:
-            if (n <= 64) return launch_dense_agg<1, 1, STAGED>(ch, p, agg, grid, smem, st);
-            if (n <= 128) return launch_dense_agg<2, 1, STAGED>(ch, p, agg, grid, smem, st);
-            if (n <= 256) return launch_dense_agg<4, 1, STAGED>(ch, p, agg, grid, smem, st);
-            return launch_dense_agg<8, 1, STAGED>(ch, p, agg, grid, smem, st);
-        case 2: return launch_dense_agg<8, 2, STAGED>(ch, p, agg, grid, smem, st);
-        case 4: return launch_dense_agg<8, 4, STAGED>(ch, p, agg, grid, smem, st);
-        case 8: return launch_dense_agg<8, 8, STAGED>(ch, p, agg, grid, smem, st);
-        default: return launch_dense_agg<8, 16, STAGED>(ch, p, agg, grid, smem, st);
-    }
+    if (n <= 64) return launch_dense_agg<1, 1, 4, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 128) return launch_dense_agg<1, 2, 4, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 256) return launch_dense_agg<1, 4, 8, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 512) return launch_dense_agg<1, 8, 8, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 1024) return launch_dense_agg<1, 16, 8, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 2048) return launch_dense_agg<2, 16, 4, STAGED>(ch, p, agg, grid, smem, st);
+    if (n <= 4096) return launch_dense_agg<4, 16, 2, STAGED>(ch, p, agg, grid, smem, st);
+    return launch_dense_agg<8, 16, 1, STAGED>(ch, p, agg, grid, smem, st);
 }
 
 }  // namespace
@@ -582,21 +601,17 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     } else {
         p.X = X->dense.data; p.ldx = X->dense.ld;
         const bool staged = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
-        // ring geometry: stages of about 64 KB, whole rows, one to four rows per team
-        const int teams = kDenseWarps / dense_team(cols);
-        int rpt = (int)((64 * 1024) / (cols * 8 * teams));
-        if (rpt < 1) rpt = 1;
-        if (rpt > 4) rpt = 4;
-        p.rows_per_stage = rpt * teams;
+        // ring geometry: a stage is the rows all groups work on at once
+        const DenseShape sh = dense_shape(cols);
+        p.rows_per_stage = (kDenseWarps / sh.w) * sh.r;
         const size_t stage_bytes = (size_t)p.rows_per_stage * cols * 8;
-        const size_t v_bytes = (size_t)64 * 8 * dense_team(cols) * 8;      // v, zero-padded
-        int stages = (int)((kSmemBudget - v_bytes) / stage_bytes);
-        if (stages > 4) stages = 4;
+        int stages = (int)(kSmemBudget / (stage_bytes ? stage_bytes : 1));
+        if (stages > 8) stages = 8;
         if (stages < 2) stages = 2;
         p.stages = staged ? stages : 1;
         size_t smem = staged ? stage_bytes * stages : 0;       // the ring
-        if (!staged && agg == FO_ROW_COL_T_AGG) smem = (((size_t)teams * cols + 1) & ~(size_t)1) * 8;   // team partials
-        smem += v_bytes;
+        const size_t qs_bytes = (size_t)(kDenseWarps / sh.w) * cols * 8;    // group accumulators
+        if (agg == FO_ROW_COL_T_AGG && smem < qs_bytes) smem = qs_bytes;
         const long long ntiles = (rows + p.rows_per_stage - 1) / p.rows_per_stage;
         long long grid = ntiles < sms ? ntiles : sms;
         if (grid > row_grid_cap()) grid = row_grid_cap();
