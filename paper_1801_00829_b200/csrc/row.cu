@@ -27,7 +27,13 @@ struct RowParams {
     double *partials;
     double *out;
     int stages, rows_per_stage; // dense ring geometry
+    int chain_kind;             // kChainGeneric, or a row chain the kernels evaluate inline
+    int sides_in_ring;          // dense: used sides are contiguous vectors, staged with the rows
 };
+
+// Row chains common enough to be evaluated inline instead of interpreted; the
+// arithmetic is the same, so are the bits.
+enum { kChainGeneric = 0, kChainSideTimesDot = 1, kChainDot = 2 };
 
 enum { kRowColT = 0, kRowRow = 1, kRowFull = 2 };
 
@@ -80,16 +86,27 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
 }
 
 // The chain for one row per lane: R0 = d, R(1+k) = side k of that lane's row.
-__device__ __forceinline__ double lane_chain(const DevChain &ch, double d, const double (&sv)[FO_MAX_SIDES])
+template <int NR>
+__device__ __forceinline__ double lane_chain_nr(const DevChain &ch, double d, const double (&sv)[FO_MAX_SIDES])
 {
-    RegFile<kRegs, 1> f;
+    RegFile<NR, 1> f;
     f.r[0][0] = d;
 #pragma unroll
-    for (int k = 0; k < FO_MAX_SIDES; ++k) f.r[1 + k][0] = sv[k];
-    run_chain<kRegs, 1>(ch, f);
+    for (int k = 0; k < FO_MAX_SIDES; ++k)
+        if (1 + k < NR) f.r[1 + k < NR ? 1 + k : 0][0] = sv[k];
+    run_chain<NR, 1>(ch, f);
     double o[1];
-    operand<kRegs, 1>(ch, f, ch.out[0], o);
+    operand<NR, 1>(ch, f, ch.out[0], o);
     return o[0];
+}
+
+__device__ __forceinline__ double lane_chain(const DevChain &ch, int kind, double d,
+                                             const double (&sv)[FO_MAX_SIDES])
+{
+    if (kind == kChainSideTimesDot) return sv[0] * d;
+    if (kind == kChainDot) return d;
+    if (ch.n_regs <= 4) return lane_chain_nr<4>(ch, d, sv);
+    return lane_chain_nr<kRegs>(ch, d, sv);
 }
 
 // ------------------------------------------------------------------ dense
@@ -169,21 +186,42 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
     double tsum = 0.0;
     bool timed_out = false;
 
+    // side ring: [slot][side][RPS] doubles behind the row ring (STAGED only)
+    double *side_ring = ring + (size_t)S * RPS * n;
+    const bool ring_sides = STAGED && p.sides_in_ring != 0;
+
     auto issue = [&](long long it) {
         const long long tile = blockIdx.x + it * gridDim.x;
         const int slot = (int)(it % S);
         const long long r0 = tile * RPS;
         const int nr = (int)((p.rows - r0 < RPS) ? p.rows - r0 : RPS);
         double *dst = ring + (size_t)slot * RPS * n;
-        mbar_expect_tx(&s_full[slot], (unsigned)(nr * n * 8));
+        // a ragged last tile with an odd row count cannot be a 16-byte multiple:
+        // its side values are read directly (see tile_sides)
+        const bool with_sides = ring_sides && (nr % 2 == 0);
+        unsigned bytes = (unsigned)(nr * n * 8);
+        if (with_sides) {
+#pragma unroll
+            for (int k = 0; k < FO_MAX_SIDES; ++k)
+                if ((ch.side_used >> k) & 1u) bytes += (unsigned)(nr * 8);
+        }
+        mbar_expect_tx(&s_full[slot], bytes);
         if (p.ldx == n) {
             bulk_g2s(dst, p.X + r0 * p.ldx, (unsigned)(nr * n * 8), &s_full[slot]);
         } else {
             for (int r = 0; r < nr; ++r)
                 bulk_g2s(dst + (size_t)r * n, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &s_full[slot]);
         }
+        if (with_sides) {
+#pragma unroll
+            for (int k = 0; k < FO_MAX_SIDES; ++k)
+                if ((ch.side_used >> k) & 1u)
+                    bulk_g2s(side_ring + ((size_t)slot * FO_MAX_SIDES + k) * RPS, p.sides.s[k].data + r0,
+                             (unsigned)(nr * 8), &s_full[slot]);
+        }
     };
-    // side values of the row this lane evaluates the chain for (lanes 0..R-1)
+    // side values of the row this lane evaluates the chain for (lanes 0..R-1),
+    // read straight from global memory
     auto load_tile_sides = [&](long long it, double (&sv)[FO_MAX_SIDES]) {
         const long long row = (blockIdx.x + it * gridDim.x) * RPS + grp * R + lane;
 #pragma unroll
@@ -204,7 +242,9 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
     }
 
     double sv_next[FO_MAX_SIDES];
-    load_tile_sides(0, sv_next);
+#pragma unroll
+    for (int k = 0; k < FO_MAX_SIDES; ++k) sv_next[k] = 0.0;
+    if (!ring_sides) load_tile_sides(0, sv_next);
     for (long long it = 0; it < my_tiles; ++it) {
         const long long r0 = (blockIdx.x + it * gridDim.x) * RPS;
         const int slot = (int)(it % S);
@@ -212,9 +252,20 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
         double sv[FO_MAX_SIDES];
 #pragma unroll
         for (int k = 0; k < FO_MAX_SIDES; ++k) sv[k] = sv_next[k];
-        load_tile_sides(it + 1, sv_next);       // one tile ahead: hidden behind this tile's work
+        if (!ring_sides) load_tile_sides(it + 1, sv_next);   // a tile ahead (a ring is better: see host)
         if (STAGED) {
             if (!mbar_wait(&s_full[slot], (unsigned)((it / S) & 1))) timed_out = true;
+        }
+        if (ring_sides) {
+            const int nr = (int)((p.rows - r0 < RPS) ? p.rows - r0 : RPS);
+            if (nr % 2 == 0) {
+#pragma unroll
+                for (int k = 0; k < FO_MAX_SIDES; ++k)
+                    sv[k] = (lane < R && ((ch.side_used >> k) & 1u))
+                                ? side_ring[((size_t)slot * FO_MAX_SIDES + k) * RPS + grp * R + lane] : 0.0;
+            } else {
+                load_tile_sides(it, sv);
+            }
         }
         // rows of this group into registers, partial dot products
         double2 x[R][NCH];
@@ -254,7 +305,7 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
 #pragma unroll
             for (int k = 0; k < W; ++k) d += s_part[par][grp * W + k][lane];
         }
-        const double t = lane_chain(ch, d, sv);
+        const double t = lane_chain(ch, p.chain_kind, d, sv);
         if (AGG == kRowColT) {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
@@ -386,7 +437,7 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
             const double dall = __shfl_sync(0xffffffffu, d, (lane & 3) * 8);
             if ((lane >> 2) == it) dmine = dall;
         }
-        const double t = lane_chain(ch, dmine, sv);
+        const double t = lane_chain(ch, p.chain_kind, dmine, sv);
         if (AGG == kRowRow) {
             if (have) p.out[myrow] = t;
         } else if (AGG == kRowFull) {
@@ -558,6 +609,13 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     if (cols > kCsrMaxCols) return FO_ERR_UNSUPPORTED;
     if (!csr && cols > kDenseMaxCols) return FO_ERR_UNSUPPORTED;
 
+    // row chains evaluated inline: t = side0 * d (either operand order) and t = d
+    p.chain_kind = kChainGeneric;
+    if (ch.n_ops == 0 && ch.out[0] == 0) p.chain_kind = kChainDot;
+    if (ch.n_ops == 1 && ch.ops[0].opcode == FO_OP_MUL && ch.out[0] == ch.ops[0].dst &&
+        ((ch.ops[0].a == 0 && ch.ops[0].b == 1) || (ch.ops[0].a == 1 && ch.ops[0].b == 0)))
+        p.chain_kind = kChainSideTimesDot;
+
     rc = check_workspace(ws, ws_bytes, row_ws_bytes(cols, agg));
     if (rc != FO_OK) return rc;
     p.head = (WsHead *)ws;
@@ -605,11 +663,18 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
         const DenseShape sh = dense_shape(cols);
         p.rows_per_stage = (kDenseWarps / sh.w) * sh.r;
         const size_t stage_bytes = (size_t)p.rows_per_stage * cols * 8;
-        int stages = (int)(kSmemBudget / (stage_bytes ? stage_bytes : 1));
+        int stages = (int)(kSmemBudget / (stage_bytes + (size_t)FO_MAX_SIDES * p.rows_per_stage * 8));
         if (stages > 8) stages = 8;
         if (stages < 2) stages = 2;
         p.stages = staged ? stages : 1;
+        // used sides ride in the ring when they are contiguous, 16-byte aligned vectors
+        p.sides_in_ring = staged ? 1 : 0;
+        for (int k = 0; k < n_sides; ++k)
+            if (((ch.side_used >> k) & 1u) && (p.sides.s[k].ld != 1 || !aligned16(p.sides.s[k].data)))
+                p.sides_in_ring = 0;
+        if (ch.side_used == 0) p.sides_in_ring = 0;
         size_t smem = staged ? stage_bytes * stages : 0;       // the ring
+        if (staged) smem += (size_t)stages * FO_MAX_SIDES * p.rows_per_stage * 8;   // side ring
         const size_t qs_bytes = (size_t)(kDenseWarps / sh.w) * cols * 8;    // group accumulators
         if (agg == FO_ROW_COL_T_AGG && smem < qs_bytes) smem = qs_bytes;
         const long long ntiles = (rows + p.rows_per_stage - 1) / p.rows_per_stage;
