@@ -52,7 +52,8 @@ typedef enum fo_status {
     FO_ERR_UNSUPPORTED = -4,    /* variant or size outside what the kernels cover */
     FO_ERR_WORKSPACE = -5,      /* ws NULL, misaligned or too small */
     FO_ERR_CUDA = -6,           /* the CUDA runtime refused the launch */
-    FO_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait ran out (see fo_query_device_status) */
+    FO_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait ran out (see fo_query_device_status) */
+    FO_ERR_STATIC_LIMIT = -8    /* fused_cell_static: the call needs more than the built-in scratch */
 } fo_status;
 
 /* ---------------------------------------------------------------- matrices */
@@ -194,6 +195,40 @@ int fused_cell(const fo_chain *chain, const fo_mat *X,
                const fo_side *sides, int n_sides,
                const double *scalars, int n_scalars,
                int agg, double *out, void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------- Cell, built-in scratch
+ * (No counterpart in the paper: a deployment variant of fused_cell.)
+ *
+ * Some callers cannot obtain device memory at the point where they need a fused
+ * operator: code that runs inside a region where another component owns the
+ * allocator, callbacks that must not call cudaMalloc or a framework allocator
+ * (an allocation may synchronise the device, or is simply forbidden there), and
+ * hosts whose memory pool is handed out once at start-up.  For them this entry
+ * point takes no workspace: the scratch is a 1 MiB array that lives inside the
+ * library image on every GPU that loads it, from load until the process exits.
+ *
+ * Same arguments, results and bits as fused_cell (dense X; all four variants).
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Limit: the call must need at most fused_cell_static_limit_bytes() (1 MiB)
+ *     of scratch, i.e. fused_cell_workspace_bytes(X, agg) <= that.  This always
+ *     holds for no_agg, row_agg and full_agg.  col_agg keeps one partial row of
+ *     `cols` doubles per row panel (up to about 1200 panels for tall matrices),
+ *     so it fits for, e.g., 1000 x 1000 or 1 000 000 x 100 but not for
+ *     1 000 000 x 1000.  Beyond the limit: FO_ERR_STATIC_LIMIT, nothing is launched.
+ *   - The first call on each device looks up the array's device address (a
+ *     one-time runtime query, with that device current).  Make that first call
+ *     outside any stream capture.
+ *   - Every call on a device shares the one array, which keeps what the last
+ *     call left in it.  The kernels leave its control words zeroed for the next
+ *     call and overwrite the rest before reading it, so calls in sequence on one
+ *     stream need no clearing; calls that may overlap on the GPU (different
+ *     streams, different threads) race on it and must be serialised by the caller.
+ */
+int fused_cell_static(const fo_chain *chain, const fo_mat *X,
+                      const fo_side *sides, int n_sides,
+                      const double *scalars, int n_scalars,
+                      int agg, double *out, void *stream);
+size_t fused_cell_static_limit_bytes(void);
 
 /* ------------------------------------------------------------------ MAgg
  * Table 1, MAgg template; Section 5.2 "Multi-Aggregate Operations".

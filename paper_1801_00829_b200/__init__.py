@@ -4,12 +4,12 @@ The work happens in ``libfusedops.so`` (CUDA, sm_100a; C ABI in
 ``include/fusedops.h``); this package is the thin ctypes binding around it.
 """
 from .binding import (  # noqa: F401
-    CSR, FusedOpsError, device_status, force_interpreter, fused_cell, fused_magg, fused_outer, fused_row,
+    CSR, FusedOpsError, device_status, force_interpreter, fused_cell, fused_cell_static, fused_magg, fused_outer, fused_row,
     load_library, make_chain, workspace,
 )
 from .roofline import algorithmic_bytes, ideal_seconds  # noqa: F401
 
 __all__ = [
-    "CSR", "FusedOpsError", "device_status", "force_interpreter", "fused_cell", "fused_magg", "fused_outer",
+    "CSR", "FusedOpsError", "device_status", "force_interpreter", "fused_cell", "fused_cell_static", "fused_magg", "fused_outer",
     "fused_row", "load_library", "make_chain", "workspace", "algorithmic_bytes", "ideal_seconds",
 ]

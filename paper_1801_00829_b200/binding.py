@@ -37,7 +37,7 @@ ACCESS = {"cell": 0, "row": 1, "col": 2}
 
 STATUS = {0: "FO_OK", -1: "FO_ERR_NULL", -2: "FO_ERR_SHAPE", -3: "FO_ERR_CHAIN",
           -4: "FO_ERR_UNSUPPORTED", -5: "FO_ERR_WORKSPACE", -6: "FO_ERR_CUDA",
-          -7: "FO_ERR_DEVICE_TIMEOUT"}
+          -7: "FO_ERR_DEVICE_TIMEOUT", -8: "FO_ERR_STATIC_LIMIT"}
 
 
 class FusedOpsError(RuntimeError):
@@ -79,6 +79,7 @@ EXPORTS = [
     "fused_cell_workspace_bytes", "fused_magg_workspace_bytes", "fused_row_workspace_bytes",
     "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
+    "fused_cell_static", "fused_cell_static_limit_bytes",
 ]
 
 _lib = None
@@ -117,6 +118,10 @@ def load_library(path=None):
         lib.fo_status_string.restype = C.c_char_p
         lib.fo_last_cuda_error.argtypes = []
         lib.fo_last_cuda_error.restype = C.c_int
+        lib.fused_cell_static.argtypes = [chain_p, mat_p, side_p, i32, scal_p, i32, i32, dp, vp]
+        lib.fused_cell_static.restype = C.c_int
+        lib.fused_cell_static_limit_bytes.argtypes = []
+        lib.fused_cell_static_limit_bytes.restype = C.c_size_t
         lib.fo_set_force_interpreter.argtypes = [C.c_int]
         lib.fo_set_force_interpreter.restype = C.c_int
         if path is None:
@@ -335,6 +340,28 @@ def fused_cell(steps, output, X, sides=(), scalars=(), agg="full", out=None):
     _check(lib.fused_cell(C.byref(ch), C.byref(m), sarr, len(sides), sc, len(scalars), a,
                           C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
                           _stream(dev)), "fused_cell")
+    return out
+
+
+def fused_cell_static(steps, output, X, sides=(), scalars=(), agg="full", out=None):
+    """fused_cell for callers that may not allocate device memory for scratch: the
+    library's built-in 1 MiB scratch array is used instead of a workspace tensor.
+    Raises FusedOpsError(FO_ERR_STATIC_LIMIT) if the call would need more.  Calls
+    that can overlap on the GPU must not use it concurrently.  Such callers pass
+    `out` themselves; it is only created here as a convenience for tests."""
+    lib = load_library()
+    sides = list(sides)
+    ch, keep = make_chain(steps, output)
+    m = _mat(X)
+    rows, cols = X.shape
+    dev = X.device
+    a = CELL_AGG[agg]
+    if out is None:
+        shape = {"full": (1,), "row": (rows,), "col": (cols,), "none": (rows, cols)}[agg]
+        out = torch.empty(shape, dtype=torch.float64, device=dev)
+    sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
+    _check(lib.fused_cell_static(C.byref(ch), C.byref(m), sarr, len(sides), sc, len(scalars), a,
+                                 C.c_void_p(out.data_ptr()), _stream(dev)), "fused_cell_static")
     return out
 
 

@@ -486,7 +486,60 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
 
 }  // namespace fo
 
+namespace fo {
+namespace {
+
+// Scratch of fused_cell_static: one array per GPU that loads the library, held
+// until the process exits.  Zero-initialised at load, which is the state the
+// ticket counters need; every call leaves them at zero again.
+constexpr size_t kStaticWsBytes = 1u << 20;
+static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
+
+// Device address of g_static_ws on the current device (NULL on failure).  In host
+// code the symbol's name is only a handle: the address a kernel can use has to
+// be asked for, once per device, with that device current.
+void *static_ws_address()
+{
+    static void *cached[64] = {nullptr};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= 64) {
+        cuda_fail(e != cudaSuccess ? e : cudaErrorInvalidDevice);
+        return nullptr;
+    }
+    if (!cached[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress((void **)&ptr, g_static_ws);
+        if (e != cudaSuccess) {
+            cuda_fail(e);
+            return nullptr;
+        }
+        cached[dev] = ptr;
+    }
+    return cached[dev];
+}
+
+}  // namespace
+}  // namespace fo
+
 extern "C" {
+
+int fused_cell_static(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
+                      const double *scalars, int n_scalars, int agg, double *out, void *stream)
+{
+    if (!X) return FO_ERR_NULL;
+    if (agg < FO_CELL_NO_AGG || agg > FO_CELL_FULL_AGG) return FO_ERR_UNSUPPORTED;
+    if (X->kind != FO_DENSE) return (X->kind == FO_CSR) ? FO_ERR_UNSUPPORTED : FO_ERR_SHAPE;
+    if (X->dense.rows < 0 || X->dense.cols < 0) return FO_ERR_SHAPE;
+    const size_t need = fo::cell_ws_bytes(X->dense.rows, X->dense.cols, agg, 1);
+    if (need > fo::kStaticWsBytes) return FO_ERR_STATIC_LIMIT;
+    void *ws = fo::static_ws_address();
+    if (!ws) return FO_ERR_CUDA;
+    return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, false, out, ws,
+                        fo::kStaticWsBytes, stream);
+}
+
+size_t fused_cell_static_limit_bytes(void) { return fo::kStaticWsBytes; }
 
 int fo_set_force_interpreter(int on)
 {

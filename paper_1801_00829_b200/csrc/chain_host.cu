@@ -212,6 +212,7 @@ const char *fo_status_string(int status)
         case FO_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case FO_ERR_CUDA: return "CUDA runtime error at launch";
         case FO_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        case FO_ERR_STATIC_LIMIT: return "the call needs more scratch than the built-in array holds";
         default: return "unknown status";
     }
 }

@@ -34,11 +34,11 @@ def test_header_functions_are_exported(lib):
 
 def test_status_strings(lib):
     seen = set()
-    for code in range(0, -8, -1):
+    for code in range(0, -9, -1):
         s = lib.fo_status_string(code).decode()
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 8
+    assert len(seen) == 9
     assert lib.fo_status_string(-99).decode() == "unknown status"
 
 
