@@ -11,6 +11,8 @@
 //   cell_rows_kernel  general case (leading dimensions, row / column vector
 //                     sides): a warp per row (no_agg, row_agg, full_agg, MAgg);
 //   cell_cols_kernel  col_agg: a thread per column pair, a CTA per panel of rows.
+#include <stdlib.h>
+
 #include "spec.cuh"
 
 namespace fo {
@@ -293,10 +295,28 @@ __global__ void fill_zero_kernel(double *out, long long n)
 // ------------------------------------------------------------------ host
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
+// CTAs per SM of the streaming kernels.  FUSEDOPS_CELL_CTAS_PER_SM (1..8, read once)
+// overrides the default; it is a tuning knob, results do not depend on it beyond
+// the order of the per-CTA partial sums.
+int cell_ctas_per_sm()
+{
+    static int cached = 0;
+    if (cached == 0) {
+        int v = 3;        // measured: 2-3 is best for 10-100 MB inputs, larger inputs do not care
+        const char *e = getenv("FUSEDOPS_CELL_CTAS_PER_SM");
+        if (e) {
+            const int x = atoi(e);
+            if (x >= 1 && x <= 8) v = x;
+        }
+        cached = v;
+    }
+    return cached;
+}
+
 // Grid of a streaming kernel: every CTA gets work, at most `cap` CTAs.
 int stream_grid(long long units, int sms)
 {
-    const long long cap = (long long)(sms > 0 ? sms : 148) * 8;
+    const long long cap = (long long)(sms > 0 ? sms : 148) * cell_ctas_per_sm();
     long long g = units < cap ? units : cap;
     if (g > kMaxPartials) g = kMaxPartials;
     if (g < 1) g = 1;

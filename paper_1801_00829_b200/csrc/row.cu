@@ -55,6 +55,10 @@ __device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned
                  "r"(bytes)
                  : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity)
 {
     unsigned ok;
@@ -121,8 +125,9 @@ __device__ __forceinline__ double lane_chain(const DevChain &ch, int kind, doubl
 // that row, and the warp adds t_r * X_r into its accumulator columns.
 // STAGED: rows arrive through the shared-memory ring; otherwise lanes load
 // their pairs straight from global memory (any alignment, any cols).
-constexpr int kDenseThreads = 512;
+constexpr int kDenseThreads = 512;                 // compute threads
 constexpr int kDenseWarps = kDenseThreads / 32;
+constexpr int kDenseBlock = kDenseThreads + 32;    // plus the warp that feeds the ring
 
 // Sums R values per lane over the 32 lanes of a warp in a fixed order.  On
 // return v[0] holds, in every lane l, the total of value number (l >> (5 - log2 R)).
@@ -154,11 +159,11 @@ struct Log2<1> {
 };
 
 template <int NCH, int W, int R, int AGG, bool STAGED>
-__global__ void __launch_bounds__(kDenseThreads, 1)
+__global__ void __launch_bounds__(kDenseBlock, 1)
 row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    __shared__ unsigned long long s_full[8];
+    __shared__ unsigned long long s_full[8], s_empty[8];
     __shared__ double s_part[2][kDenseWarps][8];     // [parity][warp][row of the group]
     __shared__ double s_red[32];
     __shared__ unsigned int s_flag;
@@ -167,7 +172,8 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
     constexpr int RPS = GROUPS * R;                  // rows per stage
     constexpr int SH = 5 - Log2<R>::value;           // lane l holds row (l >> SH) after the butterfly
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int grp = warp / W, w = warp % W;
+    const bool feeder = warp == kDenseWarps;         // warp 16 only moves data
+    const int grp = (warp % kDenseWarps) / W, w = warp % W;
     const int n = (int)p.cols;
     const int S = p.stages;
     double *ring = reinterpret_cast<double *>(smem_raw);
@@ -232,20 +238,29 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
 
     if (STAGED) {
         if (threadIdx.x == 0) {
-            for (int s = 0; s < S; ++s) mbar_init(&s_full[s], 1);
+            for (int s = 0; s < S; ++s) {
+                mbar_init(&s_full[s], 1);
+                mbar_init(&s_empty[s], kDenseWarps);
+            }
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         __syncthreads();
-        if (threadIdx.x == 0)
-            for (long long it = 0; it < S && it < my_tiles; ++it) issue(it);
+        // the feeding warp refills a slot as soon as every compute warp has taken
+        // its pieces of the slot's rows into registers
+        if (feeder && lane == 0) {
+            for (long long it = 0; it < my_tiles; ++it) {
+                if (it >= S && !mbar_wait(&s_empty[it % S], (unsigned)(((it / S) - 1) & 1))) timed_out = true;
+                issue(it);
+            }
+        }
     }
 
     double sv_next[FO_MAX_SIDES];
 #pragma unroll
     for (int k = 0; k < FO_MAX_SIDES; ++k) sv_next[k] = 0.0;
     if (!ring_sides) load_tile_sides(0, sv_next);
-    for (long long it = 0; it < my_tiles; ++it) {
+    for (long long it = 0; it < my_tiles && !feeder; ++it) {
         const long long r0 = (blockIdx.x + it * gridDim.x) * RPS;
         const int slot = (int)(it % S);
         const int par = (int)(it & 1);
@@ -292,20 +307,39 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
             }
             part[r] = d0 + d1;
         }
+        // rows and side values are in registers: hand the slot back to the feeder
+        if (STAGED) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_empty[slot]);
+        }
         warp_sum_multi<R>(part, lane);
         if ((lane & ((1 << SH) - 1)) == 0) s_part[par][warp][lane >> SH] = part[0];
-        __syncthreads();
-        // every thread holds its pieces in registers: the slot can be refilled
-        if (STAGED) {
-            if (threadIdx.x == 0 && it + S < my_tiles) issue(it + S);
-        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kDenseThreads) : "memory");     // the compute warps
         // lane r: dot product of row r (warps of the group in order), then the chain
         double d = 0.0;
         if (lane < R) {
 #pragma unroll
             for (int k = 0; k < W; ++k) d += s_part[par][grp * W + k][lane];
         }
-        const double t = lane_chain(ch, p.chain_kind, d, sv);
+        double t;
+        if (p.chain_kind == kChainSideTimesDot) {
+            t = sv[0] * d;
+        } else if (p.chain_kind == kChainDot) {
+            t = d;
+        } else {
+            // general chain: one warp-wide evaluation per row (lane 0 holds d, lane 1 + k side k)
+            t = 0.0;
+            for (int r = 0; r < R; ++r) {
+                double mine = __shfl_sync(0xffffffffu, d, r);
+#pragma unroll
+                for (int k = 0; k < FO_MAX_SIDES; ++k) {
+                    const double sk = __shfl_sync(0xffffffffu, sv[k], r);
+                    if (lane == 1 + k) mine = sk;
+                }
+                const double tr = warp_chain(ch, mine, lane);
+                if (lane == r) t = tr;
+            }
+        }
         if (AGG == kRowColT) {
 #pragma unroll
             for (int r = 0; r < R; ++r) {
@@ -334,11 +368,11 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
             const int col = 64 * (c * W + w) + 2 * lane;
-            if (col < n) qs[(size_t)grp * n + col] = q[c].x;
-            if (col + 1 < n) qs[(size_t)grp * n + col + 1] = q[c].y;
+            if (!feeder && col < n) qs[(size_t)grp * n + col] = q[c].x;
+            if (!feeder && col + 1 < n) qs[(size_t)grp * n + col + 1] = q[c].y;
         }
         __syncthreads();
-        for (int j = threadIdx.x; j < n; j += kDenseThreads) {
+        for (int j = threadIdx.x; j < n; j += kDenseBlock) {
             double s = 0.0;
 #pragma unroll
             for (int g = 0; g < GROUPS; ++g) s += qs[(size_t)g * n + j];
@@ -506,7 +540,7 @@ cudaError_t launch_dense_agg(const DevChain &ch, const RowParams &p, int agg, in
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kern<<<grid, kDenseThreads, smem, st>>>(ch, p);
+        kern<<<grid, kDenseBlock, smem, st>>>(ch, p);
         return cudaGetLastError();
     };
     if (agg == FO_ROW_COL_T_AGG) return go(row_dense_kernel<NCH, W, R, kRowColT, STAGED>);
