@@ -9,6 +9,9 @@
 // of the rows, of v and of the output accumulator, all in registers.  CSR X: a
 // warp per block of 32 rows, an 8-lane group per row; v and the output
 // accumulator live in shared memory.
+#include <stdio.h>
+#include <stdlib.h>
+
 #include "chain.cuh"
 
 namespace fo {
@@ -128,6 +131,7 @@ __device__ __forceinline__ double lane_chain(const DevChain &ch, int kind, doubl
 constexpr int kDenseThreads = 512;                 // compute threads
 constexpr int kDenseWarps = kDenseThreads / 32;
 constexpr int kDenseBlock = kDenseThreads + 32;    // plus the warp that feeds the ring
+constexpr int kDenseMaxSlots = 64;                 // ring slots of all groups together
 
 // Sums R values per lane over the 32 lanes of a warp in a fixed order.  On
 // return v[0] holds, in every lane l, the total of value number (l >> (5 - log2 R)).
@@ -163,47 +167,55 @@ __global__ void __launch_bounds__(kDenseBlock, 1)
 row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    __shared__ unsigned long long s_full[8], s_empty[8];
+    __shared__ unsigned long long s_full[kDenseMaxSlots], s_empty[kDenseMaxSlots];
     __shared__ double s_part[2][kDenseWarps][8];     // [parity][warp][row of the group]
     __shared__ double s_red[32];
     __shared__ unsigned int s_flag;
 
+    // The 16 compute warps form GROUPS independent groups of W warps.  A group has
+    // its own ring slots, barriers and sequence of tiles (R rows each), so the
+    // groups drift apart and one group's barrier and reduction latency is covered
+    // by the others' work.
     constexpr int GROUPS = kDenseWarps / W;
-    constexpr int RPS = GROUPS * R;                  // rows per stage
     constexpr int SH = 5 - Log2<R>::value;           // lane l holds row (l >> SH) after the butterfly
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool feeder = warp == kDenseWarps;         // warp 16 only moves data
-    const int grp = (warp % kDenseWarps) / W, w = warp % W;
+    const int w = warp % W;
+    // a feeder lane serves the group of its lane number
+    const int grp = feeder ? (lane < GROUPS ? lane : 0) : warp / W;
     const int n = (int)p.cols;
-    const int S = p.stages;
-    double *ring = reinterpret_cast<double *>(smem_raw);
-    const long long ntiles = (p.rows + RPS - 1) / RPS;
-    const long long my_tiles = (ntiles > blockIdx.x) ? (ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int S = p.stages;                          // ring slots per group
+    double *ring = reinterpret_cast<double *>(smem_raw) + (size_t)grp * S * R * n;
+    // side ring: [group][slot][side][R] doubles behind all the row rings (STAGED only)
+    double *side_ring = reinterpret_cast<double *>(smem_raw) + (size_t)GROUPS * S * R * n
+                        + (size_t)grp * S * FO_MAX_SIDES * R;
+    unsigned long long *full = s_full + grp * S, *empty = s_empty + grp * S;
+    const bool ring_sides = STAGED && p.sides_in_ring != 0;
+
+    // tiles of R rows are dealt round-robin to the (CTA, group) pairs
+    const long long ntiles = (p.rows + R - 1) / R;
+    const long long me = (long long)blockIdx.x * GROUPS + grp, stride = (long long)gridDim.x * GROUPS;
+    const long long my_tiles = (ntiles > me) ? (ntiles - me + stride - 1) / stride : 0;
 
     // this lane's columns: pair (col, col + 1) of chunk c
     double2 vreg[NCH], q[NCH];
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
         const int col = 64 * (c * W + w) + 2 * lane;
-        vreg[c].x = col < n ? __ldg(p.v + col) : 0.0;
-        vreg[c].y = col + 1 < n ? __ldg(p.v + col + 1) : 0.0;
+        vreg[c].x = (!feeder && col < n) ? __ldg(p.v + col) : 0.0;
+        vreg[c].y = (!feeder && col + 1 < n) ? __ldg(p.v + col + 1) : 0.0;
         q[c] = make_double2(0.0, 0.0);
     }
     double tsum = 0.0;
     bool timed_out = false;
 
-    // side ring: [slot][side][RPS] doubles behind the row ring (STAGED only)
-    double *side_ring = ring + (size_t)S * RPS * n;
-    const bool ring_sides = STAGED && p.sides_in_ring != 0;
-
     auto issue = [&](long long it) {
-        const long long tile = blockIdx.x + it * gridDim.x;
         const int slot = (int)(it % S);
-        const long long r0 = tile * RPS;
-        const int nr = (int)((p.rows - r0 < RPS) ? p.rows - r0 : RPS);
-        double *dst = ring + (size_t)slot * RPS * n;
+        const long long r0 = (me + it * stride) * R;
+        const int nr = (int)((p.rows - r0 < R) ? p.rows - r0 : R);
+        double *dst = ring + (size_t)slot * R * n;
         // a ragged last tile with an odd row count cannot be a 16-byte multiple:
-        // its side values are read directly (see tile_sides)
+        // its side values are read directly (see load_tile_sides)
         const bool with_sides = ring_sides && (nr % 2 == 0);
         unsigned bytes = (unsigned)(nr * n * 8);
         if (with_sides) {
@@ -211,25 +223,25 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
             for (int k = 0; k < FO_MAX_SIDES; ++k)
                 if ((ch.side_used >> k) & 1u) bytes += (unsigned)(nr * 8);
         }
-        mbar_expect_tx(&s_full[slot], bytes);
+        mbar_expect_tx(&full[slot], bytes);
         if (p.ldx == n) {
-            bulk_g2s(dst, p.X + r0 * p.ldx, (unsigned)(nr * n * 8), &s_full[slot]);
+            bulk_g2s(dst, p.X + r0 * p.ldx, (unsigned)(nr * n * 8), &full[slot]);
         } else {
             for (int r = 0; r < nr; ++r)
-                bulk_g2s(dst + (size_t)r * n, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &s_full[slot]);
+                bulk_g2s(dst + (size_t)r * n, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &full[slot]);
         }
         if (with_sides) {
 #pragma unroll
             for (int k = 0; k < FO_MAX_SIDES; ++k)
                 if ((ch.side_used >> k) & 1u)
-                    bulk_g2s(side_ring + ((size_t)slot * FO_MAX_SIDES + k) * RPS, p.sides.s[k].data + r0,
-                             (unsigned)(nr * 8), &s_full[slot]);
+                    bulk_g2s(side_ring + ((size_t)slot * FO_MAX_SIDES + k) * R, p.sides.s[k].data + r0,
+                             (unsigned)(nr * 8), &full[slot]);
         }
     };
     // side values of the row this lane evaluates the chain for (lanes 0..R-1),
     // read straight from global memory
     auto load_tile_sides = [&](long long it, double (&sv)[FO_MAX_SIDES]) {
-        const long long row = (blockIdx.x + it * gridDim.x) * RPS + grp * R + lane;
+        const long long row = (me + it * stride) * R + lane;
 #pragma unroll
         for (int k = 0; k < FO_MAX_SIDES; ++k)
             sv[k] = (lane < R && it < my_tiles && row < p.rows && ((ch.side_used >> k) & 1u))
@@ -238,67 +250,58 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
 
     if (STAGED) {
         if (threadIdx.x == 0) {
-            for (int s = 0; s < S; ++s) {
+            for (int s = 0; s < GROUPS * S; ++s) {
                 mbar_init(&s_full[s], 1);
-                mbar_init(&s_empty[s], kDenseWarps);
+                mbar_init(&s_empty[s], W);
             }
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         __syncthreads();
-        // the feeding warp refills a slot as soon as every compute warp has taken
-        // its pieces of the slot's rows into registers
-        if (feeder && lane == 0) {
+        // the feeding warp, one lane per group: refill a slot as soon as every warp
+        // of the group has taken its pieces of the slot's rows into registers
+        if (feeder && lane < GROUPS) {
             for (long long it = 0; it < my_tiles; ++it) {
-                if (it >= S && !mbar_wait(&s_empty[it % S], (unsigned)(((it / S) - 1) & 1))) timed_out = true;
+                if (it >= S && !mbar_wait(&empty[it % S], (unsigned)(((it / S) - 1) & 1))) timed_out = true;
                 issue(it);
             }
         }
     }
 
-    double sv_next[FO_MAX_SIDES];
-#pragma unroll
-    for (int k = 0; k < FO_MAX_SIDES; ++k) sv_next[k] = 0.0;
-    if (!ring_sides) load_tile_sides(0, sv_next);
     for (long long it = 0; it < my_tiles && !feeder; ++it) {
-        const long long r0 = (blockIdx.x + it * gridDim.x) * RPS;
+        const long long r0 = (me + it * stride) * R;
         const int slot = (int)(it % S);
         const int par = (int)(it & 1);
         double sv[FO_MAX_SIDES];
-#pragma unroll
-        for (int k = 0; k < FO_MAX_SIDES; ++k) sv[k] = sv_next[k];
-        if (!ring_sides) load_tile_sides(it + 1, sv_next);   // a tile ahead (a ring is better: see host)
+        const int nr = (int)((p.rows - r0 < R) ? p.rows - r0 : R);
+        // strided or unaligned side vectors (and a ragged odd last tile) cannot ride
+        // in the ring: their values are requested here, ahead of the wait
+        if (!(ring_sides && nr % 2 == 0)) load_tile_sides(it, sv);
         if (STAGED) {
-            if (!mbar_wait(&s_full[slot], (unsigned)((it / S) & 1))) timed_out = true;
+            if (!mbar_wait(&full[slot], (unsigned)((it / S) & 1))) timed_out = true;
         }
-        if (ring_sides) {
-            const int nr = (int)((p.rows - r0 < RPS) ? p.rows - r0 : RPS);
-            if (nr % 2 == 0) {
+        if (ring_sides && nr % 2 == 0) {
 #pragma unroll
-                for (int k = 0; k < FO_MAX_SIDES; ++k)
-                    sv[k] = (lane < R && ((ch.side_used >> k) & 1u))
-                                ? side_ring[((size_t)slot * FO_MAX_SIDES + k) * RPS + grp * R + lane] : 0.0;
-            } else {
-                load_tile_sides(it, sv);
-            }
+            for (int k = 0; k < FO_MAX_SIDES; ++k)
+                sv[k] = (lane < R && ((ch.side_used >> k) & 1u))
+                            ? side_ring[((size_t)slot * FO_MAX_SIDES + k) * R + lane] : 0.0;
         }
-        // rows of this group into registers, partial dot products
+        // rows of this tile into registers, partial dot products
         double2 x[R][NCH];
         double part[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const int rl = grp * R + r;
-            const bool have = r0 + rl < p.rows;
+            const bool have = r0 + r < p.rows;
             double d0 = 0.0, d1 = 0.0;
 #pragma unroll
             for (int c = 0; c < NCH; ++c) {
                 const int col = 64 * (c * W + w) + 2 * lane;
                 if (STAGED) {
-                    const double *rowp = ring + ((size_t)slot * RPS + rl) * n;
+                    const double *rowp = ring + ((size_t)slot * R + r) * n;
                     x[r][c] = (have && col < n) ? *reinterpret_cast<const double2 *>(rowp + col)
                                                 : make_double2(0.0, 0.0);
                 } else {
-                    const double *rowp = p.X + (r0 + rl) * p.ldx;
+                    const double *rowp = p.X + (r0 + r) * p.ldx;
                     x[r][c].x = (have && col < n) ? ld_stream1(rowp + col) : 0.0;
                     x[r][c].y = (have && col + 1 < n) ? ld_stream1(rowp + col + 1) : 0.0;
                 }
@@ -310,11 +313,15 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
         // rows and side values are in registers: hand the slot back to the feeder
         if (STAGED) {
             __syncwarp();
-            if (lane == 0) mbar_arrive(&s_empty[slot]);
+            if (lane == 0) mbar_arrive(&empty[slot]);
         }
         warp_sum_multi<R>(part, lane);
         if ((lane & ((1 << SH) - 1)) == 0) s_part[par][warp][lane >> SH] = part[0];
-        asm volatile("bar.sync 1, %0;" ::"n"(kDenseThreads) : "memory");     // the compute warps
+        if (W > 1) {
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "n"(W * 32) : "memory");   // the group's warps
+        } else {
+            __syncwarp();
+        }
         // lane r: dot product of row r (warps of the group in order), then the chain
         double d = 0.0;
         if (lane < R) {
@@ -351,7 +358,7 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
                 }
             }
         } else {
-            const long long row = r0 + grp * R + lane;
+            const long long row = r0 + lane;
             if (w == 0 && lane < R && row < p.rows) {
                 if (AGG == kRowRow) p.out[row] = t;
                 else tsum += t;
@@ -365,11 +372,12 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
         // groups -> CTA: fixed order over groups, through shared memory
         __syncthreads();
         double *qs = reinterpret_cast<double *>(smem_raw);      // GROUPS * n doubles
+        const int cgrp = warp / W;
 #pragma unroll
         for (int c = 0; c < NCH; ++c) {
             const int col = 64 * (c * W + w) + 2 * lane;
-            if (!feeder && col < n) qs[(size_t)grp * n + col] = q[c].x;
-            if (!feeder && col + 1 < n) qs[(size_t)grp * n + col + 1] = q[c].y;
+            if (!feeder && col < n) qs[(size_t)cgrp * n + col] = q[c].x;
+            if (!feeder && col + 1 < n) qs[(size_t)cgrp * n + col + 1] = q[c].y;
         }
         __syncthreads();
         for (int j = threadIdx.x; j < n; j += kDenseBlock) {
@@ -555,13 +563,28 @@ struct DenseShape {
     int nch, w, r;
 };
 
+// Shapes that are compiled.  FUSEDOPS_DENSE_SHAPE="nch,w,r" (read per call; a
+// tuning knob) picks one of them if it covers the column count.
+const DenseShape kDenseShapes[] = {{1, 1, 4}, {1, 2, 4}, {1, 4, 8}, {1, 8, 8}, {1, 16, 8}, {2, 16, 4},
+                                   {4, 16, 2}, {8, 16, 1}, {2, 8, 4}, {4, 4, 2}, {8, 2, 1}, {4, 4, 1}, {2, 8, 2}, {2, 4, 4}, {4, 8, 2}, {1, 1, 8}, {1, 2, 8}};
+
 DenseShape dense_shape(long long n)
 {
-    if (n <= 64) return {1, 1, 4};
-    if (n <= 128) return {1, 2, 4};
+    const char *e = getenv("FUSEDOPS_DENSE_SHAPE");
+    if (e) {
+        int a = 0, b = 0, c = 0;
+        if (sscanf(e, "%d,%d,%d", &a, &b, &c) == 3)
+            for (const DenseShape &k : kDenseShapes)
+                if (k.nch == a && k.w == b && k.r == c && (long long)64 * a * b >= n) return k;
+    }
+    // measured on B200: several small independent groups beat one large group
+    // (1000 columns: {4,4,2} 6.6 TB/s, {2,8,4} 6.4, {1,16,8} 5.1)
+    // (512: {1,8,8} 6.2 vs {2,4,4} 5.9; 2048: {2,16,4} 6.0 vs {4,8,2} 5.1)
+    if (n <= 64) return {1, 1, 8};
+    if (n <= 128) return {1, 2, 8};
     if (n <= 256) return {1, 4, 8};
     if (n <= 512) return {1, 8, 8};
-    if (n <= 1024) return {1, 16, 8};
+    if (n <= 1024) return {4, 4, 2};
     if (n <= 2048) return {2, 16, 4};
     if (n <= 4096) return {4, 16, 2};
     return {8, 16, 1};
@@ -571,15 +594,14 @@ template <bool STAGED>
 cudaError_t launch_dense(const DevChain &ch, const RowParams &p, int agg, int grid, size_t smem,
                          cudaStream_t st)
 {
-    const long long n = p.cols;
-    if (n <= 64) return launch_dense_agg<1, 1, 4, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 128) return launch_dense_agg<1, 2, 4, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 256) return launch_dense_agg<1, 4, 8, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 512) return launch_dense_agg<1, 8, 8, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 1024) return launch_dense_agg<1, 16, 8, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 2048) return launch_dense_agg<2, 16, 4, STAGED>(ch, p, agg, grid, smem, st);
-    if (n <= 4096) return launch_dense_agg<4, 16, 2, STAGED>(ch, p, agg, grid, smem, st);
-    return launch_dense_agg<8, 16, 1, STAGED>(ch, p, agg, grid, smem, st);
+    const DenseShape k = dense_shape(p.cols);
+#define FO_SHAPE(A, B, C) \
+    if (k.nch == A && k.w == B && k.r == C) return launch_dense_agg<A, B, C, STAGED>(ch, p, agg, grid, smem, st);
+    FO_SHAPE(1, 1, 4) FO_SHAPE(1, 2, 4) FO_SHAPE(1, 4, 8) FO_SHAPE(1, 8, 8) FO_SHAPE(1, 16, 8)
+    FO_SHAPE(2, 16, 4) FO_SHAPE(4, 16, 2) FO_SHAPE(8, 16, 1) FO_SHAPE(2, 8, 4) FO_SHAPE(4, 4, 2)
+    FO_SHAPE(8, 2, 1) FO_SHAPE(4, 4, 1) FO_SHAPE(2, 8, 2) FO_SHAPE(2, 4, 4) FO_SHAPE(4, 8, 2) FO_SHAPE(1, 1, 8) FO_SHAPE(1, 2, 8)
+#undef FO_SHAPE
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace
@@ -693,12 +715,14 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     } else {
         p.X = X->dense.data; p.ldx = X->dense.ld;
         const bool staged = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
-        // ring geometry: a stage is the rows all groups work on at once
+        // ring geometry: every group of warps has its own ring of `stages` slots of r rows
         const DenseShape sh = dense_shape(cols);
-        p.rows_per_stage = (kDenseWarps / sh.w) * sh.r;
-        const size_t stage_bytes = (size_t)p.rows_per_stage * cols * 8;
-        int stages = (int)(kSmemBudget / (stage_bytes + (size_t)FO_MAX_SIDES * p.rows_per_stage * 8));
+        const int groups = kDenseWarps / sh.w;
+        p.rows_per_stage = sh.r;
+        const size_t slot_bytes = (size_t)sh.r * cols * 8 + (size_t)FO_MAX_SIDES * sh.r * 8;
+        int stages = (int)(kSmemBudget / (slot_bytes * groups));
         if (stages > 8) stages = 8;
+        if (stages * groups > kDenseMaxSlots) stages = kDenseMaxSlots / groups;
         if (stages < 2) stages = 2;
         p.stages = staged ? stages : 1;
         // used sides ride in the ring when they are contiguous, 16-byte aligned vectors
@@ -707,12 +731,12 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
             if (((ch.side_used >> k) & 1u) && (p.sides.s[k].ld != 1 || !aligned16(p.sides.s[k].data)))
                 p.sides_in_ring = 0;
         if (ch.side_used == 0) p.sides_in_ring = 0;
-        size_t smem = staged ? stage_bytes * stages : 0;       // the ring
-        if (staged) smem += (size_t)stages * FO_MAX_SIDES * p.rows_per_stage * 8;   // side ring
-        const size_t qs_bytes = (size_t)(kDenseWarps / sh.w) * cols * 8;    // group accumulators
+        size_t smem = staged ? slot_bytes * groups * stages : 0;     // the rings
+        const size_t qs_bytes = (size_t)groups * cols * 8;           // group accumulators
         if (agg == FO_ROW_COL_T_AGG && smem < qs_bytes) smem = qs_bytes;
-        const long long ntiles = (rows + p.rows_per_stage - 1) / p.rows_per_stage;
-        long long grid = ntiles < sms ? ntiles : sms;
+        const long long ntiles = (rows + sh.r - 1) / sh.r;
+        long long grid = (ntiles + groups - 1) / groups;
+        if (grid > sms) grid = sms;
         if (grid > row_grid_cap()) grid = row_grid_cap();
         if (grid < 1) grid = 1;
         e = staged ? launch_dense<true>(ch, p, agg, (int)grid, smem, st)
