@@ -30,71 +30,26 @@ struct OuterParams {
 
 enum { kOutFull = 0, kOutNone = 1, kOutRight = 2 };
 
-// L2 eviction policies: rows of V are gathered again and again and should stay in
-// L2; X and U are read once and should not push them out.
-__device__ __forceinline__ unsigned long long policy_evict_last()
-{
-    unsigned long long pol;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ unsigned long long policy_evict_first()
-{
-    unsigned long long pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ double2 ldg2_hint(const double *p, unsigned long long pol)
-{
-    double2 r;
-    asm volatile("ld.global.nc.L2::cache_hint.v2.f64 {%0, %1}, [%2], %3;"
-                 : "=d"(r.x), "=d"(r.y) : "l"(p), "l"(pol));
-    return r;
-}
-__device__ __forceinline__ double ldg1_hint(const double *p, unsigned long long pol)
-{
-    double r;
-    asm volatile("ld.global.nc.L2::cache_hint.f64 %0, [%1], %2;" : "=d"(r) : "l"(p), "l"(pol));
-    return r;
-}
-__device__ __forceinline__ int ldgi_hint(const int *p, unsigned long long pol)
-{
-    int r;
-    asm volatile("ld.global.nc.L2::cache_hint.s32 %0, [%1], %2;" : "=r"(r) : "l"(p), "l"(pol));
-    return r;
-}
-
-// The pair (col, col + 1) of a factor row of length n; elements at or beyond n
-// read as 0.  ALIGNED: the row start is 16-byte aligned and n is even, so a pair
-// is either whole or absent and one 128-bit load fetches it.
 template <bool ALIGNED>
-__device__ __forceinline__ double2 ld_pair(const double *row, int col, int n, unsigned long long pol)
+__device__ __forceinline__ double2 ld_pair_cached(const double *row, int col, int n)
 {
-    if (ALIGNED) {
-        if (col < n) return ldg2_hint(row + col, pol);
-        return make_double2(0.0, 0.0);
+    if (col + 1 < n) {
+        if (ALIGNED) return __ldg(reinterpret_cast<const double2 *>(row + col));
+        return make_double2(__ldg(row + col), __ldg(row + col + 1));
     }
-    if (col + 1 < n) return make_double2(ldg1_hint(row + col, pol), ldg1_hint(row + col + 1, pol));
-    if (col < n) return make_double2(ldg1_hint(row + col, pol), 0.0);
+    if (col < n) return make_double2(__ldg(row + col), 0.0);
     return make_double2(0.0, 0.0);
-}
-
-template <int NR>
-__device__ __forceinline__ double outer_chain_nr(const DevChain &ch, double a, double d)
-{
-    RegFile<NR, 1> f;
-    f.r[0][0] = a;
-    f.r[1][0] = d;
-    run_chain<NR, 1>(ch, f);
-    double o[1];
-    operand<NR, 1>(ch, f, ch.out[0], o);
-    return o[0];
 }
 
 __device__ __forceinline__ double outer_chain(const DevChain &ch, double a, double d)
 {
-    if (ch.n_regs <= 4) return outer_chain_nr<4>(ch, a, d);
-    return outer_chain_nr<kRegs>(ch, a, d);
+    RegFile<kRegs, 1> f;
+    f.r[0][0] = a;
+    f.r[1][0] = d;
+    run_chain<kRegs, 1>(ch, f);
+    double o[1];
+    operand<kRegs, 1>(ch, f, ch.out[0], o);
+    return o[0];
 }
 
 // First row r in [0, rows] with rowptr[r] >= target.
@@ -136,7 +91,6 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
     const int l8 = lane & 7, grp = lane >> 3;
     const unsigned full = 0xffffffffu;
     const int rank = p.rank;
-    const unsigned long long keep = policy_evict_last(), once = policy_evict_first();
     double acc = 0.0;
 
     for (long long row = row_lo + warp; row < row_hi; row += kThreads / 32) {
@@ -145,15 +99,15 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
         const double *urow = p.U + row * p.ldu;
 #pragma unroll
         for (int c = 0; c < NK2; ++c) {
-            u[c] = (beg < end) ? ld_pair<ALIGNED>(urow, 16 * c + 2 * l8, rank, once)
+            u[c] = (beg < end) ? ld_pair_cached<ALIGNED>(urow, 16 * c + 2 * l8, rank)
                                : make_double2(0.0, 0.0);
             racc[c] = make_double2(0.0, 0.0);
         }
         for (int c0 = beg; c0 < end; c0 += 32) {
             const int cnt = (end - c0 < 32) ? end - c0 : 32;
             const bool valid = lane < cnt;
-            const int jmine = valid ? ldgi_hint(p.colidx + c0 + lane, once) : 0;
-            const double amine = valid ? ldg1_hint(p.vals + c0 + lane, once) : 0.0;
+            const int jmine = valid ? __ldg(p.colidx + c0 + lane) : 0;
+            const double amine = valid ? __ldg(p.vals + c0 + lane) : 0.0;
             double dmine = 0.0;
             const int nit = (cnt + 3) >> 2;
             for (int it = 0; it < nit; it += 2) {
@@ -166,8 +120,8 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
                 double2 xA[NK2], xB[NK2];
 #pragma unroll
                 for (int c = 0; c < NK2; ++c) {
-                    xA[c] = actA ? ld_pair<ALIGNED>(vA, 16 * c + 2 * l8, rank, keep) : make_double2(0.0, 0.0);
-                    xB[c] = actB ? ld_pair<ALIGNED>(vB, 16 * c + 2 * l8, rank, keep) : make_double2(0.0, 0.0);
+                    xA[c] = actA ? ld_pair_cached<ALIGNED>(vA, 16 * c + 2 * l8, rank) : make_double2(0.0, 0.0);
+                    xB[c] = actB ? ld_pair_cached<ALIGNED>(vB, 16 * c + 2 * l8, rank) : make_double2(0.0, 0.0);
                 }
                 double dA = 0.0, dB = 0.0;
 #pragma unroll
@@ -205,7 +159,7 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
                     if (act) {
 #pragma unroll
                         for (int c = 0; c < NK2; ++c) {
-                            const double2 x = ld_pair<ALIGNED>(vj, 16 * c + 2 * l8, rank, keep);
+                            const double2 x = ld_pair_cached<ALIGNED>(vj, 16 * c + 2 * l8, rank);
                             racc[c].x = fma(ww, x.x, racc[c].x);
                             racc[c].y = fma(ww, x.y, racc[c].y);
                         }
@@ -325,8 +279,7 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
 
     const int sms = sm_count();
     if (sms <= 0) return cuda_fail(cudaErrorNoDevice);
-    const bool aligned = aligned16(U->data) && aligned16(V->data) && U->ld % 2 == 0 && V->ld % 2 == 0 &&
-                         rank % 2 == 0;
+    const bool aligned = aligned16(U->data) && aligned16(V->data) && U->ld % 2 == 0 && V->ld % 2 == 0;
     long long grid = (long long)sms * 8;
     const long long by_rows = (X->rows + 7) / 8;
     if (grid > by_rows) grid = by_rows;
