@@ -7,6 +7,8 @@
 // The row U_i sits in registers, spread over the 8 lanes of a group; the four
 // groups of a warp take different stored cells of the row and gather their V_j
 // rows with 128-bit loads (V is read many times and stays in L2).
+#include <stdlib.h>
+
 #include "chain.cuh"
 
 namespace fo {
@@ -193,6 +195,165 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
     }
 }
 
+// ------------------------------------------------------------------ staged
+// The same work with the V rows landing in shared memory first.  A warp owns a
+// buffer of 16 rows; for half a chunk (16 stored cells) it issues all the 16-byte
+// asynchronous copies of the 16 V rows at once, waits for them, and only then
+// forms the dot products from shared memory.  The copies need no registers, so a
+// warp keeps 16 rows (12.8 KB at rank 100) in flight instead of 8, and the right_mm
+// variant reuses the staged rows instead of gathering them twice.
+// Needs 16-byte aligned factor rows and an even rank (a row piece is one 16-byte copy).
+constexpr int kStageRows = 16;
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
+{
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+
+template <int NK2, int AGG>
+__global__ void __launch_bounds__(kThreads, 2)
+outer_staged_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ double s_red[32];
+    __shared__ unsigned int s_flag;
+    __shared__ long long s_rows[2];
+
+    if (threadIdx.x == 0) {
+        const long long G = gridDim.x, b = blockIdx.x;
+        s_rows[0] = (b == 0) ? 0 : lower_row(p.rowptr, p.rows, (p.nnz * b) / G);
+        s_rows[1] = (b == G - 1) ? p.rows : lower_row(p.rowptr, p.rows, (p.nnz * (b + 1)) / G);
+    }
+    __syncthreads();
+    const long long row_lo = s_rows[0], row_hi = s_rows[1];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int l8 = lane & 7, grp = lane >> 3;
+    const unsigned full = 0xffffffffu;
+    const int rank = p.rank;                       // even
+    double *buf = reinterpret_cast<double *>(smem_raw) + (size_t)warp * kStageRows * rank;
+    double acc = 0.0;
+
+    for (long long row = row_lo + warp; row < row_hi; row += kThreads / 32) {
+        const int beg = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
+        double2 u[NK2], racc[NK2];
+        const double *urow = p.U + row * p.ldu;
+#pragma unroll
+        for (int c = 0; c < NK2; ++c) {
+            const int col = 16 * c + 2 * l8;
+            u[c] = (beg < end && col < rank) ? __ldg(reinterpret_cast<const double2 *>(urow + col))
+                                             : make_double2(0.0, 0.0);
+            racc[c] = make_double2(0.0, 0.0);
+        }
+        for (int c0 = beg; c0 < end; c0 += 32) {
+            const int cnt = (end - c0 < 32) ? end - c0 : 32;
+            const bool valid = lane < cnt;
+            const int jmine = valid ? __ldg(p.colidx + c0 + lane) : 0;
+            const double amine = valid ? __ldg(p.vals + c0 + lane) : 0.0;
+            double dmine = 0.0, wmine = 0.0;
+            for (int h = 0; h < 2 && 16 * h < cnt; ++h) {
+                // land the V rows of cells 16h .. 16h+15: group grp takes cells 16h + 4i + grp
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int sidx = 16 * h + 4 * i + grp;
+                    const int j = __shfl_sync(full, jmine, sidx);
+                    if (sidx < cnt) {
+                        const double *vj = p.V + (long long)j * p.ldv;
+                        double *dst = buf + (4 * i + grp) * rank;
+#pragma unroll
+                        for (int c = 0; c < NK2; ++c) {
+                            const int col = 16 * c + 2 * l8;
+                            if (col < rank) cp_async16(dst + col, vj + col);
+                        }
+                    }
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int sidx = 16 * h + 4 * i + grp;
+                    const double *src = buf + (4 * i + grp) * rank;
+                    double d = 0.0;
+                    if (sidx < cnt) {
+#pragma unroll
+                        for (int c = 0; c < NK2; ++c) {
+                            const int col = 16 * c + 2 * l8;
+                            if (col < rank) {
+                                const double2 x = *reinterpret_cast<const double2 *>(src + col);
+                                d = fma(u[c].x, x.x, d);
+                                d = fma(u[c].y, x.y, d);
+                            }
+                        }
+                    }
+                    d += __shfl_xor_sync(full, d, 4);
+                    d += __shfl_xor_sync(full, d, 2);
+                    d += __shfl_xor_sync(full, d, 1);
+                    // cell s of the chunk was handled by group (s & 3) in trip (s >> 2)
+                    const double all = __shfl_sync(full, d, (lane & 3) * 8);
+                    if ((lane >> 2) == 4 * h + i) dmine = all;
+                }
+                if (AGG == kOutRight) {
+                    // the chain's values for this half, then O_i += w * V_j from the staged rows
+                    const double w = outer_chain(ch, amine, dmine);
+                    if ((lane >> 4) == h) wmine = w;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int sidx = 16 * h + 4 * i + grp;
+                        const double ww = __shfl_sync(full, w, sidx);
+                        const double *src = buf + (4 * i + grp) * rank;
+                        if (sidx < cnt) {
+#pragma unroll
+                            for (int c = 0; c < NK2; ++c) {
+                                const int col = 16 * c + 2 * l8;
+                                if (col < rank) {
+                                    const double2 x = *reinterpret_cast<const double2 *>(src + col);
+                                    racc[c].x = fma(ww, x.x, racc[c].x);
+                                    racc[c].y = fma(ww, x.y, racc[c].y);
+                                }
+                            }
+                        }
+                    }
+                }
+                __syncwarp();          // the buffer is overwritten by the next half
+            }
+            if (AGG != kOutRight) {
+                const double w = outer_chain(ch, amine, dmine);
+                if (AGG == kOutFull) {
+                    if (valid) acc += w;
+                } else {
+                    if (valid) p.out[c0 + lane] = w;
+                }
+            }
+            (void)wmine;
+        }
+        if (AGG == kOutRight) {
+            // the four groups hold partial rows: add them in a fixed order
+#pragma unroll
+            for (int c = 0; c < NK2; ++c) {
+                racc[c].x += __shfl_xor_sync(full, racc[c].x, 8);
+                racc[c].y += __shfl_xor_sync(full, racc[c].y, 8);
+                racc[c].x += __shfl_xor_sync(full, racc[c].x, 16);
+                racc[c].y += __shfl_xor_sync(full, racc[c].y, 16);
+                const int col = 16 * c + 2 * l8;
+                if (grp == 0) {
+                    if (col < rank) p.out[row * rank + col] = racc[c].x;
+                    if (col + 1 < rank) p.out[row * rank + col + 1] = racc[c].y;
+                }
+            }
+        }
+    }
+
+    if (AGG == kOutFull) {
+        double v1[1] = {acc};
+        block_sum<1>(v1, s_red);
+        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
+    }
+}
+
 __global__ void outer_fill_zero_kernel(double *out, long long n)
 {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -216,6 +377,22 @@ cudaError_t launch_outer(const DevChain &ch, const OuterParams &p, int agg, bool
     else FO_GO(kOutRight);
 #undef FO_GO
     return cudaGetLastError();
+}
+
+template <int NK2>
+cudaError_t launch_outer_staged(const DevChain &ch, const OuterParams &p, int agg, int grid,
+                                cudaStream_t st)
+{
+    const size_t smem = (size_t)(kThreads / 32) * kStageRows * p.rank * sizeof(double);
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, kThreads, smem, st>>>(ch, p);
+        return cudaGetLastError();
+    };
+    if (agg == FO_OUTER_FULL_AGG) return go(outer_staged_kernel<NK2, kOutFull>);
+    if (agg == FO_OUTER_NO_AGG) return go(outer_staged_kernel<NK2, kOutNone>);
+    return go(outer_staged_kernel<NK2, kOutRight>);
 }
 
 }  // namespace
@@ -288,6 +465,16 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
 
     cudaError_t e;
     const int nk2 = (rank + 15) / 16;
+    // factor rows that are 16-byte aligned pieces go through the staged kernel
+    const bool staged = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && !getenv("FUSEDOPS_OUTER_DIRECT");
+    if (staged) {
+        if (nk2 <= 1) e = launch_outer_staged<1>(ch, p, agg, (int)grid, st);
+        else if (nk2 <= 2) e = launch_outer_staged<2>(ch, p, agg, (int)grid, st);
+        else if (nk2 <= 4) e = launch_outer_staged<4>(ch, p, agg, (int)grid, st);
+        else if (nk2 <= 7) e = launch_outer_staged<7>(ch, p, agg, (int)grid, st);
+        else e = launch_outer_staged<8>(ch, p, agg, (int)grid, st);
+        return e == cudaSuccess ? FO_OK : cuda_fail(e);
+    }
     if (nk2 <= 1) e = launch_outer<1>(ch, p, agg, aligned, (int)grid, st);
     else if (nk2 <= 2) e = launch_outer<2>(ch, p, agg, aligned, (int)grid, st);
     else if (nk2 <= 4) e = launch_outer<4>(ch, p, agg, aligned, (int)grid, st);
