@@ -36,6 +36,17 @@ WD = [("mul", "t0", "side0", "d")]
 WSLOSS = [("ne", "t0", "a", 0.0), ("sub", "t1", "a", "d"), ("mul", "t2", "t1", "t1"),
           ("mul", "t3", "t0", "t2")]
 
+# dram__bytes_read.sum + dram__bytes_write.sum per unit of work, from the ncu captures summarised
+# under profiles/ (row_dense: 200 000 x 1000 capture, per row; traffic grows in proportion to the
+# rows).  A kernel that changed since its capture is listed as None.
+NCU_DRAM_BYTES_PER_UNIT = {
+    "cell": 24.013e6 / 1e6,                      # per cell (3 inputs)
+    "magg": (480.018e6 + 3.807e6) / 2e7,         # per cell (3 inputs)
+    "row_dense": (1601.676e6 + 7.674e6) / 2e5,   # per row of 1000 columns
+    "row_csr": (264.058e6 + 4.077e6) / 19998162, # per stored cell (2 000 000 x 1000 @ 0.01 capture)
+    "outer": None,                               # kernel changed since the capture
+}
+
 FULL = {
     "cell": dict(rows=1000, cols=1000),
     "magg": dict(rows=1_000_000, cols=100),
@@ -186,6 +197,60 @@ class Step:
             self.run(name)
             if events is not None:
                 events[i][1].record()
+
+
+def time_variants(fo, step, shapes, reps=10):
+    """Other variants of the four templates on the inputs already resident (not part
+    of the timed step): CUDA events, `reps` runs each after 2 warm-ups, inputs larger
+    than L2.  Returns {name: {ms, gbs, bytes}}."""
+    import torch
+    d = step.d
+    mr, mc = shapes["magg"]["rows"], shapes["magg"]["cols"]
+    rr, rc = shapes["row_dense"]["rows"], shapes["row_dense"]["cols"]
+    orow, rank = shapes["outer"]["rows"], shapes["outer"]["rank"]
+    nnz5 = step.csr5.nnz
+    sides = [("cell", d["magg.Y"]), ("cell", d["magg.Z"])]
+    dev = d["magg.X"].device
+    o_row = torch.empty(mr, dtype=torch.float64, device=dev)
+    o_col = torch.empty(mc, dtype=torch.float64, device=dev)
+    o_all = torch.empty((mr, mc), dtype=torch.float64, device=dev)
+    o_one = torch.empty(1, dtype=torch.float64, device=dev)
+    o_rr = torch.empty(rr, dtype=torch.float64, device=dev)
+    o_nnz = torch.empty(nnz5, dtype=torch.float64, device=dev)
+    o_right = torch.empty((orow, rank), dtype=torch.float64, device=dev)
+    generic = [("sub", "t0", "a", "side0"), ("abs", "t1", "t0"), ("fma", "t2", "t1", "side1", 0.5)]
+    in3 = 3 * 8 * mr * mc
+    outer_in = 12 * nnz5 + 4 * (orow + 1) + 8 * rank * (orow + shapes["outer"]["cols"])
+    cases = [
+        ("cell_row_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="row", out=o_row), in3 + 8 * mr),
+        ("cell_col_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="col", out=o_col), in3 + 8 * mc),
+        ("cell_no_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="none", out=o_all), in3 + 8 * mr * mc),
+        ("cell_full_agg_interpreted_chain",
+         lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="full", out=o_one), in3 + 8),
+        ("row_dense_row_agg", lambda: fo.fused_row(WD, "t0", d["row_dense.X"], d["row_dense.v"],
+                                                   [("row", d["row_dense.w"])], agg="row", out=o_rr),
+         8 * rr * rc + 16 * rr + 8 * rc),
+        ("row_dense_full_agg", lambda: fo.fused_row(WD, "t0", d["row_dense.X"], d["row_dense.v"],
+                                                    [("row", d["row_dense.w"])], agg="full", out=o_one),
+         8 * rr * rc + 8 * rr + 8 * rc),
+        ("outer_no_agg", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
+                                                agg="none", out=o_nnz), outer_in + 8 * nnz5),
+        ("outer_right_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
+                                                  agg="right", out=o_right), outer_in + 8 * orow * rank),
+    ]
+    res = {}
+    for name, fn, nbytes in cases:
+        for _ in range(2):
+            fn()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, b in ev:
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize()
+        ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
+        res[name] = {"ms": ms, "bytes": nbytes, "gbs": nbytes / (ms * 1e-3) / 1e9}
+    return res
 
 
 # ---------------------------------------------------------------------- clocks
@@ -495,10 +560,17 @@ def run_ours(args):
     per_op["row_csr"]["nnz_per_s"] = nnz4 / (per_op["row_csr"]["ms"] * 1e-3)
     per_op["outer"]["nnz_per_s"] = nnz5 / (per_op["outer"]["ms"] * 1e-3)
     dominant = max(sorted(step.enabled), key=lambda n: per_op[n]["ms"])
-    traffic = None
+    units = {"cell": shapes["cell"]["rows"] * shapes["cell"]["cols"],
+             "magg": shapes["magg"]["rows"] * shapes["magg"]["cols"],
+             "row_dense": shapes["row_dense"]["rows"], "row_csr": nnz4, "outer": nnz5}
+    per_unit = NCU_DRAM_BYTES_PER_UNIT.get(dominant)
+    traffic = per_unit * units[dominant] if per_unit is not None and args.frac == 1.0 else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": per_op[dominant]["gbs"], "peak": peak_gbs,
                 "peak_kind": peak_kind, "unit": "GB/s", "frac": per_op[dominant]["gbs"] / peak_gbs,
-                "traffic": traffic}
+                "traffic": traffic, "algorithmic_bytes": nbytes[dominant]}
+    roofline_per_op = {n: {"bound": "hbm", "achieved": per_op[n]["gbs"], "peak": peak_gbs, "unit": "GB/s",
+                           "frac": per_op[n]["gbs"] / peak_gbs, "algorithmic_bytes": nbytes[n]}
+                       for n in OPS if n in step.enabled}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -515,11 +587,15 @@ def run_ours(args):
                 "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
         "gpu_launches": gpu_launches,
         "roofline": roofline,
+        "roofline_per_op": roofline_per_op,
         "per_op": per_op,
         "device_status": status,
         "results": {k: [float(x) for x in v.reshape(-1)[:3]] for k, v in results.items()},
         "input_generation_s": t_gen,
     }
+
+    if not args.no_variants and step.enabled == set(OPS):
+        line["variants"] = time_variants(fo, step, shapes)
 
     # ---- CPU baseline: the checker on a bounded sample, rank 0 at N = 1 only
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -544,14 +620,15 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--frac", type=float, default=1.0, help="scale the row counts (debugging)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-frac", type=float, default=0.5, help="sample of the workloads the CPU baseline runs")
+    ap.add_argument("--cpu-frac", type=float, default=1.0, help="sample of the workloads the CPU baseline runs")
     ap.add_argument("--ref-frac", type=float, default=0.01, help="sample per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the untimed-step variant measurements")
     ap.add_argument("--full-outer", action="store_true", help="keep the Outer workload at full size under --frac")
     ap.add_argument("--ops", default="", help="comma-separated subset of the five operators (profiling)")
     ap.add_argument("--interp", action="store_true", help="run Cell / MAgg chains through the interpreter")
