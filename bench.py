@@ -219,14 +219,24 @@ def time_variants(fo, step, shapes, reps=10):
     o_nnz = torch.empty(nnz5, dtype=torch.float64, device=dev)
     o_right = torch.empty((orow, rank), dtype=torch.float64, device=dev)
     generic = [("sub", "t0", "a", "side0"), ("abs", "t1", "t0"), ("fma", "t2", "t1", "side1", 0.5)]
+
+    def interpreted(fn):
+        fo.force_interpreter(True)
+        try:
+            fn()
+        finally:
+            fo.force_interpreter(False)
+
     in3 = 3 * 8 * mr * mc
     outer_in = 12 * nnz5 + 4 * (orow + 1) + 8 * rank * (orow + shapes["outer"]["cols"])
     cases = [
         ("cell_row_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="row", out=o_row), in3 + 8 * mr),
         ("cell_col_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="col", out=o_col), in3 + 8 * mc),
         ("cell_no_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="none", out=o_all), in3 + 8 * mr * mc),
-        ("cell_full_agg_interpreted_chain",
+        ("cell_full_agg_runtime_compiled_chain",
          lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="full", out=o_one), in3 + 8),
+        ("cell_full_agg_interpreted_chain", lambda: interpreted(
+            lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="full", out=o_one)), in3 + 8),
         ("row_dense_row_agg", lambda: fo.fused_row(WD, "t0", d["row_dense.X"], d["row_dense.v"],
                                                    [("row", d["row_dense.w"])], agg="row", out=o_rr),
          8 * rr * rc + 16 * rr + 8 * rc),

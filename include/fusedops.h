@@ -174,6 +174,28 @@ int fo_last_cuda_error(void);
  * (process-wide; for tests and measurements).  Returns the previous setting. */
 int fo_set_force_interpreter(int on);
 
+/* Run-time specialisation (the paper's template expansion to source, compilation
+ * and plan cache, Section 2.1 "Codegen Architecture").  A Cell / MAgg chain over
+ * contiguous inputs (full_agg, MAgg, no_agg) that has no built-in specialisation
+ * is written out as straight-line code inside the library's streaming kernel,
+ * compiled for the current GPU with NVRTC on first use (a few hundred ms) and
+ * cached by its translated program for the life of the process; later calls
+ * with the same chain - whatever the values of its scalars and immediates - reuse
+ * it.  Results are bit-identical to the interpreter's.  NVRTC and the driver
+ * library are loaded on demand; if they are missing or a compilation fails the
+ * interpreter runs instead, so behaviour never depends on them.
+ *   fo_set_jit(on)   switches the mechanism (default on); returns the old setting.
+ *   fo_jit_stats()   kernels compiled, specialised launches, failed compilations so
+ *                    far; returns 1 if NVRTC and the driver library are usable.
+ *   fo_jit_compile_check()  generates and compiles (for sm_100a, without loading or
+ *                    launching: no GPU needed) the kernel of a Cell chain; FO_OK,
+ *                    a chain error, FO_ERR_UNSUPPORTED without NVRTC; the compiler
+ *                    log is copied to `log`. */
+int fo_set_jit(int on);
+int fo_jit_stats(int *compiled, int *launches, int *failures);
+int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int store,
+                         char *log, size_t log_bytes);
+
 /* ------------------------------------------------------------------ Cell
  * Table 1, Cell template; Section 2.2 cell-wise listing.
  * For every cell (i, j) of a dense main input X (for a CSR main input: every

@@ -5,11 +5,11 @@ The work happens in ``libfusedops.so`` (CUDA, sm_100a; C ABI in
 """
 from .binding import (  # noqa: F401
     CSR, FusedOpsError, device_status, force_interpreter, fused_cell, fused_cell_static, fused_magg, fused_outer, fused_row,
-    load_library, make_chain, workspace,
+    jit_compile_check, jit_stats, load_library, make_chain, set_jit, workspace,
 )
 from .roofline import algorithmic_bytes, ideal_seconds  # noqa: F401
 
 __all__ = [
     "CSR", "FusedOpsError", "device_status", "force_interpreter", "fused_cell", "fused_cell_static", "fused_magg", "fused_outer",
-    "fused_row", "load_library", "make_chain", "workspace", "algorithmic_bytes", "ideal_seconds",
+    "fused_row", "jit_compile_check", "jit_stats", "set_jit", "load_library", "make_chain", "workspace", "algorithmic_bytes", "ideal_seconds",
 ]

@@ -80,6 +80,7 @@ EXPORTS = [
     "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
+    "fo_set_jit", "fo_jit_stats", "fo_jit_compile_check",
 ]
 
 _lib = None
@@ -122,6 +123,13 @@ def load_library(path=None):
         lib.fused_cell_static.restype = C.c_int
         lib.fused_cell_static_limit_bytes.argtypes = []
         lib.fused_cell_static_limit_bytes.restype = C.c_size_t
+        lib.fo_set_jit.argtypes = [C.c_int]
+        lib.fo_set_jit.restype = C.c_int
+        ip = C.POINTER(C.c_int)
+        lib.fo_jit_stats.argtypes = [ip, ip, ip]
+        lib.fo_jit_stats.restype = C.c_int
+        lib.fo_jit_compile_check.argtypes = [chain_p, i32, i32, i32, C.c_char_p, sz]
+        lib.fo_jit_compile_check.restype = C.c_int
         lib.fo_set_force_interpreter.argtypes = [C.c_int]
         lib.fo_set_force_interpreter.restype = C.c_int
         if path is None:
@@ -308,6 +316,27 @@ def force_interpreter(on):
     """Route every Cell / MAgg chain through the interpreter (True) or let known
     chains use their compile-time specialisation (False).  Returns the old setting."""
     return bool(load_library().fo_set_force_interpreter(1 if on else 0))
+
+
+def set_jit(on):
+    """Switches run-time specialisation of Cell / MAgg chains on or off; returns the old setting."""
+    return bool(load_library().fo_set_jit(1 if on else 0))
+
+
+def jit_stats():
+    """(usable, kernels compiled, specialised launches, failed compilations)."""
+    a, b, c = C.c_int(0), C.c_int(0), C.c_int(0)
+    ok = load_library().fo_jit_stats(C.byref(a), C.byref(b), C.byref(c))
+    return bool(ok), a.value, b.value, c.value
+
+
+def jit_compile_check(steps, outputs, n_sides=0, n_scalars=0, store=False):
+    """Generates and compiles the specialised kernel of a Cell chain without running
+    it (no GPU needed).  Returns (status, compiler log)."""
+    ch, keep = make_chain(steps, outputs)
+    log = C.create_string_buffer(1 << 16)
+    rc = load_library().fo_jit_compile_check(C.byref(ch), n_sides, n_scalars, 1 if store else 0, log, len(log))
+    return rc, log.value.decode(errors="replace")
 
 
 def device_status(device=None):

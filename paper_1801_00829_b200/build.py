@@ -54,7 +54,7 @@ def is_stale() -> bool:
 def _compile_one(src: str, verbose: bool) -> str:
     obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
     log = obj + ".log"
-    cmd = [_nvcc()] + NVCC_FLAGS + ["-I", INCLUDE, "-c", src, "-o", obj]
+    cmd = [_nvcc()] + NVCC_FLAGS + ["-I", INCLUDE, "-I", OBJ_DIR, "-c", src, "-o", obj]
     res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
     with open(log, "w") as fh:
         fh.write(res.stdout)
@@ -65,16 +65,39 @@ def _compile_one(src: str, verbose: bool) -> str:
     return obj
 
 
+JIT_HEADERS = ["common.cuh", "cell_flat.cuh"]      # what a run-time specialised kernel is made of
+
+
+def _write_jit_source() -> None:
+    """Embeds the headers the run-time compiled kernels consist of as a C++ string
+    literal (_build/jit_source.inc), without their #include / #pragma once lines."""
+    chunks = []
+    for name in JIT_HEADERS:
+        with open(os.path.join(CSRC, name)) as fh:
+            lines = [l for l in fh.read().splitlines()
+                     if not l.lstrip().startswith("#include") and not l.lstrip().startswith("#pragma once")]
+        chunks.append("// ---- %s\n" % name + "\n".join(lines) + "\n")
+    text = "".join(chunks)
+    assert ')FOJIT"' not in text
+    out = []
+    step = 8000                                   # keep each literal well below compiler limits
+    for i in range(0, len(text), step):
+        out.append('R"FOJIT(' + text[i:i + step] + ')FOJIT"\n')
+    with open(os.path.join(OBJ_DIR, "jit_source.inc"), "w") as fh:
+        fh.write("".join(out))
+
+
 def build_library(force: bool = False, verbose: bool = False) -> str:
     """Compile (if needed) and return the path of libfusedops.so."""
     if not force and not is_stale():
         return LIB_PATH
     os.makedirs(OBJ_DIR, exist_ok=True)
+    _write_jit_source()
     srcs = _sources()
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, len(srcs))) as pool:
         objs = list(pool.map(lambda s: _compile_one(s, verbose), srcs))
     tmp = LIB_PATH + ".tmp%d" % os.getpid()
-    cmd = [_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs
+    cmd = [_nvcc(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs + ["-ldl"]
     res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
     if res.returncode != 0:
         raise RuntimeError("link failed:\n%s" % res.stdout[-4000:])

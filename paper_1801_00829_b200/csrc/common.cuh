@@ -1,11 +1,16 @@
 // Shared device/host helpers of the fused-operator kernels (sm_100a).
 #pragma once
 
+// This header is also compiled at run time (NVRTC) as part of specialised
+// kernels; there the system headers are not available, so the few fixed-width
+// types and the FO_* limits are supplied by the generated source instead.
+#ifndef __CUDACC_RTC__
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <string.h>
 
 #include "../../include/fusedops.h"
+#endif
 
 namespace fo {
 
@@ -67,6 +72,7 @@ struct DevSides {
     DevSide s[FO_MAX_SIDES];
 };
 
+#ifndef __CUDACC_RTC__
 // Host: validate a chain for a template and translate it (chain_host.cu).
 enum ChainUse { kUseCell, kUseRow, kUseOuter };
 int translate_chain(const fo_chain *chain, ChainUse use, int n_sides,
@@ -76,6 +82,7 @@ int translate_chain(const fo_chain *chain, ChainUse use, int n_sides,
 int check_workspace(const void *ws, size_t ws_bytes, size_t need);
 int cuda_fail(cudaError_t e);
 int sm_count();
+#endif
 
 #ifdef __CUDACC__
 // ------------------------------------------------------------ device helpers

@@ -1,0 +1,309 @@
+// Run-time specialisation of Cell / MAgg chains: the analogue of the paper's
+// template expansion to source code, compilation and plan cache (Section 2.1,
+// "Codegen Architecture").  A chain that has no built-in specialisation is
+// written out as a straight-line C++ functor, placed into the same flat
+// streaming kernel the library compiles ahead of time (cell_flat.cuh), compiled
+// for the current device with NVRTC and cached by the chain's translated program.
+// NVRTC and the driver API are looked up with dlopen at first use; if either is
+// missing, or a compilation fails, the caller falls back to the interpreter.
+#include <dlfcn.h>
+#include <stdio.h>
+
+#include <mutex>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "cell_flat.cuh"
+#include "jit.h"
+
+namespace fo {
+
+namespace {
+
+const char kSkeleton[] =
+#include "jit_source.inc"
+    ;
+
+// ---- the few NVRTC / driver entry points used, declared here so that neither
+// library is needed at link time
+typedef struct _nvrtcProgram *nvrtcProgram;
+typedef int (*nvrtcCreateProgram_t)(nvrtcProgram *, const char *, const char *, int, const char *const *,
+                                    const char *const *);
+typedef int (*nvrtcCompileProgram_t)(nvrtcProgram, int, const char *const *);
+typedef int (*nvrtcGetSize_t)(nvrtcProgram, size_t *);
+typedef int (*nvrtcGetData_t)(nvrtcProgram, char *);
+typedef int (*nvrtcDestroyProgram_t)(nvrtcProgram *);
+typedef struct CUmod_st *CUmodule;
+typedef struct CUfunc_st *CUfunction;
+typedef int (*cuModuleLoadData_t)(CUmodule *, const void *);
+typedef int (*cuModuleGetFunction_t)(CUfunction *, CUmodule, const char *);
+typedef int (*cuLaunchKernel_t)(CUfunction, unsigned, unsigned, unsigned, unsigned, unsigned, unsigned,
+                                unsigned, void *, void **, void **);
+
+struct Api {
+    bool nvrtc_ok = false, driver_ok = false;
+    nvrtcCreateProgram_t create = nullptr;
+    nvrtcCompileProgram_t compile = nullptr;
+    nvrtcGetSize_t cubin_size = nullptr, log_size = nullptr;
+    nvrtcGetData_t cubin = nullptr, log = nullptr;
+    nvrtcDestroyProgram_t destroy = nullptr;
+    cuModuleLoadData_t load = nullptr;
+    cuModuleGetFunction_t getfn = nullptr;
+    cuLaunchKernel_t launch = nullptr;
+};
+
+void *open_first(const char *const *names)
+{
+    for (; *names; ++names) {
+        void *h = dlopen(*names, RTLD_NOW | RTLD_GLOBAL);
+        if (h) return h;
+    }
+    return nullptr;
+}
+
+Api &api()
+{
+    static Api a;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        const char *nv[] = {"libnvrtc.so.12", "libnvrtc.so", "/usr/local/cuda/lib64/libnvrtc.so.12",
+                            "/usr/local/cuda/lib64/libnvrtc.so", nullptr};
+        if (void *h = open_first(nv)) {
+            a.create = (nvrtcCreateProgram_t)dlsym(h, "nvrtcCreateProgram");
+            a.compile = (nvrtcCompileProgram_t)dlsym(h, "nvrtcCompileProgram");
+            a.cubin_size = (nvrtcGetSize_t)dlsym(h, "nvrtcGetCUBINSize");
+            a.cubin = (nvrtcGetData_t)dlsym(h, "nvrtcGetCUBIN");
+            a.log_size = (nvrtcGetSize_t)dlsym(h, "nvrtcGetProgramLogSize");
+            a.log = (nvrtcGetData_t)dlsym(h, "nvrtcGetProgramLog");
+            a.destroy = (nvrtcDestroyProgram_t)dlsym(h, "nvrtcDestroyProgram");
+            a.nvrtc_ok = a.create && a.compile && a.cubin_size && a.cubin && a.log_size && a.log && a.destroy;
+        }
+        const char *cu[] = {"libcuda.so.1", "libcuda.so", nullptr};
+        if (void *h = open_first(cu)) {
+            a.load = (cuModuleLoadData_t)dlsym(h, "cuModuleLoadData");
+            a.getfn = (cuModuleGetFunction_t)dlsym(h, "cuModuleGetFunction");
+            a.launch = (cuLaunchKernel_t)dlsym(h, "cuLaunchKernel");
+            a.driver_ok = a.load && a.getfn && a.launch;
+        }
+    });
+    return a;
+}
+
+std::mutex g_mutex;
+std::unordered_map<std::string, CUfunction> g_cache;      // key: device + translated program
+bool g_enabled = true;
+int g_compiled = 0, g_launches = 0, g_failures = 0;
+std::string g_last_log;
+
+// ---- source generation
+std::string operand_text(int opnd)
+{
+    char buf[32];
+    if (opnd & 0x80) snprintf(buf, sizeof(buf), "c[%d]", opnd & 0x7f);
+    else snprintf(buf, sizeof(buf), "R%d", opnd);
+    return buf;
+}
+
+std::string op_text(const DevOp &op)
+{
+    const std::string a = operand_text(op.a), b = operand_text(op.b), c = operand_text(op.c);
+    switch (op.opcode) {
+        case FO_OP_MOV: return a;
+        case FO_OP_NEG: return "-" + a;
+        case FO_OP_ABS: return "fabs(" + a + ")";
+        case FO_OP_SQRT: return "sqrt(" + a + ")";
+        case FO_OP_EXP: return "exp(" + a + ")";
+        case FO_OP_LOG: return "log(" + a + ")";
+        case FO_OP_SQ: return a + " * " + a;
+        case FO_OP_ADD: return a + " + " + b;
+        case FO_OP_SUB: return a + " - " + b;
+        case FO_OP_MUL: return a + " * " + b;
+        case FO_OP_DIV: return a + " / " + b;
+        case FO_OP_MIN: return "fmin(" + a + ", " + b + ")";
+        case FO_OP_MAX: return "fmax(" + a + ", " + b + ")";
+        case FO_OP_POW: return "pow(" + a + ", " + b + ")";
+        case FO_OP_EQ: return a + " == " + b + " ? 1.0 : 0.0";
+        case FO_OP_NE: return a + " != " + b + " ? 1.0 : 0.0";
+        case FO_OP_LT: return a + " < " + b + " ? 1.0 : 0.0";
+        case FO_OP_LE: return a + " <= " + b + " ? 1.0 : 0.0";
+        case FO_OP_GT: return a + " > " + b + " ? 1.0 : 0.0";
+        case FO_OP_GE: return a + " >= " + b + " ? 1.0 : 0.0";
+        case FO_OP_SEL: return a + " != 0.0 ? " + b + " : " + c;
+        case FO_OP_FMA: return "fma(" + a + ", " + b + ", " + c + ")";
+        default: return "0.0";
+    }
+}
+
+std::string generate_source(const DevChain &ch, bool store)
+{
+    char buf[512];
+    std::string s;
+    // what the system headers and fusedops.h provide in the ahead-of-time build
+    snprintf(buf, sizeof(buf),
+             "typedef unsigned char uint8_t;\ntypedef int int32_t;\ntypedef unsigned int uint32_t;\n"
+             "#define FO_MAX_OPS %d\n#define FO_MAX_TMPS %d\n#define FO_MAX_SIDES %d\n"
+             "#define FO_MAX_SCALARS %d\n#define FO_MAX_OUT %d\n",
+             FO_MAX_OPS, FO_MAX_TMPS, FO_MAX_SIDES, FO_MAX_SCALARS, FO_MAX_OUT);
+    s += buf;
+    s += kSkeleton;
+    snprintf(buf, sizeof(buf),
+             "static_assert(sizeof(fo::DevChain) == %zu, \"chain layout\");\n"
+             "static_assert(sizeof(fo::CellParams) == %zu, \"parameter layout\");\n",
+             sizeof(DevChain), sizeof(CellParams));
+    s += buf;
+    s += "struct JitFn {\n";
+    snprintf(buf, sizeof(buf), "    static constexpr unsigned kSideMask = %uu;\n    static constexpr int kOut = %d;\n",
+             ch.side_used, ch.n_out);
+    s += buf;
+    s += "    __device__ __forceinline__ static void eval(const double *in, const double *c, double *o)\n    {\n";
+    for (int r = 0; r < ch.tmp_base; ++r) {
+        snprintf(buf, sizeof(buf), "        const double R%d = in[%d];\n", r, r);
+        s += buf;
+    }
+    for (int r = ch.tmp_base; r < ch.n_regs; ++r) {
+        snprintf(buf, sizeof(buf), "        double R%d;\n", r);
+        s += buf;
+    }
+    for (int k = 0; k < ch.n_ops; ++k) {
+        snprintf(buf, sizeof(buf), "        R%d = ", ch.ops[k].dst);
+        s += buf;
+        s += op_text(ch.ops[k]) + ";\n";
+    }
+    for (int k = 0; k < ch.n_out; ++k) {
+        snprintf(buf, sizeof(buf), "        o[%d] = ", k);
+        s += buf;
+        s += operand_text(ch.out[k]) + ";\n";
+    }
+    s += "        (void)c; (void)in;\n    }\n};\n";
+    snprintf(buf, sizeof(buf),
+             "extern \"C\" __global__ void __launch_bounds__(%d)\n"
+             "fo_jit_flat(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::CellParams p)\n"
+             "{\n    fo::cell_flat_body<fo::EvalFn<JitFn>, %d, %s>(ch, p);\n}\n",
+             kThreads, ch.n_out, store ? "true" : "false");
+    s += buf;
+    return s;
+}
+
+std::string cache_key(const DevChain &ch, bool store, int dev)
+{
+    std::string k;
+    k.append((const char *)&dev, sizeof(dev));
+    k.push_back(store ? 1 : 0);
+    k.append((const char *)&ch.n_ops, sizeof(int32_t));
+    k.append((const char *)&ch.n_out, sizeof(int32_t));
+    k.append((const char *)&ch.n_regs, sizeof(int32_t));
+    k.append((const char *)&ch.tmp_base, sizeof(int32_t));
+    k.append((const char *)&ch.side_used, sizeof(uint32_t));
+    k.append((const char *)ch.out, sizeof(ch.out));
+    k.append((const char *)ch.ops, sizeof(DevOp) * (size_t)ch.n_ops);
+    return k;
+}
+
+// Compiles `src` for `arch`; returns the CUBIN (empty on failure, log in g_last_log).
+std::vector<char> compile(const std::string &src, const std::string &arch)
+{
+    std::vector<char> cubin;
+    Api &a = api();
+    nvrtcProgram prog = nullptr;
+    if (a.create(&prog, src.c_str(), "fo_jit.cu", 0, nullptr, nullptr) != 0) {
+        g_last_log = "nvrtcCreateProgram failed";
+        return cubin;
+    }
+    const std::string archopt = "--gpu-architecture=" + arch;
+    const char *opts[] = {archopt.c_str(), "--std=c++17", "--fmad=false"};
+    const int rc = a.compile(prog, 3, opts);
+    size_t n = 0;
+    if (a.log_size(prog, &n) == 0 && n > 1) {
+        g_last_log.resize(n);
+        a.log(prog, &g_last_log[0]);
+    } else {
+        g_last_log.clear();
+    }
+    if (rc == 0 && a.cubin_size(prog, &n) == 0 && n > 0) {
+        cubin.resize(n);
+        if (a.cubin(prog, cubin.data()) != 0) cubin.clear();
+    }
+    a.destroy(&prog);
+    return cubin;
+}
+
+}  // namespace
+
+bool jit_enabled() { return g_enabled; }
+
+int jit_launch_flat(const DevChain &ch, const CellParams &p, bool store, int grid, cudaStream_t st)
+{
+    Api &a = api();
+    if (!g_enabled || !a.nvrtc_ok || !a.driver_ok) return kJitUnavailable;
+    int dev = 0, major = 0, minor = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess)
+        return kJitUnavailable;
+    CUfunction fn = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        const std::string key = cache_key(ch, store, dev);
+        auto it = g_cache.find(key);
+        if (it != g_cache.end()) {
+            fn = it->second;
+        } else {
+            char arch[32];
+            snprintf(arch, sizeof(arch), "sm_%d%d%s", major, minor, major >= 9 ? "a" : "");
+            const std::vector<char> cubin = compile(generate_source(ch, store), arch);
+            CUmodule mod = nullptr;
+            if (!cubin.empty() && a.load(&mod, cubin.data()) == 0 && a.getfn(&fn, mod, "fo_jit_flat") == 0) {
+                ++g_compiled;
+            } else {
+                fn = nullptr;
+                ++g_failures;
+            }
+            g_cache.emplace(key, fn);         // a failed chain is not compiled again
+        }
+        if (fn) ++g_launches;
+    }
+    if (!fn) return kJitUnavailable;
+    void *args[2] = {(void *)&ch, (void *)&p};
+    const int rc = a.launch(fn, (unsigned)grid, 1, 1, kThreads, 1, 1, 0, (void *)st, args, nullptr);
+    return rc == 0 ? FO_OK : cuda_fail(cudaErrorLaunchFailure);
+}
+
+}  // namespace fo
+
+extern "C" {
+
+int fo_set_jit(int on)
+{
+    std::lock_guard<std::mutex> lock(fo::g_mutex);
+    const int prev = fo::g_enabled ? 1 : 0;
+    fo::g_enabled = on != 0;
+    return prev;
+}
+
+int fo_jit_stats(int *compiled, int *launches, int *failures)
+{
+    std::lock_guard<std::mutex> lock(fo::g_mutex);
+    if (compiled) *compiled = fo::g_compiled;
+    if (launches) *launches = fo::g_launches;
+    if (failures) *failures = fo::g_failures;
+    return (fo::api().nvrtc_ok && fo::api().driver_ok) ? 1 : 0;
+}
+
+int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int store, char *log,
+                         size_t log_bytes)
+{
+    using namespace fo;
+    if (log && log_bytes) log[0] = 0;
+    double scalars[FO_MAX_SCALARS] = {0};
+    DevChain ch;
+    const int rc = translate_chain(chain, kUseCell, n_sides, scalars, n_scalars, 1, FO_MAX_OUT, &ch);
+    if (rc != FO_OK) return rc;
+    if (!api().nvrtc_ok) return FO_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const std::vector<char> cubin = compile(generate_source(ch, store != 0), "sm_100a");
+    if (log && log_bytes) snprintf(log, log_bytes, "%s", g_last_log.c_str());
+    return cubin.empty() ? FO_ERR_CHAIN : FO_OK;
+}
+
+}  // extern "C"

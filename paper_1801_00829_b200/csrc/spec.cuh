@@ -10,6 +10,7 @@
 // runs through the interpreter.  Both give bit-identical results.
 #pragma once
 
+#include "cell_flat.cuh"
 #include "chain.cuh"
 
 namespace fo {
@@ -27,7 +28,6 @@ enum SpecId {
 // Host: specialisation matching a translated Cell / MAgg chain, or kSpecNone.
 int match_cell_spec(const DevChain &ch);
 
-constexpr int kIn = 1 + FO_MAX_SIDES;      // input slots: a, side0..side3
 
 template <int NR>
 struct EvalInterp {
@@ -67,26 +67,30 @@ struct SpecFn;
 
 template <>
 struct SpecFn<kSpecMul2> {
-    static constexpr int kSides = 1, kOut = 1;
-    __device__ __forceinline__ static void eval(const double *in, double *o) { o[0] = in[0] * in[1]; }
+    static constexpr unsigned kSideMask = 1u;
+    static constexpr int kOut = 1;
+    __device__ __forceinline__ static void eval(const double *in, const double *, double *o) { o[0] = in[0] * in[1]; }
 };
 template <>
 struct SpecFn<kSpecMul3> {
-    static constexpr int kSides = 2, kOut = 1;
-    __device__ __forceinline__ static void eval(const double *in, double *o)
+    static constexpr unsigned kSideMask = 3u;
+    static constexpr int kOut = 1;
+    __device__ __forceinline__ static void eval(const double *in, const double *, double *o)
     {
         o[0] = (in[0] * in[1]) * in[2];
     }
 };
 template <>
 struct SpecFn<kSpecSq> {
-    static constexpr int kSides = 0, kOut = 1;
-    __device__ __forceinline__ static void eval(const double *in, double *o) { o[0] = in[0] * in[0]; }
+    static constexpr unsigned kSideMask = 0u;
+    static constexpr int kOut = 1;
+    __device__ __forceinline__ static void eval(const double *in, const double *, double *o) { o[0] = in[0] * in[0]; }
 };
 template <>
 struct SpecFn<kSpecMagg2> {
-    static constexpr int kSides = 2, kOut = 2;
-    __device__ __forceinline__ static void eval(const double *in, double *o)
+    static constexpr unsigned kSideMask = 3u;
+    static constexpr int kOut = 2;
+    __device__ __forceinline__ static void eval(const double *in, const double *, double *o)
     {
         o[0] = in[0] * in[1];
         o[1] = in[0] * in[2];
@@ -94,8 +98,9 @@ struct SpecFn<kSpecMagg2> {
 };
 template <>
 struct SpecFn<kSpecMagg3> {
-    static constexpr int kSides = 2, kOut = 3;
-    __device__ __forceinline__ static void eval(const double *in, double *o)
+    static constexpr unsigned kSideMask = 3u;
+    static constexpr int kOut = 3;
+    __device__ __forceinline__ static void eval(const double *in, const double *, double *o)
     {
         o[0] = in[0] * in[1];
         o[1] = in[0] * in[2];
@@ -104,26 +109,6 @@ struct SpecFn<kSpecMagg3> {
 };
 
 template <int ID>
-struct EvalSpec {
-    using Fn = SpecFn<ID>;
-    static constexpr bool kInterp = false;
-    static constexpr int kOutMax = Fn::kOut;
-    __device__ __forceinline__ static bool uses_side(const DevChain &, int k) { return k < Fn::kSides; }
-    template <int V, int NOUT>
-    __device__ __forceinline__ static void run(const DevChain &, const double (&in)[kIn][V],
-                                               double (&o)[NOUT][V])
-    {
-        static_assert(NOUT >= Fn::kOut, "accumulator count");
-#pragma unroll
-        for (int i = 0; i < V; ++i) {
-            double x[kIn], y[Fn::kOut];
-#pragma unroll
-            for (int k = 0; k < kIn; ++k) x[k] = (k <= Fn::kSides) ? in[k][i] : 0.0;
-            Fn::eval(x, y);
-#pragma unroll
-            for (int k = 0; k < NOUT; ++k) o[k][i] = (k < Fn::kOut) ? y[k < Fn::kOut ? k : 0] : 0.0;
-        }
-    }
-};
+using EvalSpec = EvalFn<SpecFn<ID>>;
 
 }  // namespace fo

@@ -1,0 +1,103 @@
+"""Run-time specialised Cell / MAgg chains: the generated kernels compile (checked
+without a GPU) and, on a GPU, give the interpreter's bits, are cached by chain, and
+do not depend on the values of scalars and immediates."""
+import numpy as np
+import pytest
+
+import datagen
+import oracle
+from util import assert_close, to_dev
+
+import paper_1801_00829_b200 as fo
+
+CHAINS = {
+    "abs-fma": ([("sub", "t0", "a", "side0"), ("abs", "t1", "t0"), ("fma", "t2", "t1", "side1", 0.5)], ["t2"], 2, 0),
+    "scalars": ([("mul", "t0", "a", "s0"), ("add", "t1", "t0", "s1"), ("max", "t2", "t1", "side0")], ["t2"], 1, 2),
+    "cmp-sel": ([("gt", "t0", "a", "side0"), ("sel", "t1", "t0", "a", "side0"), ("min", "t2", "t1", 0.75)], ["t2"], 1, 0),
+    "math": ([("abs", "t0", "a"), ("add", "t1", "t0", 1.0), ("log", "t2", "t1"), ("exp", "t3", "t2"),
+              ("sqrt", "t4", "t3"), ("pow", "t5", "t4", 1.5), ("div", "t6", "t5", "t1"), ("neg", "t7", "t6")],
+             ["t7"], 0, 0),
+    "only-side1": ([("mul", "t0", "a", "side1")], ["t0"], 2, 0),
+    "magg5": ([("mul", "t0", "a", "side0"), ("sub", "t1", "a", "side0"), ("sq", "t2", "t1"),
+               ("eq", "t3", "a", "side0"), ("ne", "t4", "a", 0.0)], ["t0", "t1", "t2", "t3", "t4"], 1, 0),
+    "passthrough": ([], ["a"], 0, 0),
+}
+
+
+@pytest.mark.parametrize("name", sorted(CHAINS))
+@pytest.mark.parametrize("store", [False, True])
+def test_generated_kernels_compile_without_a_gpu(name, store):
+    steps, outs, n_sides, n_scalars = CHAINS[name]
+    if store and len(outs) > 1:
+        pytest.skip("no_agg has one result")
+    rc, log = fo.jit_compile_check(steps, outs, n_sides, n_scalars, store)
+    if rc == -4:
+        pytest.skip("NVRTC not available here")
+    assert rc == 0, log
+    assert "error" not in log
+
+
+def test_compile_check_rejects_bad_chain():
+    rc, _ = fo.jit_compile_check([("mul", "t0", "a", "t3")], ["t0"])
+    assert rc == -3
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", sorted(CHAINS))
+def test_jit_equals_interpreter_bitwise_and_checker(name):
+    steps, outs, n_sides, n_scalars = CHAINS[name]
+    rows, cols = 1031, 517                      # full tiles and a ragged tail
+    X = datagen.uniform(61, 0, rows * cols, -1.0, 2.0).reshape(rows, cols)
+    S = [datagen.uniform(61, 2 + k, rows * cols, -1.0, 2.0).reshape(rows, cols) for k in range(n_sides)]
+    scalars = [1.25, -0.5][:n_scalars]
+    sides_h = [("cell", s) for s in S]
+    Xd, sides = to_dev(X), [("cell", to_dev(s)) for s in S]
+    usable, c0, l0, f0 = fo.jit_stats()
+    if not usable:
+        pytest.skip("NVRTC or the driver library is not usable here")
+    got = fo.fused_magg(steps, outs, Xd, sides, scalars).cpu().numpy()
+    usable, c1, l1, f1 = fo.jit_stats()
+    assert f1 == f0, "a specialised kernel failed to compile"
+    assert l1 == l0 + 1 and c1 in (c0, c0 + 1)
+    again = fo.fused_magg(steps, outs, Xd, sides, scalars).cpu().numpy()
+    assert fo.jit_stats()[1] == c1                                   # cached: nothing compiled again
+    assert again.tobytes() == got.tobytes()
+    try:
+        fo.force_interpreter(True)
+        slow = fo.fused_magg(steps, outs, Xd, sides, scalars).cpu().numpy()
+    finally:
+        fo.force_interpreter(False)
+    assert got.tobytes() == slow.tobytes()
+    ref = oracle.magg(steps, outs, X, sides_h, scalars)
+    absref = oracle.magg(steps + [("abs", "t%d" % k, o) for k, o in enumerate(outs)],
+                         ["t%d" % k for k in range(len(outs))], X, sides_h, scalars)
+    assert_close(got, ref, absscale=absref + 1.0, what=name)
+    if len(outs) == 1:                                               # no_agg through the same mechanism
+        e = fo.fused_cell(steps, outs[0], Xd, sides, scalars, agg="none").cpu().numpy()
+        assert_close(e, oracle.cell(steps, outs[0], X, sides_h, scalars, agg="none"), what=name + " none")
+
+
+@pytest.mark.gpu
+def test_jit_kernel_is_reused_for_other_constants_and_can_be_switched_off():
+    rows, cols = 300, 700
+    X = datagen.normal(62, 0, rows * cols).reshape(rows, cols)
+    Xd = to_dev(X)
+    if not fo.jit_stats()[0]:
+        pytest.skip("NVRTC or the driver library is not usable here")
+
+    def chain(k):
+        return [("mul", "t0", "a", "s0"), ("add", "t1", "t0", k)]
+
+    a = fo.fused_cell(chain(2.0), "t1", Xd, scalars=[3.0]).item()
+    compiled = fo.jit_stats()[1]
+    b = fo.fused_cell(chain(-7.0), "t1", Xd, scalars=[0.25]).item()
+    assert fo.jit_stats()[1] == compiled                             # same program, other constants
+    assert_close([a], [oracle.cell(chain(2.0), "t1", X, scalars=[3.0])], absscale=np.abs(X).sum() * 3 + 2 * X.size)
+    assert_close([b], [oracle.cell(chain(-7.0), "t1", X, scalars=[0.25])], absscale=np.abs(X).sum() + 7 * X.size)
+    launches = fo.jit_stats()[2]
+    try:
+        fo.set_jit(False)
+        c = fo.fused_cell(chain(-7.0), "t1", Xd, scalars=[0.25]).item()
+    finally:
+        fo.set_jit(True)
+    assert fo.jit_stats()[2] == launches and c == b                  # interpreter, same bits
