@@ -123,24 +123,30 @@ cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
 }
 
 // ------------------------------------------------------------------ cols
-// grid.x: tiles of 512 columns; grid.y: row panels.  A thread owns a column pair
-// and walks its panel two rows at a time.
+// grid.x: tiles of 2 * cx columns; grid.y: row panels.  The 256 threads of a CTA
+// form cx column pairs by 256 / cx row lanes (cx = p.cx, a power of two <= 256,
+// chosen so that narrow matrices still fill the CTA); a thread owns a column pair
+// and walks every (256 / cx)-th row of its panel, two rows per chain evaluation;
+// the row lanes are then added in order through shared memory.
 template <class EVAL, bool ALIGNED>
 __global__ void __launch_bounds__(kThreads)
 cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ CellParams p)
 {
     __shared__ unsigned int s_flag;
-    const long long col = (long long)blockIdx.x * 512 + 2 * threadIdx.x;
+    __shared__ double2 s_lane[kThreads];
+    const int cx = p.cx, ry = kThreads / cx;
+    const int tx = threadIdx.x & (cx - 1), ty = threadIdx.x / cx;
+    const long long col = ((long long)blockIdx.x * cx + tx) * 2;
     const long long per = (p.rows + p.panels - 1) / p.panels;
     const long long r0 = (long long)blockIdx.y * per;
     const long long r1 = (r0 + per < p.rows) ? r0 + per : p.rows;
     double a0 = 0.0, a1 = 0.0;
 
     if (col < p.cols) {
-        for (long long row = r0; row < r1; row += 2) {
-            const bool two = row + 1 < r1;
+        for (long long row = r0 + ty; row < r1; row += 2 * ry) {
+            const bool two = row + ry < r1;
             double in[kIn][kV];
-            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, col, row + 1, col, two, in);
+            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, col, row + ry, col, two, in);
             double o[1][kV];
             EVAL::template run<kV, 1>(ch, in, o);
             a0 += o[0][0];
@@ -150,6 +156,18 @@ cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
                 a1 += o[0][3];
             }
         }
+    }
+    if (ry > 1) {
+        s_lane[threadIdx.x] = make_double2(a0, a1);
+        __syncthreads();
+        if (ty == 0) {
+            for (int k = 1; k < ry; ++k) {
+                a0 += s_lane[k * cx + tx].x;
+                a1 += s_lane[k * cx + tx].y;
+            }
+        }
+    }
+    if (col < p.cols && ty == 0) {
         if (p.panels == 1) {
             p.out[col] = a0;
             if (col + 1 < p.cols) p.out[col + 1] = a1;
@@ -161,7 +179,7 @@ cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
     }
     if (p.panels == 1) return;
     // the last panel of this column tile to finish adds the tile's partials, panel 0 first
-    if (take_ticket(&p.head->group[blockIdx.x], (unsigned)p.panels, &s_flag) && col < p.cols) {
+    if (take_ticket(&p.head->group[blockIdx.x], (unsigned)p.panels, &s_flag) && col < p.cols && ty == 0) {
         double s0 = 0.0, s1 = 0.0;
         const bool two = col + 1 < p.cols;
         for (int g = 0; g < p.panels; ++g) {
@@ -213,9 +231,17 @@ int stream_grid(long long units, int sms)
 
 // Row panels of the column-aggregation kernel: enough CTAs to fill the GPU, at
 // least 32 rows per panel, one ticket per column tile.
+// Column pairs a CTA covers: 256, or fewer for narrow matrices (a power of two).
+int col_cx(long long cols)
+{
+    int cx = 256;
+    while (cx > 8 && (long long)cx >= cols) cx >>= 1;      // smallest power of two with 2 * cx >= cols
+    return cx;
+}
+
 int col_panels(long long rows, long long cols)
 {
-    const long long tiles = (cols + 511) / 512;
+    const long long tiles = (cols + 2 * col_cx(cols) - 1) / (2 * col_cx(cols));
     if (tiles > kMaxGroups) return 1;
     long long p = (148 * 8 + tiles - 1) / tiles;
     const long long maxp = (rows + 31) / 32;
@@ -248,7 +274,7 @@ cudaError_t launch_cell(const DevChain &ch, const CellParams &p, int agg, bool f
 {
     if (agg == FO_CELL_COL_AGG) {
         if constexpr (NOUT == 1) {
-            const dim3 g((unsigned)((p.cols + 511) / 512), (unsigned)p.panels);
+            const dim3 g((unsigned)((p.cols + 2 * p.cx - 1) / (2 * p.cx)), (unsigned)p.panels);
             if (aligned) cell_cols_kernel<EVAL, true><<<g, kThreads, 0, st>>>(ch, p);
             else cell_cols_kernel<EVAL, false><<<g, kThreads, 0, st>>>(ch, p);
         }
@@ -368,6 +394,7 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     int grid;
     if (agg == FO_CELL_COL_AGG) {
         p.panels = col_panels(xd.rows, xd.cols);
+        p.cx = col_cx(xd.cols);
         grid = 0;
     } else if (flat) {
         grid = stream_grid((ncells + 1023) >> 10, sms);

@@ -18,7 +18,7 @@ struct CellParams {
     double *partials;
     double *out;
     int panels;           // cell_cols_kernel: number of row panels
-    int pad;
+    int cx;               // cell_cols_kernel: column pairs per CTA
 };
 
 constexpr int kV = 4;     // cells per thread per chain evaluation
