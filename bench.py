@@ -263,6 +263,87 @@ def time_variants(fo, step, shapes, reps=10):
     return res
 
 
+def _event_times(fn, reps, warm=2, before=None):
+    """Milliseconds of `reps` runs of fn() (CUDA events on the current stream) after `warm` untimed runs;
+    before() runs untimed ahead of every timed run."""
+    import torch
+    for _ in range(warm):
+        fn()
+    out = []
+    for _ in range(reps):
+        if before is not None:
+            before()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        out.append(a.elapsed_time(b))
+    return out
+
+
+def machine_probes(fo, step, shapes):
+    """Rates the rooflines are quoted against besides the copy peak: a read-only streaming sum through
+    the Cell kernel, whole-row gathers from an L2-resident matrix, and fp64 multiply-add issue."""
+    import torch
+    d = step.d
+    dev = d["row_dense.X"].device
+    one = torch.empty(1, dtype=torch.float64, device=dev)
+    X = d["row_dense.X"]
+    ms = min(_event_times(lambda: fo.fused_cell([("mov", "t0", "a")], "t0", X, agg="full", out=one), 5))
+    res = {"stream_sum_gbs": X.numel() * 8 / (ms * 1e-3) / 1e9,
+           "stream_sum": "sum(X) over the %dx%d Row input, Cell kernel" % tuple(X.shape)}
+    V = d["outer.V"]
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    n = 10_000_000
+    out = torch.empty(fo.probe_out_len(), dtype=torch.float64, device=dev)
+    for label, nrows in (("l2_gather_gbs", min(V.shape[0], 40_000)), ("gather_all_rows_gbs", V.shape[0])):
+        idx = torch.randint(0, nrows, (n,), generator=g, device=dev, dtype=torch.int32)
+        moved = [0]
+
+        def run(idx=idx):
+            moved[0] = fo.probe_l2_gather(V, idx, out)
+        ms = min(_event_times(run, 5))
+        res[label] = moved[0] / (ms * 1e-3) / 1e9
+        res[label + "_rows"] = nrows
+    res["l2_gather"] = ("%d random rows of %d doubles from the first rows of V (%.0f MB resident set, resp. "
+                        "all of V)" % (n, V.shape[1], 40_000 * V.shape[1] * 8 / 1e6))
+    flops = [0]
+
+    def fma():
+        flops[0] = fo.probe_fp64_fma(20_000, out)
+    ms = min(_event_times(fma, 5))
+    res["fp64_fma_tflops"] = flops[0] / (ms * 1e-3) / 1e12
+    return res
+
+
+def size_sweep(fo, device, cols=1000, rows_list=(1_000, 10_000, 100_000, 1_000_000), reps=10):
+    """Cell sum(X*Y*Z) and the three-aggregate MAgg over rows x 1000 inputs, rows from 1e3 to 1e6
+    (Section 5.2's sweep), cold L2: a 512 MB buffer is overwritten before every timed run."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(11)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+    one = torch.empty(1, dtype=torch.float64, device=device)
+    three = torch.empty(3, dtype=torch.float64, device=device)
+    res = []
+    for rows in rows_list:
+        X, Y, Z = (torch.rand((rows, cols), generator=g, dtype=torch.float64, device=device) for _ in range(3))
+        sides = [("cell", Y), ("cell", Z)]
+        nbytes = 3 * 8 * rows * cols
+        entry = {"rows": rows, "cols": cols, "bytes": nbytes}
+        for name, fn in (("cell", lambda: fo.fused_cell(XYZ, "t1", X, sides, out=one)),
+                         ("magg", lambda: fo.fused_magg(MAGG3, ["t0", "t1", "t2"], X, sides, out=three))):
+            ms = _event_times(fn, reps, before=flush.zero_)
+            entry[name] = {"us_min": min(ms) * 1e3, "us_median": statistics.median(ms) * 1e3,
+                           "us_mean": statistics.mean(ms) * 1e3,
+                           "gbs_at_median": nbytes / (statistics.median(ms) * 1e-3) / 1e9}
+        res.append(entry)
+        del X, Y, Z
+    return res
+
+
 # ---------------------------------------------------------------------- clocks
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
@@ -357,6 +438,32 @@ def oracle_step(np_inputs, shapes):
     r["outer"] = oracle.outer_wsloss_masked(X5, h["outer.U"], h["outer.V"])
     t["outer"] = time.perf_counter() - t0
     return t, r
+
+
+def oracle_single_thread(np_inputs, shapes):
+    """Cell and Outer legs of the checker with the numeric libraries held to one thread."""
+    import oracle
+    h = np_inputs
+    try:
+        from threadpoolctl import threadpool_limits
+        limit = threadpool_limits(limits=1)
+    except Exception:
+        limit = None
+    try:
+        t = {}
+        t0 = time.perf_counter()
+        oracle.sum_xyz(h["cell.X"], h["cell.Y"], h["cell.Z"])
+        t["cell"] = time.perf_counter() - t0
+        s = shapes["outer"]
+        X5 = dict(rows=s["rows"], cols=s["cols"], rowptr=h["outer.rowptr"], colidx=h["outer.colidx"],
+                  vals=h["outer.vals"])
+        t0 = time.perf_counter()
+        oracle.outer_wsloss_masked(X5, h["outer.U"], h["outer.V"])
+        t["outer"] = time.perf_counter() - t0
+    finally:
+        if limit is not None:
+            limit.restore_original_limits()
+    return t
 
 
 def host_threads():
@@ -564,8 +671,9 @@ def run_ours(args):
     for name in OPS:
         ms = statistics.mean(per_op_ms[name])
         gbs = nbytes[name] / (ms * 1e-3) / 1e9
-        per_op[name] = {"ms": ms, "ms_min": min(per_op_ms[name]), "bytes": nbytes[name], "gbs": gbs,
-                        "frac_of_" + peak_kind: gbs / peak_gbs}
+        per_op[name] = {"ms": ms, "ms_min": min(per_op_ms[name]), "ms_median": statistics.median(per_op_ms[name]),
+                        "bytes": nbytes[name], "gbs": gbs, "frac_of_" + peak_kind: gbs / peak_gbs,
+                        "frac_of_nominal_8000": gbs / 8000.0}
     nnz4, nnz5 = int(host["row_csr.vals"].numel()), int(host["outer.vals"].numel())
     per_op["row_csr"]["nnz_per_s"] = nnz4 / (per_op["row_csr"]["ms"] * 1e-3)
     per_op["outer"]["nnz_per_s"] = nnz5 / (per_op["outer"]["ms"] * 1e-3)
@@ -606,6 +714,20 @@ def run_ours(args):
 
     if not args.no_variants and step.enabled == set(OPS):
         line["variants"] = time_variants(fo, step, shapes)
+        probes = machine_probes(fo, step, shapes)
+        line["probes"] = probes
+        for n in roofline_per_op:
+            roofline_per_op[n]["frac_of_stream_sum"] = per_op[n]["gbs"] / probes["stream_sum_gbs"]
+        # Outer: the slowest of compulsory bytes / HBM, gathered V rows / L2 gather rate, FMAs / fp64 rate
+        rank5 = shapes["outer"]["rank"]
+        terms = {"hbm": nbytes["outer"] / (peak_gbs * 1e9) * 1e3,
+                 "l2_gather": nnz5 * rank5 * 8 / (probes["l2_gather_gbs"] * 1e9) * 1e3,
+                 "fp64_fma": 2.0 * nnz5 * rank5 / (probes["fp64_fma_tflops"] * 1e12) * 1e3}
+        binding = max(terms, key=terms.get)
+        roofline_per_op["outer"].update({"bound_terms_ms": terms, "binding_term": binding,
+                                         "frac_of_binding_term": terms[binding] / per_op["outer"]["ms"]})
+        if args.frac == 1.0 and world == 1:
+            line["size_sweep"] = size_sweep(fo, device)
 
     # ---- CPU baseline: the checker on a bounded sample, rank 0 at N = 1 only
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -620,6 +742,13 @@ def run_ours(args):
                 args.cpu_frac, sample_description(cshapes)),
             "seconds": cdt, "per_op_gbs": {k: cbytes[k] / ct[k] / 1e9 for k in OPS},
         }
+        # one thread, configs 1 and 5 (Outer on a sixteenth of the sample's rows)
+        shost, sshapes = row_sample(chost, cshapes, 1.0 / 16)
+        sbytes = algorithmic_bytes(sshapes, shost)
+        st = oracle_single_thread(numpy_inputs(shost), sshapes)
+        line["cpu_baseline"]["single_thread_gbs"] = {k: sbytes[k] / st[k] / 1e9 for k in st}
+        line["cpu_baseline"]["single_thread_sample"] = "cell full size; outer %d rows x %d" % (
+            sshapes["outer"]["rows"], sshapes["outer"]["cols"])
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

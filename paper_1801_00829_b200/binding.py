@@ -81,6 +81,7 @@ EXPORTS = [
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
     "fo_set_jit", "fo_jit_stats", "fo_jit_compile_check",
+    "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_fp64_fma", "fo_chain_describe",
 ]
 
 _lib = None
@@ -132,6 +133,14 @@ def load_library(path=None):
         lib.fo_jit_compile_check.restype = C.c_int
         lib.fo_set_force_interpreter.argtypes = [C.c_int]
         lib.fo_set_force_interpreter.restype = C.c_int
+        lib.fo_chain_describe.argtypes = [chain_p, i32, i32, scal_p, i32, i32, C.c_char_p, sz]
+        lib.fo_chain_describe.restype = C.c_int
+        lib.fo_probe_out_len.argtypes = []
+        lib.fo_probe_out_len.restype = C.c_size_t
+        lib.fo_probe_l2_gather.argtypes = [C.POINTER(fo_dense), vp, C.c_longlong, dp, vp]
+        lib.fo_probe_l2_gather.restype = C.c_int
+        lib.fo_probe_fp64_fma.argtypes = [C.c_longlong, dp, vp]
+        lib.fo_probe_fp64_fma.restype = C.c_int
         if path is None:
             _lib = lib
         return lib
@@ -337,6 +346,41 @@ def jit_compile_check(steps, outputs, n_sides=0, n_scalars=0, store=False):
     log = C.create_string_buffer(1 << 16)
     rc = load_library().fo_jit_compile_check(C.byref(ch), n_sides, n_scalars, 1 if store else 0, log, len(log))
     return rc, log.value.decode(errors="replace")
+
+
+def chain_describe(steps, outputs, use="cell", n_sides=0, scalars=(), k=0):
+    """The k-th result of a chain as an expression over its inputs (host only)."""
+    ch, keep = make_chain(steps, outputs)
+    text = C.create_string_buffer(8192)
+    _check(load_library().fo_chain_describe(C.byref(ch), {"cell": 0, "row": 1, "outer": 2}[use], n_sides,
+                                            _scalars(scalars), len(scalars), k, text, len(text)),
+           "fo_chain_describe")
+    return text.value.decode()
+
+
+def probe_l2_gather(V, idx, out=None):
+    """Gathers the rows idx (int32) of the dense matrix V once; returns the bytes moved.
+    Time it with events on the current stream."""
+    lib = load_library()
+    assert V.dtype == torch.float64 and V.dim() == 2 and idx.dtype == torch.int32 and idx.is_contiguous()
+    if out is None:
+        out = torch.empty(lib.fo_probe_out_len(), dtype=torch.float64, device=V.device)
+    vs = _dense_struct(V)
+    _check(lib.fo_probe_l2_gather(C.byref(vs), C.c_void_p(idx.data_ptr()), idx.numel(),
+                                  C.c_void_p(out.data_ptr()), _stream(V.device)), "fo_probe_l2_gather")
+    return idx.numel() * V.shape[1] * 8
+
+
+def probe_fp64_fma(iters, out):
+    """Runs 8 * iters multiply-adds per launched thread; returns the flop count."""
+    lib = load_library()
+    _check(lib.fo_probe_fp64_fma(int(iters), C.c_void_p(out.data_ptr()), _stream(out.device)),
+           "fo_probe_fp64_fma")
+    return 16 * int(iters) * lib.fo_probe_out_len()
+
+
+def probe_out_len():
+    return int(load_library().fo_probe_out_len())
 
 
 def device_status(device=None):

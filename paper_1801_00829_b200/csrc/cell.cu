@@ -426,6 +426,8 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
 
 }  // namespace
 
+bool force_interpreter() { return g_force_interpreter; }
+
 }  // namespace fo
 
 namespace fo {

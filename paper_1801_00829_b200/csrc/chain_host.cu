@@ -3,6 +3,8 @@
 // utilities shared by the entry points.
 #include <string.h>
 
+#include <string>
+
 #include "common.cuh"
 
 namespace fo {
@@ -168,6 +170,39 @@ int translate_chain(const fo_chain *chain, ChainUse use, int n_sides,
     return FO_OK;
 }
 
+int chain_expression(const DevChain &ch, int k, char *text, size_t cap)
+{
+    static const char *const names[FO_OP_COUNT_] = {
+        "mov", "neg", "abs", "sqrt", "exp", "log", "sq", "add", "sub", "mul", "div",
+        "min", "max", "pow", "eq", "ne", "lt", "le", "gt", "ge", "sel", "fma"};
+    std::string reg[kRegs + 1];
+    for (int r = 0; r < kRegs + 1; ++r) reg[r] = "r" + std::to_string(r);
+    auto operand_text = [&](int o) -> std::string {
+        if (o & 0x80) return "k" + std::to_string(o & 0x7f);
+        return (o >= 0 && o <= kRegs) ? reg[o] : std::string("?");
+    };
+    const size_t limit = 4096;       // shared subexpressions are written out again: bound the growth
+    for (int s = 0; s < ch.n_ops; ++s) {
+        const DevOp &op = ch.ops[s];
+        if (op.opcode >= FO_OP_COUNT_ || op.dst > kRegs) return -1;
+        const std::string a = operand_text(op.a);
+        std::string e;
+        if (op.opcode == FO_OP_MOV) e = a;
+        else if (op.opcode == FO_OP_SQ) e = "mul(" + a + "," + a + ")";
+        else if (op.opcode < FO_OP_ADD) e = std::string(names[op.opcode]) + "(" + a + ")";
+        else if (op.opcode == FO_OP_SEL || op.opcode == FO_OP_FMA)
+            e = std::string(names[op.opcode]) + "(" + a + "," + operand_text(op.b) + "," + operand_text(op.c) + ")";
+        else e = std::string(names[op.opcode]) + "(" + a + "," + operand_text(op.b) + ")";
+        if (e.size() > limit) return -1;
+        reg[op.dst] = e;
+    }
+    if (k < 0 || k >= ch.n_out) return -1;
+    const std::string out = operand_text(ch.out[k]);
+    if (out.size() + 1 > cap) return -1;
+    memcpy(text, out.c_str(), out.size() + 1);
+    return 0;
+}
+
 int check_workspace(const void *ws, size_t ws_bytes, size_t need)
 {
     if (!ws) return FO_ERR_WORKSPACE;
@@ -237,6 +272,18 @@ int fo_query_device_status(const void *ws, void *stream, int *status)
     if (e != cudaSuccess) return fo::cuda_fail(e);
     *status = words[1] ? FO_ERR_DEVICE_TIMEOUT : FO_OK;
     return FO_OK;
+}
+
+int fo_chain_describe(const fo_chain *chain, int use, int n_sides, const double *scalars, int n_scalars,
+                      int k, char *text, size_t cap)
+{
+    if (!chain || !text || cap == 0) return FO_ERR_NULL;
+    if (use < 0 || use > 2) return FO_ERR_SHAPE;
+    fo::DevChain ch;
+    const int rc = fo::translate_chain(chain, (fo::ChainUse)use, n_sides, scalars, n_scalars, 1, FO_MAX_OUT, &ch);
+    if (rc != FO_OK) return rc;
+    if (k < 0 || k >= ch.n_out) return FO_ERR_SHAPE;
+    return fo::chain_expression(ch, k, text, cap) == 0 ? FO_OK : FO_ERR_SHAPE;
 }
 
 }  // extern "C"

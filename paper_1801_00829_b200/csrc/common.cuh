@@ -79,6 +79,18 @@ int translate_chain(const fo_chain *chain, ChainUse use, int n_sides,
                     const double *scalars, int n_scalars, int min_out, int max_out,
                     DevChain *out);
 
+// Host: the k-th result of a translated chain written out as an expression over
+// its inputs, e.g. "mul(ne(r0,k0),mul(sub(r0,r1),sub(r0,r1)))": rN is input
+// register N, kN entry N of the constant table; sq(x) is written mul(x,x).  Two
+// chains with the same text do the same arithmetic in the same order, whatever
+// temporaries they were written with.  Writes at most cap - 1 characters;
+// returns 0, or -1 if the text does not fit.
+int chain_expression(const DevChain &ch, int k, char *text, size_t cap);
+
+// True while fo_set_force_interpreter(1) is in effect: every chain goes through
+// the general interpreter (cell.cu).
+bool force_interpreter();
+
 int check_workspace(const void *ws, size_t ws_bytes, size_t need);
 int cuda_fail(cudaError_t e);
 int sm_count();

@@ -7,6 +7,7 @@
 // The row U_i sits in registers, spread over the 8 lanes of a group; the four
 // groups of a warp take different stored cells of the row and gather their V_j
 // rows with 128-bit loads (V is read many times and stays in L2).
+#include <stdio.h>
 #include <stdlib.h>
 
 #include "chain.cuh"
@@ -20,7 +21,8 @@ struct OuterParams {
     const int *colidx;
     const double *vals;
     long long rows, cols, nnz;
-    int rank, pad;
+    int rank;
+    int chain_kind;              // kOuterGeneric or a chain evaluated inline
     const double *U;
     long long ldu;
     const double *V;
@@ -28,9 +30,16 @@ struct OuterParams {
     WsHead *head;
     double *partials;
     double *out;
+    int kconst;                  // constant-table index an inline chain reads
+    int pad;
 };
 
 enum { kOutFull = 0, kOutNone = 1, kOutRight = 2 };
+
+// Chains evaluated inline, in the chain's own operation order (same bits as the
+// interpreter): the weighted squared loss of Eq. 1, (a != 0) * (a - d)^2, and the
+// sparse micro-benchmark expression of Section 5.2, a * log(d + eps).
+enum { kOuterGeneric = 0, kOuterWsloss = 1, kOuterXlogd = 2 };
 
 template <bool ALIGNED>
 __device__ __forceinline__ double2 ld_pair_cached(const double *row, int col, int n)
@@ -43,8 +52,15 @@ __device__ __forceinline__ double2 ld_pair_cached(const double *row, int col, in
     return make_double2(0.0, 0.0);
 }
 
-__device__ __forceinline__ double outer_chain(const DevChain &ch, double a, double d)
+__device__ __forceinline__ double outer_chain(const DevChain &ch, int kind, int kc, double a, double d)
 {
+    if (kind == kOuterWsloss) {
+        const double t0 = a != 0.0 ? 1.0 : 0.0;
+        const double t1 = a - d;
+        const double t2 = t1 * t1;
+        return t0 * t2;
+    }
+    if (kind == kOuterXlogd) return a * slow_log(d + ch.consts[kc]);
     RegFile<kRegs, 1> f;
     f.r[0][0] = a;
     f.r[1][0] = d;
@@ -145,7 +161,7 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
                 if ((lane >> 2) == it) dmine = allA;
                 if ((lane >> 2) == it + 1) dmine = allB;
             }
-            const double w = outer_chain(ch, amine, dmine);
+            const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
             if (AGG == kOutFull) {
                 if (valid) acc += w;
             } else if (AGG == kOutNone) {
@@ -296,7 +312,7 @@ outer_staged_kernel(const __grid_constant__ DevChain ch, const __grid_constant__
                 }
                 if (AGG == kOutRight) {
                     // the chain's values for this half, then O_i += w * V_j from the staged rows
-                    const double w = outer_chain(ch, amine, dmine);
+                    const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
                     if ((lane >> 4) == h) wmine = w;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
@@ -319,7 +335,7 @@ outer_staged_kernel(const __grid_constant__ DevChain ch, const __grid_constant__
                 __syncwarp();          // the buffer is overwritten by the next half
             }
             if (AGG != kOutRight) {
-                const double w = outer_chain(ch, amine, dmine);
+                const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
                 if (AGG == kOutFull) {
                     if (valid) acc += w;
                 } else {
@@ -395,6 +411,31 @@ cudaError_t launch_outer_staged(const DevChain &ch, const OuterParams &p, int ag
     return go(outer_staged_kernel<NK2, kOutRight>);
 }
 
+// Recognises the chains that outer_chain() evaluates inline by the text of the
+// translated program's result (chain_expression); multiplication and addition
+// commute bit for bit, so both operand orders count.
+int outer_chain_kind(const DevChain &ch, int *kconst)
+{
+    char e[160];
+    *kconst = 0;
+    if (chain_expression(ch, 0, e, sizeof(e)) != 0) return kOuterGeneric;
+    auto match = [&](const char *pattern, int *k) -> bool {
+        int n = 0;
+        *k = -1;
+        return sscanf(e, pattern, k, &n) == 1 && n > 0 && e[n] == 0 && *k >= 0 && *k < kConsts;
+    };
+    int k;
+    if ((match("mul(ne(r0,k%d),mul(sub(r0,r1),sub(r0,r1)))%n", &k) ||
+         match("mul(mul(sub(r0,r1),sub(r0,r1)),ne(r0,k%d))%n", &k)) && ch.consts[k] == 0.0)
+        return kOuterWsloss;
+    if (match("mul(r0,log(add(r1,k%d)))%n", &k) || match("mul(r0,log(add(k%d,r1)))%n", &k) ||
+        match("mul(log(add(r1,k%d)),r0)%n", &k) || match("mul(log(add(k%d,r1)),r0)%n", &k)) {
+        *kconst = k;
+        return kOuterXlogd;
+    }
+    return kOuterGeneric;
+}
+
 }  // namespace
 
 }  // namespace fo
@@ -441,6 +482,7 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     p.head = (WsHead *)ws;
     p.partials = (double *)((char *)ws + sizeof(WsHead));
     p.out = out;
+    p.chain_kind = fo::force_interpreter() ? fo::kOuterGeneric : fo::outer_chain_kind(ch, &p.kconst);
     cudaStream_t st = (cudaStream_t)stream;
 
     if (X->nnz == 0 || X->rows == 0) {

@@ -189,3 +189,26 @@ def test_cost_model_worked_example():
     assert abs(ideal_seconds(nbytes, float(vals["gb_per_s"])) - float(vals["seconds"])) < 1e-12
     assert algorithmic_bytes("cell", rows=1000, cols=1000, n_inputs=3) == 24_000_008
     assert algorithmic_bytes("row_dense", rows=10**6, cols=1000) == 8 * 10**9 + 8 * 10**6 + 16000
+
+
+def test_chain_describe_writes_the_arithmetic_not_the_temporaries():
+    import paper_1801_00829_b200 as fo
+    from paper_1801_00829_b200.binding import FusedOpsError
+    wsloss = [("ne", "t0", "a", 0.0), ("sub", "t1", "a", "d"), ("mul", "t2", "t1", "t1"), ("mul", "t3", "t0", "t2")]
+    renamed = [("ne", "t7", "a", 0.0), ("sub", "t0", "a", "d"), ("sq", "t0", "t0"), ("mul", "t1", "t7", "t0")]
+    a = fo.chain_describe(wsloss, "t3", use="outer")
+    b = fo.chain_describe(renamed, "t1", use="outer")
+    assert a == b == "mul(ne(r0,k8),mul(sub(r0,r1),sub(r0,r1)))"       # Eq. 1; sq(x) reads mul(x,x)
+    assert fo.chain_describe([("mul", "t0", "a", "side0"), ("mul", "t1", "t0", "side1")], "t1",
+                             use="cell", n_sides=2) == "mul(mul(r0,r1),r2)"
+    assert fo.chain_describe([("mul", "t0", "side0", "d")], "t0", use="row", n_sides=1) == "mul(r1,r0)"
+    assert fo.chain_describe([("add", "t0", "d", "s0"), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")], "t2",
+                             use="outer", scalars=[1e-15]) == "mul(r0,log(add(r1,k0)))"
+    # several outputs, and an output that is an input
+    magg = [("mul", "t0", "a", "side0"), ("mul", "t1", "a", "a")]
+    assert fo.chain_describe(magg, ["t0", "t1"], use="cell", n_sides=1, k=1) == "mul(r0,r0)"
+    assert fo.chain_describe([], "a", use="cell") == "r0"
+    with pytest.raises(FusedOpsError):
+        fo.chain_describe(magg, ["t0", "t1"], use="cell", n_sides=1, k=2)
+    with pytest.raises(FusedOpsError):
+        fo.chain_describe([("mul", "t0", "a", "side3")], "t0", use="cell", n_sides=1)

@@ -368,3 +368,28 @@ def test_specialised_chains_equal_interpreter_bitwise(fo, name, chain, outs, nsi
                 fo.force_interpreter(False)
             assert f1.tobytes() == f2.tobytes(), (name, agg)
             assert_close(f1, r, absscale=a, what="%s %s" % (name, agg))
+
+
+@pytest.mark.parametrize("name,chain,out,scalars", [
+    ("wsloss", WSLOSS, "t3", []),
+    ("wsloss-commuted", [("sub", "t0", "a", "d"), ("sq", "t5", "t0"), ("ne", "t1", "a", 0.0),
+                         ("mul", "t0", "t5", "t1")], "t0", []),
+    ("xlogd", [("add", "t0", "d", "s0"), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")], "t2", [2.5]),
+    ("xlogd-imm", [("add", "t0", 2.5, "d"), ("log", "t1", "t0"), ("mul", "t2", "t1", "a")], "t2", []),
+    ("not-inline", [("sub", "t0", "a", "d"), ("abs", "t1", "t0")], "t1", []),
+])
+@pytest.mark.parametrize("agg", ["full", "none", "right"])
+def test_outer_inline_chains_equal_interpreter_bitwise(fo, name, chain, out, scalars, agg):
+    w = datagen.outer_workload(300, 257, 20, 0.05, seed=77)
+    U, V = w["U"], w["V"]
+    X, Ud, Vd = csr_to_dev(w), to_dev(U), to_dev(V)
+    try:
+        fo.force_interpreter(False)
+        fast = fo.fused_outer(chain, out, X, Ud, Vd, scalars, agg=agg).cpu().numpy()
+        fo.force_interpreter(True)
+        slow = fo.fused_outer(chain, out, X, Ud, Vd, scalars, agg=agg).cpu().numpy()
+    finally:
+        fo.force_interpreter(False)
+    assert fast.tobytes() == slow.tobytes(), (name, agg)
+    ref = oracle.outer(chain, out, host_csr(w), U, V, scalars, mode="masked", agg=agg)
+    assert_close(fast, np.asarray(ref).reshape(fast.shape), what="%s %s" % (name, agg))
