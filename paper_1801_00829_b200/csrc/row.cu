@@ -12,6 +12,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <type_traits>
+
 #include "chain.cuh"
 
 namespace fo {
@@ -401,15 +403,17 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
 // A warp takes blocks of 32 consecutive rows.  Row offsets, side values and the
 // chain are handled one row per lane (coalesced loads, one chain evaluation for
 // 32 rows); the block's stored cells - one contiguous piece of colidx / vals -
-// are first copied into the warp's slice of shared memory with coalesced loads,
-// then an 8-lane group walks each row: dot product against v (shared memory),
-// and for col_t_agg the scatter  acc[col] += t * val  into the CTA's shared
-// accumulator.  Two groups may hit the same column at the same time, so the
-// scatter uses shared-memory atomics (their order is not fixed).
+// are first copied into the warp's slice of shared memory with coalesced loads.
+// Then G lanes share a row (G = 2 .. 32 by the matrix's mean row length, so
+// that a row takes a few trips): 32 / G rows at a time, every group walks its
+// row with the same, warp-uniform trip count - dot product against v (shared
+// memory), and for col_t_agg the scatter  acc[col] += t * val  into the CTA's
+// shared accumulator.  Two lanes may hit the same column at the same time, so
+// the scatter uses shared-memory atomics (their order is not fixed).
 constexpr int kCsrStage = 512;            // stored cells a warp can stage per block of rows
 
-template <int AGG>
-__global__ void __launch_bounds__(kThreads)
+template <int AGG, int G>
+__global__ void __launch_bounds__(kThreads, 3)
 row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -417,7 +421,7 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
     __shared__ unsigned int s_flag;
     const long long n = p.cols;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int l8 = lane & 7, grp = lane >> 3;
+    const int lg = lane & (G - 1), grp = lane / G;
 
     double *vs = reinterpret_cast<double *>(smem_raw);
     double *qs = vs + n;                                       // col_t_agg only
@@ -460,24 +464,34 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
         }
         __syncwarp();
 
+        // G lanes per row: 32 / G rows at a time, G trips
         double dmine = 0.0;
-        for (int it = 0; it < 8; ++it) {
-            const int rr = it * 4 + grp;
+#pragma unroll 1
+        for (int it = 0; it < G; ++it) {
+            const int rr = it * (32 / G) + grp;
             const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
             const int end = __shfl_sync(0xffffffffu, end_l, rr);
             double d = 0.0;
             if (staged) {
-                for (int q0 = beg - base + l8; q0 < end - base; q0 += 8) d = fma(sx[q0], vs[sc[q0]], d);
+                // the same trip count in all groups: no divergent loop
+                const int trips = __reduce_max_sync(0xffffffffu, (end - beg + G - 1) / G);
+                int q0 = beg - base + lg;
+                const int qe = end - base;
+                for (int s = 0; s < trips; ++s, q0 += G) {
+                    const bool ok = q0 < qe;
+                    const int qq = ok ? q0 : 0;
+                    const double x = ok ? sx[qq] : 0.0;
+                    d = fma(x, vs[sc[qq]], d);
+                }
             } else {
-                for (int q0 = beg + l8; q0 < end; q0 += 8)
+                for (int q0 = beg + lg; q0 < end; q0 += G)
                     d = fma(__ldg(p.vals + q0), vs[__ldg(p.colidx + q0)], d);
             }
-            d += __shfl_xor_sync(0xffffffffu, d, 4);
-            d += __shfl_xor_sync(0xffffffffu, d, 2);
-            d += __shfl_xor_sync(0xffffffffu, d, 1);
-            // row rr's dot product sits in group (rr & 3); lane rr keeps it
-            const double dall = __shfl_sync(0xffffffffu, d, (lane & 3) * 8);
-            if ((lane >> 2) == it) dmine = dall;
+#pragma unroll
+            for (int o = G / 2; o >= 1; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+            // row rr's dot product sits in group (rr mod groups); lane rr keeps it
+            const double dall = __shfl_sync(0xffffffffu, d, (lane & (32 / G - 1)) * G);
+            if (lane / (32 / G) == it) dmine = dall;
         }
         const double t = lane_chain(ch, p.chain_kind, dmine, sv);
         if (AGG == kRowRow) {
@@ -485,16 +499,20 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
         } else if (AGG == kRowFull) {
             if (have) tsum += t;
         } else {
-            for (int it = 0; it < 8; ++it) {
-                const int rr = it * 4 + grp;
+#pragma unroll 1
+            for (int it = 0; it < G; ++it) {
+                const int rr = it * (32 / G) + grp;
                 const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
                 const int end = __shfl_sync(0xffffffffu, end_l, rr);
                 const double tt = __shfl_sync(0xffffffffu, t, rr);
                 if (staged) {
-                    for (int q0 = beg - base + l8; q0 < end - base; q0 += 8)
-                        atomicAdd(&qs[sc[q0]], tt * sx[q0]);
+                    const int trips = __reduce_max_sync(0xffffffffu, (end - beg + G - 1) / G);
+                    int q0 = beg - base + lg;
+                    const int qe = end - base;
+                    for (int s = 0; s < trips; ++s, q0 += G)
+                        if (q0 < qe) atomicAdd(&qs[sc[q0]], tt * sx[q0]);
                 } else {
-                    for (int q0 = beg + l8; q0 < end; q0 += 8)
+                    for (int q0 = beg + lg; q0 < end; q0 += G)
                         atomicAdd(&qs[__ldg(p.colidx + q0)], tt * __ldg(p.vals + q0));
                 }
             }
@@ -709,9 +727,19 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
             kern<<<(unsigned)grid, kThreads, smem, st>>>(ch, p);
             return cudaGetLastError();
         };
-        if (agg == FO_ROW_COL_T_AGG) e = go(row_csr_kernel<kRowColT>);
-        else if (agg == FO_ROW_ROW_AGG) e = go(row_csr_kernel<kRowRow>);
-        else e = go(row_csr_kernel<kRowFull>);
+        auto by_agg = [&](auto g) -> cudaError_t {
+            constexpr int G = decltype(g)::value;
+            if (agg == FO_ROW_COL_T_AGG) return go(row_csr_kernel<kRowColT, G>);
+            if (agg == FO_ROW_ROW_AGG) return go(row_csr_kernel<kRowRow, G>);
+            return go(row_csr_kernel<kRowFull, G>);
+        };
+        // lanes per row from the mean row length: about four trips for a typical row
+        const double mean_len = rows > 0 ? (double)X->csr.nnz / (double)rows : 0.0;
+        if (mean_len <= 12.0) e = by_agg(std::integral_constant<int, 2>());
+        else if (mean_len <= 24.0) e = by_agg(std::integral_constant<int, 4>());
+        else if (mean_len <= 48.0) e = by_agg(std::integral_constant<int, 8>());
+        else if (mean_len <= 96.0) e = by_agg(std::integral_constant<int, 16>());
+        else e = by_agg(std::integral_constant<int, 32>());
     } else {
         p.X = X->dense.data; p.ldx = X->dense.ld;
         const bool staged = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;

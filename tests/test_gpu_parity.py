@@ -237,7 +237,9 @@ def test_row_dense_variants_strided_unaligned(fo, agg):
 
 
 @pytest.mark.parametrize("rows,cols,density", [(100000, 1000, 0.01), (5000, 64, 0.2), (300, 4000, 0.001),
-                                               (17, 9, 0.5), (1000, 1000, 0.0)])
+                                               (17, 9, 0.5), (1000, 1000, 0.0),
+                                               # mean row lengths 36, 80 and 200: 8, 16 and 32 lanes per row
+                                               (3000, 600, 0.06), (2000, 800, 0.1), (1500, 2000, 0.1)])
 def test_row_csr_col_t(fo, rows, cols, density):
     w = datagen.row_csr_workload(rows, cols, density, seed=3)
     Xh = host_csr(w)
@@ -249,9 +251,10 @@ def test_row_csr_col_t(fo, rows, cols, density):
 
 
 @pytest.mark.parametrize("agg", ["row", "full"])
-def test_row_csr_other_aggs_and_dense_agreement(fo, agg):
+@pytest.mark.parametrize("density", [0.02, 0.05, 0.12, 0.5])
+def test_row_csr_other_aggs_and_dense_agreement(fo, agg, density):
     rows, cols = 2500, 300
-    w = datagen.row_csr_workload(rows, cols, 0.05, seed=33)
+    w = datagen.row_csr_workload(rows, cols, density, seed=33)
     Xh = host_csr(w)
     ref = oracle.row(WD, "t0", Xh, w["v"], [("row", w["w"])], agg=agg)
     got = fo.fused_row(WD, "t0", csr_to_dev(w), to_dev(w["v"]), [("row", to_dev(w["w"]))], agg=agg)
