@@ -43,7 +43,7 @@ NCU_DRAM_BYTES_PER_UNIT = {
     "cell": 24.013e6 / 1e6,                      # per cell (3 inputs)
     "magg": (480.018e6 + 3.807e6) / 2e7,         # per cell (3 inputs)
     "row_dense": (1601.676e6 + 7.674e6) / 2e5,   # per row of 1000 columns
-    "row_csr": (264.058e6 + 4.077e6) / 19998162, # per stored cell (2 000 000 x 1000 @ 0.01 capture)
+    "row_csr": (264.058e6 + 3.779e6) / 19998162, # per stored cell (2 000 000 x 1000 @ 0.01 capture)
     "outer": (1382.994e6 + 3.550e6) / 9996322,   # per stored cell (full-size capture, staged kernel)
 }
 
