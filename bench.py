@@ -248,6 +248,25 @@ def time_variants(fo, step, shapes, reps=10):
         ("outer_right_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
                                                   agg="right", out=o_right), outer_in + 8 * orow * rank),
     ]
+    # sparse-safe Cell / MAgg (Section 5.2's sparse variants): X at density 0.1 as the CSR driver,
+    # dense Y and Z read at the stored cells
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    mask = torch.rand((mr, mc), generator=g, device=dev) < 0.1
+    counts = mask.sum(dim=1, dtype=torch.int32)
+    rowptr = torch.zeros(mr + 1, dtype=torch.int32, device=dev)
+    rowptr[1:] = torch.cumsum(counts, 0)
+    colidx = mask.nonzero()[:, 1].to(torch.int32).contiguous()
+    Xs = fo.CSR(mr, mc, rowptr, colidx, d["magg.X"][mask].contiguous())
+    del mask
+    o_three = torch.empty(3, dtype=torch.float64, device=dev)
+    sparse_in = 12 * Xs.nnz + 4 * (mr + 1) + 16 * Xs.nnz       # X once, one Y and one Z value per stored cell
+    cases += [
+        ("cell_csr_full_agg_density_0.1", lambda: fo.fused_cell(XYZ, "t1", Xs, sides, agg="full", out=o_one),
+         sparse_in + 8),
+        ("magg_csr_density_0.1", lambda: fo.fused_magg(MAGG3, ["t0", "t1", "t2"], Xs, sides, out=o_three),
+         sparse_in + 24),
+    ]
     res = {}
     for name, fn, nbytes in cases:
         for _ in range(2):

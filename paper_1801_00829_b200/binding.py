@@ -445,7 +445,7 @@ def fused_magg(steps, outputs, X, sides=(), scalars=(), out=None):
     outputs = list(outputs)
     ch, keep = make_chain(steps, outputs)
     m = _mat(X)
-    rows, cols = X.shape
+    rows, cols = (X.rows, X.cols) if isinstance(X, CSR) else X.shape
     dev = X.device
     if out is None:
         out = torch.empty(len(outputs), dtype=torch.float64, device=dev)

@@ -15,6 +15,7 @@
 
 #include "cell_flat.cuh"
 #include "jit.h"
+#include "cell_csr.h"
 #include "spec.cuh"
 
 namespace fo {
@@ -326,7 +327,10 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     if (!chain || !X || !out) return FO_ERR_NULL;
     if (n_sides > 0 && !sides) return FO_ERR_NULL;
     if (agg < FO_CELL_NO_AGG || agg > FO_CELL_FULL_AGG) return FO_ERR_UNSUPPORTED;
-    if (X->kind != FO_DENSE) return (X->kind == FO_CSR) ? FO_ERR_UNSUPPORTED : FO_ERR_SHAPE;
+    if (X->kind == FO_CSR)
+        return run_cell_csr(chain, X->csr, sides, n_sides, scalars, n_scalars, agg, magg, out, ws, ws_bytes,
+                            stream);
+    if (X->kind != FO_DENSE) return FO_ERR_SHAPE;
     const fo_dense &xd = X->dense;
     int rc = check_dense(xd);
     if (rc != FO_OK) return rc;
@@ -494,14 +498,17 @@ int fo_set_force_interpreter(int on)
 
 size_t fused_cell_workspace_bytes(const fo_mat *X, int agg)
 {
-    if (!X || X->kind != FO_DENSE || X->dense.rows < 0 || X->dense.cols < 0) return 0;
-    if (agg < FO_CELL_NO_AGG || agg > FO_CELL_FULL_AGG) return 0;
+    if (!X || agg < FO_CELL_NO_AGG || agg > FO_CELL_FULL_AGG) return 0;
+    if (X->kind == FO_CSR) return fo::cell_csr_ws_bytes(agg, 1);
+    if (X->kind != FO_DENSE || X->dense.rows < 0 || X->dense.cols < 0) return 0;
     return fo::cell_ws_bytes(X->dense.rows, X->dense.cols, agg, 1);
 }
 
 size_t fused_magg_workspace_bytes(const fo_mat *X, int n_out)
 {
-    if (!X || X->kind != FO_DENSE || n_out < 1 || n_out > FO_MAX_OUT) return 0;
+    if (!X || n_out < 1 || n_out > FO_MAX_OUT) return 0;
+    if (X->kind == FO_CSR) return fo::cell_csr_ws_bytes(FO_CELL_FULL_AGG, n_out);
+    if (X->kind != FO_DENSE) return 0;
     return fo::cell_ws_bytes(X->dense.rows, X->dense.cols, FO_CELL_FULL_AGG, n_out);
 }
 

@@ -1,0 +1,229 @@
+// Cell and MAgg templates over a CSR main input: the sparse-safe binding of
+// Table 1 / Section 2.2 - the chain runs on the stored cells only, side inputs
+// are read at each stored cell's (row, column).
+//
+// A warp takes blocks of 32 consecutive rows; G lanes share a row (G from the
+// matrix's mean row length), 32 / G rows at a time, with a warp-uniform trip
+// count.  The cells of a block are one contiguous piece of colidx / vals, so the
+// loads of neighbouring groups fall into the same cache lines.  Aggregation:
+//   full  per-lane sums -> CTA -> workspace partial -> last CTA (fixed order);
+//   row   the G lanes of a row are added by a shuffle tree (fixed order);
+//   none  one value per stored cell, in X's pattern;
+//   col   out[col] += value with global fp64 atomics after zeroing `out`
+//         (the order of these additions is not fixed).
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <type_traits>
+
+#include "cell_csr.h"
+#include "spec.cuh"
+
+namespace fo {
+
+namespace {
+
+struct CsrCellParams {
+    const int *rowptr;
+    const int *colidx;
+    const double *vals;
+    long long rows, cols;
+    DevSides sides;
+    WsHead *head;
+    double *partials;
+    double *out;
+    int agg;                 // FO_CELL_*
+    int pad;
+};
+
+template <class EVAL, int NOUT, int G>
+__global__ void __launch_bounds__(kThreads)
+cell_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ CsrCellParams p)
+{
+    __shared__ double s_red[NOUT * 32];
+    __shared__ unsigned int s_flag;
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int lg = lane & (G - 1), grp = lane / G;
+    const int agg = p.agg;
+    double acc[NOUT];
+#pragma unroll
+    for (int k = 0; k < NOUT; ++k) acc[k] = 0.0;
+
+    const long long nblocks = (p.rows + 31) >> 5;
+    const long long warp0 = (long long)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    const long long nwarps = (long long)gridDim.x * (kThreads / 32);
+
+    for (long long blk = warp0; blk < nblocks; blk += nwarps) {
+        const long long myrow = (blk << 5) + lane;
+        const int beg_l = __ldg(p.rowptr + (myrow < p.rows ? myrow : p.rows));
+        const int end_l = __ldg(p.rowptr + (myrow + 1 < p.rows ? myrow + 1 : p.rows));
+#pragma unroll 1
+        for (int it = 0; it < G; ++it) {
+            const int rr = it * (32 / G) + grp;
+            const long long row = (blk << 5) + rr;
+            const int beg = __shfl_sync(full, beg_l, rr);
+            const int end = __shfl_sync(full, end_l, rr);
+            const int trips = __reduce_max_sync(full, (end - beg + G - 1) / G);
+            // sides indexed by the row: one value for the whole row
+            double srow[FO_MAX_SIDES];
+#pragma unroll
+            for (int k = 0; k < FO_MAX_SIDES; ++k)
+                srow[k] = (EVAL::uses_side(ch, k) && p.sides.s[k].access == FO_AT_ROW && beg < end)
+                              ? __ldg(p.sides.s[k].data + row * p.sides.s[k].ld) : 0.0;
+            double rowacc = 0.0;
+            int q = beg + lg;
+            for (int s = 0; s < trips; ++s, q += G) {
+                const bool ok = q < end;
+                const int j = ok ? __ldg(p.colidx + q) : 0;
+                double in[kIn][1];
+                in[0][0] = ok ? __ldg(p.vals + q) : 0.0;
+#pragma unroll
+                for (int k = 0; k < FO_MAX_SIDES; ++k) {
+                    double v = 0.0;
+                    if (EVAL::uses_side(ch, k)) {
+                        const DevSide sd = p.sides.s[k];
+                        if (sd.access == FO_AT_ROW) v = srow[k];
+                        else if (ok) v = __ldg(sd.data + (sd.access == FO_AT_CELL ? row * sd.ld + j : (long long)j));
+                    }
+                    in[1 + k][0] = v;
+                }
+                double o[NOUT][1];
+                EVAL::template run<1, NOUT>(ch, in, o);
+                if (agg == FO_CELL_FULL_AGG) {
+#pragma unroll
+                    for (int k = 0; k < NOUT; ++k) acc[k] += ok ? o[k][0] : 0.0;
+                } else if (agg == FO_CELL_ROW_AGG) {
+                    rowacc += ok ? o[0][0] : 0.0;
+                } else if (agg == FO_CELL_NO_AGG) {
+                    if (ok) p.out[q] = o[0][0];
+                } else {
+                    if (ok) atomicAdd(p.out + j, o[0][0]);
+                }
+            }
+            if (agg == FO_CELL_ROW_AGG) {
+#pragma unroll
+                for (int o2 = G / 2; o2 >= 1; o2 >>= 1) rowacc += __shfl_xor_sync(full, rowacc, o2);
+                if (lg == 0 && row < p.rows) p.out[row] = rowacc;
+            }
+        }
+    }
+
+    if (agg == FO_CELL_FULL_AGG) {
+        block_sum<NOUT>(acc, s_red);
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int k = 0; k < NOUT; ++k)
+                if (k < ch.n_out) p.partials[(size_t)blockIdx.x * ch.n_out + k] = acc[k];
+        }
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, ch.n_out, p.out, s_red);
+    }
+}
+
+__global__ void csr_fill_zero_kernel(double *out, long long n)
+{
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+         i += (long long)gridDim.x * blockDim.x)
+        out[i] = 0.0;
+}
+
+cudaError_t fill_zero(double *out, long long n, cudaStream_t st)
+{
+    if (n <= 0) return cudaSuccess;
+    const long long b = (n + 255) / 256;
+    csr_fill_zero_kernel<<<(unsigned)(b > 1024 ? 1024 : b), 256, 0, st>>>(out, n);
+    return cudaGetLastError();
+}
+
+template <class EVAL, int NOUT>
+cudaError_t launch_by_group(const DevChain &ch, const CsrCellParams &p, double mean_len, int grid,
+                            cudaStream_t st)
+{
+    if (mean_len <= 12.0) cell_csr_kernel<EVAL, NOUT, 2><<<grid, kThreads, 0, st>>>(ch, p);
+    else if (mean_len <= 48.0) cell_csr_kernel<EVAL, NOUT, 8><<<grid, kThreads, 0, st>>>(ch, p);
+    else cell_csr_kernel<EVAL, NOUT, 32><<<grid, kThreads, 0, st>>>(ch, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t cell_csr_ws_bytes(int agg, int n_out)
+{
+    if (agg == FO_CELL_FULL_AGG) return sizeof(WsHead) + (size_t)kMaxPartials * (size_t)n_out * sizeof(double);
+    return sizeof(WsHead);
+}
+
+int run_cell_csr(const fo_chain *chain, const fo_csr &X, const fo_side *sides, int n_sides,
+                 const double *scalars, int n_scalars, int agg, bool magg, double *out, void *ws,
+                 size_t ws_bytes, void *stream)
+{
+    if (X.rows < 0 || X.cols < 0 || X.nnz < 0) return FO_ERR_SHAPE;
+    if (X.nnz > 0x7fffffffLL) return FO_ERR_UNSUPPORTED;
+    if (!X.rowptr) return FO_ERR_NULL;
+    if (X.nnz > 0 && (!X.colidx || !X.vals)) return FO_ERR_NULL;
+
+    DevChain ch;
+    int rc = translate_chain(chain, kUseCell, n_sides, scalars, n_scalars, 1, magg ? FO_MAX_OUT : 1, &ch);
+    if (rc != FO_OK) return rc;
+
+    CsrCellParams p;
+    memset(&p, 0, sizeof(p));
+    p.rowptr = X.rowptr; p.colidx = X.colidx; p.vals = X.vals;
+    p.rows = X.rows; p.cols = X.cols;
+    p.agg = agg;
+    p.sides.n = n_sides;
+    for (int k = 0; k < n_sides; ++k) {
+        const fo_side &s = sides[k];
+        if (s.m.rows < 0 || s.m.cols < 0 || s.m.ld < s.m.cols) return FO_ERR_SHAPE;
+        if (s.m.rows > 0 && s.m.cols > 0 && !s.m.data) return FO_ERR_NULL;
+        switch (s.access) {
+            case FO_AT_CELL: if (s.m.rows != X.rows || s.m.cols != X.cols) return FO_ERR_SHAPE; break;
+            case FO_AT_ROW: if (s.m.rows != X.rows || s.m.cols != 1) return FO_ERR_SHAPE; break;
+            case FO_AT_COL: if (s.m.rows != 1 || s.m.cols != X.cols) return FO_ERR_SHAPE; break;
+            default: return FO_ERR_SHAPE;
+        }
+        p.sides.s[k].data = s.m.data;
+        p.sides.s[k].ld = s.m.ld;
+        p.sides.s[k].access = s.access;
+    }
+    rc = check_workspace(ws, ws_bytes, cell_csr_ws_bytes(agg, ch.n_out));
+    if (rc != FO_OK) return rc;
+    p.head = (WsHead *)ws;
+    p.partials = (double *)((char *)ws + sizeof(WsHead));
+    p.out = out;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    // empty sums, and the accumulator of the atomic column sums
+    cudaError_t e = cudaSuccess;
+    if (agg == FO_CELL_COL_AGG) e = fill_zero(out, X.cols, st);
+    if (X.nnz == 0 || X.rows == 0) {
+        if (agg == FO_CELL_FULL_AGG) e = fill_zero(out, ch.n_out, st);
+        else if (agg == FO_CELL_ROW_AGG) e = fill_zero(out, X.rows, st);
+        return e == cudaSuccess ? FO_OK : cuda_fail(e);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    const int sms = sm_count();
+    if (sms <= 0) return cuda_fail(cudaErrorNoDevice);
+    const long long nblocks = (X.rows + 31) / 32;
+    long long grid = (nblocks + kThreads / 32 - 1) / (kThreads / 32);
+    if (grid > (long long)sms * 8) grid = (long long)sms * 8;
+    if (grid > kMaxPartials) grid = kMaxPartials;
+    const double mean_len = (double)X.nnz / (double)X.rows;
+
+    switch (force_interpreter() ? kSpecNone : match_cell_spec(ch)) {
+        case kSpecMul2: e = launch_by_group<EvalSpec<kSpecMul2>, 1>(ch, p, mean_len, (int)grid, st); break;
+        case kSpecMul3: e = launch_by_group<EvalSpec<kSpecMul3>, 1>(ch, p, mean_len, (int)grid, st); break;
+        case kSpecSq: e = launch_by_group<EvalSpec<kSpecSq>, 1>(ch, p, mean_len, (int)grid, st); break;
+        case kSpecMagg2: e = launch_by_group<EvalSpec<kSpecMagg2>, 2>(ch, p, mean_len, (int)grid, st); break;
+        case kSpecMagg3: e = launch_by_group<EvalSpec<kSpecMagg3>, 3>(ch, p, mean_len, (int)grid, st); break;
+        default:
+            if (ch.n_out == 1) e = launch_by_group<EvalInterp<kRegs>, 1>(ch, p, mean_len, (int)grid, st);
+            else e = launch_by_group<EvalInterp<kRegs>, FO_MAX_OUT>(ch, p, mean_len, (int)grid, st);
+    }
+    return e == cudaSuccess ? FO_OK : cuda_fail(e);
+}
+
+}  // namespace fo
