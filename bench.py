@@ -218,6 +218,8 @@ def time_variants(fo, step, shapes, reps=10):
     o_rr = torch.empty(rr, dtype=torch.float64, device=dev)
     o_nnz = torch.empty(nnz5, dtype=torch.float64, device=dev)
     o_right = torch.empty((orow, rank), dtype=torch.float64, device=dev)
+    ocol = shapes["outer"]["cols"]
+    o_left = torch.empty((ocol, rank), dtype=torch.float64, device=dev)
     generic = [("sub", "t0", "a", "side0"), ("abs", "t1", "t0"), ("fma", "t2", "t1", "side1", 0.5)]
 
     def interpreted(fn):
@@ -247,6 +249,8 @@ def time_variants(fo, step, shapes, reps=10):
                                                 agg="none", out=o_nnz), outer_in + 8 * nnz5),
         ("outer_right_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
                                                   agg="right", out=o_right), outer_in + 8 * orow * rank),
+        ("outer_left_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
+                                                 agg="left", out=o_left), outer_in + 8 * ocol * rank),
     ]
     # sparse-safe Cell / MAgg (Section 5.2's sparse variants): X at density 0.1 as the CSR driver,
     # dense Y and Z read at the stored cells

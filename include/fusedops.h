@@ -305,6 +305,9 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v,
  *   FO_OUTER_NO_AGG  : out[p] = w of stored cell p          (nnz doubles)
  *   FO_OUTER_RIGHT_MM: out[i * rank + c] = sum_j w_ij V_jc  (rows x rank, packed)
  *   FO_OUTER_LEFT_MM : out[j * rank + c] = sum_i w_ij U_ic  (cols x rank, packed)
+ * FO_OUTER_LEFT_MM adds into rows of `out` shared by all rows of X: global
+ * atomics on a zeroed result, so the order of its additions is not fixed; the
+ * other variants are bit-reproducible.
  * U V^T is never formed; cells that are not stored cost nothing.  Stored
  * zeros ARE visited (a chain tests a != 0 itself, as the listing does).
  * rank <= 256.  Errors: FO_ERR_SHAPE if U.rows != X.rows, V.rows != X.cols or

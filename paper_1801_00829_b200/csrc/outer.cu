@@ -34,7 +34,7 @@ struct OuterParams {
     int pad;
 };
 
-enum { kOutFull = 0, kOutNone = 1, kOutRight = 2 };
+enum { kOutFull = 0, kOutNone = 1, kOutRight = 2, kOutLeft = 3 };
 
 // Chains evaluated inline, in the chain's own operation order (same bits as the
 // interpreter): the weighted squared loss of Eq. 1, (a != 0) * (a - d)^2, and the
@@ -166,6 +166,23 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
                 if (valid) acc += w;
             } else if (AGG == kOutNone) {
                 if (valid) p.out[c0 + lane] = w;
+            } else if (AGG == kOutLeft) {
+                // second walk over the chunk: O_j += w_ij * U_i.  Rows of O are shared by
+                // all warps, so the additions are global atomics (their order is not fixed).
+                for (int it = 0; it < nit; ++it) {
+                    const int src = it * 4 + grp;
+                    const int j = __shfl_sync(full, jmine, src & 31);
+                    const double ww = __shfl_sync(full, w, src & 31);
+                    double *oj = p.out + (long long)j * rank;
+                    if (src < cnt) {
+#pragma unroll
+                        for (int c = 0; c < NK2; ++c) {
+                            const int col = 16 * c + 2 * l8;
+                            if (col < rank) atomicAdd(oj + col, ww * u[c].x);
+                            if (col + 1 < rank) atomicAdd(oj + col + 1, ww * u[c].y);
+                        }
+                    }
+                }
             } else {
                 // second walk over the chunk: O_i += w_ij * V_j (rows of V come from cache)
                 for (int it = 0; it < nit; ++it) {
@@ -390,6 +407,7 @@ cudaError_t launch_outer(const DevChain &ch, const OuterParams &p, int agg, bool
     } while (0)
     if (agg == FO_OUTER_FULL_AGG) FO_GO(kOutFull);
     else if (agg == FO_OUTER_NO_AGG) FO_GO(kOutNone);
+    else if (agg == FO_OUTER_LEFT_MM) FO_GO(kOutLeft);
     else FO_GO(kOutRight);
 #undef FO_GO
     return cudaGetLastError();
@@ -455,8 +473,8 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
 {
     using namespace fo;
     if (!chain || !X || !U || !V || !out) return FO_ERR_NULL;
-    if (agg == FO_OUTER_LEFT_MM) return FO_ERR_UNSUPPORTED;
-    if (agg != FO_OUTER_FULL_AGG && agg != FO_OUTER_NO_AGG && agg != FO_OUTER_RIGHT_MM)
+    if (agg != FO_OUTER_FULL_AGG && agg != FO_OUTER_NO_AGG && agg != FO_OUTER_RIGHT_MM &&
+        agg != FO_OUTER_LEFT_MM)
         return FO_ERR_UNSUPPORTED;
     if (X->rows < 0 || X->cols < 0 || X->nnz < 0) return FO_ERR_SHAPE;
     if (X->nnz >= (1ll << 31)) return FO_ERR_UNSUPPORTED;
@@ -485,15 +503,19 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     p.chain_kind = fo::force_interpreter() ? fo::kOuterGeneric : fo::outer_chain_kind(ch, &p.kconst);
     cudaStream_t st = (cudaStream_t)stream;
 
-    if (X->nnz == 0 || X->rows == 0) {
+    const bool empty = X->nnz == 0 || X->rows == 0;
+    if (empty || agg == FO_OUTER_LEFT_MM) {
+        // empty sums; left_mm accumulates into a zeroed result
         const long long nout = agg == FO_OUTER_FULL_AGG ? 1
-                             : agg == FO_OUTER_RIGHT_MM ? X->rows * rank : 0;
+                             : agg == FO_OUTER_RIGHT_MM ? X->rows * rank
+                             : agg == FO_OUTER_LEFT_MM ? X->cols * rank : 0;
         if (nout > 0) {
             const long long b = (nout + 255) / 256;
             outer_fill_zero_kernel<<<(unsigned)(b > 1024 ? 1024 : b), 256, 0, st>>>(out, nout);
         }
         const cudaError_t e = cudaGetLastError();
-        return e == cudaSuccess ? FO_OK : cuda_fail(e);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (empty) return FO_OK;
     }
 
     const int sms = sm_count();
@@ -508,7 +530,8 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     cudaError_t e;
     const int nk2 = (rank + 15) / 16;
     // factor rows that are 16-byte aligned pieces go through the staged kernel
-    const bool staged = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && !getenv("FUSEDOPS_OUTER_DIRECT");
+    const bool staged = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && agg != FO_OUTER_LEFT_MM &&
+                        !getenv("FUSEDOPS_OUTER_DIRECT");
     if (staged) {
         if (nk2 <= 1) e = launch_outer_staged<1>(ch, p, agg, (int)grid, st);
         else if (nk2 <= 2) e = launch_outer_staged<2>(ch, p, agg, (int)grid, st);

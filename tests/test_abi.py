@@ -160,7 +160,7 @@ def test_row_and_outer_argument_errors(lib):
     u2 = B.fo_dense()
     u2.rows, u2.cols, u2.ld, u2.data = 11, 4, 4, 0x8000
     assert outer(uu=u2) == -2                             # U.rows != X.rows
-    assert outer(agg=0) == -4                             # left_mm not provided
+    assert outer(agg=7) == -4                             # no such variant
     x2 = B.fo_csr()
     x2.rows, x2.cols, x2.nnz = 10, 12, 1 << 31
     x2.rowptr, x2.colidx, x2.vals = 0x5000, 0x6000, 0x7000

@@ -286,8 +286,8 @@ def test_outer_full_agg(fo, rows, cols, rank, density):
         assert_close(got.cpu().numpy(), [oracle.outer_wsloss_dense(Xh, w["U"], w["V"])])
 
 
-@pytest.mark.parametrize("agg", ["none", "right"])
-@pytest.mark.parametrize("rank", [5, 100])
+@pytest.mark.parametrize("agg", ["none", "right", "left"])
+@pytest.mark.parametrize("rank", [5, 100, 200])
 def test_outer_other_aggs(fo, agg, rank):
     w, Xh = outer_case(700, 900, rank, 0.02, seed=14)
     chain = [("ne", "t0", "a", 0.0), ("mul", "t1", "t0", "d")]          # (X != 0) * (U V^T), Eq. 1
