@@ -249,6 +249,9 @@ def time_variants(fo, step, shapes, reps=10):
                                                 agg="none", out=o_nnz), outer_in + 8 * nnz5),
         ("outer_right_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
                                                   agg="right", out=o_right), outer_in + 8 * orow * rank),
+        ("outer_x_log_uvt_plus_eps", lambda: fo.fused_outer(
+            [("add", "t0", "d", "s0"), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")], "t2", step.csr5,
+            d["outer.U"], d["outer.V"], [10.0], agg="full", out=o_one), outer_in + 8),
         ("outer_left_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
                                                  agg="left", out=o_left), outer_in + 8 * ocol * rank),
     ]
