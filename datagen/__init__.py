@@ -100,10 +100,11 @@ def csr_bernoulli(seed, stream, rows, cols, density, lo=0.0, hi=1.0, row0=0):
 
 from .workloads import (  # noqa: E402
     cell_workload, magg_workload, row_dense_workload, row_csr_workload, outer_workload,
+    row_b1_workload,
 )
 
 __all__ = [
     "build", "uniform", "normal", "csr_bernoulli",
     "cell_workload", "magg_workload", "row_dense_workload", "row_csr_workload",
-    "outer_workload",
+    "outer_workload", "row_b1_workload",
 ]

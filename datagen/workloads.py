@@ -78,6 +78,20 @@ def outer_workload(rows=100_000, cols=100_000, rank=100, density=0.001, seed=4):
     }
 
 
+def row_b1_workload(rows=1_000_000, cols=1000, k=2, seed=5, out=None):
+    """Row template with a matrix-valued row intermediate: X dense N(0,1)
+    (rows x cols), V dense N(0,1) (cols x k), and P (rows x k) uniform[0, 1/(k+1))
+    - entries shaped like the first k of k+1 class probabilities, so that a
+    row of P sums to less than one."""
+    g = _gen()
+    out = out or {}
+    return {
+        "X": g.normal(seed, 0, rows * cols, out=out.get("X")).reshape(rows, cols),
+        "V": g.normal(seed, 2, cols * k).reshape(cols, k),
+        "P": g.uniform(seed, 3, rows * k, 0.0, 1.0 / (k + 1), out=out.get("P")).reshape(rows, k),
+    }
+
+
 def csr_to_dense(rows, cols, rowptr, colidx, vals):
     """Scatter a CSR matrix into a dense array (format conversion only)."""
     d = np.zeros((rows, cols), dtype=np.float64)

@@ -20,12 +20,15 @@ Outer template.  Every function below is covered by at least one of them.
 
 Chains.  A scalar operator chain is a list of steps ``(op, dst, a[, b[, c]])``:
 ``dst`` is a temporary name ``"t0".."t7"``; operands are ``"a"`` (main-input
-value), ``"d"`` (Row: the row's dot product; Outer: U_i . V_j), ``"sideK"``,
+value), ``"d"`` (Row: the row's dot product, for the B1 variants one entry of the row's
+product with the side matrix; Outer: U_i . V_j), ``"rowsum"`` (B1 variants: the
+row sum of the first chain), ``"sideK"``,
 ``"sK"`` (K-th scalar), ``"tK"`` or a Python float.  Outputs are operand names.
 """
 from .ops import (
     OPS, eval_chain, full_sum, row_sums, col_sums,
-    cell, magg, row, outer,
+    cell, magg, row, row_b1, outer,
+    mmchain, mlogreg_inner,
     sum_xyz, magg_xy_xz_xx, row_chain_dense, row_chain_csr,
     outer_wsloss_dense, outer_wsloss_masked,
     csr_row_ids,
@@ -33,7 +36,7 @@ from .ops import (
 
 __all__ = [
     "OPS", "eval_chain", "full_sum", "row_sums", "col_sums",
-    "cell", "magg", "row", "outer",
+    "cell", "magg", "row", "row_b1", "outer", "mmchain", "mlogreg_inner",
     "sum_xyz", "magg_xy_xz_xx", "row_chain_dense", "row_chain_csr",
     "outer_wsloss_dense", "outer_wsloss_masked", "csr_row_ids",
 ]

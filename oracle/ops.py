@@ -10,7 +10,10 @@ Paper passages followed:
   MAgg  - Table 1 and "Multi-Aggregate Operations" in Section 5.2: several
           full aggregates over shared inputs, returned as a k x 1 column.
   Row   - Fig. 1(b) / "Row Operations" in Section 5.2: X^T (w * (X v)) is the
-          unfused sequence  t1 = X v ; t2 = w * t1 ; q = X^T t2.
+          unfused sequence  t1 = X v ; t2 = w * t1 ; q = X^T t2.  With a side
+          matrix instead of v (Table 1, the *_B1 variants; Eq. 2 and its row-wise
+          listing in Section 2.2) the row intermediate is a k-vector:
+          D = X V ; T = chains(D, sides, rowSums) ; H = X^T T.
   Outer - Fig. 1(d), Eq. 1 and the outer-product listing of Section 2.2: for
           every stored X_ij the scalar chain sees a = X_ij and d = U_i . V_j;
           unfused, d is the dense product U V^T masked by X's pattern.
@@ -259,6 +262,73 @@ def row(chain, output, X, v, sides=(), scalars=(), agg="col_t"):
     if agg == "full":
         return full_sum(t)
     raise ValueError(agg)
+
+
+def row_b1(pre, pre_out, post, post_out, X, B, sides=(), scalars=(), agg="col_t"):
+    """Row template with a matrix-valued row intermediate (Table 1: the *_B1
+    variants; the row-wise listing of Section 2.2 for Eq. 2; "Row Operations" in
+    Section 5.2 for t(X) %*% (X %*% V)).  X is dense m x n, B dense n x k.
+
+    D  = X B                     first scan of X: m x k (the listing's vectMatMult)
+    P  = pre(d = D, sides)       m x k, and  s = rowSums(P)  (vectSum); skipped
+                                 when `pre` is None
+    T  = post(d = D, sides, rowsum = s broadcast over the k columns)   m x k
+    agg "col_t": H = X^T T       second scan of X: n x k (vectOuterMultAdd)
+        "none" : T itself        m x k
+    Sides: ("cell", m x k) read at (row, class), ("row", m) read at the row,
+    ("col", k) read at the class.
+    """
+    X = np.asarray(X, dtype=np.float64)
+    B = np.asarray(B, dtype=np.float64)
+    m, n = X.shape
+    assert B.shape[0] == n
+    k = B.shape[1]
+    D = X @ B
+    env = {"d": D}
+    for j, (access, arr) in enumerate(sides):
+        arr = np.asarray(arr, dtype=np.float64)
+        if access == "cell":
+            assert arr.shape == (m, k)
+            env["side%d" % j] = arr
+        elif access == "row":
+            assert arr.shape == (m,)
+            env["side%d" % j] = arr.reshape(m, 1)
+        elif access == "col":
+            assert arr.shape == (k,)
+            env["side%d" % j] = arr.reshape(1, k)
+        else:
+            raise ValueError(access)
+    for j, s in enumerate(scalars):
+        env["s%d" % j] = np.float64(s)
+    if pre is not None:
+        (P,) = eval_chain(pre, [pre_out], env, (m, k))
+        env["rowsum"] = row_sums(P).reshape(m, 1)
+    (T,) = eval_chain(post, [post_out], env, (m, k))
+    if agg == "col_t":
+        return X.T @ T
+    if agg == "none":
+        return T
+    raise ValueError(agg)
+
+
+def mmchain(X, V):
+    """t(X) %*% (X %*% V) with its m x k intermediate (Section 5.2, "Row
+    Operations": the matrix-matrix multiplication chain)."""
+    T1 = X @ V
+    return X.T @ T1
+
+
+def mlogreg_inner(X, V, P):
+    """Eq. 2, written out one basic operator at a time (P stands for P[,1:k],
+    m x k; V is n x k):
+        Q = P * (X V);   H = X^T (Q - P * rowSums(Q))
+    """
+    T1 = X @ V
+    Q = P * T1
+    s = row_sums(Q).reshape(-1, 1)
+    T2 = P * s
+    T3 = Q - T2
+    return X.T @ T3
 
 
 # --------------------------------------------------------------------------

@@ -263,6 +263,111 @@ def test_row_other_aggregations():
     assert np.allclose(q, rat_row_chain(X, v, np.ones(8)), rtol=1e-13, atol=1e-15)
 
 
+# ------------------------------------------------------------------ Row, matrix-valued intermediates
+MLR_PRE = [("mul", "t0", "side0", "d")]
+MLR_POST = [("mul", "t0", "side0", "d"), ("mul", "t1", "side0", "rowsum"), ("sub", "t2", "t0", "t1")]
+
+
+def rat_mlogreg(X, V, P):
+    """Eq. 2 in exact rationals: H_jc = sum_i X_ij (Q_ic - P_ic * sum_c' Q_ic'), Q = P * (X V)."""
+    m, n = X.shape
+    k = V.shape[1]
+    H = [[F(0)] * k for _ in range(n)]
+    for i in range(m):
+        D = [sum((F(float(X[i, j])) * F(float(V[j, c])) for j in range(n)), F(0)) for c in range(k)]
+        Q = [F(float(P[i, c])) * D[c] for c in range(k)]
+        s = sum(Q, F(0))
+        T = [Q[c] - F(float(P[i, c])) * s for c in range(k)]
+        for j in range(n):
+            for c in range(k):
+                H[j][c] += F(float(X[i, j])) * T[c]
+    return np.array([[float(x) for x in r] for r in H])
+
+
+def test_row_b1_bruteforce_rational():
+    for (m, n, k) in [(7, 5, 3), (4, 9, 2), (1, 3, 4), (6, 1, 1), (5, 4, 5)]:
+        w = datagen.row_b1_workload(m, n, k, seed=5)
+        X, V, P = w["X"], w["V"], w["P"]
+        ref = rat_mlogreg(X, V, P)
+        aX, aV = np.abs(X), np.abs(V)
+        scale = aX.T @ (2.0 * P * (aX @ aV) + 1e-300)
+        got = oracle.mlogreg_inner(X, V, P)
+        assert got.shape == (n, k)
+        assert np.all(np.abs(got - ref) <= 4e-15 * scale)
+        # the generic two-chain form states the same expression
+        got2 = oracle.row_b1(MLR_PRE, "t0", MLR_POST, "t2", X, V, [("cell", P)], agg="col_t")
+        assert np.all(np.abs(got2 - ref) <= 4e-15 * scale)
+        # no aggregation: the m x k row intermediates themselves
+        T = oracle.row_b1(MLR_PRE, "t0", MLR_POST, "t2", X, V, [("cell", P)], agg="none")
+        D = X @ V
+        for i in range(m):
+            Q = [F(float(P[i, c])) * F(float(D[i, c])) for c in range(k)]
+            s = float(sum(Q, F(0)))
+            for c in range(k):
+                want = float(P[i, c]) * float(D[i, c]) - float(P[i, c]) * s
+                assert abs(T[i, c] - want) <= 1e-14 * (abs(want) + abs(s))
+
+
+def test_row_b1_probability_rows_give_zero_column_total():
+    # if every row of P sums to one, sum_c (Q_ic - P_ic * rowSums(Q)_i) = 0, so the
+    # columns of H add up to the zero vector: a sign or index slip in Eq. 2 breaks it
+    m, n, k = 40, 6, 4
+    w = datagen.row_b1_workload(m, n, k, seed=6)
+    P = w["P"] / w["P"].sum(axis=1, keepdims=True)
+    H = oracle.mlogreg_inner(w["X"], w["V"], P)
+    scale = np.abs(w["X"]).T @ (P * (np.abs(w["X"]) @ np.abs(w["V"]))).sum(axis=1)
+    assert np.all(np.abs(H.sum(axis=1)) <= 1e-13 * scale)
+    assert np.max(np.abs(H)) > 1e-3            # and H itself is not zero
+
+
+def test_row_b1_mmchain_special_cases():
+    m, n, k = 11, 6, 3
+    w = datagen.row_b1_workload(m, n, k, seed=7)
+    X, V = w["X"], w["V"]
+    H = oracle.mmchain(X, V)
+    # column c of t(X) (X V) is the vector chain with v = V[:, c]
+    for c in range(k):
+        ref = rat_row_chain(X, V[:, c], np.ones(m))
+        assert np.allclose(H[:, c], ref, rtol=1e-13, atol=1e-14)
+    # generic form with the identity chain
+    H2 = oracle.row_b1(None, None, [], "d", X, V, agg="col_t")
+    assert H2.tolist() == H.tolist()
+    # X = I: t(I) (I V) = V exactly
+    E = np.eye(n)
+    assert oracle.mmchain(E, V).tolist() == V.tolist()
+    # a one-column V is the Row template's vector form (col_t_agg), bit for bit
+    q = oracle.row([], "d", X, V[:, 0], agg="col_t")
+    assert oracle.mmchain(X, V[:, :1])[:, 0].tolist() == q.tolist()
+    # a non-square X: transposing the first factor would not even have the right shape
+    assert H.shape == (n, k)
+    # small integers: every intermediate exact
+    Xi = np.arange(1, 1 + m * n, dtype=np.float64).reshape(m, n) % 7 - 3
+    Vi = np.arange(1, 1 + n * k, dtype=np.float64).reshape(n, k) % 5 - 2
+    Hi = oracle.mmchain(Xi, Vi)
+    want = [[sum(int(Xi[i, j]) * sum(int(Xi[i, l]) * int(Vi[l, c]) for l in range(n)) for i in range(m))
+             for c in range(k)] for j in range(n)]
+    assert Hi.tolist() == [[float(x) for x in r] for r in want]
+
+
+def test_row_b1_side_kinds_and_scalars():
+    # T_ic = (d * rowvec_c + colvec_i) * s0 - rowsum, rowsum = sum_c d * rowvec_c
+    m, n, k = 5, 4, 3
+    w = datagen.row_b1_workload(m, n, k, seed=8)
+    X, V = w["X"], w["V"]
+    cvec = datagen.normal(8, 9, m)            # read at the row
+    rvec = datagen.normal(8, 10, k)           # read at the class
+    pre = [("mul", "t0", "d", "side0")]
+    post = [("mul", "t0", "d", "side0"), ("add", "t1", "t0", "side1"), ("mul", "t2", "t1", "s0"),
+            ("sub", "t3", "t2", "rowsum")]
+    T = oracle.row_b1(pre, "t0", post, "t3", X, V, [("col", rvec), ("row", cvec)], [2.5], agg="none")
+    D = X @ V
+    for i in range(m):
+        rs = fsum_exact([D[i, c] * rvec[c] for c in range(k)])
+        for c in range(k):
+            want = (D[i, c] * rvec[c] + cvec[i]) * 2.5 - rs
+            assert abs(T[i, c] - want) <= 1e-14 * (abs(want) + abs(rs) + 1.0)
+
+
 def test_row_csr_equals_dense_and_bruteforce():
     m, n = 40, 25
     w_ = datagen.row_csr_workload(m, n, 0.2, seed=3)
