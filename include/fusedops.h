@@ -135,11 +135,12 @@ typedef struct fo_chain {
 /* ------------------------------------------------------ template variants */
 /* Cell (Table 1: no_agg, row_agg, col_agg, full_agg) */
 enum { FO_CELL_NO_AGG = 0, FO_CELL_ROW_AGG = 1, FO_CELL_COL_AGG = 2, FO_CELL_FULL_AGG = 3 };
-/* Row (Table 1).  Implemented: ROW_AGG (one value per row), FULL_AGG, COL_T_AGG
- * (the n x 1 vector sum_i t_i * X_i^T).  NO_AGG, COL_AGG and the *_B1 variants
- * return FO_ERR_UNSUPPORTED. */
+/* Row (Table 1).  fused_row implements ROW_AGG (one value per row), FULL_AGG and
+ * COL_T_AGG (the n x 1 vector sum_i t_i * X_i^T); NO_AGG and COL_AGG return
+ * FO_ERR_UNSUPPORTED.  The *_B1 variants (row intermediates that are k-vectors,
+ * from a product with a side matrix) belong to fused_row_b1. */
 enum { FO_ROW_NO_AGG = 0, FO_ROW_ROW_AGG = 1, FO_ROW_COL_AGG = 2, FO_ROW_FULL_AGG = 3,
-       FO_ROW_COL_T_AGG = 4 };
+       FO_ROW_COL_T_AGG = 4, FO_ROW_NO_AGG_B1 = 5, FO_ROW_COL_AGG_B1_T = 6 };
 /* Outer (Table 1: left_mm, right_mm, no_agg, full_agg) */
 enum { FO_OUTER_LEFT_MM = 0, FO_OUTER_RIGHT_MM = 1, FO_OUTER_NO_AGG = 2, FO_OUTER_FULL_AGG = 3 };
 
@@ -150,6 +151,7 @@ size_t fused_cell_workspace_bytes(const fo_mat *X, int agg);
 size_t fused_magg_workspace_bytes(const fo_mat *X, int n_out);
 size_t fused_row_workspace_bytes(const fo_mat *X, int agg);
 size_t fused_outer_workspace_bytes(const fo_csr *X, int rank, int agg);
+size_t fused_row_b1_workspace_bytes(const fo_mat *X, int k, int agg);
 
 /* Clears the control words at the head of a workspace (asynchronous on `stream`).
  * Needed once after allocation, and again after a call returned
@@ -295,6 +297,38 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v,
               const fo_side *sides, int n_sides,
               const double *scalars, int n_scalars,
               int agg, double *out, void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------- Row, matrix-valued intermediates
+ * Table 1, Row template, variants no_agg_B1 / col_agg_B1; Eq. 2 and the row-wise
+ * operator listing of Section 2.2 (RowType COL_AGG_B1_T); Section 5.2 "Row
+ * Operations" (t(X) %*% (X %*% V)) and "Hybrid Algorithms" (k = 2 .. 32).
+ * One pass over the rows of a dense X (rows x n).  B is a dense n x k side
+ * matrix, 1 <= k <= FO_B1_MAX_K.  For row i:
+ *     D_ic = X_i . B[:, c]                       c = 0 .. k-1  (the listing's vectMatMult)
+ *     s_i  = sum_c pre(d = D_ic, sides, scalars)               (vectSum; pre may be NULL)
+ *     T_ic = post(d = D_ic, sides, s_i, scalars)
+ *   FO_ROW_COL_AGG_B1_T: out[j * k + c] = sum_i X_ij T_ic   (n x k, packed; vectOuterMultAdd)
+ *   FO_ROW_NO_AGG_B1   : out[i * k + c] = T_ic              (rows x k, packed)
+ * In both chains FO_DOT names D_ic.  Sides: FO_AT_CELL sides are rows x k and
+ * are read at (i, c); FO_AT_ROW sides rows x 1, read at (i); FO_AT_COL sides
+ * 1 x k, read at (c).  In `post`, FO_ROWSUM(n_sides) names s_i: it takes the
+ * side slot right behind the call's own sides, so with `pre` given at most
+ * FO_MAX_SIDES - 1 sides can be passed; without `pre` that operand is invalid.
+ * With pre = NULL and an empty post chain whose result is FO_DOT this is
+ * t(X) %*% (X %*% B); with one FO_AT_CELL side P, pre = P * d and
+ * post = P * d - P * s it is Eq. 2.
+ * Limits (FO_ERR_UNSUPPORTED beyond them): dense X only; k <= 32; the columns
+ * a group of warps can hold shrink as k grows (n <= 4096 for k <= 2, 2048 for
+ * k <= 4, 1024 for k <= 8, 512 for k <= 16, 256 for k <= 32); for col_agg_B1_T
+ * n * k <= 24576 (the CTA's output tile lives in shared memory).
+ * Bit-reproducible for given shapes.
+ */
+#define FO_B1_MAX_K 32
+#define FO_ROWSUM(n_sides)  FO_SIDE(n_sides)
+int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, const fo_dense *B,
+                 const fo_side *sides, int n_sides,
+                 const double *scalars, int n_scalars,
+                 int agg, double *out, void *ws, size_t ws_bytes, void *stream);
 
 /* ----------------------------------------------------------------- Outer
  * Table 1, Outer template; Fig. 1(d), Eq. 1 and the outer-product listing of

@@ -4,7 +4,7 @@ The work happens in ``libfusedops.so`` (CUDA, sm_100a; C ABI in
 ``include/fusedops.h``); this package is the thin ctypes binding around it.
 """
 from .binding import (  # noqa: F401
-    CSR, FusedOpsError, chain_describe, device_status, force_interpreter, fused_cell, fused_cell_static, fused_magg, fused_outer, fused_row,
+    CSR, FusedOpsError, chain_describe, device_status, force_interpreter, fused_cell, fused_cell_static, fused_magg, fused_outer, fused_row, fused_row_b1,
     jit_compile_check, jit_stats, load_library, make_chain, probe_fp64_fma, probe_l2_gather, probe_out_len, set_jit,
     workspace,
 )
@@ -12,6 +12,6 @@ from .roofline import algorithmic_bytes, ideal_seconds  # noqa: F401
 
 __all__ = [
     "CSR", "FusedOpsError", "chain_describe", "device_status", "force_interpreter", "fused_cell", "fused_cell_static", "fused_magg", "fused_outer",
-    "fused_row", "jit_compile_check", "jit_stats", "set_jit", "load_library", "make_chain", "workspace", "algorithmic_bytes", "ideal_seconds",
+    "fused_row", "fused_row_b1", "jit_compile_check", "jit_stats", "set_jit", "load_library", "make_chain", "workspace", "algorithmic_bytes", "ideal_seconds",
     "probe_fp64_fma", "probe_l2_gather", "probe_out_len",
 ]

@@ -32,6 +32,7 @@ ARITY = {**{n: 1 for n in ("mov", "neg", "abs", "sqrt", "exp", "log", "sq")},
 
 CELL_AGG = {"none": 0, "row": 1, "col": 2, "full": 3}
 ROW_AGG = {"none": 0, "row": 1, "col": 2, "full": 3, "col_t": 4}
+ROW_B1_AGG = {"none": 5, "col_t": 6}
 OUTER_AGG = {"left": 0, "right": 1, "none": 2, "full": 3}
 ACCESS = {"cell": 0, "row": 1, "col": 2}
 
@@ -75,7 +76,8 @@ class fo_chain(C.Structure):
 
 
 EXPORTS = [
-    "fused_cell", "fused_magg", "fused_row", "fused_outer",
+    "fused_cell", "fused_magg", "fused_row", "fused_outer", "fused_row_b1",
+    "fused_row_b1_workspace_bytes",
     "fused_cell_workspace_bytes", "fused_magg_workspace_bytes", "fused_row_workspace_bytes",
     "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
@@ -103,8 +105,12 @@ def load_library(path=None):
         lib.fused_row.argtypes = [chain_p, mat_p, dp, side_p, i32, scal_p, i32, i32, dp, vp, sz, vp]
         lib.fused_outer.argtypes = [chain_p, C.POINTER(fo_csr), C.POINTER(fo_dense),
                                     C.POINTER(fo_dense), scal_p, i32, i32, dp, vp, sz, vp]
-        for f in (lib.fused_cell, lib.fused_magg, lib.fused_row, lib.fused_outer):
+        lib.fused_row_b1.argtypes = [chain_p, chain_p, mat_p, C.POINTER(fo_dense), side_p, i32, scal_p, i32,
+                                     i32, dp, vp, sz, vp]
+        for f in (lib.fused_cell, lib.fused_magg, lib.fused_row, lib.fused_outer, lib.fused_row_b1):
             f.restype = C.c_int
+        lib.fused_row_b1_workspace_bytes.argtypes = [mat_p, i32, i32]
+        lib.fused_row_b1_workspace_bytes.restype = C.c_size_t
         lib.fused_cell_workspace_bytes.argtypes = [mat_p, i32]
         lib.fused_magg_workspace_bytes.argtypes = [mat_p, i32]
         lib.fused_row_workspace_bytes.argtypes = [mat_p, i32]
@@ -159,8 +165,11 @@ def _check(status, what):
 
 
 # ------------------------------------------------------------------ marshalling
-def _operand(x, allow_imm=True):
-    """Operand name -> (operand byte, immediate or None)."""
+def _operand(x, allow_imm=True, rowsum_side=None):
+    """Operand name -> (operand byte, immediate or None).  "rowsum" (second chain of
+    fused_row_b1) is the side slot `rowsum_side`, right behind the call's own sides."""
+    if x == "rowsum" and rowsum_side is not None:
+        return 0x40 | int(rowsum_side), None
     if isinstance(x, (int, float)) and not isinstance(x, bool):
         if not allow_imm:
             raise ValueError("an output cannot be an immediate")
@@ -180,7 +189,7 @@ def _operand(x, allow_imm=True):
     raise ValueError("bad operand %r" % (x,))
 
 
-def make_chain(steps, outputs):
+def make_chain(steps, outputs, rowsum_side=None):
     """Builds the fo_chain for `steps` and `outputs`; returns (chain, keepalive)."""
     steps = list(steps)
     outputs = [outputs] if isinstance(outputs, (str, float, int)) else list(outputs)
@@ -200,7 +209,7 @@ def make_chain(steps, outputs):
         imm = None
         enc = []
         for s in srcs:
-            b, im = _operand(s)
+            b, im = _operand(s, rowsum_side=rowsum_side)
             if im is not None:
                 if imm is not None and imm != im:
                     raise ValueError("a step can carry one immediate value")
@@ -214,7 +223,7 @@ def make_chain(steps, outputs):
     ch.n_out = len(outputs)
     ch.ops = C.cast(ops, C.POINTER(fo_op))
     for k, o in enumerate(outputs):
-        ch.out[k] = _operand(o, allow_imm=False)[0]
+        ch.out[k] = _operand(o, allow_imm=False, rowsum_side=rowsum_side)[0]
     return ch, ops
 
 
@@ -477,6 +486,35 @@ def fused_row(steps, output, X, v, sides=(), scalars=(), agg="col_t", out=None):
     _check(lib.fused_row(C.byref(ch), C.byref(m), C.c_void_p(v.data_ptr()), sarr, len(sides), sc,
                          len(scalars), a, C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()),
                          ws.numel(), _stream(dev)), "fused_row")
+    return out
+
+
+def fused_row_b1(pre, pre_out, post, post_out, X, B, sides=(), scalars=(), agg="col_t", out=None):
+    """Row template with a matrix-valued row intermediate (side matrix B, n x k).
+    `pre` may be None; in `post` the operand "rowsum" names the row sum of `pre`.
+    Returns (cols, k) for agg "col_t", (rows, k) for "none"."""
+    lib = load_library()
+    sides = list(sides)
+    post_ch, keep2 = make_chain(post, post_out, rowsum_side=len(sides) if pre is not None else None)
+    pre_ref = None
+    if pre is not None:
+        pre_ch, keep1 = make_chain(pre, pre_out)
+        pre_ref = C.byref(pre_ch)
+    m = _mat(X)
+    rows, cols = X.shape
+    dev = X.device
+    a = ROW_B1_AGG[agg]
+    assert B.dtype == torch.float64 and B.dim() == 2
+    k = B.shape[1]
+    bs = _dense_struct(B)
+    if out is None:
+        out = torch.empty((cols, k) if agg == "col_t" else (rows, k), dtype=torch.float64, device=dev)
+    need = lib.fused_row_b1_workspace_bytes(C.byref(m), k, a)
+    ws = workspace(dev, max(need, 16384))
+    sarr, sc = _sides(sides, rows, k), _scalars(scalars)
+    _check(lib.fused_row_b1(pre_ref, C.byref(post_ch), C.byref(m), C.byref(bs), sarr, len(sides), sc,
+                            len(scalars), a, C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()),
+                            ws.numel(), _stream(dev)), "fused_row_b1")
     return out
 
 

@@ -15,6 +15,7 @@
 #include <type_traits>
 
 #include "chain.cuh"
+#include "ptx.cuh"
 
 namespace fo {
 
@@ -43,56 +44,6 @@ enum { kChainGeneric = 0, kChainSideTimesDot = 1, kChainDot = 2 };
 enum { kRowColT = 0, kRowRow = 1, kRowFull = 2 };
 
 constexpr int kWarps = kThreads / 32;
-constexpr unsigned kWaitLimit = 1u << 22;     // polls of one mbarrier wait before giving up
-
-// ---------------------------------------------------------------- PTX helpers
-__device__ __forceinline__ unsigned smem_u32(const void *p)
-{
-    return (unsigned)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
-                 "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long *bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: returns false (and the caller records it) if the phase never completes.
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity)
-{
-    for (unsigned i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-// Bulk asynchronous copy global -> shared; completion is counted on `bar`.
-// src, dst 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes,
-                                         unsigned long long *bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-        : "memory");
-}
 
 // The chain for one row per lane: R0 = d, R(1+k) = side k of that lane's row.
 template <int NR>
@@ -134,35 +85,6 @@ constexpr int kDenseThreads = 512;                 // compute threads
 constexpr int kDenseWarps = kDenseThreads / 32;
 constexpr int kDenseBlock = kDenseThreads + 32;    // plus the warp that feeds the ring
 constexpr int kDenseMaxSlots = 64;                 // ring slots of all groups together
-
-// Sums R values per lane over the 32 lanes of a warp in a fixed order.  On
-// return v[0] holds, in every lane l, the total of value number (l >> (5 - log2 R)).
-template <int R>
-__device__ __forceinline__ void warp_sum_multi(double (&v)[R], int lane)
-{
-    int mask = 16;
-#pragma unroll
-    for (int half = R / 2; half >= 1; half /= 2) {
-        const bool up = (lane & mask) != 0;
-#pragma unroll
-        for (int i = 0; i < half; ++i) {
-            const double send = up ? v[i] : v[i + half];
-            const double keep = up ? v[i + half] : v[i];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
-        }
-        mask >>= 1;
-    }
-    for (; mask >= 1; mask >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], mask);
-}
-
-template <int R>
-struct Log2 {
-    static constexpr int value = 1 + Log2<R / 2>::value;
-};
-template <>
-struct Log2<1> {
-    static constexpr int value = 0;
-};
 
 template <int NCH, int W, int R, int AGG, bool STAGED>
 __global__ void __launch_bounds__(kDenseBlock, 1)

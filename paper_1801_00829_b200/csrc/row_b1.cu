@@ -1,0 +1,595 @@
+// Row template with matrix-valued row intermediates (Table 1: no_agg_B1 /
+// col_agg_B1; Eq. 2 and its row-wise listing in Section 2.2; Section 5.2 "Row
+// Operations", t(X) %*% (X %*% V)).  Per row i of a dense X and a side matrix
+// B (n x k):  D_i = X_i B  (k values),  s_i = sum_c pre(D_ic),  T_ic = post(D_ic, s_i),
+// then  out += X_i^T T_i  (n x k)  or  out[i] = T_i.
+//
+// The row is read from HBM once.  A CTA's 16 warps form independent groups; a
+// group streams its tiles of R rows through its own shared-memory ring with
+// bulk asynchronous copies (bounded waits): once the group's barrier of a tile
+// has been passed every warp holds its pieces of the tile in registers, so one
+// elected lane refills that slot right away - nobody waits for a free slot.  Inside a group W warps
+// split the columns and KW warps split the k classes into slices of KL; a lane
+// keeps its column pairs of the tile's rows in registers for both uses, takes
+// B (transposed, zero-padded) from shared memory, and owns the output
+// accumulators of (its columns) x (its class slice) in registers.
+#include <stdio.h>
+#include <stdlib.h>
+
+#include "chain.cuh"
+#include "ptx.cuh"
+
+namespace fo {
+
+namespace {
+
+struct B1Params {
+    const double *X;
+    long long rows, cols, ldx;
+    const double *B;            // n x k, row-major
+    long long ldb;
+    int k;
+    DevSides sides;
+    WsHead *head;
+    double *partials;
+    double *out;
+    int stages;                 // ring slots per group
+    int W, KW;                  // warps of a group across columns / across class slices
+    int chain_kind;
+    int has_pre;
+    unsigned side_used;         // sides read by either chain
+};
+
+// Chains evaluated inline (same arithmetic, same order, same bits as the interpreter).
+enum { kB1Generic = 0, kB1Identity = 1, kB1Mlogreg = 2 };
+enum { kB1ColT = 0, kB1None = 1 };
+
+constexpr int kB1Warps = 16;
+constexpr int kB1Block = kB1Warps * 32;            // 4 warps per SM sub-partition: 128 registers a thread
+constexpr int kB1MaxSlots = 64;
+constexpr int kB1MaxTile = 64;                     // R * (padded k) values of one tile
+
+// The chain for one (row, class) value per lane: R0 = d, R(1 + j) = side j.
+// Out of line: the interpreter's register file must not weigh on the streaming
+// loop, which the common chains (evaluated inline) never leave.
+__device__ __noinline__ double b1_lane_chain(const DevChain &ch, double d, double s0, double s1, double s2,
+                                             double s3)
+{
+    RegFile<kRegs, 1> f;
+    f.r[0][0] = d;
+    f.r[1][0] = s0;
+    f.r[2][0] = s1;
+    f.r[3][0] = s2;
+    f.r[4][0] = s3;
+    run_chain<kRegs, 1>(ch, f);
+    double o[1];
+    operand<kRegs, 1>(ch, f, ch.out[0], o);
+    return o[0];
+}
+
+// GENERIC: the chains go through the interpreter; otherwise only the chains
+// evaluated inline exist in the kernel, and no call weighs on the streaming loop.
+template <int NCH, int R, int KL, int AGG, bool STAGED, bool GENERIC>
+__global__ void __launch_bounds__(kB1Block, 1)
+row_b1_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ DevChain post,
+              const __grid_constant__ B1Params p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ unsigned long long s_full[kB1MaxSlots];
+    __shared__ __align__(16) double s_part[2][kB1Warps * R * KL];  // [parity][warp][row, local class]
+    __shared__ __align__(16) double s_T[kB1Warps][kB1MaxTile];     // every warp's copy of the tile's T
+    __shared__ unsigned int s_flag;
+
+    constexpr int M = R * KL;                        // partial sums a warp forms per tile
+    constexpr int SH = 5 - Log2<M>::value;           // lane l holds value (l >> SH) after the butterfly
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int W = p.W, KW = p.KW, GW = W * KW;       // warps per group
+    const int GROUPS = kB1Warps / GW;
+    const int KP = KL * KW;                          // padded class count
+    const int MT = R * KP;                           // T values per tile
+    const int grp = warp / GW;
+    const int wig = warp % GW, w_cls = wig / W, w_col = wig % W;
+    const int n = (int)p.cols, k = p.k;
+    const int nB = 64 * NCH * W;                     // padded row length of B^T
+    const int S = p.stages;
+
+    double *ring = reinterpret_cast<double *>(smem_raw) + (size_t)grp * S * R * n;
+    double *BT = reinterpret_cast<double *>(smem_raw) + (size_t)GROUPS * S * R * n;   // KP x nB
+    unsigned long long *full = s_full + grp * S;
+
+    const long long ntiles = (p.rows + R - 1) / R;
+    const long long me = (long long)blockIdx.x * GROUPS + grp, stride = (long long)gridDim.x * GROUPS;
+    const long long my_tiles = (ntiles > me) ? (ntiles - me + stride - 1) / stride : 0;
+
+    // B^T, zero beyond n columns and k classes
+    for (int e = threadIdx.x; e < KP * nB; e += kB1Block) {
+        const int c = e / nB, j = e - c * nB;
+        BT[e] = (c < k && j < n) ? __ldg(p.B + (long long)j * p.ldb + c) : 0.0;
+    }
+
+    double2 q[KL][NCH];
+#pragma unroll
+    for (int cl = 0; cl < KL; ++cl)
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) q[cl][c] = make_double2(0.0, 0.0);
+    bool timed_out = false;
+
+    auto issue = [&](long long it) {
+        const int slot = (int)(it % S);
+        const long long r0 = (me + it * stride) * R;
+        const int nr = (int)((p.rows - r0 < R) ? p.rows - r0 : R);
+        double *dst = ring + (size_t)slot * R * n;
+        mbar_expect_tx(&full[slot], (unsigned)(nr * n * 8));
+        if (p.ldx == n) {
+            bulk_g2s(dst, p.X + r0 * p.ldx, (unsigned)(nr * n * 8), &full[slot]);
+        } else {
+            for (int r = 0; r < nr; ++r)
+                bulk_g2s(dst + (size_t)r * n, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &full[slot]);
+        }
+    };
+
+    if (STAGED) {
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < GROUPS * S; ++s) mbar_init(&s_full[s], 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+    }
+    __syncthreads();
+    const bool elected = wig == 0 && lane == 0;      // the lane that feeds its group's ring
+    if (STAGED && elected)
+        for (long long it = 0; it < my_tiles && it < S; ++it) issue(it);
+
+    // what does not change from tile to tile: this lane's columns, and the two
+    // (row, class) entries of a tile - entries lane and lane + 32 - it evaluates
+    // the chains for
+    int colv[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) colv[c] = 64 * (c * W + w_col) + 2 * lane;
+    int er[2], ec[2], esrc[2];
+    bool ein[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int idx = lane + 32 * u;
+        er[u] = idx / KP;
+        ec[u] = idx - er[u] * KP;
+        ein[u] = idx < MT;
+        esrc[u] = ein[u] ? (grp * GW + (ec[u] / KL) * W) * M + er[u] * KL + (ec[u] % KL) : 0;
+    }
+    const double *bt_mine = BT + (size_t)(w_cls * KL) * nB;
+    const double *t_mine = &s_T[warp][w_cls * KL];
+
+    int slot = 0;
+    unsigned phase = 0;
+    long long r0 = me * R;
+    const long long r0_step = stride * R;
+    for (long long it = 0; it < my_tiles; ++it, r0 += r0_step) {
+        const int par = (int)(it & 1);
+
+        // side values of this lane's entries, requested ahead of the wait
+        double sv[2][FO_MAX_SIDES];
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int j = 0; j < FO_MAX_SIDES; ++j) sv[u][j] = 0.0;
+        if (p.side_used != 0) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const long long row = r0 + er[u];
+                const bool ok = ein[u] && ec[u] < k && row < p.rows;
+#pragma unroll
+                for (int j = 0; j < FO_MAX_SIDES; ++j) {
+                    if (ok && ((p.side_used >> j) & 1u)) {
+                        const DevSide &sd = p.sides.s[j];
+                        const long long off = sd.access == FO_AT_CELL ? row * sd.ld + ec[u]
+                                              : sd.access == FO_AT_ROW ? row * sd.ld : (long long)ec[u];
+                        sv[u][j] = __ldg(sd.data + off);
+                    }
+                }
+            }
+        }
+
+        if (STAGED) {
+            if (!mbar_wait(&full[slot], phase)) timed_out = true;
+        }
+        // this lane's column pairs of the tile's rows
+        double2 x[R][NCH];
+        const double *tile = ring + (size_t)slot * R * n;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const bool have = r0 + r < p.rows;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                const int col = colv[c];
+                if (STAGED) {
+                    x[r][c] = (have && col < n) ? *reinterpret_cast<const double2 *>(tile + (size_t)r * n + col)
+                                                : make_double2(0.0, 0.0);
+                } else {
+                    const double *rowp = p.X + (r0 + r) * p.ldx;
+                    x[r][c].x = (have && col < n) ? ld_stream1(rowp + col) : 0.0;
+                    x[r][c].y = (have && col + 1 < n) ? ld_stream1(rowp + col + 1) : 0.0;
+                }
+            }
+        }
+
+        // partial products with this warp's class slice of B
+        double part[M];
+#pragma unroll
+        for (int i = 0; i < M; ++i) part[i] = 0.0;
+#pragma unroll
+        for (int cl = 0; cl < KL; ++cl) {
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                const double2 b = *reinterpret_cast<const double2 *>(bt_mine + (size_t)cl * nB + colv[c]);
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    part[r * KL + cl] = fma(x[r][c].x, b.x, part[r * KL + cl]);
+                    part[r * KL + cl] = fma(x[r][c].y, b.y, part[r * KL + cl]);
+                }
+            }
+        }
+        warp_sum_multi<M>(part, lane);
+        double *mypart = &s_part[par][0];
+        if ((lane & ((1 << SH) - 1)) == 0) mypart[warp * M + (lane >> SH)] = part[0];
+        if (GW > 1) {
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(GW * 32) : "memory");
+        } else {
+            __syncwarp();
+        }
+        // the tile now lives in the group's registers: its slot takes the tile S ahead
+        if (STAGED && elected && it + S < my_tiles) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue(it + S);
+        }
+        if (++slot == S) { slot = 0; phase ^= 1u; }
+
+        // every warp of the group: D of the whole tile (column warps in order), the
+        // two chains, T into the warp's own copy
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (32 * u < MT) {                        // uniform
+                const bool ok = ein[u] && ec[u] < k && r0 + er[u] < p.rows;
+                double d = 0.0;
+                if (ein[u]) {
+                    const double *src = mypart + esrc[u];
+                    for (int wc = 0; wc < W; ++wc) d += src[wc * M];
+                }
+                double t;
+                if (p.chain_kind == kB1Identity) {
+                    t = d;
+                } else {
+                    double rowsum = 0.0;
+                    if (p.has_pre) {
+                        double pv;
+                        if (!GENERIC || p.chain_kind == kB1Mlogreg) pv = sv[u][0] * d;
+                        else pv = b1_lane_chain(pre, d, sv[u][0], sv[u][1], sv[u][2], sv[u][3]);
+                        rowsum = ok ? pv : 0.0;
+                        // classes of a row sit in KP consecutive lanes
+                        for (int o = 1; o < KP && o < 32; o <<= 1)
+                            rowsum += __shfl_xor_sync(0xffffffffu, rowsum, o);
+                    }
+                    if (!GENERIC || p.chain_kind == kB1Mlogreg) {
+                        t = sv[u][0] * d - sv[u][0] * rowsum;
+                    } else {
+                        double s2[FO_MAX_SIDES];
+#pragma unroll
+                        for (int j = 0; j < FO_MAX_SIDES; ++j)
+                            s2[j] = (p.has_pre && j == p.sides.n) ? rowsum : sv[u][j];
+                        t = b1_lane_chain(post, d, s2[0], s2[1], s2[2], s2[3]);
+                    }
+                }
+                t = ok ? t : 0.0;
+                if (ein[u]) s_T[warp][lane + 32 * u] = t;
+                if (AGG == kB1None && wig == 0 && ok) p.out[(r0 + er[u]) * k + ec[u]] = t;
+            }
+        }
+
+        if (AGG == kB1ColT) {
+            __syncwarp();
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+#pragma unroll
+                for (int cl = 0; cl < KL; cl += 2) {
+                    const double2 tt = *reinterpret_cast<const double2 *>(t_mine + r * KP + cl);
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        q[cl][c].x = fma(tt.x, x[r][c].x, q[cl][c].x);
+                        q[cl][c].y = fma(tt.x, x[r][c].y, q[cl][c].y);
+                        q[cl + 1][c].x = fma(tt.y, x[r][c].x, q[cl + 1][c].x);
+                        q[cl + 1][c].y = fma(tt.y, x[r][c].y, q[cl + 1][c].y);
+                    }
+                }
+            }
+        }
+    }
+
+    if (STAGED && timed_out) atomicExch(&p.head->status, 1u);
+
+    if (AGG == kB1ColT) {
+        // groups -> CTA through shared memory, groups in index order; then the
+        // CTA's n x k tile goes to the workspace and the last CTAs add them up
+        double *qs = reinterpret_cast<double *>(smem_raw);
+        for (int g = 0; g < GROUPS; ++g) {
+            __syncthreads();
+            if (warp / GW == g) {
+#pragma unroll
+                for (int cl = 0; cl < KL; ++cl) {
+                    const int c = w_cls * KL + cl;
+#pragma unroll
+                    for (int ch = 0; ch < NCH; ++ch) {
+                        const int col = 64 * (ch * W + w_col) + 2 * lane;
+                        if (c < k && col < n) {
+                            double *dst = qs + (size_t)col * k + c;
+                            *dst = (g == 0) ? q[cl][ch].x : *dst + q[cl][ch].x;
+                        }
+                        if (c < k && col + 1 < n) {
+                            double *dst = qs + (size_t)(col + 1) * k + c;
+                            *dst = (g == 0) ? q[cl][ch].y : *dst + q[cl][ch].y;
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        const long long width = (long long)n * k;
+        for (long long j = threadIdx.x; j < width; j += kB1Block)
+            p.partials[(size_t)blockIdx.x * width + j] = qs[j];
+        reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * width, width, p.out,
+                                 &s_flag);
+    }
+}
+
+__global__ void b1_fill_zero_kernel(double *out, long long n)
+{
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
+         i += (long long)gridDim.x * blockDim.x)
+        out[i] = 0.0;
+}
+
+// ------------------------------------------------------------------- host
+constexpr size_t kB1SmemBudget = 200 * 1024;       // dynamic shared memory of one CTA
+constexpr long long kB1MaxOutTile = 24576;         // n * k doubles of a CTA's output tile (192 KB)
+
+int b1_grid_cap() { return 148 * 2; }              // bound used for workspace sizing
+
+size_t b1_ws_bytes(long long cols, int k, int agg)
+{
+    if (agg == FO_ROW_COL_AGG_B1_T)
+        return sizeof(WsHead) + (size_t)(b1_grid_cap() + b1_grid_cap() / kGroup + 1) * (size_t)cols * (size_t)k * sizeof(double);
+    return sizeof(WsHead);
+}
+
+// Kernel shape for n columns and k classes: column pairs per lane (nch), rows
+// per tile (r), classes per warp (kl) - the compiled combinations - and the
+// group layout (w warps across columns, kw across class slices).
+struct B1Shape {
+    int nch, r, kl, w, kw;
+};
+
+const int kB1Compiled[][3] = {{1, 8, 2}, {2, 4, 2}, {4, 2, 2}, {1, 4, 4}, {2, 2, 4}, {1, 2, 8}};
+
+int pow2_at_least(long long v)
+{
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// Fills in w and kw for a compiled (nch, r, kl); false if the shape cannot hold the problem.
+bool b1_complete(B1Shape &s, long long n, int k)
+{
+    const int kp = pow2_at_least(k < 2 ? 2 : k);
+    if (s.kl > kp) return false;
+    s.kw = kp / s.kl;
+    s.w = pow2_at_least((n + 64 * s.nch - 1) / (64 * s.nch));
+    if (s.w < 1) s.w = 1;
+    if (s.w * s.kw > kB1Warps) return false;
+    if (s.r * s.kl * s.kw > kB1MaxTile) return false;
+    // B^T plus at least two ring slots per group must fit in shared memory
+    const size_t bt = (size_t)s.kl * s.kw * 64 * s.nch * s.w * 8, slot = (size_t)s.r * n * 8;
+    if (bt + 2 * slot * (kB1Warps / (s.w * s.kw)) > kB1SmemBudget) return false;
+    return true;
+}
+
+bool b1_shape(long long n, int k, B1Shape *out)
+{
+    // FUSEDOPS_B1_SHAPE="nch,r,kl" (read per call; a tuning knob) picks a compiled shape
+    const char *e = getenv("FUSEDOPS_B1_SHAPE");
+    if (e) {
+        int a = 0, b = 0, c = 0;
+        if (sscanf(e, "%d,%d,%d", &a, &b, &c) == 3)
+            for (const auto &t : kB1Compiled)
+                if (t[0] == a && t[1] == b && t[2] == c) {
+                    B1Shape s = {a, b, c, 0, 0};
+                    if (b1_complete(s, n, k)) { *out = s; return true; }
+                }
+    }
+    const int kp = pow2_at_least(k < 2 ? 2 : k);
+    // measured on B200 (t(X) (X V) and the Eq. 2 chain; 100, 500 and 1000 columns,
+    // k = 2 .. 32): two column pairs per lane beat one (half as many partial sums
+    // to combine per multiply-add); two classes: {2,4,2}; more: {2,2,4}, and
+    // {4,2,2} for 8 classes over more than 512 columns
+    const int pref2[][3] = {{2, 4, 2}, {4, 2, 2}, {1, 8, 2}};
+    const int pref4[][3] = {{2, 2, 4}, {2, 4, 2}, {1, 4, 4}};
+    const int pref8w[][3] = {{4, 2, 2}, {2, 2, 4}, {1, 2, 8}};
+    const int (*pref)[3] = kp <= 2 ? pref2 : (kp == 8 && n > 512) ? pref8w : pref4;
+    if (kp <= 2 && n <= 64) {
+        B1Shape s = {1, 8, 2, 0, 0};
+        if (b1_complete(s, n, k)) { *out = s; return true; }
+    }
+    for (int i = 0; i < 3; ++i) {
+        B1Shape s = {pref[i][0], pref[i][1], pref[i][2], 0, 0};
+        if (b1_complete(s, n, k)) { *out = s; return true; }
+    }
+    for (const auto &t : kB1Compiled) {
+        B1Shape s = {t[0], t[1], t[2], 0, 0};
+        if (b1_complete(s, n, k)) { *out = s; return true; }
+    }
+    return false;
+}
+
+template <int NCH, int R, int KL>
+cudaError_t b1_launch_shape(const DevChain &pre, const DevChain &post, const B1Params &p, int agg,
+                            bool staged, int grid, size_t smem, cudaStream_t st)
+{
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, kB1Block, smem, st>>>(pre, post, p);
+        return cudaGetLastError();
+    };
+    const bool generic = p.chain_kind == kB1Generic;
+    if (agg == FO_ROW_COL_AGG_B1_T) {
+        if (generic)
+            return staged ? go(row_b1_kernel<NCH, R, KL, kB1ColT, true, true>)
+                          : go(row_b1_kernel<NCH, R, KL, kB1ColT, false, true>);
+        return staged ? go(row_b1_kernel<NCH, R, KL, kB1ColT, true, false>)
+                      : go(row_b1_kernel<NCH, R, KL, kB1ColT, false, false>);
+    }
+    if (generic)
+        return staged ? go(row_b1_kernel<NCH, R, KL, kB1None, true, true>)
+                      : go(row_b1_kernel<NCH, R, KL, kB1None, false, true>);
+    return staged ? go(row_b1_kernel<NCH, R, KL, kB1None, true, false>)
+                  : go(row_b1_kernel<NCH, R, KL, kB1None, false, false>);
+}
+
+bool b1_aligned16(const void *q) { return ((uintptr_t)q & 15u) == 0; }
+
+}  // namespace
+
+}  // namespace fo
+
+extern "C" {
+
+size_t fused_row_b1_workspace_bytes(const fo_mat *X, int k, int agg)
+{
+    if (!X || X->kind != FO_DENSE || k < 1 || k > FO_B1_MAX_K) return 0;
+    if (agg != FO_ROW_COL_AGG_B1_T && agg != FO_ROW_NO_AGG_B1) return 0;
+    if (X->dense.cols < 0) return 0;
+    return fo::b1_ws_bytes(X->dense.cols, k, agg);
+}
+
+int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, const fo_dense *B,
+                 const fo_side *sides, int n_sides, const double *scalars, int n_scalars,
+                 int agg, double *out, void *ws, size_t ws_bytes, void *stream)
+{
+    using namespace fo;
+    if (!post || !X || !B) return FO_ERR_NULL;
+    if (n_sides > 0 && !sides) return FO_ERR_NULL;
+    if (agg != FO_ROW_COL_AGG_B1_T && agg != FO_ROW_NO_AGG_B1) return FO_ERR_UNSUPPORTED;
+    if (X->kind == FO_CSR) return FO_ERR_UNSUPPORTED;
+    if (X->kind != FO_DENSE) return FO_ERR_SHAPE;
+    const long long rows = X->dense.rows, cols = X->dense.cols;
+    if (rows < 0 || cols < 0 || X->dense.ld < cols) return FO_ERR_SHAPE;
+    if (rows > 0 && cols > 0 && !X->dense.data) return FO_ERR_NULL;
+    if (B->rows != cols || B->cols < 1 || B->ld < B->cols) return FO_ERR_SHAPE;
+    if (B->cols > FO_B1_MAX_K) return FO_ERR_UNSUPPORTED;
+    if (cols > 0 && !B->data) return FO_ERR_NULL;
+    const int k = (int)B->cols;
+    if (!out && (agg == FO_ROW_COL_AGG_B1_T ? cols : rows) > 0) return FO_ERR_NULL;
+    if (n_sides < 0 || n_sides > FO_MAX_SIDES) return FO_ERR_UNSUPPORTED;
+    if (pre && n_sides + 1 > FO_MAX_SIDES) return FO_ERR_UNSUPPORTED;
+
+    // the second chain sees the row sum of the first as one more side input
+    DevChain chpre, chpost;
+    memset(&chpre, 0, sizeof(chpre));
+    int rc;
+    if (pre) {
+        rc = translate_chain(pre, kUseRow, n_sides, scalars, n_scalars, 1, 1, &chpre);
+        if (rc != FO_OK) return rc;
+    }
+    rc = translate_chain(post, kUseRow, n_sides + (pre ? 1 : 0), scalars, n_scalars, 1, 1, &chpost);
+    if (rc != FO_OK) return rc;
+
+    B1Params p;
+    memset(&p, 0, sizeof(p));
+    p.rows = rows; p.cols = cols; p.X = X->dense.data; p.ldx = X->dense.ld;
+    p.B = B->data; p.ldb = B->ld; p.k = k;
+    p.has_pre = pre ? 1 : 0;
+    p.sides.n = n_sides;
+    for (int j = 0; j < n_sides; ++j) {
+        const fo_side &s = sides[j];
+        if (s.access == FO_AT_CELL) {
+            if (s.m.rows != rows || s.m.cols != k || s.m.ld < k) return FO_ERR_SHAPE;
+        } else if (s.access == FO_AT_ROW) {
+            if (s.m.rows != rows || s.m.cols != 1 || s.m.ld < 1) return FO_ERR_SHAPE;
+        } else if (s.access == FO_AT_COL) {
+            if (s.m.rows != 1 || s.m.cols != k) return FO_ERR_SHAPE;
+        } else {
+            return FO_ERR_SHAPE;
+        }
+        if (rows > 0 && !s.m.data) return FO_ERR_NULL;
+        p.sides.s[j].data = s.m.data;
+        p.sides.s[j].ld = s.m.ld;
+        p.sides.s[j].access = s.access;
+    }
+    p.side_used = (chpre.side_used | chpost.side_used) & ((1u << n_sides) - 1u);
+
+    if (agg == FO_ROW_COL_AGG_B1_T && cols * k > kB1MaxOutTile) return FO_ERR_UNSUPPORTED;
+    B1Shape sh;
+    if (!b1_shape(cols, k, &sh)) return FO_ERR_UNSUPPORTED;
+
+    // chains evaluated inline: the identity (t(X) (X B)) and the inner loop of Eq. 2
+    p.chain_kind = kB1Generic;
+    if (!pre && chpost.n_ops == 0 && chpost.out[0] == 0) p.chain_kind = kB1Identity;
+    if (pre && n_sides == 1 && sides[0].access == FO_AT_CELL) {
+        char e1[96], e2[96];
+        if (chain_expression(chpre, 0, e1, sizeof(e1)) == 0 && chain_expression(chpost, 0, e2, sizeof(e2)) == 0) {
+            const bool pre_ok = !strcmp(e1, "mul(r1,r0)") || !strcmp(e1, "mul(r0,r1)");
+            const bool post_ok = !strcmp(e2, "sub(mul(r1,r0),mul(r1,r2))") || !strcmp(e2, "sub(mul(r0,r1),mul(r1,r2))") ||
+                                 !strcmp(e2, "sub(mul(r1,r0),mul(r2,r1))") || !strcmp(e2, "sub(mul(r0,r1),mul(r2,r1))");
+            if (pre_ok && post_ok) p.chain_kind = kB1Mlogreg;
+        }
+    }
+
+    rc = check_workspace(ws, ws_bytes, b1_ws_bytes(cols, k, agg));
+    if (rc != FO_OK) return rc;
+    p.head = (WsHead *)ws;
+    p.partials = (double *)((char *)ws + sizeof(WsHead));
+    p.out = out;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    if (rows == 0 || (cols == 0 && agg == FO_ROW_COL_AGG_B1_T)) {
+        const long long nout = agg == FO_ROW_COL_AGG_B1_T ? cols * k : 0;
+        if (nout > 0) {
+            const long long b = (nout + 255) / 256;
+            b1_fill_zero_kernel<<<(unsigned)(b > 1024 ? 1024 : b), 256, 0, st>>>(out, nout);
+        }
+        const cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? FO_OK : cuda_fail(e);
+    }
+
+    const int sms = sm_count();
+    if (sms <= 0) return cuda_fail(cudaErrorNoDevice);
+    const bool staged = b1_aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
+    const int groups = kB1Warps / (sh.w * sh.kw);
+    p.W = sh.w; p.KW = sh.kw;
+    const size_t bt_bytes = (size_t)sh.kl * sh.kw * 64 * sh.nch * sh.w * 8;
+    const size_t slot_bytes = (size_t)sh.r * cols * 8;
+    int stages = 0;
+    if (staged) {
+        if (bt_bytes + 2 * slot_bytes * groups > kB1SmemBudget) return FO_ERR_UNSUPPORTED;
+        stages = (int)((kB1SmemBudget - bt_bytes) / (slot_bytes * groups));
+        if (stages > 8) stages = 8;
+        if (stages * groups > kB1MaxSlots) stages = kB1MaxSlots / groups;
+    }
+    p.stages = stages;
+    size_t smem = bt_bytes + slot_bytes * groups * stages;
+    const size_t qs_bytes = agg == FO_ROW_COL_AGG_B1_T ? (size_t)cols * k * 8 : 0;
+    if (smem < qs_bytes) smem = qs_bytes;
+    const long long ntiles = (rows + sh.r - 1) / sh.r;
+    long long grid = (ntiles + groups - 1) / groups;
+    if (grid > sms) grid = sms;
+    if (grid > b1_grid_cap()) grid = b1_grid_cap();
+    if (grid < 1) grid = 1;
+
+    cudaError_t e = cudaErrorInvalidValue;
+#define FO_B1(A, B_, C) \
+    if (sh.nch == A && sh.r == B_ && sh.kl == C) \
+        e = b1_launch_shape<A, B_, C>(chpre, chpost, p, agg, staged, (int)grid, smem, st);
+    FO_B1(1, 8, 2) FO_B1(2, 4, 2) FO_B1(4, 2, 2) FO_B1(1, 4, 4) FO_B1(2, 2, 4) FO_B1(1, 2, 8)
+#undef FO_B1
+    return e == cudaSuccess ? FO_OK : cuda_fail(e);
+}
+
+}  // extern "C"
