@@ -274,6 +274,29 @@ def time_variants(fo, step, shapes, reps=10):
         ("magg_csr_density_0.1", lambda: fo.fused_magg(MAGG3, ["t0", "t1", "t2"], Xs, sides, out=o_three),
          sparse_in + 24),
     ]
+    # Row template with matrix-valued row intermediates (Section 5.2: t(X) %*% (X %*% V) with
+    # V 1000 x 2 on the dense Row input; the Eq. 2 inner loop for k classes on the 100-column input)
+    MLR_PRE = [("mul", "t0", "side0", "d")]
+    MLR_POST = [("mul", "t0", "side0", "d"), ("mul", "t1", "side0", "rowsum"), ("sub", "t2", "t0", "t1")]
+    g.manual_seed(6)
+    V2 = torch.randn((rc, 2), generator=g, dtype=torch.float64, device=dev)
+    P2 = torch.rand((rr, 2), generator=g, dtype=torch.float64, device=dev) / 3.0
+    o_h2 = torch.empty((rc, 2), dtype=torch.float64, device=dev)
+    cases += [
+        ("row_b1_mmchain_k2", lambda: fo.fused_row_b1(None, None, [], "d", d["row_dense.X"], V2, out=o_h2),
+         8 * rr * rc + 2 * 8 * rc * 2),
+        ("row_b1_mlogreg_k2", lambda: fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", d["row_dense.X"], V2,
+                                                      [("cell", P2)], out=o_h2),
+         8 * rr * rc + 8 * rr * 2 + 2 * 8 * rc * 2),
+    ]
+    for kk in (2, 8, 32):
+        Vk = torch.randn((mc, kk), generator=g, dtype=torch.float64, device=dev)
+        Pk = torch.rand((mr, kk), generator=g, dtype=torch.float64, device=dev) / (kk + 1)
+        o_hk = torch.empty((mc, kk), dtype=torch.float64, device=dev)
+        cases.append(("row_b1_mlogreg_100cols_k%d" % kk,
+                      lambda Vk=Vk, Pk=Pk, o_hk=o_hk: fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", d["magg.X"], Vk,
+                                                                      [("cell", Pk)], out=o_hk),
+                      8 * mr * mc + 8 * mr * kk + 2 * 8 * mc * kk))
     res = {}
     for name, fn, nbytes in cases:
         for _ in range(2):
@@ -286,6 +309,9 @@ def time_variants(fo, step, shapes, reps=10):
         torch.cuda.synchronize()
         ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
         res[name] = {"ms": ms, "bytes": nbytes, "gbs": nbytes / (ms * 1e-3) / 1e9}
+        if name.startswith("row_b1_mlogreg_100cols_k"):
+            kk = int(name.rsplit("k", 1)[1])
+            res[name]["fp64_tflops"] = 4.0 * mr * mc * kk / (ms * 1e-3) / 1e12
     return res
 
 

@@ -35,6 +35,7 @@ struct B1Params {
     double *out;
     int stages;                 // ring slots per group
     int W, KW;                  // warps of a group across columns / across class slices
+    int ns;                     // tensor-core variant: row stride of a tile in shared memory
     int chain_kind;
     int has_pre;
     unsigned side_used;         // sides read by either chain
@@ -339,6 +340,259 @@ row_b1_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ DevC
     }
 }
 
+// ------------------------------------------------------- tensor-core variant
+// The two products of a tile - D = X_tile B (8 rows x 8 classes, summed over the
+// columns) and H += X_tile^T T (8 columns x 8 classes, summed over the 8 rows) -
+// are small dense fp64 contractions, so they run as m8n8k4 double-precision
+// matrix multiply-accumulates: one instruction does the work of eight warp-wide
+// multiply-adds and sums over its k dimension by itself, which removes the
+// partial-sum exchange that bounds the kernel above once k > 2.
+//
+// 8 warps per CTA.  A group of W x KB warps shares a ring of 8-row tiles; warp
+// (w, cb) owns the columns [w * 8 NCB, (w + 1) * 8 NCB) and the classes
+// [8 cb, 8 cb + 8): its fragments of B (one register per 4-column step) and its
+// tile of the output (two registers per 8-column block) stay in registers.
+// Rows sit in shared memory with a stride of ns doubles, ns = 4 (mod 8), so
+// that both ways of reading a tile - 8 rows x 4 columns, 4 rows x 8 columns -
+// touch every bank once.  Rows beyond the matrix and columns beyond n read
+// zeros or stale finite values whose partner operand is zero.
+__device__ __forceinline__ void dmma_8x8x4(double &c0, double &c1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
+
+constexpr int kMmaWarps = 8;
+constexpr int kMmaBlock = kMmaWarps * 32;
+constexpr int kMmaMaxSlots = 32;
+
+template <int NCB, int AGG, bool GENERIC>
+__global__ void __launch_bounds__(kMmaBlock, 1)
+row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ DevChain post,
+                  const __grid_constant__ B1Params p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ unsigned long long s_full[kMmaMaxSlots];
+    __shared__ __align__(16) double s_D[2][kMmaWarps][64];    // partial D of every warp (W > 1)
+    __shared__ double s_rs[2][kMmaWarps][8];                  // row sums of every class block (KB > 1)
+    __shared__ double s_T[kMmaWarps][64];
+    __shared__ unsigned int s_flag;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int W = p.W, KB = p.KW, GW = W * KB, GROUPS = kMmaWarps / GW;
+    const int grp = warp / GW, wig = warp % GW, cb = wig / W, w = wig % W;
+    const int n = (int)p.cols, k = p.k, ns = p.ns, S = p.stages;
+    const int lq = lane >> 2, lr = lane & 3;                   // fragment coordinates
+    const int col0 = w * NCB * 8;
+
+    double *ring = reinterpret_cast<double *>(smem_raw) + (size_t)grp * S * 8 * ns;
+    unsigned long long *full = s_full + grp * S;
+    const long long ntiles = (p.rows + 7) / 8;
+    const long long me = (long long)blockIdx.x * GROUPS + grp, stride = (long long)gridDim.x * GROUPS;
+    const long long my_tiles = (ntiles > me) ? (ntiles - me + stride - 1) / stride : 0;
+
+    // fragments of B: step s covers columns col0 + 4 s .. + 3
+    double bfrag[2 * NCB];
+#pragma unroll
+    for (int s = 0; s < 2 * NCB; ++s) {
+        const int j = col0 + 4 * s + lr, c = cb * 8 + lq;
+        bfrag[s] = (j < n && c < k) ? __ldg(p.B + (long long)j * p.ldb + c) : 0.0;
+    }
+    double acc[NCB][2];
+#pragma unroll
+    for (int jb = 0; jb < NCB; ++jb) acc[jb][0] = acc[jb][1] = 0.0;
+
+    // the rings start as zeros: padding columns and the rows of a ragged last
+    // tile are never written by a copy
+    {
+        double *all = reinterpret_cast<double *>(smem_raw);
+        const int total = GROUPS * S * 8 * ns + 8;               // and the slack behind the last tile
+        for (int e = threadIdx.x; e < total; e += kMmaBlock) all[e] = 0.0;
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < GROUPS * S; ++s) mbar_init(&s_full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+
+    bool timed_out = false;
+    auto issue = [&](long long it, int slot) {
+        const long long r0 = (me + it * stride) * 8;
+        const int nr = (int)((p.rows - r0 < 8) ? p.rows - r0 : 8);
+        double *dst = ring + (size_t)slot * 8 * ns;
+        mbar_expect_tx(&full[slot], (unsigned)(nr * n * 8));
+        if (p.ldx == n && ns == n) {
+            bulk_g2s(dst, p.X + r0 * p.ldx, (unsigned)(nr * n * 8), &full[slot]);
+        } else {
+            for (int r = 0; r < nr; ++r)
+                bulk_g2s(dst + (size_t)r * ns, p.X + (r0 + r) * p.ldx, (unsigned)(n * 8), &full[slot]);
+        }
+    };
+    const bool elected = wig == 0 && lane == 0;
+    if (elected)
+        for (int it = 0; it < S && it < my_tiles; ++it) issue(it, it);
+
+    const int c0 = cb * 8 + 2 * lr;                            // this lane's two classes (c0, c0 + 1)
+    int slot = 0, prev_slot = 0;
+    unsigned phase = 0;
+    long long r0 = me * 8;
+    const long long r0_step = stride * 8;
+    for (long long it = 0; it < my_tiles; ++it, r0 += r0_step) {
+        const int par = (int)(it & 1);
+        const long long row = r0 + lq;
+        const bool ok0 = row < p.rows && c0 < k, ok1 = row < p.rows && c0 + 1 < k;
+
+        double sv0[FO_MAX_SIDES], sv1[FO_MAX_SIDES];
+#pragma unroll
+        for (int j = 0; j < FO_MAX_SIDES; ++j) sv0[j] = sv1[j] = 0.0;
+        if (p.side_used != 0) {
+#pragma unroll
+            for (int j = 0; j < FO_MAX_SIDES; ++j) {
+                if ((p.side_used >> j) & 1u) {
+                    const DevSide &sd = p.sides.s[j];
+                    const long long base = sd.access == FO_AT_CELL ? row * sd.ld + c0
+                                           : sd.access == FO_AT_ROW ? row * sd.ld : (long long)c0;
+                    const int step = sd.access == FO_AT_ROW ? 0 : 1;
+                    if (ok0) sv0[j] = __ldg(sd.data + base);
+                    if (ok1) sv1[j] = __ldg(sd.data + base + step);
+                }
+            }
+        }
+
+        if (!mbar_wait(&full[slot], phase)) timed_out = true;
+        const double *tile = ring + (size_t)slot * 8 * ns;
+
+        // D = X_tile B over this warp's columns
+        double d0 = 0.0, d1 = 0.0;
+        {
+            const double *arow = tile + (size_t)lq * ns + col0 + lr;
+#pragma unroll
+            for (int s = 0; s < 2 * NCB; ++s)
+                if (col0 + 4 * s < n) dmma_8x8x4(d0, d1, arow[4 * s], bfrag[s]);
+        }
+        if (W > 1) *reinterpret_cast<double2 *>(&s_D[par][warp][2 * lane]) = make_double2(d0, d1);
+        if (GW > 1) {
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(GW * 32) : "memory");
+            // every warp of the group is past its use of the previous tile
+            if (elected && it > 0 && it - 1 + S < my_tiles) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                issue(it - 1 + S, prev_slot);
+            }
+        }
+        if (W > 1) {
+            d0 = d1 = 0.0;
+            for (int ww = 0; ww < W; ++ww) {
+                const double2 v = *reinterpret_cast<const double2 *>(&s_D[par][grp * GW + cb * W + ww][2 * lane]);
+                d0 += v.x;
+                d1 += v.y;
+            }
+        }
+
+        double t0, t1;
+        if (p.chain_kind == kB1Identity) {
+            t0 = d0;
+            t1 = d1;
+        } else {
+            double rowsum = 0.0;
+            if (p.has_pre) {
+                double p0, p1;
+                if (!GENERIC || p.chain_kind == kB1Mlogreg) {
+                    p0 = sv0[0] * d0;
+                    p1 = sv1[0] * d1;
+                } else {
+                    p0 = b1_lane_chain(pre, d0, sv0[0], sv0[1], sv0[2], sv0[3]);
+                    p1 = b1_lane_chain(pre, d1, sv1[0], sv1[1], sv1[2], sv1[3]);
+                }
+                rowsum = (ok0 ? p0 : 0.0) + (ok1 ? p1 : 0.0);
+                rowsum += __shfl_xor_sync(0xffffffffu, rowsum, 1);
+                rowsum += __shfl_xor_sync(0xffffffffu, rowsum, 2);
+                if (KB > 1) {
+                    if (w == 0 && lr == 0) s_rs[par][grp * KB + cb][lq] = rowsum;
+                    asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(GW * 32) : "memory");
+                    rowsum = 0.0;
+                    for (int b = 0; b < KB; ++b) rowsum += s_rs[par][grp * KB + b][lq];
+                }
+            }
+            if (!GENERIC || p.chain_kind == kB1Mlogreg) {
+                t0 = sv0[0] * d0 - sv0[0] * rowsum;
+                t1 = sv1[0] * d1 - sv1[0] * rowsum;
+            } else {
+                double a0[FO_MAX_SIDES], a1[FO_MAX_SIDES];
+#pragma unroll
+                for (int j = 0; j < FO_MAX_SIDES; ++j) {
+                    const bool rs = p.has_pre && j == p.sides.n;
+                    a0[j] = rs ? rowsum : sv0[j];
+                    a1[j] = rs ? rowsum : sv1[j];
+                }
+                t0 = b1_lane_chain(post, d0, a0[0], a0[1], a0[2], a0[3]);
+                t1 = b1_lane_chain(post, d1, a1[0], a1[1], a1[2], a1[3]);
+            }
+        }
+        t0 = ok0 ? t0 : 0.0;
+        t1 = ok1 ? t1 : 0.0;
+
+        if (AGG == kB1None) {
+            if (w == 0 && ok0) p.out[row * k + c0] = t0;
+            if (w == 0 && ok1) p.out[row * k + c0 + 1] = t1;
+        } else {
+            // T from accumulator layout (row lq, classes 2 lr, 2 lr + 1) to operand
+            // layout (rows lr and lr + 4, class lq) through the warp's own scratch
+            s_T[warp][lq * 8 + 2 * lr] = t0;
+            s_T[warp][lq * 8 + 2 * lr + 1] = t1;
+            __syncwarp();
+            const double tf0 = s_T[warp][lr * 8 + lq], tf1 = s_T[warp][(4 + lr) * 8 + lq];
+            const double *a0p = tile + (size_t)lr * ns + col0 + lq;
+            const double *a1p = a0p + (size_t)4 * ns;
+#pragma unroll
+            for (int jb = 0; jb < NCB; ++jb) {
+                if (col0 + 8 * jb < n) {
+                    dmma_8x8x4(acc[jb][0], acc[jb][1], a0p[8 * jb], tf0);
+                    dmma_8x8x4(acc[jb][0], acc[jb][1], a1p[8 * jb], tf1);
+                }
+            }
+        }
+        if (GW == 1) {
+            __syncwarp();
+            if (elected && it + S < my_tiles) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                issue(it + S, slot);
+            }
+        }
+        prev_slot = slot;
+        if (++slot == S) { slot = 0; phase ^= 1u; }
+    }
+
+    if (timed_out) atomicExch(&p.head->status, 1u);
+
+    if (AGG == kB1ColT) {
+        double *qs = reinterpret_cast<double *>(smem_raw);
+        for (int g = 0; g < GROUPS; ++g) {
+            __syncthreads();
+            if (grp == g) {
+#pragma unroll
+                for (int jb = 0; jb < NCB; ++jb) {
+                    const int j = col0 + 8 * jb + lq;
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const int c = c0 + i;
+                        if (j < n && c < k) {
+                            double *dst = qs + (size_t)j * k + c;
+                            *dst = (g == 0) ? acc[jb][i] : *dst + acc[jb][i];
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        const long long width = (long long)n * k;
+        for (long long j = threadIdx.x; j < width; j += kMmaBlock)
+            p.partials[(size_t)blockIdx.x * width + j] = qs[j];
+        reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * width, width, p.out,
+                                 &s_flag);
+    }
+}
+
 __global__ void b1_fill_zero_kernel(double *out, long long n)
 {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -453,6 +707,45 @@ cudaError_t b1_launch_shape(const DevChain &pre, const DevChain &post, const B1P
                   : go(row_b1_kernel<NCH, R, KL, kB1None, false, false>);
 }
 
+// Tensor-core variant: column blocks per warp (compiled: 8, 14, 16, 20), warps
+// across the columns and class blocks of 8; w * kb <= 8 warps.
+struct MmaShape {
+    int ncb, w, kb;
+};
+
+bool b1_mma_shape(long long n, int k, MmaShape *out)
+{
+    const int kb = pow2_at_least((k + 7) / 8);
+    if (kb > kMmaWarps || n < 2) return false;
+    const int ncbs[] = {8, 14, 16, 20};
+    for (int w = 1; w * kb <= kMmaWarps; w *= 2)
+        for (int ncb : ncbs)
+            if ((long long)8 * ncb * w >= n) {
+                *out = MmaShape{ncb, w, kb};
+                return true;
+            }
+    return false;
+}
+
+// Row stride of a tile in shared memory: the smallest ns >= n with ns = 4 (mod 8).
+int b1_mma_stride(long long n) { return (int)(n + ((4 - n % 8) + 8) % 8); }
+
+template <int NCB>
+cudaError_t b1_mma_launch(const DevChain &pre, const DevChain &post, const B1Params &p, int agg,
+                          int grid, size_t smem, cudaStream_t st)
+{
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, kMmaBlock, smem, st>>>(pre, post, p);
+        return cudaGetLastError();
+    };
+    const bool generic = p.chain_kind == kB1Generic;
+    if (agg == FO_ROW_COL_AGG_B1_T)
+        return generic ? go(row_b1_mma_kernel<NCB, kB1ColT, true>) : go(row_b1_mma_kernel<NCB, kB1ColT, false>);
+    return generic ? go(row_b1_mma_kernel<NCB, kB1None, true>) : go(row_b1_mma_kernel<NCB, kB1None, false>);
+}
+
 bool b1_aligned16(const void *q) { return ((uintptr_t)q & 15u) == 0; }
 
 }  // namespace
@@ -562,6 +855,37 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
     const int sms = sm_count();
     if (sms <= 0) return cuda_fail(cudaErrorNoDevice);
     const bool staged = b1_aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
+    // tensor-core variant where its layout fits (FUSEDOPS_B1_MMA=0 / 1 forces the choice)
+    {
+        MmaShape ms;
+        const char *env = getenv("FUSEDOPS_B1_MMA");
+        const bool want = env ? env[0] != '0' : (k > 2 || cols <= 160);
+        if (want && staged && b1_mma_shape(cols, k, &ms)) {
+            const int groups = kMmaWarps / (ms.w * ms.kb);
+            const int ns = b1_mma_stride(cols);
+            const size_t slot_bytes = (size_t)8 * ns * 8;
+            const size_t budget = 208 * 1024;
+            int stages = (int)((budget - 64) / (slot_bytes * groups));
+            if (stages > 6) stages = 6;
+            if (stages * groups > kMmaMaxSlots) stages = kMmaMaxSlots / groups;
+            if (stages >= 2) {
+                p.W = ms.w; p.KW = ms.kb; p.ns = ns; p.stages = stages;
+                size_t smem = slot_bytes * groups * stages + 64;      // 8 doubles of slack behind the rings
+                const size_t qs_bytes = agg == FO_ROW_COL_AGG_B1_T ? (size_t)cols * k * 8 : 0;
+                if (smem < qs_bytes) smem = qs_bytes;
+                const long long ntiles = (rows + 7) / 8;
+                long long grid = (ntiles + groups - 1) / groups;
+                if (grid > sms) grid = sms;
+                if (grid < 1) grid = 1;
+                cudaError_t e = cudaErrorInvalidValue;
+                if (ms.ncb == 8) e = b1_mma_launch<8>(chpre, chpost, p, agg, (int)grid, smem, st);
+                else if (ms.ncb == 14) e = b1_mma_launch<14>(chpre, chpost, p, agg, (int)grid, smem, st);
+                else if (ms.ncb == 16) e = b1_mma_launch<16>(chpre, chpost, p, agg, (int)grid, smem, st);
+                else if (ms.ncb == 20) e = b1_mma_launch<20>(chpre, chpost, p, agg, (int)grid, smem, st);
+                return e == cudaSuccess ? FO_OK : cuda_fail(e);
+            }
+        }
+    }
     const int groups = kB1Warps / (sh.w * sh.kw);
     p.W = sh.w; p.KW = sh.kw;
     const size_t bt_bytes = (size_t)sh.kl * sh.kw * 64 * sh.nch * sh.w * 8;

@@ -167,6 +167,44 @@ def test_row_and_outer_argument_errors(lib):
     assert outer(xx=x2) == -4
 
 
+def test_row_b1_argument_errors(lib):
+    # every error is found on the host, before anything is launched (no GPU here)
+    pre, k1 = B.make_chain([("mul", "t0", "side0", "d")], "t0")
+    post, k2 = B.make_chain([("mul", "t0", "side0", "rowsum")], "t0", rowsum_side=1)
+    ident, k3 = B.make_chain([], "d")
+    sc = (C.c_double * 8)()
+
+    def dense(rows, cols, ld=None, data=0x9000):
+        d = B.fo_dense()
+        d.rows, d.cols, d.ld, d.data = rows, cols, ld or cols, data
+        return d
+
+    def call(mat, bmat, agg=6, sides=None, ns=0, prec=None, postc=ident, ws_bytes=1 << 30):
+        sarr = sides if sides is not None else (B.fo_side * 1)()
+        return lib.fused_row_b1(C.byref(prec) if prec is not None else None, C.byref(postc), C.byref(mat),
+                                C.byref(bmat), sarr, ns, sc, 0, agg, C.c_void_p(0x2000),
+                                C.c_void_p(0x10000), ws_bytes, None)
+
+    m = dense_mat(10, 100)
+    assert call(m, dense(100, 33)) == -4                    # more than 32 classes
+    assert call(m, dense(99, 2)) == -2                      # B.rows != X.cols
+    assert call(m, dense(100, 2), agg=4) == -4              # not a B1 variant
+    assert call(dense_mat(10, 5000), dense(5000, 2)) == -4  # too wide
+    assert call(dense_mat(10, 2000), dense(2000, 16)) == -4  # n * k beyond the output tile
+    assert call(m, dense(100, 2), ws_bytes=1024) == -5
+    one = (B.fo_side * 1)(side(10, 2, 0))
+    bad = (B.fo_side * 1)(side(10, 3, 0))
+    assert call(m, dense(100, 2), sides=bad, ns=1, prec=pre, postc=post) == -2   # cell side must be rows x k
+    assert call(m, dense(100, 2), sides=one, ns=1, prec=None, postc=post) == -3  # row sum without a first chain
+    x = B.fo_mat()
+    x.kind = 1
+    assert call(x, dense(100, 2)) == -4                     # CSR main input not provided
+    # workspace: one n x k tile per CTA and per group of CTAs for col_agg_B1_T, the head alone otherwise
+    assert lib.fused_row_b1_workspace_bytes(C.byref(m), 2, 5) == 16384
+    assert lib.fused_row_b1_workspace_bytes(C.byref(m), 2, 6) > 16384 + 148 * 100 * 2 * 8
+    assert lib.fused_row_b1_workspace_bytes(C.byref(m), 0, 6) == 0
+
+
 def test_make_chain_rejects_bad_text():
     with pytest.raises(ValueError):
         B.make_chain([("frobnicate", "t0", "a")], "t0")

@@ -27,6 +27,19 @@ def fo():
     return fo_
 
 
+@pytest.fixture(params=["fma", "mma"])
+def path(request):
+    """Runs a test once on the multiply-add kernels and once with the tensor-core
+    kernels preferred (they take over wherever their layout fits)."""
+    old = os.environ.get("FUSEDOPS_B1_MMA")
+    os.environ["FUSEDOPS_B1_MMA"] = "0" if request.param == "fma" else "1"
+    yield request.param
+    if old is None:
+        del os.environ["FUSEDOPS_B1_MMA"]
+    else:
+        os.environ["FUSEDOPS_B1_MMA"] = old
+
+
 def mm_scale(X, V):
     aX = np.abs(X)
     return aX.T @ (aX @ np.abs(V))
@@ -41,11 +54,11 @@ def mlr_scale(X, V, P):
 # (rows, cols, k): k = 1..32, narrow and wide rows, odd sizes, ragged last tiles
 SHAPES = [(2000, 1000, 2), (5000, 100, 2), (3001, 100, 4), (3000, 100, 8), (2500, 100, 16), (1501, 100, 32),
           (777, 64, 3), (513, 200, 5), (1000, 512, 16), (600, 1024, 8), (300, 2048, 4), (150, 4096, 2),
-          (97, 31, 7), (64, 2, 1), (1, 10, 2), (5, 1, 3), (1200, 256, 32), (40, 999, 2), (333, 250, 24)]
+          (97, 31, 7), (64, 2, 1), (900, 102, 9), (700, 160, 20), (500, 500, 12), (650, 1000, 8), (800, 64, 32), (300, 230, 17), (1, 10, 2), (5, 1, 3), (1200, 256, 32), (40, 999, 2), (333, 250, 24)]
 
 
 @pytest.mark.parametrize("rows,cols,k", SHAPES)
-def test_b1_mmchain(fo, rows, cols, k):
+def test_b1_mmchain(fo, path, rows, cols, k):
     w = datagen.row_b1_workload(rows, cols, k, seed=5)
     ref = oracle.mmchain(w["X"], w["V"])
     got = fo.fused_row_b1(None, None, [], "d", to_dev(w["X"]), to_dev(w["V"]), agg="col_t")
@@ -55,7 +68,7 @@ def test_b1_mmchain(fo, rows, cols, k):
 
 
 @pytest.mark.parametrize("rows,cols,k", SHAPES)
-def test_b1_mlogreg(fo, rows, cols, k):
+def test_b1_mlogreg(fo, path, rows, cols, k):
     w = datagen.row_b1_workload(rows, cols, k, seed=6)
     X, V, P = w["X"], w["V"], w["P"]
     ref = oracle.mlogreg_inner(X, V, P)
@@ -71,7 +84,7 @@ def test_b1_mlogreg(fo, rows, cols, k):
 
 
 @pytest.mark.parametrize("rows,cols,k", [(1000, 100, 3), (700, 1000, 2), (400, 300, 8), (90, 64, 32)])
-def test_b1_generic_chains_all_side_kinds(fo, rows, cols, k):
+def test_b1_generic_chains_all_side_kinds(fo, path, rows, cols, k):
     # T_ic = (d * rvec_c + cvec_i * P_ic) * s0 - exp(-|rowsum|),  rowsum = sum_c P_ic * d
     w = datagen.row_b1_workload(rows, cols, k, seed=7)
     X, V, P = w["X"], w["V"], w["P"]
@@ -97,7 +110,7 @@ def test_b1_generic_chains_all_side_kinds(fo, rows, cols, k):
     assert fo.device_status() == 0
 
 
-def test_b1_inline_and_interpreted_chains_agree_bitwise(fo):
+def test_b1_inline_and_interpreted_chains_agree_bitwise(fo, path):
     # the Eq. 2 chains are evaluated inline; the same arithmetic written with an extra
     # (no-op) step goes through the interpreter and must give the same bits
     rows, cols, k = 4000, 100, 4
@@ -119,7 +132,9 @@ def test_b1_every_compiled_shape(fo, shape):
     rows, cols = 3000 + r - 1, 200
     w = datagen.row_b1_workload(rows, cols, k, seed=9)
     old = os.environ.get("FUSEDOPS_B1_SHAPE")
+    old_mma = os.environ.get("FUSEDOPS_B1_MMA")
     os.environ["FUSEDOPS_B1_SHAPE"] = shape
+    os.environ["FUSEDOPS_B1_MMA"] = "0"
     try:
         for kk in (k, 2 * k):
             ww = w if kk == k else datagen.row_b1_workload(rows, cols, kk, seed=9)
@@ -128,14 +143,15 @@ def test_b1_every_compiled_shape(fo, shape):
             got = fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", to_dev(X), to_dev(V), [("cell", to_dev(P))])
             assert_close(got.cpu().numpy(), ref, absscale=mlr_scale(X, V, P), what="shape %s k=%d" % (shape, kk))
     finally:
-        if old is None:
-            del os.environ["FUSEDOPS_B1_SHAPE"]
-        else:
-            os.environ["FUSEDOPS_B1_SHAPE"] = old
+        for name, val in (("FUSEDOPS_B1_SHAPE", old), ("FUSEDOPS_B1_MMA", old_mma)):
+            if val is None:
+                del os.environ[name]
+            else:
+                os.environ[name] = val
     assert fo.device_status() == 0
 
 
-def test_b1_strided_unaligned_inputs(fo):
+def test_b1_strided_unaligned_inputs(fo, path):
     rows, cols, ld, k, ldv = 333, 120, 130, 3, 5
     flat = datagen.normal(5, 0, rows * ld + 1)
     Vflat = datagen.normal(5, 2, cols * ldv)
@@ -153,7 +169,7 @@ def test_b1_strided_unaligned_inputs(fo):
     assert fo.device_status() == 0
 
 
-def test_b1_many_tiles_per_group(fo):
+def test_b1_many_tiles_per_group(fo, path):
     # far more tiles than ring slots: every slot is refilled many times
     rows, cols, k = 60011, 100, 2
     w = datagen.row_b1_workload(rows, cols, k, seed=10)
