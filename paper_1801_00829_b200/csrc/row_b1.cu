@@ -362,15 +362,16 @@ __device__ __forceinline__ void dmma_8x8x4(double &c0, double &c1, double a, dou
                  : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
 
-constexpr int kMmaWarps = 8;
-constexpr int kMmaBlock = kMmaWarps * 32;
+constexpr int kMmaMaxWarps = 16;
 constexpr int kMmaMaxSlots = 32;
 
-template <int NCB, int AGG, bool GENERIC>
-__global__ void __launch_bounds__(kMmaBlock, 1)
+// NW warps per CTA (8 are compiled: up to 255 registers a thread).
+template <int NW, int NCB, int AGG, bool GENERIC>
+__global__ void __launch_bounds__(NW * 32, 1)
 row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ DevChain post,
                   const __grid_constant__ B1Params p)
 {
+    constexpr int kMmaWarps = NW, kMmaBlock = NW * 32;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ unsigned long long s_full[kMmaMaxSlots];
     __shared__ __align__(16) double s_D[2][kMmaWarps][64];    // partial D of every warp (W > 1)
@@ -434,6 +435,29 @@ row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ 
         for (int it = 0; it < S && it < my_tiles; ++it) issue(it, it);
 
     const int c0 = cb * 8 + 2 * lr;                            // this lane's two classes (c0, c0 + 1)
+    // side values of the entries (row lq, classes c0 and c0 + 1) of the tile at tile_r0;
+    // the inline chains only ever read side 0
+    constexpr int NS = GENERIC ? FO_MAX_SIDES : 1;
+    auto load_sides = [&](long long tile_r0, double (&a)[NS], double (&b)[NS]) {
+#pragma unroll
+        for (int j = 0; j < NS; ++j) a[j] = b[j] = 0.0;
+        if (p.side_used == 0) return;
+        const long long row = tile_r0 + lq;
+        const bool okr = row < p.rows;
+#pragma unroll
+        for (int j = 0; j < NS; ++j) {
+            if ((p.side_used >> j) & 1u) {
+                const DevSide &sd = p.sides.s[j];
+                const long long base = sd.access == FO_AT_CELL ? row * sd.ld + c0
+                                       : sd.access == FO_AT_ROW ? row * sd.ld : (long long)c0;
+                const int step = sd.access == FO_AT_ROW ? 0 : 1;
+                if (okr && c0 < k) a[j] = __ldg(sd.data + base);
+                if (okr && c0 + 1 < k) b[j] = __ldg(sd.data + base + step);
+            }
+        }
+    };
+    double nsv0[NS], nsv1[NS];
+    load_sides(me * 8, nsv0, nsv1);
     int slot = 0, prev_slot = 0;
     unsigned phase = 0;
     long long r0 = me * 8;
@@ -443,33 +467,31 @@ row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ 
         const long long row = r0 + lq;
         const bool ok0 = row < p.rows && c0 < k, ok1 = row < p.rows && c0 + 1 < k;
 
-        double sv0[FO_MAX_SIDES], sv1[FO_MAX_SIDES];
+        // side values of this tile (requested while the previous tile was worked on)
+        double sv0[NS], sv1[NS];
 #pragma unroll
-        for (int j = 0; j < FO_MAX_SIDES; ++j) sv0[j] = sv1[j] = 0.0;
-        if (p.side_used != 0) {
-#pragma unroll
-            for (int j = 0; j < FO_MAX_SIDES; ++j) {
-                if ((p.side_used >> j) & 1u) {
-                    const DevSide &sd = p.sides.s[j];
-                    const long long base = sd.access == FO_AT_CELL ? row * sd.ld + c0
-                                           : sd.access == FO_AT_ROW ? row * sd.ld : (long long)c0;
-                    const int step = sd.access == FO_AT_ROW ? 0 : 1;
-                    if (ok0) sv0[j] = __ldg(sd.data + base);
-                    if (ok1) sv1[j] = __ldg(sd.data + base + step);
-                }
-            }
+        for (int j = 0; j < NS; ++j) {
+            sv0[j] = nsv0[j];
+            sv1[j] = nsv1[j];
         }
+        load_sides(r0 + r0_step, nsv0, nsv1);
 
         if (!mbar_wait(&full[slot], phase)) timed_out = true;
         const double *tile = ring + (size_t)slot * 8 * ns;
 
         // D = X_tile B over this warp's columns
-        double d0 = 0.0, d1 = 0.0;
+        // (four independent accumulator pairs: consecutive steps do not wait for each other)
+        double d0, d1;
         {
+            double da[4][2];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) da[i][0] = da[i][1] = 0.0;
             const double *arow = tile + (size_t)lq * ns + col0 + lr;
 #pragma unroll
             for (int s = 0; s < 2 * NCB; ++s)
-                if (col0 + 4 * s < n) dmma_8x8x4(d0, d1, arow[4 * s], bfrag[s]);
+                if (col0 + 4 * s < n) dmma_8x8x4(da[s & 3][0], da[s & 3][1], arow[4 * s], bfrag[s]);
+            d0 = (da[0][0] + da[1][0]) + (da[2][0] + da[3][0]);
+            d1 = (da[0][1] + da[1][1]) + (da[2][1] + da[3][1]);
         }
         if (W > 1) *reinterpret_cast<double2 *>(&s_D[par][warp][2 * lane]) = make_double2(d0, d1);
         if (GW > 1) {
@@ -501,8 +523,8 @@ row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ 
                     p0 = sv0[0] * d0;
                     p1 = sv1[0] * d1;
                 } else {
-                    p0 = b1_lane_chain(pre, d0, sv0[0], sv0[1], sv0[2], sv0[3]);
-                    p1 = b1_lane_chain(pre, d1, sv1[0], sv1[1], sv1[2], sv1[3]);
+                    p0 = b1_lane_chain(pre, d0, sv0[0], sv0[NS > 1 ? 1 : 0], sv0[NS > 2 ? 2 : 0], sv0[NS > 3 ? 3 : 0]);
+                    p1 = b1_lane_chain(pre, d1, sv1[0], sv1[NS > 1 ? 1 : 0], sv1[NS > 2 ? 2 : 0], sv1[NS > 3 ? 3 : 0]);
                 }
                 rowsum = (ok0 ? p0 : 0.0) + (ok1 ? p1 : 0.0);
                 rowsum += __shfl_xor_sync(0xffffffffu, rowsum, 1);
@@ -522,8 +544,8 @@ row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ 
 #pragma unroll
                 for (int j = 0; j < FO_MAX_SIDES; ++j) {
                     const bool rs = p.has_pre && j == p.sides.n;
-                    a0[j] = rs ? rowsum : sv0[j];
-                    a1[j] = rs ? rowsum : sv1[j];
+                    a0[j] = rs ? rowsum : sv0[j < NS ? j : 0];
+                    a1[j] = rs ? rowsum : sv1[j < NS ? j : 0];
                 }
                 t0 = b1_lane_chain(post, d0, a0[0], a0[1], a0[2], a0[3]);
                 t1 = b1_lane_chain(post, d1, a1[0], a1[1], a1[2], a1[3]);
@@ -713,12 +735,22 @@ struct MmaShape {
     int ncb, w, kb;
 };
 
-bool b1_mma_shape(long long n, int k, MmaShape *out)
+bool b1_mma_shape(long long n, int k, int nw, MmaShape *out)
 {
     const int kb = pow2_at_least((k + 7) / 8);
-    if (kb > kMmaWarps || n < 2) return false;
+    if (kb > nw || n < 2) return false;
+    // FUSEDOPS_B1_MMA_SHAPE="ncb,w" (read per call; a tuning knob)
+    const char *e = getenv("FUSEDOPS_B1_MMA_SHAPE");
+    if (e) {
+        int a = 0, b = 0;
+        if (sscanf(e, "%d,%d", &a, &b) == 2 && (a == 8 || a == 14 || a == 16 || a == 20) && b >= 1 &&
+            (b & (b - 1)) == 0 && b * kb <= nw && (long long)8 * a * b >= n) {
+            *out = MmaShape{a, b, kb};
+            return true;
+        }
+    }
     const int ncbs[] = {8, 14, 16, 20};
-    for (int w = 1; w * kb <= kMmaWarps; w *= 2)
+    for (int w = 1; w * kb <= nw; w *= 2)
         for (int ncb : ncbs)
             if ((long long)8 * ncb * w >= n) {
                 *out = MmaShape{ncb, w, kb};
@@ -730,10 +762,11 @@ bool b1_mma_shape(long long n, int k, MmaShape *out)
 // Row stride of a tile in shared memory: the smallest ns >= n with ns = 4 (mod 8).
 int b1_mma_stride(long long n) { return (int)(n + ((4 - n % 8) + 8) % 8); }
 
-template <int NCB>
+template <int NW, int NCB>
 cudaError_t b1_mma_launch(const DevChain &pre, const DevChain &post, const B1Params &p, int agg,
                           int grid, size_t smem, cudaStream_t st)
 {
+    constexpr int kMmaBlock = NW * 32;
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -742,8 +775,8 @@ cudaError_t b1_mma_launch(const DevChain &pre, const DevChain &post, const B1Par
     };
     const bool generic = p.chain_kind == kB1Generic;
     if (agg == FO_ROW_COL_AGG_B1_T)
-        return generic ? go(row_b1_mma_kernel<NCB, kB1ColT, true>) : go(row_b1_mma_kernel<NCB, kB1ColT, false>);
-    return generic ? go(row_b1_mma_kernel<NCB, kB1None, true>) : go(row_b1_mma_kernel<NCB, kB1None, false>);
+        return generic ? go(row_b1_mma_kernel<NW, NCB, kB1ColT, true>) : go(row_b1_mma_kernel<NW, NCB, kB1ColT, false>);
+    return generic ? go(row_b1_mma_kernel<NW, NCB, kB1None, true>) : go(row_b1_mma_kernel<NW, NCB, kB1None, false>);
 }
 
 bool b1_aligned16(const void *q) { return ((uintptr_t)q & 15u) == 0; }
@@ -860,8 +893,12 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
         MmaShape ms;
         const char *env = getenv("FUSEDOPS_B1_MMA");
         const bool want = env ? env[0] != '0' : (k > 2 || cols <= 160);
-        if (want && staged && b1_mma_shape(cols, k, &ms)) {
-            const int groups = kMmaWarps / (ms.w * ms.kb);
+        // 8 warps (two per scheduler, up to 255 registers each) measured faster than 16
+        // warps of 128 registers in every layout tried: 0.81 against 1.06 ms at best for
+        // 5 000 000 x 100, k = 8
+        const int nw = 8;
+        if (want && staged && b1_mma_shape(cols, k, nw, &ms)) {
+            const int groups = nw / (ms.w * ms.kb);
             const int ns = b1_mma_stride(cols);
             const size_t slot_bytes = (size_t)8 * ns * 8;
             const size_t budget = 208 * 1024;
@@ -878,10 +915,10 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
                 if (grid > sms) grid = sms;
                 if (grid < 1) grid = 1;
                 cudaError_t e = cudaErrorInvalidValue;
-                if (ms.ncb == 8) e = b1_mma_launch<8>(chpre, chpost, p, agg, (int)grid, smem, st);
-                else if (ms.ncb == 14) e = b1_mma_launch<14>(chpre, chpost, p, agg, (int)grid, smem, st);
-                else if (ms.ncb == 16) e = b1_mma_launch<16>(chpre, chpost, p, agg, (int)grid, smem, st);
-                else if (ms.ncb == 20) e = b1_mma_launch<20>(chpre, chpost, p, agg, (int)grid, smem, st);
+                if (ms.ncb == 8) e = b1_mma_launch<8, 8>(chpre, chpost, p, agg, (int)grid, smem, st);
+                else if (ms.ncb == 14) e = b1_mma_launch<8, 14>(chpre, chpost, p, agg, (int)grid, smem, st);
+                else if (ms.ncb == 16) e = b1_mma_launch<8, 16>(chpre, chpost, p, agg, (int)grid, smem, st);
+                else if (ms.ncb == 20) e = b1_mma_launch<8, 20>(chpre, chpost, p, agg, (int)grid, smem, st);
                 return e == cudaSuccess ? FO_OK : cuda_fail(e);
             }
         }
