@@ -778,6 +778,23 @@ def run_ours(args):
         binding = max(terms, key=terms.get)
         roofline_per_op["outer"].update({"bound_terms_ms": terms, "binding_term": binding,
                                          "frac_of_binding_term": terms[binding] / per_op["outer"]["ms"]})
+        # the paper's cost model (Section 4.3: write time + max(read time, compute time)) fed with
+        # this machine's measured rates: predicted time of each fused operator and of the plan of
+        # basic operators it replaces, next to the measured time
+        gf = probes["fp64_fma_tflops"] * 1e3
+        cm = {}
+        for n in OPS:
+            kw = dict(shapes[n])
+            if n == "row_csr":
+                kw["nnz"] = nnz4
+            if n == "outer":
+                kw["nnz"] = nnz5
+            kw = {k2: v2 for k2, v2 in kw.items() if k2 in ("rows", "cols", "nnz", "rank")}
+            fused = fo.plan_cost([fo.operator_sizes(n, **kw)], peak_gbs, peak_gbs, gf) * 1e3
+            unfused = fo.plan_cost(fo.unfused_plan_sizes(n, **kw), peak_gbs, peak_gbs, gf) * 1e3
+            cm[n] = {"predicted_fused_ms": fused, "predicted_unfused_ms": unfused,
+                     "measured_ms": per_op[n]["ms"], "measured_over_predicted": per_op[n]["ms"] / fused}
+        line["cost_model"] = cm
         if args.frac == 1.0 and world == 1:
             line["size_sweep"] = size_sweep(fo, device)
 

@@ -8,10 +8,12 @@ from .binding import (  # noqa: F401
     jit_compile_check, jit_stats, load_library, make_chain, probe_fp64_fma, probe_l2_gather, probe_out_len, set_jit,
     workspace,
 )
-from .roofline import algorithmic_bytes, ideal_seconds  # noqa: F401
+from .roofline import (  # noqa: F401
+    algorithmic_bytes, ideal_seconds, operator_cost, operator_sizes, plan_cost, unfused_plan_sizes,
+)
 
 __all__ = [
     "CSR", "FusedOpsError", "chain_describe", "device_status", "force_interpreter", "fused_cell", "fused_cell_static", "fused_magg", "fused_outer",
-    "fused_row", "fused_row_b1", "jit_compile_check", "jit_stats", "set_jit", "load_library", "make_chain", "workspace", "algorithmic_bytes", "ideal_seconds",
+    "fused_row", "fused_row_b1", "jit_compile_check", "jit_stats", "set_jit", "load_library", "make_chain", "workspace", "algorithmic_bytes", "ideal_seconds", "operator_cost", "operator_sizes", "plan_cost", "unfused_plan_sizes",
     "probe_fp64_fma", "probe_l2_gather", "probe_out_len",
 ]

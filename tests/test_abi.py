@@ -250,3 +250,33 @@ def test_chain_describe_writes_the_arithmetic_not_the_temporaries():
         fo.chain_describe(magg, ["t0", "t1"], use="cell", n_sides=1, k=2)
     with pytest.raises(FusedOpsError):
         fo.chain_describe([("mul", "t0", "a", "side3")], "t0", use="cell", n_sides=1)
+
+
+def test_cost_model_form_and_plans():
+    # Section 4.3: C = sum over operators of T_w + max(T_r, T_c)
+    from paper_1801_00829_b200 import operator_cost, operator_sizes, plan_cost, unfused_plan_sizes
+    # the worked example is the read term of an I/O-bound operator with nothing to write
+    assert abs(operator_cost(1e9 * 8, 0, 0, 32, 32, 1) - 0.25) < 1e-12
+    # compute-bound: the larger of read and compute counts, the write time adds
+    assert abs(operator_cost(8e9, 16e9, 230.4e9 * 2, 32, 32, 230.4) - (0.5 + 2.0)) < 1e-12
+    # a fused Cell operator reads its three inputs once; the unfused plan also writes and
+    # re-reads two intermediates: 3 reads against 5 reads + 2 writes of m*n doubles
+    kw = dict(rows=1000, cols=1000)
+    r, w, f = operator_sizes("cell", **kw)
+    assert (r, w) == (24_000_000, 8)
+    ops = unfused_plan_sizes("cell", **kw)
+    assert sum(o[0] for o in ops) == 5 * 8_000_000 and sum(o[1] for o in ops) == 2 * 8_000_000 + 8
+    fused = plan_cost([(r, w, f)], 32, 32, 230.4)
+    unfused = plan_cost(ops, 32, 32, 230.4)
+    assert abs(unfused / fused - 7.0 / 3.0) < 1e-3          # bandwidth-bound on both sides
+    # the Row chain: fusion removes the second scan of X, the model's factor of two (Section 5.2)
+    kw = dict(rows=10 ** 6, cols=1000)
+    fused = plan_cost([operator_sizes("row_dense", **kw)], 32, 32, 230.4)
+    unfused = plan_cost(unfused_plan_sizes("row_dense", **kw), 32, 32, 230.4)
+    assert 1.99 < unfused / fused < 2.01
+    # the Outer operator: the unfused plan's cost does not depend on the number of stored
+    # cells, the fused one's is proportional to it - orders of magnitude at low density
+    kw = dict(rows=20000, cols=20000, rank=100)
+    hi = plan_cost(unfused_plan_sizes("outer", nnz=40000, **kw), 32, 32, 230.4)
+    lo = plan_cost([operator_sizes("outer", nnz=40000, **kw)], 32, 32, 230.4)
+    assert hi / lo > 1000
