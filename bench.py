@@ -397,6 +397,80 @@ def size_sweep(fo, device, cols=1000, rows_list=(1_000, 10_000, 100_000, 1_000_0
 
 
 # ---------------------------------------------------------------------- clocks
+def _device_csr(fo, rows, cols, density, g, device, lo=0.0, hi=1.0, chunk_rows=None):
+    """A Bernoulli(density) CSR matrix built on the device (values uniform[lo, hi)), row chunk by
+    row chunk so that the dense mask of a chunk stays small."""
+    import torch
+    if density >= 1.0:
+        rowptr = (torch.arange(rows + 1, device=device, dtype=torch.int64) * cols).to(torch.int32)
+        colidx = torch.arange(cols, device=device, dtype=torch.int32).repeat(rows)
+        vals = torch.rand(rows * cols, generator=g, dtype=torch.float64, device=device) * (hi - lo) + lo
+        return fo.CSR(rows, cols, rowptr, colidx, vals)
+    chunk_rows = chunk_rows or max(1, (64 << 20) // cols)
+    counts, cols_l = [], []
+    for r0 in range(0, rows, chunk_rows):
+        nr = min(chunk_rows, rows - r0)
+        mask = torch.rand((nr, cols), generator=g, device=device) < density
+        counts.append(mask.sum(dim=1, dtype=torch.int32))
+        cols_l.append(mask.nonzero()[:, 1].to(torch.int32))
+        del mask
+    rowptr = torch.zeros(rows + 1, dtype=torch.int32, device=device)
+    rowptr[1:] = torch.cumsum(torch.cat(counts), 0)
+    colidx = torch.cat(cols_l).contiguous()
+    vals = torch.rand(colidx.numel(), generator=g, dtype=torch.float64, device=device) * (hi - lo) + lo
+    return fo.CSR(rows, cols, rowptr, colidx, vals)
+
+
+def paper_suite(fo, device, reps=5):
+    """The operator micro-benchmarks of Section 5.2 at the paper's own sizes (inputs made on the
+    device from a seeded torch generator; parity of every kernel used here is covered by the tests):
+    Cell sum(X*Y*Z), MAgg (sum(X*Y), sum(X*Z)), Row t(X)(Xv) and t(X)(XV) over x * 10^3 inputs,
+    x = 10^3 .. 10^6, dense and at sparsity 0.1; Outer sum(X * log(U t(V) + 1e-15)) over
+    2*10^4 x 2*10^4 at rank 100, sparsity 1 .. 10^-4.  Cold L2 (a 512 MB buffer is rewritten
+    before every run); times are the minimum of `reps` runs."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(12)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+    one = torch.empty(1, dtype=torch.float64, device=device)
+    two = torch.empty(2, dtype=torch.float64, device=device)
+    magg2 = [("mul", "t0", "a", "side0"), ("mul", "t1", "a", "side1")]
+    cols = 1000
+    qv = torch.empty(cols, dtype=torch.float64, device=device)
+    qm = torch.empty((cols, 2), dtype=torch.float64, device=device)
+    v = torch.randn(cols, generator=g, dtype=torch.float64, device=device)
+    V2 = torch.randn((cols, 2), generator=g, dtype=torch.float64, device=device)
+
+    def t_us(fn):
+        return min(_event_times(fn, reps, before=flush.zero_)) * 1e3
+
+    out = {"cell_magg_row": [], "outer": []}
+    for rows in (1_000, 10_000, 100_000, 1_000_000):
+        X, Y, Z = (torch.rand((rows, cols), generator=g, dtype=torch.float64, device=device) for _ in range(3))
+        sides = [("cell", Y), ("cell", Z)]
+        Xs = _device_csr(fo, rows, cols, 0.1, g, device)
+        e = {"rows": rows, "cols": cols, "dense_bytes_per_input": 8 * rows * cols, "sparse_nnz": Xs.nnz}
+        e["cell_dense_us"] = t_us(lambda: fo.fused_cell(XYZ, "t1", X, sides, out=one))
+        e["cell_sparse_us"] = t_us(lambda: fo.fused_cell(XYZ, "t1", Xs, sides, out=one))
+        e["magg_dense_us"] = t_us(lambda: fo.fused_magg(magg2, ["t0", "t1"], X, sides, out=two))
+        e["magg_sparse_us"] = t_us(lambda: fo.fused_magg(magg2, ["t0", "t1"], Xs, sides, out=two))
+        e["row_xtxv_dense_us"] = t_us(lambda: fo.fused_row([], "d", X, v, out=qv))
+        e["row_xtxv_sparse_us"] = t_us(lambda: fo.fused_row([], "d", Xs, v, out=qv))
+        e["row_xtxV2_dense_us"] = t_us(lambda: fo.fused_row_b1(None, None, [], "d", X, V2, out=qm))
+        out["cell_magg_row"].append(e)
+        del X, Y, Z, Xs, sides
+    m = 20_000
+    U = torch.rand((m, 100), generator=g, dtype=torch.float64, device=device) + 0.1
+    Vf = torch.rand((m, 100), generator=g, dtype=torch.float64, device=device) + 0.1
+    xlog = [("add", "t0", "d", 1e-15), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")]
+    for sp in (1.0, 0.1, 0.01, 0.001, 0.0001):
+        Xs = _device_csr(fo, m, m, sp, g, device, chunk_rows=2000)
+        us = t_us(lambda: fo.fused_outer(xlog, "t2", Xs, U, Vf, out=one))
+        out["outer"].append({"sparsity": sp, "nnz": Xs.nnz, "us": us, "nnz_per_s": Xs.nnz / (us * 1e-6)})
+        del Xs
+    return out
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
@@ -797,6 +871,8 @@ def run_ours(args):
         line["cost_model"] = cm
         if args.frac == 1.0 and world == 1:
             line["size_sweep"] = size_sweep(fo, device)
+        if args.paper_suite and world == 1:
+            line["paper_suite"] = paper_suite(fo, device)
 
     # ---- CPU baseline: the checker on a bounded sample, rank 0 at N = 1 only
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -839,6 +915,8 @@ def main():
     ap.add_argument("--no-variants", action="store_true", help="skip the untimed-step variant measurements")
     ap.add_argument("--full-outer", action="store_true", help="keep the Outer workload at full size under --frac")
     ap.add_argument("--ops", default="", help="comma-separated subset of the five operators (profiling)")
+    ap.add_argument("--paper-suite", action="store_true",
+                    help="also time the paper's operator micro-benchmarks at their own sizes (adds about a minute)")
     ap.add_argument("--interp", action="store_true", help="run Cell / MAgg chains through the interpreter")
     args = ap.parse_args()
     if args.impl == "reference":
