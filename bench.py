@@ -216,6 +216,7 @@ def time_variants(fo, step, shapes, reps=10):
     o_all = torch.empty((mr, mc), dtype=torch.float64, device=dev)
     o_one = torch.empty(1, dtype=torch.float64, device=dev)
     o_rr = torch.empty(rr, dtype=torch.float64, device=dev)
+    o_rn = torch.empty((rr, rc), dtype=torch.float64, device=dev)
     o_nnz = torch.empty(nnz5, dtype=torch.float64, device=dev)
     o_right = torch.empty((orow, rank), dtype=torch.float64, device=dev)
     ocol = shapes["outer"]["cols"]
@@ -245,6 +246,9 @@ def time_variants(fo, step, shapes, reps=10):
         ("row_dense_full_agg", lambda: fo.fused_row(WD, "t0", d["row_dense.X"], d["row_dense.v"],
                                                     [("row", d["row_dense.w"])], agg="full", out=o_one),
          8 * rr * rc + 8 * rr + 8 * rc),
+        ("row_dense_no_agg", lambda: fo.fused_row(WD, "t0", d["row_dense.X"], d["row_dense.v"],
+                                                  [("row", d["row_dense.w"])], agg="none", out=o_rn),
+         2 * 8 * rr * rc + 8 * rr + 8 * rc),
         ("outer_no_agg", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
                                                 agg="none", out=o_nnz), outer_in + 8 * nnz5),
         ("outer_right_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],

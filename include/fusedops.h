@@ -135,9 +135,9 @@ typedef struct fo_chain {
 /* ------------------------------------------------------ template variants */
 /* Cell (Table 1: no_agg, row_agg, col_agg, full_agg) */
 enum { FO_CELL_NO_AGG = 0, FO_CELL_ROW_AGG = 1, FO_CELL_COL_AGG = 2, FO_CELL_FULL_AGG = 3 };
-/* Row (Table 1).  fused_row implements ROW_AGG (one value per row), FULL_AGG and
- * COL_T_AGG (the n x 1 vector sum_i t_i * X_i^T); NO_AGG and COL_AGG return
- * FO_ERR_UNSUPPORTED.  The *_B1 variants (row intermediates that are k-vectors,
+/* Row (Table 1).  fused_row implements all of no_agg, row_agg, col_agg, full_agg
+ * and col_t_agg (col_agg, 1 x n, and col_t_agg, n x 1, are the same n values in
+ * memory).  The *_B1 variants (row intermediates that are k-vectors,
  * from a product with a side matrix) belong to fused_row_b1. */
 enum { FO_ROW_NO_AGG = 0, FO_ROW_ROW_AGG = 1, FO_ROW_COL_AGG = 2, FO_ROW_FULL_AGG = 3,
        FO_ROW_COL_T_AGG = 4, FO_ROW_NO_AGG_B1 = 5, FO_ROW_COL_AGG_B1_T = 6 };
@@ -285,8 +285,12 @@ int fused_magg(const fo_chain *chain, const fo_mat *X,
  *     d   = X_i . v                    (v: device, X.cols doubles)
  *     t_i = chain(d, sides read at row i, scalars)     (sides must be FO_AT_ROW)
  *   FO_ROW_COL_T_AGG: out += t_i * X_i^T   -> out[j] = sum_i t_i X_ij (cols doubles)
+ *   FO_ROW_COL_AGG  : the same n sums, read as a 1 x n row
  *   FO_ROW_ROW_AGG  : out[i] = t_i                                   (rows doubles)
  *   FO_ROW_FULL_AGG : out[0] = sum_i t_i
+ *   FO_ROW_NO_AGG   : dense X: out[i * cols + j] = t_i * X_ij  (rows x cols, packed);
+ *                     CSR X: out[p] = t_i * vals[p] for stored cell p of row i
+ *                     (nnz doubles, X's pattern)
  * With the chain  t = side0 * d  this is  t(X) %*% (w * (X %*% v)).
  * X wider than 8192 columns returns FO_ERR_UNSUPPORTED (the single-pass
  * kernels keep a row, respectively v and the output vector, on chip).

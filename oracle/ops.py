@@ -241,6 +241,9 @@ def row(chain, output, X, v, sides=(), scalars=(), agg="col_t"):
     agg "col_t": q = X^T t       second scan of X, n-vector
         "row"  : t itself        m-vector
         "full" : sum(t)
+        "none" : T = t * X       every row of X scaled by its t (dense: m x n; CSR:
+                                 the nnz new values on X's pattern)
+        "col"  : colSums(T)      the column sums of that materialised T, n-vector
     """
     m = X["rows"] if _is_csr(X) else X.shape[0]
     v = np.asarray(v, dtype=np.float64)
@@ -261,6 +264,14 @@ def row(chain, output, X, v, sides=(), scalars=(), agg="col_t"):
         return t
     if agg == "full":
         return full_sum(t)
+    if agg in ("none", "col"):
+        if _is_csr(X):
+            T = t[csr_row_ids(X["rows"], X["rowptr"])] * np.asarray(X["vals"], dtype=np.float64)
+            if agg == "none":
+                return T
+            return _segment_sum(T, np.asarray(X["colidx"], dtype=np.int64), X["cols"])
+        T = t.reshape(m, 1) * np.asarray(X, dtype=np.float64)
+        return T if agg == "none" else col_sums(T)
     raise ValueError(agg)
 
 

@@ -468,7 +468,8 @@ def fused_magg(steps, outputs, X, sides=(), scalars=(), out=None):
 
 
 def fused_row(steps, output, X, v, sides=(), scalars=(), agg="col_t", out=None):
-    """Row template.  Returns (cols,), (rows,) or (1,)."""
+    """Row template.  Returns (cols,), (rows,), (1,) or, for agg "none", (rows, cols) /
+    (nnz,) for a dense / CSR main input."""
     lib = load_library()
     sides = list(sides)
     ch, keep = make_chain(steps, output)
@@ -478,7 +479,8 @@ def fused_row(steps, output, X, v, sides=(), scalars=(), agg="col_t", out=None):
     a = ROW_AGG[agg]
     assert v.dtype == torch.float64 and v.numel() == cols and (v.numel() <= 1 or v.stride(-1) == 1)
     if out is None:
-        shape = {"col_t": (cols,), "row": (rows,), "full": (1,)}.get(agg, (1,))
+        shape = {"col_t": (cols,), "col": (cols,), "row": (rows,), "full": (1,),
+                 "none": (X.nnz,) if isinstance(X, CSR) else (rows, cols)}[agg]
         out = torch.empty(shape, dtype=torch.float64, device=dev)
     need = lib.fused_row_workspace_bytes(C.byref(m), a)
     ws = workspace(dev, max(need, 16384))

@@ -35,13 +35,14 @@ struct RowParams {
     int stages, rows_per_stage; // dense ring geometry
     int chain_kind;             // kChainGeneric, or a row chain the kernels evaluate inline
     int sides_in_ring;          // dense: used sides are contiguous vectors, staged with the rows
+    int out_vec;                // no_agg, dense: rows of `out` can be written 16 bytes at a time
 };
 
 // Row chains common enough to be evaluated inline instead of interpreted; the
 // arithmetic is the same, so are the bits.
 enum { kChainGeneric = 0, kChainSideTimesDot = 1, kChainDot = 2 };
 
-enum { kRowColT = 0, kRowRow = 1, kRowFull = 2 };
+enum { kRowColT = 0, kRowRow = 1, kRowFull = 2, kRowNone = 3 };
 
 constexpr int kWarps = kThreads / 32;
 
@@ -281,6 +282,26 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
                     q[c].y = fma(tr, x[r][c].y, q[c].y);
                 }
             }
+        } else if (AGG == kRowNone) {
+            // out_i = t_i * X_i, written from the registers that hold the row
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const double tr = __shfl_sync(0xffffffffu, t, r);
+                double *orow = p.out + (r0 + r) * (long long)n;
+                if (r0 + r < p.rows) {
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        const int col = 64 * (c * W + w) + 2 * lane;
+                        if (p.out_vec) {
+                            if (col < n)
+                                *reinterpret_cast<double2 *>(orow + col) = make_double2(tr * x[r][c].x, tr * x[r][c].y);
+                        } else {
+                            if (col < n) orow[col] = tr * x[r][c].x;
+                            if (col + 1 < n) orow[col + 1] = tr * x[r][c].y;
+                        }
+                    }
+                }
+            }
         } else {
             const long long row = r0 + lane;
             if (w == 0 && lane < R && row < p.rows) {
@@ -420,6 +441,16 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
             if (have) p.out[myrow] = t;
         } else if (AGG == kRowFull) {
             if (have) tsum += t;
+        } else if (AGG == kRowNone) {
+            // out has X's pattern: stored cell p of row i becomes t_i * vals[p]; one
+            // row after the other, the lanes across the row's cells
+            for (int rr = 0; rr < 32; ++rr) {
+                const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
+                const int end = __shfl_sync(0xffffffffu, end_l, rr);
+                const double tt = __shfl_sync(0xffffffffu, t, rr);
+                for (int q0 = beg + lane; q0 < end; q0 += 32)
+                    p.out[q0] = tt * (staged ? sx[q0 - base] : __ldg(p.vals + q0));
+            }
         } else {
 #pragma unroll 1
             for (int it = 0; it < G; ++it) {
@@ -492,6 +523,7 @@ cudaError_t launch_dense_agg(const DevChain &ch, const RowParams &p, int agg, in
         return cudaGetLastError();
     };
     if (agg == FO_ROW_COL_T_AGG) return go(row_dense_kernel<NCH, W, R, kRowColT, STAGED>);
+    if (agg == FO_ROW_NO_AGG) return go(row_dense_kernel<NCH, W, R, kRowNone, STAGED>);
     if (agg == FO_ROW_ROW_AGG) return go(row_dense_kernel<NCH, W, R, kRowRow, STAGED>);
     return go(row_dense_kernel<NCH, W, R, kRowFull, STAGED>);
 }
@@ -553,7 +585,8 @@ extern "C" {
 size_t fused_row_workspace_bytes(const fo_mat *X, int agg)
 {
     if (!X) return 0;
-    if (agg != FO_ROW_COL_T_AGG && agg != FO_ROW_ROW_AGG && agg != FO_ROW_FULL_AGG) return 0;
+    if (agg == FO_ROW_COL_AGG) agg = FO_ROW_COL_T_AGG;
+    if (agg != FO_ROW_COL_T_AGG && agg != FO_ROW_ROW_AGG && agg != FO_ROW_FULL_AGG && agg != FO_ROW_NO_AGG) return 0;
     const long long cols = X->kind == FO_DENSE ? X->dense.cols : X->kind == FO_CSR ? X->csr.cols : -1;
     if (cols < 0) return 0;
     return fo::row_ws_bytes(cols, agg);
@@ -564,10 +597,11 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
               size_t ws_bytes, void *stream)
 {
     using namespace fo;
-    if (!chain || !X || !out) return FO_ERR_NULL;
+    if (!chain || !X) return FO_ERR_NULL;
     if (n_sides > 0 && !sides) return FO_ERR_NULL;
-    if (agg == FO_ROW_NO_AGG || agg == FO_ROW_COL_AGG) return FO_ERR_UNSUPPORTED;
-    if (agg != FO_ROW_COL_T_AGG && agg != FO_ROW_ROW_AGG && agg != FO_ROW_FULL_AGG)
+    // col_agg (1 x n) and col_t_agg (n x 1) hold the same n values
+    if (agg == FO_ROW_COL_AGG) agg = FO_ROW_COL_T_AGG;
+    if (agg != FO_ROW_COL_T_AGG && agg != FO_ROW_ROW_AGG && agg != FO_ROW_FULL_AGG && agg != FO_ROW_NO_AGG)
         return FO_ERR_UNSUPPORTED;
     if (X->kind != FO_DENSE && X->kind != FO_CSR) return FO_ERR_SHAPE;
     const bool csr = X->kind == FO_CSR;
@@ -619,11 +653,15 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     p.out = out;
     cudaStream_t st = (cudaStream_t)stream;
 
-    const long long nout = agg == FO_ROW_COL_T_AGG ? cols : agg == FO_ROW_ROW_AGG ? rows : 1;
+    const long long nout = agg == FO_ROW_COL_T_AGG ? cols : agg == FO_ROW_ROW_AGG ? rows
+                           : agg == FO_ROW_NO_AGG ? (csr ? X->csr.nnz : rows * cols) : 1;
+    if (!out && nout > 0) return FO_ERR_NULL;
     if (rows == 0 || cols == 0) {
         // no rows: empty sums; no columns: d = 0 for every row, which the chain may
         // still map to a non-zero t - handled by the kernels below unless rows == 0
-        if (rows == 0 || agg == FO_ROW_COL_T_AGG) {
+        if (rows == 0 || agg == FO_ROW_COL_T_AGG || agg == FO_ROW_NO_AGG) {
+            // (no_agg without rows or columns has nothing to write)
+            if (agg == FO_ROW_NO_AGG) return FO_OK;
             if (nout > 0) {
                 const long long b = (nout + 255) / 256;
                 row_fill_zero_kernel<<<(unsigned)(b > 1024 ? 1024 : b), 256, 0, st>>>(out, nout);
@@ -652,6 +690,7 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
         auto by_agg = [&](auto g) -> cudaError_t {
             constexpr int G = decltype(g)::value;
             if (agg == FO_ROW_COL_T_AGG) return go(row_csr_kernel<kRowColT, G>);
+            if (agg == FO_ROW_NO_AGG) return go(row_csr_kernel<kRowNone, G>);
             if (agg == FO_ROW_ROW_AGG) return go(row_csr_kernel<kRowRow, G>);
             return go(row_csr_kernel<kRowFull, G>);
         };
@@ -664,6 +703,7 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
         else e = by_agg(std::integral_constant<int, 32>());
     } else {
         p.X = X->dense.data; p.ldx = X->dense.ld;
+        p.out_vec = (aligned16(out) && cols % 2 == 0) ? 1 : 0;
         const bool staged = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
         // ring geometry: every group of warps has its own ring of `stages` slots of r rows
         const DenseShape sh = dense_shape(cols);

@@ -64,7 +64,9 @@ def test_workspace_sizes(lib):
     assert lib.fused_magg_workspace_bytes(C.byref(m), 9) == 0
     r = lib.fused_row_workspace_bytes(C.byref(m), 4)
     assert r >= HEAD + 148 * 1000 * 8
-    assert lib.fused_row_workspace_bytes(C.byref(m), 0) == 0
+    assert lib.fused_row_workspace_bytes(C.byref(m), 0) == HEAD          # no_agg: control words only
+    assert lib.fused_row_workspace_bytes(C.byref(m), 2) == r             # col_agg holds what col_t_agg holds
+    assert lib.fused_row_workspace_bytes(C.byref(m), 9) == 0
     x = B.fo_csr()
     x.rows, x.cols, x.nnz = 10, 10, 5
     assert lib.fused_outer_workspace_bytes(C.byref(x), 100, 3) >= HEAD + 8
@@ -134,8 +136,8 @@ def test_row_and_outer_argument_errors(lib):
                              C.c_void_p(0x2000), C.c_void_p(0x10000), 1 << 30, None)
 
     assert row(m) == -4                                   # too wide for the single-pass kernel
-    assert row(dense_mat(10, 100), agg=0) == -4           # no_agg not provided
-    assert row(dense_mat(10, 100), agg=2) == -4           # col_agg not provided
+    assert row(dense_mat(10, 100), agg=5) == -4           # the B1 variants belong to fused_row_b1
+    assert row(dense_mat(10, 100), agg=9) == -4           # no such variant
     assert row(dense_mat(10, 100), v=0) == -1
     bad_side = (B.fo_side * 1)(side(10, 100, 0))
     assert row(dense_mat(10, 100), sides=bad_side) == -2  # Row sides are read at the row index

@@ -236,6 +236,48 @@ def test_row_dense_variants_strided_unaligned(fo, agg):
     assert_close(got.cpu().numpy(), ref, absscale=row_abs_scale(Xh, v, np.ones(rows)))
 
 
+@pytest.mark.parametrize("rows,cols", [(1000, 1000), (333, 120), (257, 129), (64, 18), (5, 1), (1, 7), (90, 4096),
+                                       (40, 8191)])
+def test_row_dense_no_agg_and_col_agg(fo, rows, cols):
+    w = datagen.row_dense_workload(rows, cols, seed=2)
+    chain = [("mul", "t0", "side0", "d"), ("add", "t1", "t0", "s0")]
+    sides_h, sides_d = [("row", w["w"])], [("row", to_dev(w["w"]))]
+    ref = oracle.row(chain, "t1", w["X"], w["v"], sides_h, [0.25], agg="none")
+    got = fo.fused_row(chain, "t1", to_dev(w["X"]), to_dev(w["v"]), sides_d, [0.25], agg="none")
+    assert tuple(got.shape) == (rows, cols)
+    tabs = (w["w"] * (np.abs(w["X"]) @ np.abs(w["v"])) + 0.25)[:, None] * np.abs(w["X"])
+    assert_close(got.cpu().numpy(), ref, absscale=tabs, what="row dense no_agg")
+    refc = oracle.row(chain, "t1", w["X"], w["v"], sides_h, [0.25], agg="col")
+    gotc = fo.fused_row(chain, "t1", to_dev(w["X"]), to_dev(w["v"]), sides_d, [0.25], agg="col")
+    assert_close(gotc.cpu().numpy(), refc, absscale=tabs.sum(axis=0), what="row dense col_agg")
+    # an output that starts 8 bytes off a 16-byte boundary
+    import torch
+    buf = torch.empty(rows * cols + 1, dtype=torch.float64, device="cuda")
+    out = buf[1:].view(rows, cols)
+    fo.fused_row(chain, "t1", to_dev(w["X"]), to_dev(w["v"]), sides_d, [0.25], agg="none", out=out)
+    assert_close(out.cpu().numpy(), ref, absscale=tabs, what="row dense no_agg, unaligned out")
+    assert fo.device_status() == 0
+
+
+@pytest.mark.parametrize("rows,cols,density", [(20000, 1000, 0.01), (5000, 64, 0.2), (300, 4000, 0.001), (17, 9, 0.5),
+                                               (2000, 800, 0.1), (100, 50, 0.0)])
+def test_row_csr_no_agg_and_col_agg(fo, rows, cols, density):
+    w = datagen.row_csr_workload(rows, cols, density, seed=3)
+    Xh = host_csr(w)
+    sides_h, sides_d = [("row", w["w"])], [("row", to_dev(w["w"]))]
+    ref = oracle.row(WD, "t0", Xh, w["v"], sides_h, agg="none")
+    got = fo.fused_row(WD, "t0", csr_to_dev(w), to_dev(w["v"]), sides_d, agg="none")
+    assert tuple(got.shape) == (len(w["vals"]),)
+    absX = dict(Xh, vals=np.abs(w["vals"]))
+    tabs = oracle.row(WD, "t0", absX, np.abs(w["v"]), sides_h, agg="none")
+    assert_close(got.cpu().numpy(), ref, absscale=tabs, what="row csr no_agg")
+    refc = oracle.row(WD, "t0", Xh, w["v"], sides_h, agg="col")
+    gotc = fo.fused_row(WD, "t0", csr_to_dev(w), to_dev(w["v"]), sides_d, agg="col")
+    assert_close(gotc.cpu().numpy(), refc, absscale=oracle.row(WD, "t0", absX, np.abs(w["v"]), sides_h, agg="col"),
+                 what="row csr col_agg")
+    assert fo.device_status() == 0
+
+
 @pytest.mark.parametrize("rows,cols,density", [(100000, 1000, 0.01), (5000, 64, 0.2), (300, 4000, 0.001),
                                                (17, 9, 0.5), (1000, 1000, 0.0),
                                                # mean row lengths 36, 80 and 200: 8, 16 and 32 lanes per row

@@ -368,6 +368,33 @@ def test_row_b1_side_kinds_and_scalars():
             assert abs(T[i, c] - want) <= 1e-14 * (abs(want) + abs(rs) + 1.0)
 
 
+def test_row_no_agg_and_col_agg():
+    m, n = 9, 6
+    w_ = datagen.row_dense_workload(m, n, seed=2)
+    X, v, w = w_["X"], w_["v"], w_["w"]
+    T = oracle.row(WD, "t0", X, v, [("row", w)], agg="none")
+    assert T.shape == (m, n)
+    for i in range(m):
+        t = float(w[i]) * float(sum(F(float(X[i, k])) * F(float(v[k])) for k in range(n)))
+        for j in range(n):
+            assert abs(T[i, j] - t * X[i, j]) <= 4e-15 * abs(t * X[i, j]) + 1e-300
+    # the column sums of the scaled rows are the transposed product: two routes to one vector
+    c = oracle.row(WD, "t0", X, v, [("row", w)], agg="col")
+    q = rat_row_chain(X, v, w)
+    scale = np.abs(X).T @ (w * (np.abs(X) @ np.abs(v)))
+    assert np.all(np.abs(c - q) <= 2e-15 * scale)
+    # CSR main input: same values on X's pattern
+    ws = datagen.row_csr_workload(30, 12, 0.3, seed=3)
+    Xs = {k: ws[k] for k in ("rows", "cols", "rowptr", "colidx", "vals")}
+    Xd = csr_to_dense(ws["rows"], ws["cols"], ws["rowptr"], ws["colidx"], ws["vals"])
+    Ts = oracle.row(WD, "t0", Xs, ws["v"], [("row", ws["w"])], agg="none")
+    Td = oracle.row(WD, "t0", Xd, ws["v"], [("row", ws["w"])], agg="none")
+    rid = oracle.csr_row_ids(ws["rows"], ws["rowptr"])
+    assert np.allclose(Ts, Td[rid, ws["colidx"]], rtol=1e-14, atol=0)
+    cs = oracle.row(WD, "t0", Xs, ws["v"], [("row", ws["w"])], agg="col")
+    assert np.allclose(cs, oracle.row(WD, "t0", Xd, ws["v"], [("row", ws["w"])], agg="col"), rtol=1e-13, atol=1e-15)
+
+
 def test_row_csr_equals_dense_and_bruteforce():
     m, n = 40, 25
     w_ = datagen.row_csr_workload(m, n, 0.2, seed=3)
