@@ -456,6 +456,12 @@ def paper_suite(fo, device, reps=5):
         e = {"rows": rows, "cols": cols, "dense_bytes_per_input": 8 * rows * cols, "sparse_nnz": Xs.nnz}
         e["cell_dense_us"] = t_us(lambda: fo.fused_cell(XYZ, "t1", X, sides, out=one))
         e["cell_sparse_us"] = t_us(lambda: fo.fused_cell(XYZ, "t1", Xs, sides, out=one))
+        Ys = _device_csr(fo, rows, cols, 0.1, g, device)
+        Zs = _device_csr(fo, rows, cols, 0.1, g, device)
+        ssides = [("cell", Ys), ("cell", Zs)]
+        e["cell_all_sparse_us"] = t_us(lambda: fo.fused_cell(XYZ, "t1", Xs, ssides, out=one))
+        e["magg_all_sparse_us"] = t_us(lambda: fo.fused_magg(magg2, ["t0", "t1"], Xs, ssides, out=two))
+        del Ys, Zs, ssides
         e["magg_dense_us"] = t_us(lambda: fo.fused_magg(magg2, ["t0", "t1"], X, sides, out=two))
         e["magg_sparse_us"] = t_us(lambda: fo.fused_magg(magg2, ["t0", "t1"], Xs, sides, out=two))
         e["row_xtxv_dense_us"] = t_us(lambda: fo.fused_row([], "d", X, v, out=qv))

@@ -82,13 +82,20 @@ typedef struct fo_mat {
  *   FO_AT_CELL: same shape as the main input, value read at (rix, cix);
  *   FO_AT_ROW : column vector (rows x 1, element i at data[i * ld]), read at (rix);
  *   FO_AT_COL : row vector (1 x cols), read at (cix).
- * Side inputs are dense.
+ * Side inputs are dense, with one exception (the sparse side inputs of Table 1's
+ * Y+-, read through getValue() in Section 5.2 "Cell Operations"): if `sparse` is
+ * not NULL the side is that CSR matrix - same shape as the main input,
+ * FO_AT_CELL, `m` ignored - and reads 0.0 wherever it stores no cell.  Sparse
+ * sides are accepted by fused_cell and fused_magg over a CSR main input (a
+ * sparse driver with sparse sides); every other call returns
+ * FO_ERR_UNSUPPORTED for them.
  */
 enum { FO_AT_CELL = 0, FO_AT_ROW = 1, FO_AT_COL = 2 };
 typedef struct fo_side {
     fo_dense m;
     int32_t access;
     int32_t reserved;
+    const fo_csr *sparse;       /* host pointer or NULL; see below */
 } fo_side;
 
 /* ------------------------------------------------------------ operator chain */

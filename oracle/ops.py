@@ -134,6 +134,10 @@ def _cell_env_dense(X, sides, scalars):
     m, n = X.shape
     env = {"a": X}
     for k, (access, arr) in enumerate(sides):
+        if _is_csr(arr):               # sparse side over a dense main input: as a dense array
+            d = np.zeros((arr["rows"], arr["cols"]), dtype=np.float64)
+            d[csr_row_ids(arr["rows"], arr["rowptr"]), np.asarray(arr["colidx"], dtype=np.int64)] = arr["vals"]
+            arr = d
         arr = np.asarray(arr, dtype=np.float64)
         if access == "cell":
             assert arr.shape == (m, n)
@@ -151,6 +155,20 @@ def _cell_env_dense(X, sides, scalars):
     return env
 
 
+def _csr_lookup(Y, rid, cid):
+    """Values of the CSR matrix Y at the cells (rid[p], cid[p]); 0.0 where Y stores
+    nothing.  Cells are matched by their row-major position row * cols + col, which
+    ascends through a CSR matrix (np.searchsorted on those keys)."""
+    n = Y["cols"]
+    ykeys = csr_row_ids(Y["rows"], Y["rowptr"]) * n + np.asarray(Y["colidx"], dtype=np.int64)
+    keys = np.asarray(rid, dtype=np.int64) * n + np.asarray(cid, dtype=np.int64)
+    yv = np.asarray(Y["vals"], dtype=np.float64)
+    if ykeys.size == 0:
+        return np.zeros(keys.shape, dtype=np.float64)
+    pos = np.minimum(np.searchsorted(ykeys, keys), ykeys.size - 1)
+    return np.where(ykeys[pos] == keys, yv[pos], 0.0)
+
+
 def _cell_env_csr(X, sides, scalars):
     """Sparse-safe binding: one value per stored cell of the main input."""
     m, n = X["rows"], X["cols"]
@@ -158,6 +176,11 @@ def _cell_env_csr(X, sides, scalars):
     cid = np.asarray(X["colidx"], dtype=np.int64)
     env = {"a": np.asarray(X["vals"], dtype=np.float64)}
     for k, (access, arr) in enumerate(sides):
+        if _is_csr(arr):               # sparse side: its value at X's stored cells, 0 where it has none
+            if access != "cell":
+                raise ValueError("a CSR side is read at (row, column)")
+            env["side%d" % k] = _csr_lookup(arr, rid, cid)
+            continue
         arr = np.asarray(arr, dtype=np.float64)
         if access == "cell":
             env["side%d" % k] = arr[rid, cid]

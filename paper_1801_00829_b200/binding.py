@@ -62,7 +62,7 @@ class fo_mat(C.Structure):
 
 
 class fo_side(C.Structure):
-    _fields_ = [("m", fo_dense), ("access", C.c_int32), ("reserved", C.c_int32)]
+    _fields_ = [("m", fo_dense), ("access", C.c_int32), ("reserved", C.c_int32), ("sparse", C.c_void_p)]
 
 
 class fo_op(C.Structure):
@@ -284,9 +284,20 @@ def _mat(X):
 
 
 def _sides(sides, rows, cols):
+    """fo_side array for [(access, tensor or CSR), ...].  A CSR side (access "cell") is
+    passed through the struct's `sparse` pointer; the structs it points to hang off the
+    returned array so that they live as long as it does."""
     arr = (fo_side * max(1, len(sides)))()
+    arr._keep = []
     for k, (access, t) in enumerate(sides):
         acc = ACCESS[access]
+        if isinstance(t, CSR):
+            assert acc == 0, "a CSR side is read at (row, column)"
+            st = t.as_struct()
+            arr._keep.append(st)
+            arr[k].sparse = C.addressof(st)
+            arr[k].access = acc
+            continue
         if acc == 0:
             arr[k].m = _dense_struct(t)
         elif acc == 1:

@@ -347,6 +347,7 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     bool aligned = aligned16(xd.data) && (xd.ld % 2 == 0);
     for (int k = 0; k < n_sides; ++k) {
         const fo_side &s = sides[k];
+        if (s.sparse) return FO_ERR_UNSUPPORTED;       // sparse sides: CSR main input of Cell / MAgg only
         rc = check_dense(s.m);
         if (rc != FO_OK) return rc;
         switch (s.access) {

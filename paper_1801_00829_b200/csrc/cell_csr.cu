@@ -35,7 +35,25 @@ struct CsrCellParams {
     double *out;
     int agg;                 // FO_CELL_*
     int pad;
+    // sparse sides (access == kAtCellSparse): sides.s[k].data holds the values
+    const int *side_rowptr[FO_MAX_SIDES];
+    const int *side_colidx[FO_MAX_SIDES];
 };
+
+constexpr int kAtCellSparse = 3;      // a CSR side input read at (row, column); 0.0 where it stores nothing
+
+// Value of a CSR side at column j of a row whose stored cells are [sb, se):
+// binary search in the row's ascending column indices.
+__device__ __forceinline__ double sparse_side_value(const int *colidx, const double *vals, int sb, int se, int j)
+{
+    int lo = sb, hi = se;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(colidx + mid) < j) lo = mid + 1;
+        else hi = mid;
+    }
+    return (lo < se && __ldg(colidx + lo) == j) ? __ldg(vals + lo) : 0.0;
+}
 
 template <class EVAL, int NOUT, int G>
 __global__ void __launch_bounds__(kThreads)
@@ -72,6 +90,14 @@ cell_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Csr
             for (int k = 0; k < FO_MAX_SIDES; ++k)
                 srow[k] = (EVAL::uses_side(ch, k) && p.sides.s[k].access == FO_AT_ROW && beg < end)
                               ? __ldg(p.sides.s[k].data + row * p.sides.s[k].ld) : 0.0;
+            // sparse sides: the row's piece of the side's cells
+            int ssb[FO_MAX_SIDES], sse[FO_MAX_SIDES];
+#pragma unroll
+            for (int k = 0; k < FO_MAX_SIDES; ++k) {
+                const bool sp = EVAL::uses_side(ch, k) && p.sides.s[k].access == kAtCellSparse && beg < end;
+                ssb[k] = sp ? __ldg(p.side_rowptr[k] + row) : 0;
+                sse[k] = sp ? __ldg(p.side_rowptr[k] + row + 1) : 0;
+            }
             double rowacc = 0.0;
             int q = beg + lg;
             for (int s = 0; s < trips; ++s, q += G) {
@@ -85,7 +111,9 @@ cell_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Csr
                     if (EVAL::uses_side(ch, k)) {
                         const DevSide sd = p.sides.s[k];
                         if (sd.access == FO_AT_ROW) v = srow[k];
-                        else if (ok) v = __ldg(sd.data + (sd.access == FO_AT_CELL ? row * sd.ld + j : (long long)j));
+                        else if (sd.access == kAtCellSparse) {
+                            if (ok) v = sparse_side_value(p.side_colidx[k], sd.data, ssb[k], sse[k], j);
+                        } else if (ok) v = __ldg(sd.data + (sd.access == FO_AT_CELL ? row * sd.ld + j : (long long)j));
                     }
                     in[1 + k][0] = v;
                 }
@@ -176,6 +204,19 @@ int run_cell_csr(const fo_chain *chain, const fo_csr &X, const fo_side *sides, i
     p.sides.n = n_sides;
     for (int k = 0; k < n_sides; ++k) {
         const fo_side &s = sides[k];
+        if (s.sparse) {
+            const fo_csr &y = *s.sparse;
+            if (s.access != FO_AT_CELL || y.rows != X.rows || y.cols != X.cols || y.nnz < 0) return FO_ERR_SHAPE;
+            if (y.nnz > 0x7fffffffLL) return FO_ERR_UNSUPPORTED;
+            if (!y.rowptr) return FO_ERR_NULL;
+            if (y.nnz > 0 && (!y.colidx || !y.vals)) return FO_ERR_NULL;
+            p.sides.s[k].data = y.vals;
+            p.sides.s[k].ld = 0;
+            p.sides.s[k].access = kAtCellSparse;
+            p.side_rowptr[k] = y.rowptr;
+            p.side_colidx[k] = y.colidx;
+            continue;
+        }
         if (s.m.rows < 0 || s.m.cols < 0 || s.m.ld < s.m.cols) return FO_ERR_SHAPE;
         if (s.m.rows > 0 && s.m.cols > 0 && !s.m.data) return FO_ERR_NULL;
         switch (s.access) {

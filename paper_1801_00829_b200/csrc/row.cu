@@ -628,6 +628,7 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     p.sides.n = n_sides;
     for (int k = 0; k < n_sides; ++k) {
         const fo_side &s = sides[k];
+        if (s.sparse) return FO_ERR_UNSUPPORTED;       // sparse sides: CSR main input of Cell / MAgg only
         if (s.access != FO_AT_ROW) return FO_ERR_SHAPE;
         if (s.m.rows != rows || s.m.cols != 1 || s.m.ld < 1) return FO_ERR_SHAPE;
         if (rows > 0 && !s.m.data) return FO_ERR_NULL;

@@ -835,6 +835,7 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
     p.sides.n = n_sides;
     for (int j = 0; j < n_sides; ++j) {
         const fo_side &s = sides[j];
+        if (s.sparse) return FO_ERR_UNSUPPORTED;       // sparse sides: CSR main input of Cell / MAgg only
         if (s.access == FO_AT_CELL) {
             if (s.m.rows != rows || s.m.cols != k || s.m.ld < k) return FO_ERR_SHAPE;
         } else if (s.access == FO_AT_ROW) {

@@ -110,6 +110,27 @@ def test_cell_argument_errors(lib):
     assert call_cell(lib, ok_chain, "t0", bad) == -2
 
 
+def test_sparse_side_is_refused_outside_the_sparse_driver_kernels(lib):
+    y = B.fo_csr()
+    y.rows, y.cols, y.nnz = 10, 10, 5
+    y.rowptr, y.colidx, y.vals = 0x5000, 0x6000, 0x7000
+    sd = (B.fo_side * 1)()
+    sd[0].access = 0
+    sd[0].sparse = C.addressof(y)
+    ch, keep = B.make_chain([("mul", "t0", "a", "side0")], "t0")
+    sc = (C.c_double * 8)()
+    m = dense_mat(10, 10)
+    assert lib.fused_cell(C.byref(ch), C.byref(m), sd, 1, sc, 0, 3, C.c_void_p(0x2000),
+                          C.c_void_p(0x10000), 1 << 24, None) == -4
+    # over a CSR main input: the side must have the main input's shape and be read at the cell
+    x = B.fo_mat()
+    x.kind = 1
+    x.csr.rows, x.csr.cols, x.csr.nnz = 10, 12, 5
+    x.csr.rowptr, x.csr.colidx, x.csr.vals = 0x5000, 0x6000, 0x7000
+    assert lib.fused_cell(C.byref(ch), C.byref(x), sd, 1, sc, 0, 3, C.c_void_p(0x2000),
+                          C.c_void_p(0x10000), 1 << 24, None) == -2
+
+
 def test_chain_limits(lib):
     m = dense_mat(4, 4)
     long_chain = [("add", "t0", "a", 1.0)] + [("add", "t0", "t0", 1.0)] * 31

@@ -112,3 +112,39 @@ def test_cell_csr_empty_matrix_and_empty_rows(fo):
     assert fo.fused_cell(chain, "t0", E, agg="row").cpu().tolist() == [0.0, 0.0, 0.0]
     assert fo.fused_cell(chain, "t0", E, agg="col").cpu().tolist() == [0.0] * 4
     assert fo.fused_magg(chain + [("mov", "t1", "a")], ["t0", "t1"], E).cpu().tolist() == [0.0, 0.0]
+
+
+@pytest.mark.parametrize("rows,cols,dx,dy", [(3000, 1000, 0.1, 0.1), (500, 64, 0.3, 0.5), (100, 4000, 0.01, 0.02),
+                                             (33, 17, 0.5, 0.0), (2000, 300, 0.02, 0.9)])
+def test_cell_csr_sparse_sides(fo, rows, cols, dx, dy):
+    """A sparse driver with sparse side inputs (Section 5.2, "Cell Operations" over sparse data)."""
+    import datagen
+    rp, ci, xv = datagen.csr_bernoulli(21, 0, rows, cols, dx, 0.5, 1.5)
+    X = dict(rows=rows, cols=cols, rowptr=rp, colidx=ci, vals=xv)
+    rp2, ci2, yv = datagen.csr_bernoulli(21, 4, rows, cols, dy, -1.0, 1.0)
+    Y = dict(rows=rows, cols=cols, rowptr=rp2, colidx=ci2, vals=yv)
+    rp3, ci3, zv = datagen.csr_bernoulli(21, 8, rows, cols, 0.5, -1.0, 1.0)
+    Z = dict(rows=rows, cols=cols, rowptr=rp3, colidx=ci3, vals=zv)
+    W = datagen.normal(21, 12, rows * cols).reshape(rows, cols)
+    Xd, Yd_, Zd_ = csr_to_dev(X), csr_to_dev(Y), csr_to_dev(Z)
+    xyz = [("mul", "t0", "a", "side0"), ("mul", "t1", "t0", "side1")]
+    absX = dict(X, vals=np.abs(xv))
+    absY = dict(Y, vals=np.abs(yv))
+    absZ = dict(Z, vals=np.abs(zv))
+    for agg in ("full", "row", "col", "none"):
+        ref = oracle.cell(xyz, "t1", X, [("cell", Y), ("cell", Z)], agg=agg)
+        got = fo.fused_cell(xyz, "t1", Xd, [("cell", Yd_), ("cell", Zd_)], agg=agg)
+        scale = oracle.cell(xyz, "t1", absX, [("cell", absY), ("cell", absZ)], agg=agg)
+        assert_close(got.cpu().numpy(), ref, absscale=scale, what="sparse sides %s" % agg)
+    # sparse and dense sides mixed, a chain that is not zero-preserving in the sparse side, MAgg
+    chain = [("add", "t0", "side0", 1.0), ("mul", "t1", "a", "t0"), ("mul", "t2", "a", "side1")]
+    ref = oracle.magg(chain, ["t1", "t2"], X, [("cell", Y), ("cell", W)])
+    got = fo.fused_magg(chain, ["t1", "t2"], Xd, [("cell", Yd_), ("cell", to_dev(W))])
+    scale = oracle.magg([("abs", "t3", "side0"), ("add", "t0", "t3", 1.0), ("mul", "t1", "a", "t0"),
+                         ("abs", "t4", "side1"), ("mul", "t2", "a", "t4")], ["t1", "t2"], absX,
+                        [("cell", Y), ("cell", W)])
+    assert_close(got.cpu().numpy(), ref, absscale=scale, what="sparse sides magg")
+    # a dense main input refuses a sparse side
+    with pytest.raises(fo.FusedOpsError) as e:
+        fo.fused_cell(xyz, "t1", to_dev(W), [("cell", Yd_), ("cell", to_dev(W))])
+    assert e.value.status == -4

@@ -178,6 +178,39 @@ def test_cell_sparse_safe_equals_dense_for_zero_preserving_chain():
 
 
 # ------------------------------------------------------------------ MAgg
+def test_cell_sparse_sides_bruteforce():
+    # a sparse driver with a sparse side: the side reads 0 wherever it stores nothing
+    m, n = 7, 9
+    rp, ci, xv = datagen.csr_bernoulli(11, 0, m, n, 0.5, 1.0, 2.0)
+    X = dict(rows=m, cols=n, rowptr=rp, colidx=ci, vals=xv)
+    rp2, ci2, yv = datagen.csr_bernoulli(11, 4, m, n, 0.4, -1.0, 1.0)
+    Y = dict(rows=m, cols=n, rowptr=rp2, colidx=ci2, vals=yv)
+    Z = datagen.normal(11, 8, m * n).reshape(m, n)
+    Yd = csr_to_dense(m, n, rp2, ci2, yv)
+    Xd = csr_to_dense(m, n, rp, ci, xv)
+    chain = [("mul", "t0", "a", "side0"), ("mul", "t1", "t0", "side1")]
+    want = sum((F(float(Xd[i, j])) * F(float(Yd[i, j])) * F(float(Z[i, j])) for i in range(m) for j in range(n)), F(0))
+    got = oracle.cell(chain, "t1", X, [("cell", Y), ("cell", Z)], agg="full")
+    assert abs(got - float(want)) <= 1e-15 * float(np.sum(np.abs(Xd * Yd * Z))) + 1e-300
+    assert 0 < np.count_nonzero(Xd * Yd) < np.count_nonzero(Xd)        # the patterns really differ
+    # same values as with the side made dense, cell by cell and for every aggregation
+    for agg in ("none", "row", "col", "full"):
+        a = oracle.cell(chain, "t1", X, [("cell", Y), ("cell", Z)], agg=agg)
+        b = oracle.cell(chain, "t1", X, [("cell", Yd), ("cell", Z)], agg=agg)
+        assert np.array_equal(np.asarray(a), np.asarray(b))
+    # a chain that is not zero-preserving in the side: a + side0 keeps a where the side is empty
+    t = oracle.cell([("add", "t0", "a", "side0")], "t0", X, [("cell", Y)], agg="none")
+    rid = oracle.csr_row_ids(m, rp)
+    assert t.tolist() == (xv + Yd[rid, ci]).tolist()
+    # an empty side
+    E = dict(rows=m, cols=n, rowptr=np.zeros(m + 1, dtype=np.int32), colidx=np.zeros(0, dtype=np.int32),
+             vals=np.zeros(0))
+    assert oracle.cell(chain, "t1", X, [("cell", E), ("cell", Z)], agg="full") == 0.0
+    # a dense main input takes the sparse side as a dense array
+    d = oracle.cell(chain, "t1", Xd, [("cell", Y), ("cell", Z)], agg="full")
+    assert abs(d - float(want)) <= 1e-15 * float(np.sum(np.abs(Xd * Yd * Z)))
+
+
 def test_magg_matches_single_aggregates_and_inequalities():
     w = datagen.magg_workload(200, 30, seed=1)
     X, Y, Z = w["X"], w["Y"], w["Z"]
