@@ -313,7 +313,7 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v,
  * Table 1, Row template, variants no_agg_B1 / col_agg_B1; Eq. 2 and the row-wise
  * operator listing of Section 2.2 (RowType COL_AGG_B1_T); Section 5.2 "Row
  * Operations" (t(X) %*% (X %*% V)) and "Hybrid Algorithms" (k = 2 .. 32).
- * One pass over the rows of a dense X (rows x n).  B is a dense n x k side
+ * One pass over the rows of X (rows x n).  B is a dense n x k side
  * matrix, 1 <= k <= FO_B1_MAX_K.  For row i:
  *     D_ic = X_i . B[:, c]                       c = 0 .. k-1  (the listing's vectMatMult)
  *     s_i  = sum_c pre(d = D_ic, sides, scalars)               (vectSum; pre may be NULL)
@@ -328,11 +328,15 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v,
  * With pre = NULL and an empty post chain whose result is FO_DOT this is
  * t(X) %*% (X %*% B); with one FO_AT_CELL side P, pre = P * d and
  * post = P * d - P * s it is Eq. 2.
- * Limits (FO_ERR_UNSUPPORTED beyond them): dense X only; k <= 32; the columns
+ * X may be CSR: the same operator over the stored cells (a row without stored
+ * cells has D_i = 0 and still passes through the chains).  Limits
+ * (FO_ERR_UNSUPPORTED beyond them): CSR X: n * k' <= 9600 with k' = k rounded up
+ * to a power of two (>= 2); dense X: k <= 32; the columns
  * a group of warps can hold shrink as k grows (n <= 4096 for k <= 2, 2048 for
  * k <= 4, 1024 for k <= 8, 512 for k <= 16, 256 for k <= 32); for col_agg_B1_T
  * n * k <= 24576 (the CTA's output tile lives in shared memory).
- * Bit-reproducible for given shapes.
+ * Bit-reproducible for given shapes over a dense X; over a CSR X the additions
+ * into the shared output tile of col_agg_B1_T are unordered.
  */
 #define FO_B1_MAX_K 32
 #define FO_ROWSUM(n_sides)  FO_SIDE(n_sides)

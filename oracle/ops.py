@@ -301,7 +301,8 @@ def row(chain, output, X, v, sides=(), scalars=(), agg="col_t"):
 def row_b1(pre, pre_out, post, post_out, X, B, sides=(), scalars=(), agg="col_t"):
     """Row template with a matrix-valued row intermediate (Table 1: the *_B1
     variants; the row-wise listing of Section 2.2 for Eq. 2; "Row Operations" in
-    Section 5.2 for t(X) %*% (X %*% V)).  X is dense m x n, B dense n x k.
+    Section 5.2 for t(X) %*% (X %*% V)).  X is m x n, dense or CSR (the listing's
+    genexecSparse binding: the same operators over the stored cells); B dense n x k.
 
     D  = X B                     first scan of X: m x k (the listing's vectMatMult)
     P  = pre(d = D, sides)       m x k, and  s = rowSums(P)  (vectSum); skipped
@@ -312,12 +313,17 @@ def row_b1(pre, pre_out, post, post_out, X, B, sides=(), scalars=(), agg="col_t"
     Sides: ("cell", m x k) read at (row, class), ("row", m) read at the row,
     ("col", k) read at the class.
     """
-    X = np.asarray(X, dtype=np.float64)
     B = np.asarray(B, dtype=np.float64)
-    m, n = X.shape
-    assert B.shape[0] == n
     k = B.shape[1]
-    D = X @ B
+    if _is_csr(X):                 # CSR rows: one sparse matrix-vector product per class
+        m, n = X["rows"], X["cols"]
+        assert B.shape[0] == n
+        D = np.stack([_matvec(X, np.ascontiguousarray(B[:, c])) for c in range(k)], axis=1)
+    else:
+        X = np.asarray(X, dtype=np.float64)
+        m, n = X.shape
+        assert B.shape[0] == n
+        D = X @ B
     env = {"d": D}
     for j, (access, arr) in enumerate(sides):
         arr = np.asarray(arr, dtype=np.float64)
@@ -339,6 +345,8 @@ def row_b1(pre, pre_out, post, post_out, X, B, sides=(), scalars=(), agg="col_t"
         env["rowsum"] = row_sums(P).reshape(m, 1)
     (T,) = eval_chain(post, [post_out], env, (m, k))
     if agg == "col_t":
+        if _is_csr(X):
+            return np.stack([_tmatvec(X, np.ascontiguousarray(T[:, c])) for c in range(k)], axis=1)
         return X.T @ T
     if agg == "none":
         return T

@@ -514,7 +514,7 @@ def fused_row_b1(pre, pre_out, post, post_out, X, B, sides=(), scalars=(), agg="
         pre_ch, keep1 = make_chain(pre, pre_out)
         pre_ref = C.byref(pre_ch)
     m = _mat(X)
-    rows, cols = X.shape
+    rows, cols = (X.rows, X.cols) if isinstance(X, CSR) else X.shape
     dev = X.device
     a = ROW_B1_AGG[agg]
     assert B.dtype == torch.float64 and B.dim() == 2

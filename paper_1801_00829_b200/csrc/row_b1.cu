@@ -16,6 +16,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <type_traits>
+
 #include "chain.cuh"
 #include "ptx.cuh"
 
@@ -615,6 +617,153 @@ row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ 
     }
 }
 
+// ------------------------------------------------------------------- CSR
+// The same operator over the stored cells of a CSR X (the listing's
+// genexecSparse).  A warp takes blocks of 32 consecutive rows and stages their
+// cells - one contiguous piece of colidx / vals - in its slice of shared memory;
+// then one row after the other: the 32 lanes are (cell slot, class) pairs,
+// 32 / KP slots x KP classes, every lane adds val * B[col][class] over its slot's
+// cells, slots are combined by shuffles, the chains run once per class, and for
+// col_agg_B1_T every (cell, class) adds val * T_class into the CTA's n x KP
+// output tile in shared memory (atomics: several warps share the tile).
+constexpr int kB1CsrThreads = 256;
+constexpr int kB1CsrWarps = kB1CsrThreads / 32;
+constexpr int kB1CsrStage = 512;           // stored cells a warp can stage per block of rows
+
+struct B1CsrParams {
+    const int *rowptr;
+    const int *colidx;
+    const double *vals;
+    long long rows, cols;
+    const double *B;
+    long long ldb;
+    int k;
+    DevSides sides;
+    WsHead *head;
+    double *partials;
+    double *out;
+    int chain_kind, has_pre;
+    unsigned side_used;
+};
+
+template <int KP, int AGG, bool GENERIC>
+__global__ void __launch_bounds__(kB1CsrThreads)
+row_b1_csr_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ DevChain post,
+                  const __grid_constant__ B1CsrParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ unsigned int s_flag;
+    constexpr int CS = 32 / KP;                       // cell slots of a warp
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = lane % KP, slot = lane / KP;
+    const int n = (int)p.cols, k = p.k;
+
+    double *Bs = reinterpret_cast<double *>(smem_raw);                   // n x KP
+    double *Hs = Bs + (size_t)n * KP;                                    // n x KP (col_agg_B1_T)
+    double *sx = Bs + (size_t)(AGG == kB1ColT ? 2 : 1) * n * KP + (size_t)warp * kB1CsrStage;
+    int *sc = reinterpret_cast<int *>(Bs + (size_t)(AGG == kB1ColT ? 2 : 1) * n * KP + (size_t)kB1CsrWarps * kB1CsrStage)
+              + (size_t)warp * kB1CsrStage;
+    for (int e = threadIdx.x; e < n * KP; e += kB1CsrThreads) {
+        const int j = e / KP, cc = e - j * KP;
+        Bs[e] = cc < k ? __ldg(p.B + (long long)j * p.ldb + cc) : 0.0;
+        if (AGG == kB1ColT) Hs[e] = 0.0;
+    }
+    __syncthreads();
+
+    const long long nblocks = (p.rows + 31) >> 5;
+    const long long warp0 = (long long)blockIdx.x * kB1CsrWarps + warp;
+    const long long nwarps = (long long)gridDim.x * kB1CsrWarps;
+    for (long long blk = warp0; blk < nblocks; blk += nwarps) {
+        const long long myrow = (blk << 5) + lane;
+        const bool have = myrow < p.rows;
+        const int beg_l = have ? __ldg(p.rowptr + myrow) : 0;
+        const int end_l = have ? __ldg(p.rowptr + myrow + 1) : beg_l;
+        const int nrows = (int)((p.rows - (blk << 5) < 32) ? p.rows - (blk << 5) : 32);
+        const int base = __shfl_sync(0xffffffffu, beg_l, 0);
+        const int total = __shfl_sync(0xffffffffu, end_l, nrows - 1) - base;
+        const bool staged = total <= kB1CsrStage;
+        if (staged) {
+            for (int e = lane; e < total; e += 32) {
+                sc[e] = __ldg(p.colidx + base + e);
+                sx[e] = __ldg(p.vals + base + e);
+            }
+        }
+        __syncwarp();
+
+        for (int rr = 0; rr < nrows; ++rr) {
+            const long long row = (blk << 5) + rr;
+            const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
+            const int end = __shfl_sync(0xffffffffu, end_l, rr);
+            const bool ok = c < k;
+            // side values of (row, class)
+            double sv[FO_MAX_SIDES];
+#pragma unroll
+            for (int j = 0; j < FO_MAX_SIDES; ++j) {
+                sv[j] = 0.0;
+                if (ok && ((p.side_used >> j) & 1u)) {
+                    const DevSide &sd = p.sides.s[j];
+                    const long long off = sd.access == FO_AT_CELL ? row * sd.ld + c
+                                          : sd.access == FO_AT_ROW ? row * sd.ld : (long long)c;
+                    sv[j] = __ldg(sd.data + off);
+                }
+            }
+            // D_c = sum over the row's cells of val * B[col][c]
+            double d = 0.0;
+            for (int q = beg + slot; q < end; q += CS) {
+                const double val = staged ? sx[q - base] : __ldg(p.vals + q);
+                const int col = staged ? sc[q - base] : __ldg(p.colidx + q);
+                d = fma(val, Bs[(size_t)col * KP + c], d);
+            }
+#pragma unroll
+            for (int o = KP; o < 32; o <<= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+
+            double t;
+            if (p.chain_kind == kB1Identity) {
+                t = d;
+            } else {
+                double rowsum = 0.0;
+                if (p.has_pre) {
+                    double pv;
+                    if (!GENERIC || p.chain_kind == kB1Mlogreg) pv = sv[0] * d;
+                    else pv = b1_lane_chain(pre, d, sv[0], sv[1], sv[2], sv[3]);
+                    rowsum = ok ? pv : 0.0;
+#pragma unroll
+                    for (int o = 1; o < KP; o <<= 1) rowsum += __shfl_xor_sync(0xffffffffu, rowsum, o);
+                }
+                if (!GENERIC || p.chain_kind == kB1Mlogreg) {
+                    t = sv[0] * d - sv[0] * rowsum;
+                } else {
+                    double s2[FO_MAX_SIDES];
+#pragma unroll
+                    for (int j = 0; j < FO_MAX_SIDES; ++j) s2[j] = (p.has_pre && j == p.sides.n) ? rowsum : sv[j];
+                    t = b1_lane_chain(post, d, s2[0], s2[1], s2[2], s2[3]);
+                }
+            }
+            if (AGG == kB1None) {
+                if (ok && slot == 0) p.out[row * k + c] = t;
+            } else if (ok) {
+                for (int q = beg + slot; q < end; q += CS) {
+                    const double val = staged ? sx[q - base] : __ldg(p.vals + q);
+                    const int col = staged ? sc[q - base] : __ldg(p.colidx + q);
+                    atomicAdd(&Hs[(size_t)col * KP + c], val * t);
+                }
+            }
+        }
+        __syncwarp();          // the slice is reused by the next block
+    }
+
+    if (AGG == kB1ColT) {
+        __syncthreads();
+        const long long width = (long long)n * k;
+        for (long long e = threadIdx.x; e < width; e += kB1CsrThreads) {
+            const long long j = e / k, cc = e - j * k;
+            p.partials[(size_t)blockIdx.x * width + e] = Hs[j * KP + cc];
+        }
+        reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * width, width, p.out,
+                                 &s_flag);
+    }
+}
+
 __global__ void b1_fill_zero_kernel(double *out, long long n)
 {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -625,6 +774,7 @@ __global__ void b1_fill_zero_kernel(double *out, long long n)
 // ------------------------------------------------------------------- host
 constexpr size_t kB1SmemBudget = 200 * 1024;       // dynamic shared memory of one CTA
 constexpr long long kB1MaxOutTile = 24576;         // n * k doubles of a CTA's output tile (192 KB)
+constexpr long long kB1CsrMaxTile = 9600;          // CSR X: n * (padded k); B and the output tile share 150 KB
 
 int b1_grid_cap() { return 148 * 2; }              // bound used for workspace sizing
 
@@ -789,10 +939,11 @@ extern "C" {
 
 size_t fused_row_b1_workspace_bytes(const fo_mat *X, int k, int agg)
 {
-    if (!X || X->kind != FO_DENSE || k < 1 || k > FO_B1_MAX_K) return 0;
+    if (!X || (X->kind != FO_DENSE && X->kind != FO_CSR) || k < 1 || k > FO_B1_MAX_K) return 0;
     if (agg != FO_ROW_COL_AGG_B1_T && agg != FO_ROW_NO_AGG_B1) return 0;
-    if (X->dense.cols < 0) return 0;
-    return fo::b1_ws_bytes(X->dense.cols, k, agg);
+    const long long cols = X->kind == FO_CSR ? X->csr.cols : X->dense.cols;
+    if (cols < 0) return 0;
+    return fo::b1_ws_bytes(cols, k, agg);
 }
 
 int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, const fo_dense *B,
@@ -803,11 +954,18 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
     if (!post || !X || !B) return FO_ERR_NULL;
     if (n_sides > 0 && !sides) return FO_ERR_NULL;
     if (agg != FO_ROW_COL_AGG_B1_T && agg != FO_ROW_NO_AGG_B1) return FO_ERR_UNSUPPORTED;
-    if (X->kind == FO_CSR) return FO_ERR_UNSUPPORTED;
-    if (X->kind != FO_DENSE) return FO_ERR_SHAPE;
-    const long long rows = X->dense.rows, cols = X->dense.cols;
-    if (rows < 0 || cols < 0 || X->dense.ld < cols) return FO_ERR_SHAPE;
-    if (rows > 0 && cols > 0 && !X->dense.data) return FO_ERR_NULL;
+    if (X->kind != FO_DENSE && X->kind != FO_CSR) return FO_ERR_SHAPE;
+    const bool csr = X->kind == FO_CSR;
+    const long long rows = csr ? X->csr.rows : X->dense.rows, cols = csr ? X->csr.cols : X->dense.cols;
+    if (rows < 0 || cols < 0) return FO_ERR_SHAPE;
+    if (csr) {
+        if (X->csr.nnz < 0 || X->csr.nnz >= (1ll << 31)) return FO_ERR_UNSUPPORTED;
+        if (!X->csr.rowptr) return FO_ERR_NULL;
+        if (X->csr.nnz > 0 && (!X->csr.colidx || !X->csr.vals)) return FO_ERR_NULL;
+    } else {
+        if (X->dense.ld < cols) return FO_ERR_SHAPE;
+        if (rows > 0 && cols > 0 && !X->dense.data) return FO_ERR_NULL;
+    }
     if (B->rows != cols || B->cols < 1 || B->ld < B->cols) return FO_ERR_SHAPE;
     if (B->cols > FO_B1_MAX_K) return FO_ERR_UNSUPPORTED;
     if (cols > 0 && !B->data) return FO_ERR_NULL;
@@ -829,7 +987,8 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
 
     B1Params p;
     memset(&p, 0, sizeof(p));
-    p.rows = rows; p.cols = cols; p.X = X->dense.data; p.ldx = X->dense.ld;
+    p.rows = rows; p.cols = cols;
+    if (!csr) { p.X = X->dense.data; p.ldx = X->dense.ld; }
     p.B = B->data; p.ldb = B->ld; p.k = k;
     p.has_pre = pre ? 1 : 0;
     p.sides.n = n_sides;
@@ -853,8 +1012,10 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
     p.side_used = (chpre.side_used | chpost.side_used) & ((1u << n_sides) - 1u);
 
     if (agg == FO_ROW_COL_AGG_B1_T && cols * k > kB1MaxOutTile) return FO_ERR_UNSUPPORTED;
-    B1Shape sh;
-    if (!b1_shape(cols, k, &sh)) return FO_ERR_UNSUPPORTED;
+    B1Shape sh = {0, 0, 0, 0, 0};
+    if (!csr && !b1_shape(cols, k, &sh)) return FO_ERR_UNSUPPORTED;
+    const int kp_csr = pow2_at_least(k < 2 ? 2 : k);
+    if (csr && cols * kp_csr > kB1CsrMaxTile) return FO_ERR_UNSUPPORTED;
 
     // chains evaluated inline: the identity (t(X) (X B)) and the inner loop of Eq. 2
     p.chain_kind = kB1Generic;
@@ -888,6 +1049,41 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
 
     const int sms = sm_count();
     if (sms <= 0) return cuda_fail(cudaErrorNoDevice);
+    if (csr) {
+        B1CsrParams q;
+        memset(&q, 0, sizeof(q));
+        q.rowptr = X->csr.rowptr; q.colidx = X->csr.colidx; q.vals = X->csr.vals;
+        q.rows = rows; q.cols = cols; q.B = B->data; q.ldb = B->ld; q.k = k;
+        q.sides = p.sides; q.head = p.head; q.partials = p.partials; q.out = out;
+        q.chain_kind = p.chain_kind; q.has_pre = p.has_pre; q.side_used = p.side_used;
+        const size_t smem = (size_t)cols * kp_csr * 8 * (agg == FO_ROW_COL_AGG_B1_T ? 2 : 1)
+                            + (size_t)kB1CsrWarps * kB1CsrStage * 12;
+        long long grid = (rows + kB1CsrThreads - 1) / kB1CsrThreads;
+        const long long cap = (long long)sms * (smem <= 100 * 1024 ? 2 : 1);
+        if (grid > cap) grid = cap;
+        if (grid > b1_grid_cap()) grid = b1_grid_cap();
+        if (grid < 1) grid = 1;
+        auto go = [&](auto kern) -> cudaError_t {
+            cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e2 != cudaSuccess) return e2;
+            kern<<<(unsigned)grid, kB1CsrThreads, smem, st>>>(chpre, chpost, q);
+            return cudaGetLastError();
+        };
+        const bool generic = p.chain_kind == kB1Generic;
+        auto by_kp = [&](auto kpc) -> cudaError_t {
+            constexpr int KP = decltype(kpc)::value;
+            if (agg == FO_ROW_COL_AGG_B1_T)
+                return generic ? go(row_b1_csr_kernel<KP, kB1ColT, true>) : go(row_b1_csr_kernel<KP, kB1ColT, false>);
+            return generic ? go(row_b1_csr_kernel<KP, kB1None, true>) : go(row_b1_csr_kernel<KP, kB1None, false>);
+        };
+        cudaError_t e2;
+        if (kp_csr == 2) e2 = by_kp(std::integral_constant<int, 2>());
+        else if (kp_csr == 4) e2 = by_kp(std::integral_constant<int, 4>());
+        else if (kp_csr == 8) e2 = by_kp(std::integral_constant<int, 8>());
+        else if (kp_csr == 16) e2 = by_kp(std::integral_constant<int, 16>());
+        else e2 = by_kp(std::integral_constant<int, 32>());
+        return e2 == cudaSuccess ? FO_OK : cuda_fail(e2);
+    }
     const bool staged = b1_aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
     // tensor-core variant where its layout fits (FUSEDOPS_B1_MMA=0 / 1 forces the choice)
     {

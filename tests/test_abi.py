@@ -221,7 +221,11 @@ def test_row_b1_argument_errors(lib):
     assert call(m, dense(100, 2), sides=one, ns=1, prec=None, postc=post) == -3  # row sum without a first chain
     x = B.fo_mat()
     x.kind = 1
-    assert call(x, dense(100, 2)) == -4                     # CSR main input not provided
+    x.csr.rows, x.csr.cols, x.csr.nnz = 10, 100, 1 << 31
+    x.csr.rowptr, x.csr.colidx, x.csr.vals = 0x5000, 0x6000, 0x7000
+    assert call(x, dense(100, 2)) == -4                     # CSR main input: nnz must fit 31 bits
+    x.csr.nnz, x.csr.cols = 50, 2000
+    assert call(x, dense(2000, 8)) == -4                    # CSR main input: n * k beyond the shared tiles
     # workspace: one n x k tile per CTA and per group of CTAs for col_agg_B1_T, the head alone otherwise
     assert lib.fused_row_b1_workspace_bytes(C.byref(m), 2, 5) == 16384
     assert lib.fused_row_b1_workspace_bytes(C.byref(m), 2, 6) > 16384 + 148 * 100 * 2 * 8

