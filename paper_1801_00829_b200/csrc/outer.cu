@@ -387,6 +387,129 @@ outer_staged_kernel(const __grid_constant__ DevChain ch, const __grid_constant__
     }
 }
 
+// ---------------------------------------------------------------- pipelined
+// full_agg / no_agg: the same staging, software-pipelined inside the warp.  The
+// warp's buffer is two halves of eight rows; a step lands the V rows of eight
+// stored cells (two per 8-lane group) in one half while the other half is being
+// reduced, and the reduction keeps four independent multiply-add chains per lane
+// (two cells, two accumulators each) instead of one.  Copy groups are committed
+// every step (an empty group at the tail) so that "all but the newest" always
+// names the step about to be used.
+template <int NK2, int AGG>
+__global__ void __launch_bounds__(kThreads, 2)
+outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ double s_red[32];
+    __shared__ unsigned int s_flag;
+    __shared__ long long s_rows[2];
+
+    if (threadIdx.x == 0) {
+        const long long G = gridDim.x, b = blockIdx.x;
+        s_rows[0] = (b == 0) ? 0 : lower_row(p.rowptr, p.rows, (p.nnz * b) / G);
+        s_rows[1] = (b == G - 1) ? p.rows : lower_row(p.rowptr, p.rows, (p.nnz * (b + 1)) / G);
+    }
+    __syncthreads();
+    const long long row_lo = s_rows[0], row_hi = s_rows[1];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int l8 = lane & 7, grp = lane >> 3;
+    const unsigned full = 0xffffffffu;
+    const int rank = p.rank;                       // even
+    double *buf = reinterpret_cast<double *>(smem_raw) + (size_t)warp * kStageRows * rank;
+    double acc = 0.0;
+
+    for (long long row = row_lo + warp; row < row_hi; row += kThreads / 32) {
+        const int beg = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
+        double2 u[NK2];
+        const double *urow = p.U + row * p.ldu;
+#pragma unroll
+        for (int c = 0; c < NK2; ++c) {
+            const int col = 16 * c + 2 * l8;
+            u[c] = (beg < end && col < rank) ? __ldg(reinterpret_cast<const double2 *>(urow + col))
+                                             : make_double2(0.0, 0.0);
+        }
+        for (int c0 = beg; c0 < end; c0 += 32) {
+            const int cnt = (end - c0 < 32) ? end - c0 : 32;
+            const bool valid = lane < cnt;
+            const int jmine = valid ? __ldg(p.colidx + c0 + lane) : 0;
+            const double amine = valid ? __ldg(p.vals + c0 + lane) : 0.0;
+            const int nsteps = (cnt + 7) >> 3;
+            double dmine = 0.0;
+
+            // step s: group grp lands the V rows of cells 8 s + grp and 8 s + 4 + grp in
+            // half (s & 1) of the buffer
+            auto issue = [&](int s) {
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int sidx = 8 * s + 4 * i + grp;
+                    const int j = __shfl_sync(full, jmine, sidx & 31);
+                    if (s < nsteps && sidx < cnt) {
+                        const double *vj = p.V + (long long)j * p.ldv;
+                        double *dst = buf + (8 * (s & 1) + 4 * i + grp) * rank;
+#pragma unroll
+                        for (int c = 0; c < NK2; ++c) {
+                            const int col = 16 * c + 2 * l8;
+                            if (col < rank) cp_async16(dst + col, vj + col);
+                        }
+                    }
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            };
+            issue(0);
+            for (int s = 0; s < nsteps; ++s) {
+                issue(s + 1);
+                asm volatile("cp.async.wait_group 1;" ::: "memory");
+                __syncwarp();
+                // two cells per group, two accumulators per cell: four independent chains
+                double dx[2] = {0.0, 0.0}, dy[2] = {0.0, 0.0};
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int sidx = 8 * s + 4 * i + grp;
+                    const double *src = buf + (8 * (s & 1) + 4 * i + grp) * rank;
+                    if (sidx < cnt) {
+#pragma unroll
+                        for (int c = 0; c < NK2; ++c) {
+                            const int col = 16 * c + 2 * l8;
+                            if (col < rank) {
+                                const double2 x = *reinterpret_cast<const double2 *>(src + col);
+                                dx[i] = fma(u[c].x, x.x, dx[i]);
+                                dy[i] = fma(u[c].y, x.y, dy[i]);
+                            }
+                        }
+                    }
+                }
+                const double d0 = dx[0] + dy[0], d1 = dx[1] + dy[1];
+                // two values over the 8 lanes of a group in three exchanges: the upper
+                // four lanes end up with the second cell's total, the lower four with the first's
+                const bool up = (lane & 4) != 0;
+                double v = (up ? d1 : d0) + __shfl_xor_sync(full, up ? d0 : d1, 4);
+                v += __shfl_xor_sync(full, v, 2);
+                v += __shfl_xor_sync(full, v, 1);
+                // cell c of the chunk was handled by group (c & 3) in trip (c >> 2)
+                const double all = __shfl_sync(full, v, (lane & 3) * 8 + ((lane >> 2) & 1) * 4);
+                if ((lane >> 3) == s) dmine = all;
+                __syncwarp();          // half (s & 1) is refilled by the issue after next
+            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
+            if (AGG == kOutFull) {
+                if (valid) acc += w;
+            } else {
+                if (valid) p.out[c0 + lane] = w;
+            }
+        }
+    }
+
+    if (AGG == kOutFull) {
+        double v1[1] = {acc};
+        block_sum<1>(v1, s_red);
+        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
+    }
+}
+
 __global__ void outer_fill_zero_kernel(double *out, long long n)
 {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -424,8 +547,11 @@ cudaError_t launch_outer_staged(const DevChain &ch, const OuterParams &p, int ag
         kern<<<grid, kThreads, smem, st>>>(ch, p);
         return cudaGetLastError();
     };
-    if (agg == FO_OUTER_FULL_AGG) return go(outer_staged_kernel<NK2, kOutFull>);
-    if (agg == FO_OUTER_NO_AGG) return go(outer_staged_kernel<NK2, kOutNone>);
+    // FUSEDOPS_OUTER_PIPE=0 keeps the batch-at-a-time kernel for full_agg / no_agg (a measuring knob)
+    const char *e = getenv("FUSEDOPS_OUTER_PIPE");
+    const bool pipe = !(e && e[0] == '0');
+    if (agg == FO_OUTER_FULL_AGG) return pipe ? go(outer_pipe_kernel<NK2, kOutFull>) : go(outer_staged_kernel<NK2, kOutFull>);
+    if (agg == FO_OUTER_NO_AGG) return pipe ? go(outer_pipe_kernel<NK2, kOutNone>) : go(outer_staged_kernel<NK2, kOutNone>);
     return go(outer_staged_kernel<NK2, kOutRight>);
 }
 
