@@ -395,6 +395,7 @@ outer_staged_kernel(const __grid_constant__ DevChain ch, const __grid_constant__
 // (two cells, two accumulators each) instead of one.  Copy groups are committed
 // every step (an empty group at the tail) so that "all but the newest" always
 // names the step about to be used.
+// NK2 = ceil(rank / 16) exactly: only the last 16-column piece of a row needs a bounds check.
 template <int NK2, int AGG>
 __global__ void __launch_bounds__(kThreads, 2)
 outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
@@ -417,6 +418,7 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
     const unsigned full = 0xffffffffu;
     const int rank = p.rank;                       // even
     double *buf = reinterpret_cast<double *>(smem_raw) + (size_t)warp * kStageRows * rank;
+    double *mybuf = buf + grp * rank + 2 * l8;     // this lane's piece of its group's first row
     double acc = 0.0;
 
     for (long long row = row_lo + warp; row < row_hi; row += kThreads / 32) {
@@ -438,20 +440,19 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
             double dmine = 0.0;
 
             // step s: group grp lands the V rows of cells 8 s + grp and 8 s + 4 + grp in
-            // half (s & 1) of the buffer
+            // half (s & 1) of the buffer.  Past the end of a ragged chunk the chunk's last
+            // cell is fetched again: no branch, and its result is never used.
             auto issue = [&](int s) {
+                if (s < nsteps) {                     // uniform
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const int sidx = 8 * s + 4 * i + grp;
-                    const int j = __shfl_sync(full, jmine, sidx & 31);
-                    if (s < nsteps && sidx < cnt) {
-                        const double *vj = p.V + (long long)j * p.ldv;
-                        double *dst = buf + (8 * (s & 1) + 4 * i + grp) * rank;
+                    for (int i = 0; i < 2; ++i) {
+                        const int sidx = 8 * s + 4 * i + grp;
+                        const int j = __shfl_sync(full, jmine, sidx < cnt ? sidx : cnt - 1);
+                        const double *vj = p.V + (long long)j * p.ldv + 2 * l8;
+                        double *dst = mybuf + ((s & 1) * 8 + 4 * i) * rank;
 #pragma unroll
-                        for (int c = 0; c < NK2; ++c) {
-                            const int col = 16 * c + 2 * l8;
-                            if (col < rank) cp_async16(dst + col, vj + col);
-                        }
+                        for (int c = 0; c < NK2; ++c)
+                            if (c < NK2 - 1 || 16 * c + 2 * l8 < rank) cp_async16(dst + 16 * c, vj + 16 * c);
                     }
                 }
                 asm volatile("cp.async.commit_group;" ::: "memory");
@@ -465,17 +466,13 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
                 double dx[2] = {0.0, 0.0}, dy[2] = {0.0, 0.0};
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
-                    const int sidx = 8 * s + 4 * i + grp;
-                    const double *src = buf + (8 * (s & 1) + 4 * i + grp) * rank;
-                    if (sidx < cnt) {
+                    const double *src = mybuf + ((s & 1) * 8 + 4 * i) * rank;
 #pragma unroll
-                        for (int c = 0; c < NK2; ++c) {
-                            const int col = 16 * c + 2 * l8;
-                            if (col < rank) {
-                                const double2 x = *reinterpret_cast<const double2 *>(src + col);
-                                dx[i] = fma(u[c].x, x.x, dx[i]);
-                                dy[i] = fma(u[c].y, x.y, dy[i]);
-                            }
+                    for (int c = 0; c < NK2; ++c) {
+                        if (c < NK2 - 1 || 16 * c + 2 * l8 < rank) {
+                            const double2 x = *reinterpret_cast<const double2 *>(src + 16 * c);
+                            dx[i] = fma(u[c].x, x.x, dx[i]);
+                            dy[i] = fma(u[c].y, x.y, dy[i]);
                         }
                     }
                 }
@@ -547,12 +544,23 @@ cudaError_t launch_outer_staged(const DevChain &ch, const OuterParams &p, int ag
         kern<<<grid, kThreads, smem, st>>>(ch, p);
         return cudaGetLastError();
     };
-    // FUSEDOPS_OUTER_PIPE=0 keeps the batch-at-a-time kernel for full_agg / no_agg (a measuring knob)
-    const char *e = getenv("FUSEDOPS_OUTER_PIPE");
-    const bool pipe = !(e && e[0] == '0');
-    if (agg == FO_OUTER_FULL_AGG) return pipe ? go(outer_pipe_kernel<NK2, kOutFull>) : go(outer_staged_kernel<NK2, kOutFull>);
-    if (agg == FO_OUTER_NO_AGG) return pipe ? go(outer_pipe_kernel<NK2, kOutNone>) : go(outer_staged_kernel<NK2, kOutNone>);
+    if (agg == FO_OUTER_FULL_AGG) return go(outer_staged_kernel<NK2, kOutFull>);
+    if (agg == FO_OUTER_NO_AGG) return go(outer_staged_kernel<NK2, kOutNone>);
     return go(outer_staged_kernel<NK2, kOutRight>);
+}
+
+// full_agg / no_agg through the pipelined kernel; NK2 is exactly ceil(rank / 16).
+template <int NK2>
+cudaError_t launch_outer_pipe(const DevChain &ch, const OuterParams &p, int agg, int grid, cudaStream_t st)
+{
+    const size_t smem = (size_t)(kThreads / 32) * kStageRows * p.rank * sizeof(double);
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, kThreads, smem, st>>>(ch, p);
+        return cudaGetLastError();
+    };
+    return agg == FO_OUTER_FULL_AGG ? go(outer_pipe_kernel<NK2, kOutFull>) : go(outer_pipe_kernel<NK2, kOutNone>);
 }
 
 // Recognises the chains that outer_chain() evaluates inline by the text of the
@@ -659,6 +667,21 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     const bool staged = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && agg != FO_OUTER_LEFT_MM &&
                         !getenv("FUSEDOPS_OUTER_DIRECT");
     if (staged) {
+        // FUSEDOPS_OUTER_PIPE=0 keeps the batch-at-a-time kernel for full_agg / no_agg (a measuring knob)
+        const char *pe = getenv("FUSEDOPS_OUTER_PIPE");
+        const bool pipe = !(pe && pe[0] == '0') && (agg == FO_OUTER_FULL_AGG || agg == FO_OUTER_NO_AGG);
+        if (pipe) {
+            switch (nk2) {
+                case 1: e = launch_outer_pipe<1>(ch, p, agg, (int)grid, st); break;
+                case 2: e = launch_outer_pipe<2>(ch, p, agg, (int)grid, st); break;
+                case 3: e = launch_outer_pipe<3>(ch, p, agg, (int)grid, st); break;
+                case 4: e = launch_outer_pipe<4>(ch, p, agg, (int)grid, st); break;
+                case 5: e = launch_outer_pipe<5>(ch, p, agg, (int)grid, st); break;
+                case 6: e = launch_outer_pipe<6>(ch, p, agg, (int)grid, st); break;
+                case 7: e = launch_outer_pipe<7>(ch, p, agg, (int)grid, st); break;
+                default: e = launch_outer_pipe<8>(ch, p, agg, (int)grid, st); break;
+            }
+        } else
         if (nk2 <= 1) e = launch_outer_staged<1>(ch, p, agg, (int)grid, st);
         else if (nk2 <= 2) e = launch_outer_staged<2>(ch, p, agg, (int)grid, st);
         else if (nk2 <= 4) e = launch_outer_staged<4>(ch, p, agg, (int)grid, st);
