@@ -253,6 +253,10 @@ def time_variants(fo, step, shapes, reps=10):
                                                 agg="none", out=o_nnz), outer_in + 8 * nnz5),
         ("outer_right_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
                                                   agg="right", out=o_right), outer_in + 8 * orow * rank),
+        # the sparsity-exploiting half of the ALS-CG update rule, Eq. 1: ((X != 0) * (U t(V))) V
+        ("outer_right_mm_als_cg", lambda: fo.fused_outer([("ne", "t0", "a", 0.0), ("mul", "t1", "t0", "d")], "t1",
+                                                         step.csr5, d["outer.U"], d["outer.V"], agg="right",
+                                                         out=o_right), outer_in + 8 * orow * rank),
         ("outer_x_log_uvt_plus_eps", lambda: fo.fused_outer(
             [("add", "t0", "d", "s0"), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")], "t2", step.csr5,
             d["outer.U"], d["outer.V"], [10.0], agg="full", out=o_one), outer_in + 8),

@@ -39,7 +39,7 @@ enum { kOutFull = 0, kOutNone = 1, kOutRight = 2, kOutLeft = 3 };
 // Chains evaluated inline, in the chain's own operation order (same bits as the
 // interpreter): the weighted squared loss of Eq. 1, (a != 0) * (a - d)^2, and the
 // sparse micro-benchmark expression of Section 5.2, a * log(d + eps).
-enum { kOuterGeneric = 0, kOuterWsloss = 1, kOuterXlogd = 2 };
+enum { kOuterGeneric = 0, kOuterWsloss = 1, kOuterXlogd = 2, kOuterMaskDot = 3 };
 
 template <bool ALIGNED>
 __device__ __forceinline__ double2 ld_pair_cached(const double *row, int col, int n)
@@ -61,6 +61,7 @@ __device__ __forceinline__ double outer_chain(const DevChain &ch, int kind, int 
         return t0 * t2;
     }
     if (kind == kOuterXlogd) return a * slow_log(d + ch.consts[kc]);
+    if (kind == kOuterMaskDot) return (a != 0.0 ? 1.0 : 0.0) * d;      // (X != 0) * (U V^T), Eq. 1
     RegFile<kRegs, 1> f;
     f.r[0][0] = a;
     f.r[1][0] = d;
@@ -431,6 +432,9 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
             u[c] = (beg < end && col < rank) ? __ldg(reinterpret_cast<const double2 *>(urow + col))
                                              : make_double2(0.0, 0.0);
         }
+        double2 racc[AGG == kOutRight ? NK2 : 1];      // right_mm: this group's share of O_i
+#pragma unroll
+        for (int c = 0; c < (AGG == kOutRight ? NK2 : 1); ++c) racc[c] = make_double2(0.0, 0.0);
         for (int c0 = beg; c0 < end; c0 += 32) {
             const int cnt = (end - c0 < 32) ? end - c0 : 32;
             const bool valid = lane < cnt;
@@ -483,17 +487,57 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
                 double v = (up ? d1 : d0) + __shfl_xor_sync(full, up ? d0 : d1, 4);
                 v += __shfl_xor_sync(full, v, 2);
                 v += __shfl_xor_sync(full, v, 1);
-                // cell c of the chunk was handled by group (c & 3) in trip (c >> 2)
-                const double all = __shfl_sync(full, v, (lane & 3) * 8 + ((lane >> 2) & 1) * 4);
-                if ((lane >> 3) == s) dmine = all;
+                if (AGG == kOutRight) {
+                    // the chain for the group's two cells (lower four lanes: the first, upper four:
+                    // the second), then O_i += w * V_j from the rows still in the buffer
+                    const int sidx = 8 * s + 4 * ((lane >> 2) & 1) + grp;
+                    const double a = __shfl_sync(full, amine, sidx & 31);
+                    double w = outer_chain(ch, p.chain_kind, p.kconst, a, v);
+                    if (sidx >= cnt) w = 0.0;         // a row fetched again at a ragged end adds nothing
+                    const double w0 = __shfl_sync(full, w, grp * 8), w1 = __shfl_sync(full, w, grp * 8 + 4);
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const double ww = i ? w1 : w0;
+                        const double *src = mybuf + ((s & 1) * 8 + 4 * i) * rank;
+#pragma unroll
+                        for (int c = 0; c < NK2; ++c) {
+                            if (c < NK2 - 1 || 16 * c + 2 * l8 < rank) {
+                                const double2 x = *reinterpret_cast<const double2 *>(src + 16 * c);
+                                racc[AGG == kOutRight ? c : 0].x = fma(ww, x.x, racc[AGG == kOutRight ? c : 0].x);
+                                racc[AGG == kOutRight ? c : 0].y = fma(ww, x.y, racc[AGG == kOutRight ? c : 0].y);
+                            }
+                        }
+                    }
+                } else {
+                    // cell c of the chunk was handled by group (c & 3) in trip (c >> 2)
+                    const double all = __shfl_sync(full, v, (lane & 3) * 8 + ((lane >> 2) & 1) * 4);
+                    if ((lane >> 3) == s) dmine = all;
+                }
                 __syncwarp();          // half (s & 1) is refilled by the issue after next
             }
             asm volatile("cp.async.wait_group 0;" ::: "memory");
-            const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
-            if (AGG == kOutFull) {
-                if (valid) acc += w;
-            } else {
-                if (valid) p.out[c0 + lane] = w;
+            if (AGG != kOutRight) {
+                const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
+                if (AGG == kOutFull) {
+                    if (valid) acc += w;
+                } else {
+                    if (valid) p.out[c0 + lane] = w;
+                }
+            }
+        }
+        if (AGG == kOutRight) {
+            // the four groups hold partial rows: add them in a fixed order
+#pragma unroll
+            for (int c = 0; c < (AGG == kOutRight ? NK2 : 1); ++c) {
+                racc[c].x += __shfl_xor_sync(full, racc[c].x, 8);
+                racc[c].y += __shfl_xor_sync(full, racc[c].y, 8);
+                racc[c].x += __shfl_xor_sync(full, racc[c].x, 16);
+                racc[c].y += __shfl_xor_sync(full, racc[c].y, 16);
+                const int col = 16 * c + 2 * l8;
+                if (grp == 0) {
+                    if (col < rank) p.out[row * rank + col] = racc[c].x;
+                    if (col + 1 < rank) p.out[row * rank + col + 1] = racc[c].y;
+                }
             }
         }
     }
@@ -549,7 +593,7 @@ cudaError_t launch_outer_staged(const DevChain &ch, const OuterParams &p, int ag
     return go(outer_staged_kernel<NK2, kOutRight>);
 }
 
-// full_agg / no_agg through the pipelined kernel; NK2 is exactly ceil(rank / 16).
+// full_agg / no_agg / right_mm through the pipelined kernel; NK2 is exactly ceil(rank / 16).
 template <int NK2>
 cudaError_t launch_outer_pipe(const DevChain &ch, const OuterParams &p, int agg, int grid, cudaStream_t st)
 {
@@ -560,7 +604,9 @@ cudaError_t launch_outer_pipe(const DevChain &ch, const OuterParams &p, int agg,
         kern<<<grid, kThreads, smem, st>>>(ch, p);
         return cudaGetLastError();
     };
-    return agg == FO_OUTER_FULL_AGG ? go(outer_pipe_kernel<NK2, kOutFull>) : go(outer_pipe_kernel<NK2, kOutNone>);
+    if (agg == FO_OUTER_FULL_AGG) return go(outer_pipe_kernel<NK2, kOutFull>);
+    if (agg == FO_OUTER_NO_AGG) return go(outer_pipe_kernel<NK2, kOutNone>);
+    return go(outer_pipe_kernel<NK2, kOutRight>);
 }
 
 // Recognises the chains that outer_chain() evaluates inline by the text of the
@@ -585,6 +631,8 @@ int outer_chain_kind(const DevChain &ch, int *kconst)
         *kconst = k;
         return kOuterXlogd;
     }
+    if ((match("mul(ne(r0,k%d),r1)%n", &k) || match("mul(r1,ne(r0,k%d))%n", &k)) && ch.consts[k] == 0.0)
+        return kOuterMaskDot;
     return kOuterGeneric;
 }
 
@@ -667,9 +715,9 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     const bool staged = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && agg != FO_OUTER_LEFT_MM &&
                         !getenv("FUSEDOPS_OUTER_DIRECT");
     if (staged) {
-        // FUSEDOPS_OUTER_PIPE=0 keeps the batch-at-a-time kernel for full_agg / no_agg (a measuring knob)
+        // FUSEDOPS_OUTER_PIPE=0 keeps the batch-at-a-time kernel (a measuring knob)
         const char *pe = getenv("FUSEDOPS_OUTER_PIPE");
-        const bool pipe = !(pe && pe[0] == '0') && (agg == FO_OUTER_FULL_AGG || agg == FO_OUTER_NO_AGG);
+        const bool pipe = !(pe && pe[0] == '0');
         if (pipe) {
             switch (nk2) {
                 case 1: e = launch_outer_pipe<1>(ch, p, agg, (int)grid, st); break;

@@ -421,6 +421,8 @@ def test_specialised_chains_equal_interpreter_bitwise(fo, name, chain, outs, nsi
                          ("mul", "t0", "t5", "t1")], "t0", []),
     ("xlogd", [("add", "t0", "d", "s0"), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")], "t2", [2.5]),
     ("xlogd-imm", [("add", "t0", 2.5, "d"), ("log", "t1", "t0"), ("mul", "t2", "t1", "a")], "t2", []),
+    ("maskdot", [("ne", "t0", "a", 0.0), ("mul", "t1", "t0", "d")], "t1", []),
+    ("maskdot-commuted", [("ne", "t3", "a", 0.0), ("mul", "t1", "d", "t3")], "t1", []),
     ("not-inline", [("sub", "t0", "a", "d"), ("abs", "t1", "t0")], "t1", []),
 ])
 @pytest.mark.parametrize("agg", ["full", "none", "right"])
