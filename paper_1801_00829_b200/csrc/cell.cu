@@ -125,8 +125,8 @@ cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
 
 // ------------------------------------------------------------------ cols
 // grid.x: tiles of 2 * cx columns; grid.y: row panels.  The 256 threads of a CTA
-// form cx column pairs by 256 / cx row lanes (cx = p.cx, a power of two <= 256,
-// chosen so that narrow matrices still fill the CTA); a thread owns a column pair
+// form cx column pairs by 256 / cx row lanes (cx = p.cx <= 256, chosen so that the
+// column tiles are equal and narrow matrices still fill the CTA); a thread owns a column pair
 // and walks every (256 / cx)-th row of its panel, two rows per chain evaluation;
 // the row lanes are then added in order through shared memory.
 template <class EVAL, bool ALIGNED>
@@ -135,15 +135,15 @@ cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
 {
     __shared__ unsigned int s_flag;
     __shared__ double2 s_lane[kThreads];
-    const int cx = p.cx, ry = kThreads / cx;
-    const int tx = threadIdx.x & (cx - 1), ty = threadIdx.x / cx;
+    const int cx = p.cx, ry = kThreads / cx;          // threads beyond cx * ry idle
+    const int tx = threadIdx.x % cx, ty = threadIdx.x / cx;
     const long long col = ((long long)blockIdx.x * cx + tx) * 2;
     const long long per = (p.rows + p.panels - 1) / p.panels;
     const long long r0 = (long long)blockIdx.y * per;
     const long long r1 = (r0 + per < p.rows) ? r0 + per : p.rows;
     double a0 = 0.0, a1 = 0.0;
 
-    if (col < p.cols) {
+    if (col < p.cols && ty < ry) {
         for (long long row = r0 + ty; row < r1; row += 2 * ry) {
             const bool two = row + ry < r1;
             double in[kIn][kV];
@@ -235,9 +235,14 @@ int stream_grid(long long units, int sms)
 // Column pairs a CTA covers: 256, or fewer for narrow matrices (a power of two).
 int col_cx(long long cols)
 {
-    int cx = 256;
-    while (cx > 8 && (long long)cx >= cols) cx >>= 1;      // smallest power of two with 2 * cx >= cols
-    return cx;
+    // column pairs per tile: all of them in one tile up to 512 columns, else as many
+    // equal tiles of at most 256 pairs as it takes - no ragged last tile, so that for,
+    // say, 100 columns 250 of the 256 threads have a column pair (50 pairs x 5 row lanes)
+    const long long half = (cols + 1) / 2;
+    const long long tiles = (half + 255) / 256;
+    long long cx = tiles > 0 ? (half + tiles - 1) / tiles : 1;
+    if (cx < 1) cx = 1;
+    return (int)cx;
 }
 
 int col_panels(long long rows, long long cols)
@@ -275,9 +280,24 @@ cudaError_t launch_cell(const DevChain &ch, const CellParams &p, int agg, bool f
 {
     if (agg == FO_CELL_COL_AGG) {
         if constexpr (NOUT == 1) {
-            const dim3 g((unsigned)((p.cols + 2 * p.cx - 1) / (2 * p.cx)), (unsigned)p.panels);
-            if (aligned) cell_cols_kernel<EVAL, true><<<g, kThreads, 0, st>>>(ch, p);
-            else cell_cols_kernel<EVAL, false><<<g, kThreads, 0, st>>>(ch, p);
+            // row panels: as many as fill every SM exactly once with the CTAs this kernel
+            // can keep resident (a second, partly filled wave would cost up to a wave's time);
+            // p.panels, which sized the workspace, is the upper bound
+            const long long tiles = (p.cols + 2 * p.cx - 1) / (2 * p.cx);
+            CellParams q = p;
+            int nb = 0;
+            const cudaError_t oe = aligned
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cell_cols_kernel<EVAL, true>, kThreads, 0)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, cell_cols_kernel<EVAL, false>, kThreads, 0);
+            const int sms = sm_count();
+            if (oe == cudaSuccess && nb > 0 && sms > 0) {
+                long long want = ((long long)sms * nb) / tiles;
+                if (want < 1) want = 1;
+                if (want < q.panels) q.panels = (int)want;
+            }
+            const dim3 g((unsigned)tiles, (unsigned)q.panels);
+            if (aligned) cell_cols_kernel<EVAL, true><<<g, kThreads, 0, st>>>(ch, q);
+            else cell_cols_kernel<EVAL, false><<<g, kThreads, 0, st>>>(ch, q);
         }
     } else if (flat) {
         if (agg == FO_CELL_NO_AGG) {
