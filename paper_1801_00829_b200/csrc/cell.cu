@@ -144,7 +144,25 @@ cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
     double a0 = 0.0, a1 = 0.0;
 
     if (col < p.cols && ty < ry) {
-        for (long long row = r0 + ty; row < r1; row += 2 * ry) {
+        long long row = r0 + ty;
+        // four rows per turn while they last: twice the loads in flight per thread
+        for (; row + 3 * ry < r1; row += 4 * ry) {
+            double in[kIn][kV], in2[kIn][kV];
+            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, col, row + ry, col, true, in);
+            load_inputs_2d<EVAL, ALIGNED>(ch, p, row + 2 * ry, col, row + 3 * ry, col, true, in2);
+            double o[1][kV], o2[1][kV];
+            EVAL::template run<kV, 1>(ch, in, o);
+            EVAL::template run<kV, 1>(ch, in2, o2);
+            a0 += o[0][0];
+            a1 += o[0][1];
+            a0 += o[0][2];
+            a1 += o[0][3];
+            a0 += o2[0][0];
+            a1 += o2[0][1];
+            a0 += o2[0][2];
+            a1 += o2[0][3];
+        }
+        for (; row < r1; row += 2 * ry) {
             const bool two = row + ry < r1;
             double in[kIn][kV];
             load_inputs_2d<EVAL, ALIGNED>(ch, p, row, col, row + ry, col, two, in);
