@@ -34,7 +34,7 @@ struct CsrCellParams {
     double *partials;
     double *out;
     int agg;                 // FO_CELL_*
-    int pad;
+    int rb;                  // rows a warp takes at a time: 32, fewer (a power of two >= 32 / G) for small inputs
     // sparse sides (access == kAtCellSparse): sides.s[k].data holds the values
     const int *side_rowptr[FO_MAX_SIDES];
     const int *side_colidx[FO_MAX_SIDES];
@@ -69,18 +69,20 @@ cell_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Csr
 #pragma unroll
     for (int k = 0; k < NOUT; ++k) acc[k] = 0.0;
 
-    const long long nblocks = (p.rows + 31) >> 5;
+    const int RB = p.rb;
+    const long long nblocks = (p.rows + RB - 1) / RB;
     const long long warp0 = (long long)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
     const long long nwarps = (long long)gridDim.x * (kThreads / 32);
+    const int nit = G * RB / 32;                     // >= 1: RB >= 32 / G
 
     for (long long blk = warp0; blk < nblocks; blk += nwarps) {
-        const long long myrow = (blk << 5) + lane;
+        const long long myrow = blk * RB + (lane < RB ? lane : RB);     // lanes past the block: an empty row
         const int beg_l = __ldg(p.rowptr + (myrow < p.rows ? myrow : p.rows));
-        const int end_l = __ldg(p.rowptr + (myrow + 1 < p.rows ? myrow + 1 : p.rows));
+        const int end_l = (lane < RB) ? __ldg(p.rowptr + (myrow + 1 < p.rows ? myrow + 1 : p.rows)) : beg_l;
 #pragma unroll 1
-        for (int it = 0; it < G; ++it) {
+        for (int it = 0; it < nit; ++it) {
             const int rr = it * (32 / G) + grp;
-            const long long row = (blk << 5) + rr;
+            const long long row = blk * RB + rr;
             const int beg = __shfl_sync(full, beg_l, rr);
             const int end = __shfl_sync(full, end_l, rr);
             const int trips = __reduce_max_sync(full, (end - beg + G - 1) / G);
@@ -248,11 +250,17 @@ int run_cell_csr(const fo_chain *chain, const fo_csr &X, const fo_side *sides, i
 
     const int sms = sm_count();
     if (sms <= 0) return cuda_fail(cudaErrorNoDevice);
-    const long long nblocks = (X.rows + 31) / 32;
+    const double mean_len = (double)X.nnz / (double)X.rows;
+    // rows a warp takes at a time: 32, or fewer when the matrix has too few rows to give every
+    // warp of the machine a block (never fewer than 32 / G, G = the lanes that share a row)
+    const int lanes_per_row = mean_len <= 12.0 ? 2 : mean_len <= 48.0 ? 8 : 32;
+    int rb = 32;
+    while (rb > 32 / lanes_per_row && (X.rows + rb - 1) / rb < (long long)sms * 16) rb >>= 1;
+    p.rb = rb;
+    const long long nblocks = (X.rows + rb - 1) / rb;
     long long grid = (nblocks + kThreads / 32 - 1) / (kThreads / 32);
     if (grid > (long long)sms * 8) grid = (long long)sms * 8;
     if (grid > kMaxPartials) grid = kMaxPartials;
-    const double mean_len = (double)X.nnz / (double)X.rows;
 
     switch (force_interpreter() ? kSpecNone : match_cell_spec(ch)) {
         case kSpecMul2: e = launch_by_group<EvalSpec<kSpecMul2>, 1>(ch, p, mean_len, (int)grid, st); break;
