@@ -36,6 +36,7 @@ struct RowParams {
     int chain_kind;             // kChainGeneric, or a row chain the kernels evaluate inline
     int sides_in_ring;          // dense: used sides are contiguous vectors, staged with the rows
     int out_vec;                // no_agg, dense: rows of `out` can be written 16 bytes at a time
+    int rb;                     // CSR: rows a warp takes at a time (32; fewer, a power of two >= 32 / G, for few rows)
 };
 
 // Row chains common enough to be evaluated inline instead of interpreted; the
@@ -377,14 +378,16 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
     }
     __syncthreads();
 
-    const long long nblocks = (p.rows + 31) >> 5;
+    const int RB = p.rb;
+    const int nit = G * RB / 32;                     // >= 1: RB >= 32 / G
+    const long long nblocks = (p.rows + RB - 1) / RB;
     const long long warp0 = (long long)blockIdx.x * kWarps + warp;
     const long long nwarps = (long long)gridDim.x * kWarps;
     double tsum = 0.0;
 
     for (long long blk = warp0; blk < nblocks; blk += nwarps) {
-        const long long myrow = (blk << 5) + lane;
-        const bool have = myrow < p.rows;
+        const long long myrow = blk * RB + lane;
+        const bool have = lane < RB && myrow < p.rows;
         const int beg_l = have ? __ldg(p.rowptr + myrow) : 0;
         const int end_l = have ? __ldg(p.rowptr + myrow + 1) : beg_l;
         double sv[FO_MAX_SIDES];
@@ -396,7 +399,7 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
         // stage the block's stored cells (skipped, and read from global memory
         // below, when the block holds more than the slice can take)
         const int base = __shfl_sync(0xffffffffu, beg_l, 0);
-        const int last_end = __shfl_sync(0xffffffffu, end_l, (int)((p.rows - (blk << 5) < 32) ? p.rows - (blk << 5) - 1 : 31));
+        const int last_end = __shfl_sync(0xffffffffu, end_l, (int)((p.rows - blk * RB < RB) ? p.rows - blk * RB - 1 : RB - 1));
         const int total = last_end - base;
         const bool staged = total <= kCsrStage;
         if (staged) {
@@ -410,7 +413,7 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
         // G lanes per row: 32 / G rows at a time, G trips
         double dmine = 0.0;
 #pragma unroll 1
-        for (int it = 0; it < G; ++it) {
+        for (int it = 0; it < nit; ++it) {
             const int rr = it * (32 / G) + grp;
             const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
             const int end = __shfl_sync(0xffffffffu, end_l, rr);
@@ -444,7 +447,7 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
         } else if (AGG == kRowNone) {
             // out has X's pattern: stored cell p of row i becomes t_i * vals[p]; one
             // row after the other, the lanes across the row's cells
-            for (int rr = 0; rr < 32; ++rr) {
+            for (int rr = 0; rr < RB; ++rr) {
                 const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
                 const int end = __shfl_sync(0xffffffffu, end_l, rr);
                 const double tt = __shfl_sync(0xffffffffu, t, rr);
@@ -453,7 +456,7 @@ row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowP
             }
         } else {
 #pragma unroll 1
-            for (int it = 0; it < G; ++it) {
+            for (int it = 0; it < nit; ++it) {
                 const int rr = it * (32 / G) + grp;
                 const int beg = __shfl_sync(0xffffffffu, beg_l, rr);
                 const int end = __shfl_sync(0xffffffffu, end_l, rr);
@@ -679,9 +682,19 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
         p.rowptr = X->csr.rowptr; p.colidx = X->csr.colidx; p.vals = X->csr.vals;
         const size_t smem = (size_t)cols * 8 * (agg == FO_ROW_COL_T_AGG ? 2 : 1)
                             + (size_t)kWarps * kCsrStage * 12;
-        long long grid = (rows + kThreads - 1) / kThreads;
+        // lanes per row from the mean row length: about four trips for a typical row
+        const double mean_len = rows > 0 ? (double)X->csr.nnz / (double)rows : 0.0;
+        const int lanes_per_row = mean_len <= 12.0 ? 2 : mean_len <= 24.0 ? 4 : mean_len <= 48.0 ? 8
+                                  : mean_len <= 96.0 ? 16 : 32;
+        // rows a warp takes at a time: 32, or fewer when there are too few rows to give every warp
+        // of the machine a block (never fewer than 32 / lanes per row)
+        int rb = 32;
+        while (rb > 32 / lanes_per_row && (rows + rb - 1) / rb < (long long)sms * 16) rb >>= 1;
+        p.rb = rb;
+        long long grid = ((rows + rb - 1) / rb + kWarps - 1) / kWarps;
         const long long cap = (long long)sms * 3 < row_grid_cap() ? (long long)sms * 3 : row_grid_cap();
         if (grid > cap) grid = cap;
+        if (grid < 1) grid = 1;
         auto go = [&](auto kern) -> cudaError_t {
             cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e2 != cudaSuccess) return e2;
@@ -695,8 +708,6 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
             if (agg == FO_ROW_ROW_AGG) return go(row_csr_kernel<kRowRow, G>);
             return go(row_csr_kernel<kRowFull, G>);
         };
-        // lanes per row from the mean row length: about four trips for a typical row
-        const double mean_len = rows > 0 ? (double)X->csr.nnz / (double)rows : 0.0;
         if (mean_len <= 12.0) e = by_agg(std::integral_constant<int, 2>());
         else if (mean_len <= 24.0) e = by_agg(std::integral_constant<int, 4>());
         else if (mean_len <= 48.0) e = by_agg(std::integral_constant<int, 8>());
