@@ -343,6 +343,88 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
     }
 }
 
+// ----------------------------------------------------------- dense, narrow
+// Rows of at most NC <= 16 columns (the tall, narrow matrices of the paper's
+// end-to-end runs: 10^8 x 10): a row is too short to spread over a warp, so a
+// thread takes whole rows.  It loads its row (16-byte loads when the layout
+// allows), forms the dot product with v held in registers, evaluates the chain
+// and keeps the n output sums in registers; the CTA adds them up in a fixed order
+// at the end.  Neighbouring lanes read neighbouring rows, so a warp's loads cover
+// one contiguous piece of X between them and every fetched sector is used.
+constexpr int kNarrowMax = 16;
+
+template <int NC, int AGG, bool VEC>
+__global__ void __launch_bounds__(kThreads)
+row_narrow_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
+{
+    __shared__ double s_red[NC * 32];
+    __shared__ unsigned int s_flag;
+    const int n = (int)p.cols;
+    double v[NC], q[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        v[j] = j < n ? __ldg(p.v + j) : 0.0;
+        q[j] = 0.0;
+    }
+    double tsum = 0.0;
+    const long long stride = (long long)gridDim.x * kThreads;
+    for (long long row = (long long)blockIdx.x * kThreads + threadIdx.x; row < p.rows; row += stride) {
+        const double *xr = p.X + row * p.ldx;
+        double x[NC];
+        if (VEC) {
+#pragma unroll
+            for (int j = 0; j < NC; j += 2) {
+                double2 t2 = make_double2(0.0, 0.0);
+                if (j < n) t2 = ld_stream2(xr + j);          // n even: the pair is inside the row
+                x[j] = t2.x;
+                x[j + 1] = t2.y;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < NC; ++j) x[j] = j < n ? ld_stream1(xr + j) : 0.0;
+        }
+        double sv[FO_MAX_SIDES];
+#pragma unroll
+        for (int k = 0; k < FO_MAX_SIDES; ++k)
+            sv[k] = ((ch.side_used >> k) & 1u) ? __ldg(p.sides.s[k].data + row * p.sides.s[k].ld) : 0.0;
+        double d0 = 0.0, d1 = 0.0;
+#pragma unroll
+        for (int j = 0; j < NC; j += 2) {
+            d0 = fma(x[j], v[j], d0);
+            d1 = fma(x[j + 1], v[j + 1], d1);
+        }
+        const double t = lane_chain(ch, p.chain_kind, d0 + d1, sv);
+        if (AGG == kRowColT) {
+#pragma unroll
+            for (int j = 0; j < NC; ++j) q[j] = fma(t, x[j], q[j]);
+        } else if (AGG == kRowRow) {
+            p.out[row] = t;
+        } else if (AGG == kRowFull) {
+            tsum += t;
+        } else {
+            double *orow = p.out + row * (long long)n;
+#pragma unroll
+            for (int j = 0; j < NC; ++j)
+                if (j < n) orow[j] = t * x[j];
+        }
+    }
+    if (AGG == kRowColT) {
+        block_sum<NC>(q, s_red);
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int j = 0; j < NC; ++j)
+                if (j < n) p.partials[(size_t)blockIdx.x * n + j] = q[j];
+        }
+        reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * n, n, p.out, &s_flag);
+    } else if (AGG == kRowFull) {
+        double v1[1] = {tsum};
+        block_sum<1>(v1, s_red);
+        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
+    }
+}
+
 // -------------------------------------------------------------------- CSR
 // A warp takes blocks of 32 consecutive rows.  Row offsets, side values and the
 // chain are handled one row per lane (coalesced loads, one chain evaluation for
@@ -716,6 +798,35 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
     } else {
         p.X = X->dense.data; p.ldx = X->dense.ld;
         p.out_vec = (aligned16(out) && cols % 2 == 0) ? 1 : 0;
+        if (cols <= kNarrowMax) {
+            // a thread per row; FUSEDOPS_ROW_NARROW=0 keeps the warp-per-row-slice kernel (a measuring knob)
+            const char *ne = getenv("FUSEDOPS_ROW_NARROW");
+            if (!(ne && ne[0] == '0')) {
+                const bool vec = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0);
+                long long grid = (rows + kThreads - 1) / kThreads;
+                const long long cap = (long long)sms * 4 < row_grid_cap() ? (long long)sms * 4 : row_grid_cap();
+                if (grid > cap) grid = cap;
+                if (grid < 1) grid = 1;
+                auto gon = [&](auto nc) -> cudaError_t {
+                    constexpr int NC = decltype(nc)::value;
+#define FO_NARROW(A)                                                                        \
+    do {                                                                                    \
+        if (vec) row_narrow_kernel<NC, A, true><<<(unsigned)grid, kThreads, 0, st>>>(ch, p);  \
+        else row_narrow_kernel<NC, A, false><<<(unsigned)grid, kThreads, 0, st>>>(ch, p);     \
+    } while (0)
+                    if (agg == FO_ROW_COL_T_AGG) FO_NARROW(kRowColT);
+                    else if (agg == FO_ROW_ROW_AGG) FO_NARROW(kRowRow);
+                    else if (agg == FO_ROW_FULL_AGG) FO_NARROW(kRowFull);
+                    else FO_NARROW(kRowNone);
+#undef FO_NARROW
+                    return cudaGetLastError();
+                };
+                e = cols <= 4 ? gon(std::integral_constant<int, 4>())
+                    : cols <= 8 ? gon(std::integral_constant<int, 8>())
+                                : gon(std::integral_constant<int, 16>());
+                return e == cudaSuccess ? FO_OK : cuda_fail(e);
+            }
+        }
         const bool staged = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
         // ring geometry: every group of warps has its own ring of `stages` slots of r rows
         const DenseShape sh = dense_shape(cols);

@@ -236,6 +236,38 @@ def test_row_dense_variants_strided_unaligned(fo, agg):
     assert_close(got.cpu().numpy(), ref, absscale=row_abs_scale(Xh, v, np.ones(rows)))
 
 
+@pytest.mark.parametrize("cols", [1, 2, 3, 4, 5, 8, 10, 13, 16])
+def test_row_dense_narrow_rows_all_variants(fo, cols):
+    """At most 16 columns: a thread takes whole rows.  Every aggregation, a chain that goes through the
+    interpreter, contiguous and strided / 8-byte-aligned inputs."""
+    rows, ld = 70001, cols + 3
+    flat = datagen.normal(31, 0, rows * ld + 1)
+    v = datagen.normal(31, 2, cols)
+    wv = datagen.uniform(31, 3, rows)
+    chain = [("mul", "t0", "side0", "d"), ("add", "t1", "t0", "s0")]
+    for layout in ("contiguous", "strided", "offset"):
+        if layout == "contiguous":
+            Xh = np.ascontiguousarray(flat[:rows * cols].reshape(rows, cols))
+            Xd = to_dev(Xh)
+        else:
+            off = 0 if layout == "strided" else 1
+            Xh = flat[off:off + rows * ld].reshape(rows, ld)[:, :cols]
+            Xd = to_dev(flat)[off:off + rows * ld].view(rows, ld)[:, :cols]
+        tabs = wv * (np.abs(Xh) @ np.abs(v)) + 0.125
+        for agg in ("col_t", "row", "full", "none"):
+            ref = oracle.row(chain, "t1", Xh, v, [("row", wv)], [0.125], agg=agg)
+            got = fo.fused_row(chain, "t1", Xd, to_dev(v), [("row", to_dev(wv))], [0.125], agg=agg)
+            scale = {"col_t": np.abs(Xh).T @ tabs, "row": tabs, "full": float(np.sum(tabs)),
+                     "none": tabs[:, None] * np.abs(Xh)}[agg]
+            assert_close(got.cpu().numpy(), ref, absscale=scale, what="narrow %d cols %s %s" % (cols, layout, agg))
+    # the weighted chain evaluated inline, and bit-reproducible
+    ref = oracle.row_chain_dense(Xh, v, wv)
+    a = fo.fused_row(WD, "t0", Xd, to_dev(v), [("row", to_dev(wv))]).cpu().numpy()
+    assert_close(a, ref, absscale=row_abs_scale(Xh, v, wv))
+    assert fo.fused_row(WD, "t0", Xd, to_dev(v), [("row", to_dev(wv))]).cpu().numpy().tobytes() == a.tobytes()
+    assert fo.device_status() == 0
+
+
 @pytest.mark.parametrize("rows,cols", [(1000, 1000), (333, 120), (257, 129), (64, 18), (5, 1), (1, 7), (90, 4096),
                                        (40, 8191)])
 def test_row_dense_no_agg_and_col_agg(fo, rows, cols):
