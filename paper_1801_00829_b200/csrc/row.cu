@@ -344,14 +344,15 @@ row_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ro
 }
 
 // ----------------------------------------------------------- dense, narrow
-// Rows of at most NC <= 16 columns (the tall, narrow matrices of the paper's
+// Rows of at most NC <= 32 columns (the tall, narrow matrices of the paper's
 // end-to-end runs: 10^8 x 10): a row is too short to spread over a warp, so a
 // thread takes whole rows.  It loads its row (16-byte loads when the layout
-// allows), forms the dot product with v held in registers, evaluates the chain
+// allows), forms the dot product with v (in registers up to 16 columns, from the
+// cache beyond), evaluates the chain
 // and keeps the n output sums in registers; the CTA adds them up in a fixed order
 // at the end.  Neighbouring lanes read neighbouring rows, so a warp's loads cover
 // one contiguous piece of X between them and every fetched sector is used.
-constexpr int kNarrowMax = 16;
+constexpr int kNarrowMax = 32;
 
 template <int NC, int AGG, bool VEC>
 __global__ void __launch_bounds__(kThreads)
@@ -360,10 +361,11 @@ row_narrow_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ R
     __shared__ double s_red[NC * 32];
     __shared__ unsigned int s_flag;
     const int n = (int)p.cols;
-    double v[NC], q[NC];
+    constexpr bool VREG = NC <= 16;               // beyond that v is read through the cache (one address per warp)
+    double v[VREG ? NC : 1], q[NC];
 #pragma unroll
     for (int j = 0; j < NC; ++j) {
-        v[j] = j < n ? __ldg(p.v + j) : 0.0;
+        if (VREG) v[VREG ? j : 0] = j < n ? __ldg(p.v + j) : 0.0;
         q[j] = 0.0;
     }
     double tsum = 0.0;
@@ -390,8 +392,10 @@ row_narrow_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ R
         double d0 = 0.0, d1 = 0.0;
 #pragma unroll
         for (int j = 0; j < NC; j += 2) {
-            d0 = fma(x[j], v[j], d0);
-            d1 = fma(x[j + 1], v[j + 1], d1);
+            const double va = VREG ? v[VREG ? j : 0] : (j < n ? __ldg(p.v + j) : 0.0);
+            const double vb = VREG ? v[VREG ? j + 1 : 0] : (j + 1 < n ? __ldg(p.v + j + 1) : 0.0);
+            d0 = fma(x[j], va, d0);
+            d1 = fma(x[j + 1], vb, d1);
         }
         const double t = lane_chain(ch, p.chain_kind, d0 + d1, sv);
         if (AGG == kRowColT) {
@@ -823,7 +827,8 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
                 };
                 e = cols <= 4 ? gon(std::integral_constant<int, 4>())
                     : cols <= 8 ? gon(std::integral_constant<int, 8>())
-                                : gon(std::integral_constant<int, 16>());
+                    : cols <= 16 ? gon(std::integral_constant<int, 16>())
+                                 : gon(std::integral_constant<int, 32>());
                 return e == cudaSuccess ? FO_OK : cuda_fail(e);
             }
         }

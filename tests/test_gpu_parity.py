@@ -236,9 +236,9 @@ def test_row_dense_variants_strided_unaligned(fo, agg):
     assert_close(got.cpu().numpy(), ref, absscale=row_abs_scale(Xh, v, np.ones(rows)))
 
 
-@pytest.mark.parametrize("cols", [1, 2, 3, 4, 5, 8, 10, 13, 16])
+@pytest.mark.parametrize("cols", [1, 2, 3, 4, 5, 8, 10, 13, 16, 17, 24, 31, 32])
 def test_row_dense_narrow_rows_all_variants(fo, cols):
-    """At most 16 columns: a thread takes whole rows.  Every aggregation, a chain that goes through the
+    """At most 32 columns: a thread takes whole rows.  Every aggregation, a chain that goes through the
     interpreter, contiguous and strided / 8-byte-aligned inputs."""
     rows, ld = 70001, cols + 3
     flat = datagen.normal(31, 0, rows * ld + 1)
