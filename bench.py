@@ -282,6 +282,17 @@ def time_variants(fo, step, shapes, reps=10):
         ("magg_csr_density_0.1", lambda: fo.fused_magg(MAGG3, ["t0", "t1", "t2"], Xs, sides, out=o_three),
          sparse_in + 24),
     ]
+    # tall, narrow dense rows (the 10-column shape of the paper's end-to-end data, Section 5.3): the MAgg
+    # input seen as (10 * rows) x 10
+    if mc % 10 == 0:
+        Xn = d["magg.X"].view(mr * (mc // 10), 10)
+        g.manual_seed(7)
+        vn = torch.randn(10, generator=g, dtype=torch.float64, device=dev)
+        wn = torch.rand(Xn.shape[0], generator=g, dtype=torch.float64, device=dev)
+        o_n = torch.empty(10, dtype=torch.float64, device=dev)
+        cases.append(("row_dense_10cols_col_t_agg",
+                      lambda: fo.fused_row(WD, "t0", Xn, vn, [("row", wn)], out=o_n),
+                      8 * Xn.shape[0] * 10 + 8 * Xn.shape[0] + 160))
     # Row template with matrix-valued row intermediates (Section 5.2: t(X) %*% (X %*% V) with
     # V 1000 x 2 on the dense Row input; the Eq. 2 inner loop for k classes on the 100-column input)
     MLR_PRE = [("mul", "t0", "side0", "d")]

@@ -377,7 +377,9 @@ row_narrow_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ R
 #pragma unroll
             for (int j = 0; j < NC; j += 2) {
                 double2 t2 = make_double2(0.0, 0.0);
-                if (j < n) t2 = ld_stream2(xr + j);          // n even: the pair is inside the row
+                // n even: the pair is inside the row.  Cached in L1 on purpose: a 32-byte sector
+                // holds two of these pairs, and the second request should not go back to L2
+                if (j < n) t2 = __ldg(reinterpret_cast<const double2 *>(xr + j));
                 x[j] = t2.x;
                 x[j + 1] = t2.y;
             }
