@@ -31,7 +31,9 @@
  *     data[i * ld + j], ld >= cols.
  *   - Sums are deterministic: for given shapes the order of every floating-point
  *     addition is fixed, so repeated calls return identical bits (exception:
- *     the CSR variant of FO_ROW_COL_T_AGG, documented at fused_row).
+ *     the variants that scatter through atomics: FO_ROW_COL_T_AGG / FO_ROW_COL_AGG and
+ *     FO_ROW_COL_AGG_B1_T over a CSR main input, FO_CELL_COL_AGG over a CSR main input,
+ *     FO_OUTER_LEFT_MM; each is documented at its call).
  */
 #ifndef FUSEDOPS_H
 #define FUSEDOPS_H
@@ -233,6 +235,9 @@ int fo_chain_describe(const fo_chain *chain, int use, int n_sides,
  * A CSR main input with a chain that is not zero-preserving gives the result
  * of the sparse-safe binding, not of the dense one; the caller decides that
  * (in the paper the compiler marks templates sparse-safe, Section 2.2).
+ * Determinism: FO_CELL_COL_AGG over a CSR X adds into `out` with global atomics on
+ * a zeroed result, so the order of its additions is not fixed; everything else
+ * is bit-reproducible.
  * Errors: FO_ERR_CHAIN if the chain uses FO_DOT; FO_ERR_SHAPE if a side does
  * not match X under its access kind; empty X (no cells) writes zeros.
  */
@@ -301,8 +306,8 @@ int fused_magg(const fo_chain *chain, const fo_mat *X,
  * With the chain  t = side0 * d  this is  t(X) %*% (w * (X %*% v)).
  * X wider than 8192 columns returns FO_ERR_UNSUPPORTED (the single-pass
  * kernels keep a row, respectively v and the output vector, on chip).
- * Determinism: bit-reproducible except FO_ROW_COL_T_AGG over CSR, whose
- * scatter-add into on-chip accumulators is unordered.
+ * Determinism: bit-reproducible except FO_ROW_COL_T_AGG / FO_ROW_COL_AGG over
+ * CSR, whose scatter-add into on-chip accumulators is unordered.
  */
 int fused_row(const fo_chain *chain, const fo_mat *X, const double *v,
               const fo_side *sides, int n_sides,
