@@ -3,6 +3,9 @@
 // Operations", t(X) %*% (X %*% V)).  Per row i of a dense X and a side matrix
 // B (n x k):  D_i = X_i B  (k values),  s_i = sum_c pre(D_ic),  T_ic = post(D_ic, s_i),
 // then  out += X_i^T T_i  (n x k)  or  out[i] = T_i.
+// Four kernels: tensor-core tiles (row_b1_mma_kernel), multiply-add tiles
+// (row_b1_kernel, described next), a thread per row for narrow matrices
+// (row_b1_narrow_kernel) and CSR rows (row_b1_csr_kernel).
 //
 // The row is read from HBM once.  A CTA's 16 warps form independent groups; a
 // group streams its tiles of R rows through its own shared-memory ring with
@@ -617,6 +620,121 @@ row_b1_mma_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ 
     }
 }
 
+// ----------------------------------------------------------------- narrow
+// Rows of at most NC <= 16 columns and at most KC <= 8 classes, NC * KC <= 64
+// (Eq. 2 on the tall, narrow matrices of the paper's end-to-end runs): a thread
+// takes whole rows.  It loads its row, forms the k products with B (shared
+// memory, every lane the same address), sums the first chain over the classes by
+// itself, and keeps the n x k output sums in registers; the CTA adds them up in
+// a fixed order at the end.
+constexpr int kB1NarrowThreads = 256;
+
+template <int NC, int KC, int AGG, bool VEC>
+__global__ void __launch_bounds__(kB1NarrowThreads)
+row_b1_narrow_kernel(const __grid_constant__ DevChain pre, const __grid_constant__ DevChain post,
+                     const __grid_constant__ B1Params p)
+{
+    __shared__ double s_B[NC * KC];
+    __shared__ double s_red[NC * KC * 32];
+    __shared__ unsigned int s_flag;
+    const int n = (int)p.cols, k = p.k;
+    for (int e = threadIdx.x; e < NC * KC; e += kB1NarrowThreads) {
+        const int j = e / KC, c = e - j * KC;
+        s_B[e] = (j < n && c < k) ? __ldg(p.B + (long long)j * p.ldb + c) : 0.0;
+    }
+    __syncthreads();
+    double h[NC * KC];
+#pragma unroll
+    for (int e = 0; e < NC * KC; ++e) h[e] = 0.0;
+
+    const long long stride = (long long)gridDim.x * kB1NarrowThreads;
+    for (long long row = (long long)blockIdx.x * kB1NarrowThreads + threadIdx.x; row < p.rows; row += stride) {
+        const double *xr = p.X + row * p.ldx;
+        double x[NC];
+        if (VEC) {
+#pragma unroll
+            for (int j = 0; j < NC; j += 2) {
+                double2 t2 = make_double2(0.0, 0.0);
+                if (j < n) t2 = __ldg(reinterpret_cast<const double2 *>(xr + j));     // n even
+                x[j] = t2.x;
+                x[j + 1] = t2.y;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < NC; ++j) x[j] = j < n ? __ldg(xr + j) : 0.0;
+        }
+        double d[KC], t[KC], sv[KC][FO_MAX_SIDES];
+#pragma unroll
+        for (int c = 0; c < KC; ++c) {
+            d[c] = 0.0;
+#pragma unroll
+            for (int j = 0; j < FO_MAX_SIDES; ++j) {
+                sv[c][j] = 0.0;
+                if (c < k && ((p.side_used >> j) & 1u)) {
+                    const DevSide &sd = p.sides.s[j];
+                    const long long off = sd.access == FO_AT_CELL ? row * sd.ld + c
+                                          : sd.access == FO_AT_ROW ? row * sd.ld : (long long)c;
+                    sv[c][j] = __ldg(sd.data + off);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < NC; ++j)
+#pragma unroll
+            for (int c = 0; c < KC; ++c) d[c] = fma(x[j], s_B[j * KC + c], d[c]);
+
+        if (p.chain_kind == kB1Identity) {
+#pragma unroll
+            for (int c = 0; c < KC; ++c) t[c] = d[c];
+        } else {
+            double rowsum = 0.0;
+            if (p.has_pre) {
+#pragma unroll
+                for (int c = 0; c < KC; ++c) {
+                    const double pv = p.chain_kind == kB1Mlogreg
+                                          ? sv[c][0] * d[c]
+                                          : b1_lane_chain(pre, d[c], sv[c][0], sv[c][1], sv[c][2], sv[c][3]);
+                    rowsum += c < k ? pv : 0.0;
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < KC; ++c) {
+                if (p.chain_kind == kB1Mlogreg) {
+                    t[c] = sv[c][0] * d[c] - sv[c][0] * rowsum;
+                } else {
+                    double s2[FO_MAX_SIDES];
+#pragma unroll
+                    for (int j = 0; j < FO_MAX_SIDES; ++j) s2[j] = (p.has_pre && j == p.sides.n) ? rowsum : sv[c][j];
+                    t[c] = b1_lane_chain(post, d[c], s2[0], s2[1], s2[2], s2[3]);
+                }
+            }
+        }
+        if (AGG == kB1None) {
+#pragma unroll
+            for (int c = 0; c < KC; ++c)
+                if (c < k) p.out[row * k + c] = t[c];
+        } else {
+#pragma unroll
+            for (int j = 0; j < NC; ++j)
+#pragma unroll
+                for (int c = 0; c < KC; ++c) h[j * KC + c] = fma(x[j], c < k ? t[c] : 0.0, h[j * KC + c]);
+        }
+    }
+    if (AGG == kB1ColT) {
+        block_sum<NC * KC>(h, s_red);
+        const long long width = (long long)n * k;
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int j = 0; j < NC; ++j)
+#pragma unroll
+                for (int c = 0; c < KC; ++c)
+                    if (j < n && c < k) p.partials[(size_t)blockIdx.x * width + (size_t)j * k + c] = h[j * KC + c];
+        }
+        reduce_columns_two_level(p.head, p.partials, p.partials + (size_t)gridDim.x * width, width, p.out,
+                                 &s_flag);
+    }
+}
+
 // ------------------------------------------------------------------- CSR
 // The same operator over the stored cells of a CSR X (the listing's
 // genexecSparse).  A warp takes blocks of 32 consecutive rows and stages their
@@ -1085,6 +1203,37 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
         return e2 == cudaSuccess ? FO_OK : cuda_fail(e2);
     }
     const bool staged = b1_aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
+    // narrow rows: a thread per row (FUSEDOPS_B1_NARROW=0 switches it off; a measuring knob)
+    {
+        const char *ne = getenv("FUSEDOPS_B1_NARROW");
+        const int nc = cols <= 8 ? 8 : 16, kc = k <= 2 ? 2 : k <= 4 ? 4 : 8;
+        if (!(ne && ne[0] == '0') && cols <= 16 && k <= 8 && nc * kc <= 64) {
+            const bool vec = b1_aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0);
+            long long grid = (rows + kB1NarrowThreads - 1) / kB1NarrowThreads;
+            const long long cap = (long long)sms * 2 < b1_grid_cap() ? (long long)sms * 2 : b1_grid_cap();
+            if (grid > cap) grid = cap;
+            if (grid < 1) grid = 1;
+            auto gon = [&](auto ncc, auto kcc) -> cudaError_t {
+                constexpr int NC = decltype(ncc)::value, KC = decltype(kcc)::value;
+                if (agg == FO_ROW_COL_AGG_B1_T) {
+                    if (vec) row_b1_narrow_kernel<NC, KC, kB1ColT, true><<<(unsigned)grid, kB1NarrowThreads, 0, st>>>(chpre, chpost, p);
+                    else row_b1_narrow_kernel<NC, KC, kB1ColT, false><<<(unsigned)grid, kB1NarrowThreads, 0, st>>>(chpre, chpost, p);
+                } else {
+                    if (vec) row_b1_narrow_kernel<NC, KC, kB1None, true><<<(unsigned)grid, kB1NarrowThreads, 0, st>>>(chpre, chpost, p);
+                    else row_b1_narrow_kernel<NC, KC, kB1None, false><<<(unsigned)grid, kB1NarrowThreads, 0, st>>>(chpre, chpost, p);
+                }
+                return cudaGetLastError();
+            };
+            using I2 = std::integral_constant<int, 2>;
+            using I4 = std::integral_constant<int, 4>;
+            using I8 = std::integral_constant<int, 8>;
+            using I16 = std::integral_constant<int, 16>;
+            cudaError_t en;
+            if (nc == 8) en = kc == 2 ? gon(I8(), I2()) : kc == 4 ? gon(I8(), I4()) : gon(I8(), I8());
+            else en = kc == 2 ? gon(I16(), I2()) : gon(I16(), I4());
+            return en == cudaSuccess ? FO_OK : cuda_fail(en);
+        }
+    }
     // tensor-core variant where its layout fits (FUSEDOPS_B1_MMA=0 / 1 forces the choice)
     {
         MmaShape ms;

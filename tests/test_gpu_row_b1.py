@@ -54,7 +54,7 @@ def mlr_scale(X, V, P):
 # (rows, cols, k): k = 1..32, narrow and wide rows, odd sizes, ragged last tiles
 SHAPES = [(2000, 1000, 2), (5000, 100, 2), (3001, 100, 4), (3000, 100, 8), (2500, 100, 16), (1501, 100, 32),
           (777, 64, 3), (513, 200, 5), (1000, 512, 16), (600, 1024, 8), (300, 2048, 4), (150, 4096, 2),
-          (97, 31, 7), (64, 2, 1), (900, 102, 9), (700, 160, 20), (500, 500, 12), (650, 1000, 8), (800, 64, 32), (300, 230, 17), (1, 10, 2), (5, 1, 3), (1200, 256, 32), (40, 999, 2), (333, 250, 24)]
+          (97, 31, 7), (64, 2, 1), (50001, 10, 2), (40001, 10, 4), (30000, 16, 4), (25000, 8, 8), (9999, 7, 3), (20000, 16, 2), (900, 102, 9), (700, 160, 20), (500, 500, 12), (650, 1000, 8), (800, 64, 32), (300, 230, 17), (1, 10, 2), (5, 1, 3), (1200, 256, 32), (40, 999, 2), (333, 250, 24)]
 
 
 @pytest.mark.parametrize("rows,cols,k", SHAPES)
@@ -83,7 +83,8 @@ def test_b1_mlogreg(fo, path, rows, cols, k):
     assert fo.device_status() == 0
 
 
-@pytest.mark.parametrize("rows,cols,k", [(1000, 100, 3), (700, 1000, 2), (400, 300, 8), (90, 64, 32)])
+@pytest.mark.parametrize("rows,cols,k", [(1000, 100, 3), (700, 1000, 2), (400, 300, 8), (90, 64, 32), (30000, 10, 3),
+                                         (20000, 5, 8)])
 def test_b1_generic_chains_all_side_kinds(fo, path, rows, cols, k):
     # T_ic = (d * rvec_c + cvec_i * P_ic) * s0 - exp(-|rowsum|),  rowsum = sum_c P_ic * d
     w = datagen.row_b1_workload(rows, cols, k, seed=7)
@@ -230,4 +231,35 @@ def test_b1_csr_rows(fo, rows, cols, k, density):
     got = fo.fused_row_b1(genpre, "t0", gen, "t1", csr_to_dev(w), to_dev(V), agg="none")
     aD = oracle.row_b1(None, None, [], "d", absX, np.abs(V), agg="none")
     assert_close(got.cpu().numpy(), ref, absscale=(aD + 1.0) * aD.sum(axis=1, keepdims=True) + 1e-300)
+    assert fo.device_status() == 0
+
+
+@pytest.mark.parametrize("cols,k", [(10, 2), (7, 4), (16, 3), (3, 8)])
+def test_b1_narrow_rows_strided_unaligned(fo, cols, k):
+    """At most 16 columns: a thread takes whole rows; strided and 8-byte-aligned inputs, and the switch back
+    to the wide kernels gives the same values within tolerance."""
+    rows, ld = 30011, cols + 3
+    flat = datagen.normal(41, 0, rows * ld + 1)
+    V = datagen.normal(41, 2, cols * k).reshape(cols, k)
+    P = datagen.uniform(41, 3, rows * k).reshape(rows, k) / (k + 1)
+    for off in (0, 1):
+        Xh = flat[off:off + rows * ld].reshape(rows, ld)[:, :cols]
+        Xd = to_dev(flat)[off:off + rows * ld].view(rows, ld)[:, :cols]
+        for agg in ("col_t", "none"):
+            ref = oracle.row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xh, V, [("cell", P)], agg=agg)
+            got = fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xd, to_dev(V), [("cell", to_dev(P))], agg=agg)
+            Q = P * (np.abs(Xh) @ np.abs(V))
+            tabs = Q + P * Q.sum(axis=1, keepdims=True)
+            assert_close(got.cpu().numpy(), ref, absscale=tabs if agg == "none" else np.abs(Xh).T @ tabs,
+                         what="b1 narrow %dx%d off=%d %s" % (cols, k, off, agg))
+    old = os.environ.get("FUSEDOPS_B1_NARROW")
+    os.environ["FUSEDOPS_B1_NARROW"] = "0"
+    try:
+        wide = fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xd, to_dev(V), [("cell", to_dev(P))]).cpu().numpy()
+    finally:
+        if old is None:
+            del os.environ["FUSEDOPS_B1_NARROW"]
+        else:
+            os.environ["FUSEDOPS_B1_NARROW"] = old
+    assert_close(wide, oracle.mlogreg_inner(Xh, V, P), absscale=mlr_scale(Xh, V, P))
     assert fo.device_status() == 0
