@@ -82,6 +82,44 @@ cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
     const long long warp0 = (long long)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
     const long long nwarps = (long long)gridDim.x * (kThreads / 32);
 
+    // Rows of at most 64 columns: a warp takes several rows at a time instead of leaving most
+    // lanes without a column.  LPR lanes (a power of two >= cols / 2) share a row, 32 / LPR rows
+    // go into the first pair of values of a lane and as many into the second.
+    if (p.cols <= 64) {
+        int lpr = 1;
+        while (2 * lpr < p.cols) lpr <<= 1;
+        const int rw = 32 / lpr, sub = lane % lpr, rsel = lane / lpr;
+        const long long ca = 2 * sub;
+        for (long long r0 = warp0 * (2 * rw); r0 < p.rows; r0 += nwarps * (2 * rw)) {
+            const long long rowa = r0 + rsel, rowb = r0 + rw + rsel;
+            const bool have_a = rowa < p.rows, have_b = rowb < p.rows;
+            const long long ra = have_a ? rowa : p.rows - 1;        // loads stay inside the matrix
+            double in[kIn][kV];
+            load_inputs_2d<EVAL, ALIGNED>(ch, p, ra, ca, rowb, ca, have_b, in);
+            double o[NOUT][kV];
+            EVAL::template run<kV, NOUT>(ch, in, o);
+            const bool valid[kV] = {have_a && ca < p.cols, have_a && ca + 1 < p.cols,
+                                    have_b && ca < p.cols, have_b && ca + 1 < p.cols};
+            if (AGG == kAggNone) {
+                double *oa = p.out + rowa * p.cols, *ob = p.out + rowb * p.cols;
+                if (valid[0]) oa[ca] = o[0][0];
+                if (valid[1]) oa[ca + 1] = o[0][1];
+                if (valid[2]) ob[ca] = o[0][2];
+                if (valid[3]) ob[ca + 1] = o[0][3];
+            } else if (AGG == kAggRow) {
+                double sa = (valid[0] ? o[0][0] : 0.0) + (valid[1] ? o[0][1] : 0.0);
+                double sb = (valid[2] ? o[0][2] : 0.0) + (valid[3] ? o[0][3] : 0.0);
+                for (int off = lpr >> 1; off >= 1; off >>= 1) {
+                    sa += __shfl_xor_sync(0xffffffffu, sa, off);
+                    sb += __shfl_xor_sync(0xffffffffu, sb, off);
+                }
+                if (sub == 0 && have_a) p.out[rowa] = sa;
+                if (sub == 0 && have_b) p.out[rowb] = sb;
+            } else {
+                add_outputs<NOUT>(o, valid, acc);
+            }
+        }
+    } else
     for (long long row = warp0; row < p.rows; row += nwarps) {
         double rowacc[NOUT];
 #pragma unroll

@@ -34,6 +34,34 @@ def dev_sides(sides):
 
 
 # ------------------------------------------------------------------ Cell
+@pytest.mark.parametrize("cols", [1, 2, 5, 10, 20, 32, 33, 63, 64, 65])
+def test_cell_narrow_rows_with_vector_sides(fo, cols):
+    """Rows of at most 64 columns share a warp in the row-wise Cell kernel: every aggregation, the three
+    side kinds (a column vector and a row vector keep the call off the flat kernel), strided inputs."""
+    rows, ld = 4099, cols + 2
+    flat = datagen.normal(51, 0, rows * ld + 1)
+    Y = datagen.normal(51, 2, rows * cols).reshape(rows, cols)
+    rvec = datagen.normal(51, 3, rows)
+    cvec = datagen.normal(51, 4, cols)
+    chain = [("mul", "t0", "a", "side0"), ("fma", "t1", "t0", "side1", "side2"), ("mul", "t2", "t1", "s0")]
+    for off in (0, 1):
+        Xh = flat[off:off + rows * ld].reshape(rows, ld)[:, :cols]
+        Xd = to_dev(flat)[off:off + rows * ld].view(rows, ld)[:, :cols]
+        sides_h = [("cell", Y), ("row", rvec), ("col", cvec)]
+        sides_d = [("cell", to_dev(Y)), ("row", to_dev(rvec)), ("col", to_dev(cvec))]
+        tabs = (np.abs(Xh * Y) * np.abs(rvec)[:, None] + np.abs(cvec)[None, :]) * 1.5
+        for agg in ("none", "row", "full"):
+            ref = oracle.cell(chain, "t2", Xh, sides_h, [1.5], agg=agg)
+            got = fo.fused_cell(chain, "t2", Xd, sides_d, [1.5], agg=agg)
+            scale = {"none": tabs, "row": tabs.sum(axis=1), "full": float(tabs.sum())}[agg]
+            assert_close(got.cpu().numpy(), np.asarray(ref), absscale=scale, what="cell narrow %d %s off=%d" % (cols, agg, off))
+    # several aggregates in one scan over the same layout
+    ref = oracle.magg(MAGG3, ["t0", "t1", "t2"], Xh, [("cell", Y), ("cell", Y)])
+    got = fo.fused_magg(MAGG3, ["t0", "t1", "t2"], Xd, [("cell", to_dev(Y)), ("cell", to_dev(Y))])
+    assert_close(got.cpu().numpy(), ref, absscale=np.array([np.abs(Xh * Y).sum(), np.abs(Xh * Y).sum(), (Xh * Xh).sum()]))
+    assert fo.device_status() == 0
+
+
 @pytest.mark.parametrize("rows,cols", [(1000, 1000), (1, 1), (1, 7), (5, 1), (33, 65), (257, 129),
                                        (1024, 1), (1, 1024), (3, 1025), (2047, 3), (64, 2048)])
 def test_cell_full_xyz(fo, rows, cols):
