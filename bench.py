@@ -236,6 +236,11 @@ def time_variants(fo, step, shapes, reps=10):
         ("cell_row_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="row", out=o_row), in3 + 8 * mr),
         ("cell_col_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="col", out=o_col), in3 + 8 * mc),
         ("cell_no_agg", lambda: fo.fused_cell(XYZ, "t1", d["magg.X"], sides, agg="none", out=o_all), in3 + 8 * mr * mc),
+        # the cell-wise operator of the ALS-CG update rule (Section 2.2): I + 1e-6 * U * r, r a column vector
+        ("cell_no_agg_scaled_add_vector_side",
+         lambda: fo.fused_cell([("mul", "t0", "a", 1e-6), ("mul", "t1", "t0", "side1"), ("add", "t2", "side0", "t1")],
+                               "t2", d["magg.X"], [("cell", d["magg.Y"]), ("row", o_row)], agg="none", out=o_all),
+         3 * 8 * mr * mc + 8 * mr),
         ("cell_full_agg_runtime_compiled_chain",
          lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="full", out=o_one), in3 + 8),
         ("cell_full_agg_interpreted_chain", lambda: interpreted(

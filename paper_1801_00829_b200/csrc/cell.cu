@@ -490,6 +490,12 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
         case kSpecSq: e = launch_cell_spec<kSpecSq>(ch, p, agg, flat, aligned, grid, st); break;
         case kSpecMagg2: e = launch_cell_spec<kSpecMagg2>(ch, p, agg, flat, aligned, grid, st); break;
         case kSpecMagg3: e = launch_cell_spec<kSpecMagg3>(ch, p, agg, flat, aligned, grid, st); break;
+        case kSpecScaledAdd: {
+            DevChain c2 = ch;                     // the straight-line code reads its constant from slot 0
+            c2.consts[0] = ch.consts[scaled_add_const(ch)];
+            e = launch_cell_spec<kSpecScaledAdd>(c2, p, agg, flat, aligned, grid, st);
+            break;
+        }
         default:
             // no built-in specialisation: a kernel compiled for this chain at run time
             // (flat streaming case), else the interpreter

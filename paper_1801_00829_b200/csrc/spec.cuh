@@ -22,11 +22,14 @@ enum SpecId {
     kSpecSq,        // a * a                             sum(X^2)
     kSpecMagg2,     // (a * side0, a * side1)            Section 5.2 multi-aggregate
     kSpecMagg3,     // (a * side0, a * side1, a * a)     Fig. 1(c)-style
+    kSpecScaledAdd, // side0 + (a * c) * side1           the cell-wise operator of Section 2.2 (I + 1e-6 * U * r)
     kSpecCount
 };
 
 // Host: specialisation matching a translated Cell / MAgg chain, or kSpecNone.
 int match_cell_spec(const DevChain &ch);
+// Host: for kSpecScaledAdd, the entry of ch.consts that holds c (the kernels read it from consts[0]).
+int scaled_add_const(const DevChain &ch);
 
 
 template <int NR>
@@ -85,6 +88,15 @@ struct SpecFn<kSpecSq> {
     static constexpr unsigned kSideMask = 0u;
     static constexpr int kOut = 1;
     __device__ __forceinline__ static void eval(const double *in, const double *, double *o) { o[0] = in[0] * in[0]; }
+};
+template <>
+struct SpecFn<kSpecScaledAdd> {
+    static constexpr unsigned kSideMask = 3u;
+    static constexpr int kOut = 1;
+    __device__ __forceinline__ static void eval(const double *in, const double *c, double *o)
+    {
+        o[0] = in[1] + (in[0] * c[0]) * in[2];
+    }
 };
 template <>
 struct SpecFn<kSpecMagg2> {

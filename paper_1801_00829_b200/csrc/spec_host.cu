@@ -63,10 +63,31 @@ bool same_program(const DevChain &a, const DevChain &b)
     return true;
 }
 
+// side0 + (a * c) * side1 with c a scalar or an immediate, in either operand order of
+// each step (multiplication and addition commute bit for bit).  Returns the constant's
+// slot, or -1.  Inputs: register 0 = a, 1 = side 0, 2 = side 1.
+int scaled_add_slot(const DevChain &ch)
+{
+    if (ch.n_ops != 3 || ch.n_out != 1 || ch.side_used != 3u) return -1;
+    const DevOp &m0 = ch.ops[0], &m1 = ch.ops[1], &ad = ch.ops[2];
+    if (m0.opcode != FO_OP_MUL || m1.opcode != FO_OP_MUL || ad.opcode != FO_OP_ADD) return -1;
+    int slot = -1;
+    if (m0.a == 0 && (m0.b & 0x80)) slot = m0.b & 0x7f;
+    else if (m0.b == 0 && (m0.a & 0x80)) slot = m0.a & 0x7f;
+    if (slot < 0 || m0.dst < ch.tmp_base) return -1;
+    if (!((m1.a == m0.dst && m1.b == 2) || (m1.b == m0.dst && m1.a == 2))) return -1;
+    if (!((ad.a == 1 && ad.b == m1.dst) || (ad.b == 1 && ad.a == m1.dst))) return -1;
+    if (ch.out[0] != ad.dst) return -1;
+    return slot;
+}
+
 }  // namespace
+
+int scaled_add_const(const DevChain &ch) { return scaled_add_slot(ch); }
 
 int match_cell_spec(const DevChain &ch)
 {
+    if (scaled_add_slot(ch) >= 0) return kSpecScaledAdd;
     for (const RefChain &r : kRefs) {
         fo_op ops[3];
         memset(ops, 0, sizeof(ops));

@@ -34,6 +34,35 @@ def dev_sides(sides):
 
 
 # ------------------------------------------------------------------ Cell
+@pytest.mark.parametrize("chain,out,scalars", [
+    ([("mul", "t0", "a", 1e-6), ("mul", "t1", "t0", "side1"), ("add", "t2", "side0", "t1")], "t2", []),
+    ([("mul", "t3", "s0", "a"), ("mul", "t1", "side1", "t3"), ("add", "t0", "t1", "side0")], "t0", [0.25]),
+])
+@pytest.mark.parametrize("rows,cols", [(3000, 20), (257, 100), (64, 1000)])
+def test_cell_scaled_add_chain_equals_interpreter_bitwise(fo, chain, out, scalars, rows, cols):
+    """The cell-wise operator of Section 2.2 (I + 1e-6 * U * r: a matrix side, a column-vector side, no
+    aggregation) runs as straight-line code; same bits as the interpreter, same values as the checker."""
+    U = datagen.normal(61, 0, rows * cols).reshape(rows, cols)
+    I = datagen.normal(61, 2, rows * cols).reshape(rows, cols)
+    r = datagen.normal(61, 3, rows)
+    for sides_h in ([("cell", I), ("row", r)], [("cell", I), ("cell", I)]):
+        sides_d = [(a, to_dev(x)) for a, x in sides_h]
+        for agg in ("none", "full"):
+            try:
+                fo.force_interpreter(False)
+                fast = fo.fused_cell(chain, out, to_dev(U), sides_d, scalars, agg=agg).cpu().numpy()
+                fo.force_interpreter(True)
+                slow = fo.fused_cell(chain, out, to_dev(U), sides_d, scalars, agg=agg).cpu().numpy()
+            finally:
+                fo.force_interpreter(False)
+            assert fast.tobytes() == slow.tobytes()
+            ref = oracle.cell(chain, out, U, sides_h, scalars, agg=agg)
+            c = scalars[0] if scalars else 1e-6
+            second = sides_h[1][1][:, None] if sides_h[1][0] == "row" else sides_h[1][1]
+            tabs = np.abs(I) + np.abs(U * c * second)
+            assert_close(fast, np.asarray(ref), absscale=tabs if agg == "none" else float(tabs.sum()))
+
+
 @pytest.mark.parametrize("cols", [1, 2, 5, 10, 20, 32, 33, 63, 64, 65])
 def test_cell_narrow_rows_with_vector_sides(fo, cols):
     """Rows of at most 64 columns share a warp in the row-wise Cell kernel: every aggregation, the three
