@@ -18,7 +18,11 @@
  *     caller.  fo_chain, fo_op, fo_side, fo_mat structs and the `scalars` array
  *     are HOST memory; they are copied at launch and may be freed on return.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
- *     the default stream).  No call allocates, frees or synchronises.
+ *     the default stream).  No call allocates, frees or synchronises, with one
+ *     documented exception: the first use of a Cell / MAgg chain that the library
+ *     specialises at run time (see fo_set_jit) compiles and loads a kernel inside
+ *     fused_cell / fused_magg unless the chain was prepared with fo_jit_prepare or
+ *     the mode forbids it.  fused_cell_static never does.
  *   - Inputs are never written.  `out` is fully overwritten.
  *   - `ws` is scratch of at least fused_*_workspace_bytes() bytes, 256-byte
  *     aligned, prepared once with fo_workspace_init(); every call leaves it
@@ -178,48 +182,35 @@ const char *fo_status_string(int status);
  * (thread-local), 0 if none. */
 int fo_last_cuda_error(void);
 
-/* Chains that match one of the library's compile-time specialisations (the
- * products and multi-aggregates of Fig. 1(a), (c)) normally run as straight-line
- * code; every other chain runs through the general interpreter.  Both give the
- * same bits.  on != 0 sends every Cell / MAgg chain through the interpreter
- * (process-wide; for tests and measurements).  Returns the previous setting. */
-int fo_set_force_interpreter(int on);
-
 /* Run-time specialisation (the paper's template expansion to source, compilation
  * and plan cache, Section 2.1 "Codegen Architecture").  A Cell / MAgg chain over
  * contiguous inputs (full_agg, MAgg, no_agg) that has no built-in specialisation
  * is written out as straight-line code inside the library's streaming kernel,
- * compiled for the current GPU with NVRTC on first use (a few hundred ms) and
- * cached by its translated program for the life of the process; later calls
- * with the same chain - whatever the values of its scalars and immediates - reuse
- * it.  Results are bit-identical to the interpreter's.  NVRTC and the driver
- * library are loaded on demand; if they are missing or a compilation fails the
- * interpreter runs instead, so behaviour never depends on them.
- *   fo_set_jit(on)   switches the mechanism (default on); returns the old setting.
- *   fo_jit_stats()   kernels compiled, specialised launches, failed compilations so
- *                    far; returns 1 if NVRTC and the driver library are usable.
- *   fo_jit_compile_check()  generates and compiles (for sm_100a, without loading or
- *                    launching: no GPU needed) the kernel of a Cell chain; FO_OK,
- *                    a chain error, FO_ERR_UNSUPPORTED without NVRTC; the compiler
- *                    log is copied to `log`. */
-int fo_set_jit(int on);
+ * compiled for the current GPU with NVRTC (a few hundred ms) and cached under its
+ * translated program, per CUDA context, for the life of the process; calls with
+ * the same chain - whatever the values of its scalars and immediates - reuse it.
+ * Results are bit-identical to the interpreter's.  NVRTC and the driver library
+ * are loaded on demand; if they are missing or a compilation fails the
+ * interpreter runs instead, so results never depend on them.
+ *   fo_set_jit(mode)  FO_JIT_OFF: never specialise.  FO_JIT_FIRST_USE (default):
+ *                     fused_cell / fused_magg compile a chain the first time they
+ *                     see it - that one call compiles, loads a module (which
+ *                     allocates) and may synchronise; do it outside stream capture.
+ *                     FO_JIT_PREPARED: the calls only look kernels up; a chain that
+ *                     was not prepared runs through the interpreter, and no call
+ *                     ever compiles, loads or allocates.  Returns the old mode.
+ *   fo_jit_prepare()  compiles, loads and caches the kernel of a chain now, for the
+ *                     current device (n_sides / n_scalars as in the later calls;
+ *                     store != 0: the no_agg form, else the aggregating form).
+ *                     FO_OK (also when it was cached already), a chain error,
+ *                     FO_ERR_UNSUPPORTED without NVRTC / the driver library,
+ *                     FO_ERR_CHAIN if the compilation or the load failed.
+ *   fo_jit_stats()    kernels compiled, specialised launches, failed compilations so
+ *                     far; returns 1 if NVRTC and the driver library are usable. */
+enum { FO_JIT_OFF = 0, FO_JIT_FIRST_USE = 1, FO_JIT_PREPARED = 2 };
+int fo_set_jit(int mode);
+int fo_jit_prepare(const fo_chain *chain, int n_sides, int n_scalars, int store);
 int fo_jit_stats(int *compiled, int *launches, int *failures);
-int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int store,
-                         char *log, size_t log_bytes);
-
-/* The k-th result of a chain written out as an expression over the inputs,
- * after validation and translation for a template (`use`: 0 Cell / MAgg,
- * 1 Row, 2 Outer), e.g. "mul(ne(r0,k0),mul(sub(r0,r1),sub(r0,r1)))" for the
- * weighted squared loss of Eq. 1.  rN: input register N (Cell: r0 = a, r1.. =
- * sides; Row: r0 = d, r1.. = sides; Outer: r0 = a, r1 = d); kN: entry N of the
- * constant table (scalars first, then immediates); sq(x) is written mul(x,x).
- * Chains with the same text do the same arithmetic in the same order; the
- * library picks its built-in straight-line evaluations by this text.  Host
- * only, no GPU needed.  Returns FO_OK, a chain error, or FO_ERR_SHAPE when the
- * text does not fit in `cap` bytes. */
-int fo_chain_describe(const fo_chain *chain, int use, int n_sides,
-                      const double *scalars, int n_scalars, int k,
-                      char *text, size_t cap);
 
 /* ------------------------------------------------------------------ Cell
  * Table 1, Cell template; Section 2.2 cell-wise listing.
@@ -258,7 +249,11 @@ int fused_cell(const fo_chain *chain, const fo_mat *X,
  * library image on every GPU that loads it, from load until the process exits.
  *
  * Same arguments, results and bits as fused_cell (dense X; all four variants).
- * It calls no cudaMalloc / cudaFree and no allocating library routine.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.  In
+ * particular it never compiles or loads a run-time specialised kernel: a chain
+ * that fused_cell or fo_jit_prepare specialised earlier is reused (a lookup),
+ * any other chain runs through the built-in straight-line code or the
+ * interpreter - same bits, lower speed.
  *   - Limit: the call must need at most fused_cell_static_limit_bytes() (1 MiB)
  *     of scratch, i.e. fused_cell_workspace_bytes(X, agg) <= that.  This always
  *     holds for no_agg, row_agg and full_agg.  col_agg keeps one partial row of
@@ -371,27 +366,6 @@ int fused_outer(const fo_chain *chain, const fo_csr *X,
                 const fo_dense *U, const fo_dense *V,
                 const double *scalars, int n_scalars,
                 int agg, double *out, void *ws, size_t ws_bytes, void *stream);
-
-/* ---------------------------------------------------------------- probes
- * Machine-rate probes (no counterpart in the paper).  The Outer template
- * (Fig. 1(d)) gathers one row of V per stored cell and does `rank` multiply-adds
- * on it, so its roofline has two terms besides HBM bandwidth: the rate at which
- * whole rows can be gathered at random from a matrix resident in L2, and the
- * fp64 multiply-add issue rate.  These calls run a kernel that does only that;
- * the caller times them with events on `stream`.
- *   fo_probe_out_len()    doubles both probes write to `out` (device; one per
- *                         launched thread, so that the work cannot be dropped).
- *   fo_probe_l2_gather()  reads rows idx[0..n) (device int32, each in [0, V.rows))
- *                         of the dense matrix V, 8 lanes per row, 16-byte loads:
- *                         n * V.cols * 8 bytes move.  V.cols and V.ld even, V.data
- *                         16-byte aligned, else FO_ERR_UNSUPPORTED.
- *   fo_probe_fp64_fma()   every one of the fo_probe_out_len() threads runs
- *                         8 * iters dependent-chain-of-8 multiply-adds from
- *                         registers: 16 * iters * fo_probe_out_len() flop.
- * Asynchronous; allocate nothing; errors as for the other calls. */
-size_t fo_probe_out_len(void);
-int fo_probe_l2_gather(const fo_dense *V, const int *idx, long long n, double *out, void *stream);
-int fo_probe_fp64_fma(long long iters, double *out, void *stream);
 
 #ifdef __cplusplus
 }

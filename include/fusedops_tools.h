@@ -1,0 +1,69 @@
+/*
+ * fusedops_tools.h - test and measurement hooks of the fused-operator library.
+ *
+ * Nothing here is needed to execute a fused operator; the product interface is
+ * fusedops.h.  These calls let tests pin the library's internal choices (which
+ * evaluation of a chain runs, what a run-time specialised kernel compiles to)
+ * and let the benchmark measure the machine rates its rooflines divide by.
+ */
+#ifndef FUSEDOPS_TOOLS_H
+#define FUSEDOPS_TOOLS_H
+
+#include "fusedops.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Chains that match one of the library's compile-time specialisations (the
+ * products and multi-aggregates of Fig. 1(a), (c)) normally run as straight-line
+ * code; every other chain runs through the general interpreter.  Both give the
+ * same bits.  on != 0 sends every Cell / MAgg chain through the interpreter
+ * (process-wide; for tests and measurements).  Returns the previous setting. */
+int fo_set_force_interpreter(int on);
+
+/* Generates and compiles (for sm_100a, without loading or launching: no GPU
+ * needed) the run-time specialised kernel of a Cell chain; FO_OK, a chain error,
+ * FO_ERR_UNSUPPORTED without NVRTC; the compiler log is copied to `log`. */
+int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int store,
+                         char *log, size_t log_bytes);
+
+/* The k-th result of a chain written out as an expression over the inputs,
+ * after validation and translation for a template (`use`: 0 Cell / MAgg,
+ * 1 Row, 2 Outer), e.g. "mul(ne(r0,k0),mul(sub(r0,r1),sub(r0,r1)))" for the
+ * weighted squared loss of Eq. 1.  rN: input register N (Cell: r0 = a, r1.. =
+ * sides; Row: r0 = d, r1.. = sides; Outer: r0 = a, r1 = d); kN: entry N of the
+ * constant table (scalars first, then immediates); sq(x) is written mul(x,x).
+ * Chains with the same text do the same arithmetic in the same order; the
+ * library picks its built-in straight-line evaluations by this text.  Host
+ * only, no GPU needed.  Returns FO_OK, a chain error, or FO_ERR_SHAPE when the
+ * text does not fit in `cap` bytes. */
+int fo_chain_describe(const fo_chain *chain, int use, int n_sides,
+                      const double *scalars, int n_scalars, int k,
+                      char *text, size_t cap);
+
+/* ---------------------------------------------------------------- probes
+ * Machine-rate probes (no counterpart in the paper).  The Outer template
+ * (Fig. 1(d)) gathers one row of V per stored cell and does `rank` multiply-adds
+ * on it, so its roofline has two terms besides HBM bandwidth: the rate at which
+ * whole rows can be gathered at random from a matrix resident in L2, and the
+ * fp64 multiply-add issue rate.  These calls run a kernel that does only that;
+ * the caller times them with events on `stream`.
+ *   fo_probe_out_len()    doubles both probes write to `out` (device; one per
+ *                         launched thread, so that the work cannot be dropped).
+ *   fo_probe_l2_gather()  reads rows idx[0..n) (device int32, each in [0, V.rows))
+ *                         of the dense matrix V, 8 lanes per row, 16-byte loads:
+ *                         n * V.cols * 8 bytes move.  V.cols and V.ld even, V.data
+ *                         16-byte aligned, else FO_ERR_UNSUPPORTED.
+ *   fo_probe_fp64_fma()   every one of the fo_probe_out_len() threads runs
+ *                         8 * iters dependent-chain-of-8 multiply-adds from
+ *                         registers: 16 * iters * fo_probe_out_len() flop.
+ * Asynchronous; allocate nothing; errors as for the other calls. */
+size_t fo_probe_out_len(void);
+int fo_probe_l2_gather(const fo_dense *V, const int *idx, long long n, double *out, void *stream);
+int fo_probe_fp64_fma(long long iters, double *out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FUSEDOPS_TOOLS_H */

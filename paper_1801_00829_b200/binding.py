@@ -82,7 +82,7 @@ EXPORTS = [
     "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
-    "fo_set_jit", "fo_jit_stats", "fo_jit_compile_check",
+    "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_compile_check",
     "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_fp64_fma", "fo_chain_describe",
 ]
 
@@ -135,6 +135,8 @@ def load_library(path=None):
         ip = C.POINTER(C.c_int)
         lib.fo_jit_stats.argtypes = [ip, ip, ip]
         lib.fo_jit_stats.restype = C.c_int
+        lib.fo_jit_prepare.argtypes = [chain_p, i32, i32, i32]
+        lib.fo_jit_prepare.restype = C.c_int
         lib.fo_jit_compile_check.argtypes = [chain_p, i32, i32, i32, C.c_char_p, sz]
         lib.fo_jit_compile_check.restype = C.c_int
         lib.fo_set_force_interpreter.argtypes = [C.c_int]
@@ -329,9 +331,13 @@ def workspace(device, nbytes):
     """A cached, initialised scratch buffer of at least nbytes on `device`."""
     if device.type != "cuda":
         raise RuntimeError("fused operators need CUDA tensors (no CPU path)")
-    key = (device.index if device.index is not None else torch.cuda.current_device())
+    # one buffer per (device, stream): calls that may overlap on the GPU must not share scratch
+    stream = torch.cuda.current_stream(device)
+    key = (device.index if device.index is not None else torch.cuda.current_device(), stream.cuda_stream)
     buf = _ws.get(key)
     if buf is None or buf.numel() < nbytes:
+        if buf is not None:
+            buf.record_stream(stream)         # kernels already queued may still use the old one
         size = max(int(nbytes), 1 << 20)
         buf = torch.empty(size, dtype=torch.uint8, device=device)
         assert buf.data_ptr() % 256 == 0
@@ -347,9 +353,21 @@ def force_interpreter(on):
     return bool(load_library().fo_set_force_interpreter(1 if on else 0))
 
 
-def set_jit(on):
-    """Switches run-time specialisation of Cell / MAgg chains on or off; returns the old setting."""
-    return bool(load_library().fo_set_jit(1 if on else 0))
+JIT_OFF, JIT_FIRST_USE, JIT_PREPARED = 0, 1, 2
+
+
+def set_jit(mode):
+    """Mode of the run-time specialisation of Cell / MAgg chains: JIT_OFF (False),
+    JIT_FIRST_USE (True; compile a chain when it is first seen), JIT_PREPARED (only
+    kernels made by jit_prepare or earlier calls; nothing is compiled inside a
+    call).  Returns the old mode."""
+    return int(load_library().fo_set_jit(int(mode)))
+
+
+def jit_prepare(steps, outputs, n_sides=0, n_scalars=0, store=False):
+    """Compiles and caches the run-time specialised kernel of a chain for the current device."""
+    ch, keep = make_chain(steps, outputs)
+    _check(load_library().fo_jit_prepare(C.byref(ch), n_sides, n_scalars, 1 if store else 0), "fo_jit_prepare")
 
 
 def jit_stats():

@@ -13,6 +13,8 @@
 //   cell_cols_kernel  col_agg: a thread per column pair, a CTA per panel of rows.
 #include <stdlib.h>
 
+#include <atomic>
+
 #include "cell_flat.cuh"
 #include "jit.h"
 #include "cell_csr.h"
@@ -398,7 +400,7 @@ bool g_force_interpreter = false;
 // Common body of fused_cell and fused_magg.
 int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
              const double *scalars, int n_scalars, int agg, bool magg, double *out, void *ws,
-             size_t ws_bytes, void *stream)
+             size_t ws_bytes, void *stream, bool may_compile)
 {
     if (!chain || !X || !out) return FO_ERR_NULL;
     if (n_sides > 0 && !sides) return FO_ERR_NULL;
@@ -500,7 +502,7 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
             // no built-in specialisation: a kernel compiled for this chain at run time
             // (flat streaming case), else the interpreter
             if (!g_force_interpreter && flat && (agg == FO_CELL_FULL_AGG || agg == FO_CELL_NO_AGG)) {
-                const int jrc = jit_launch_flat(ch, p, agg == FO_CELL_NO_AGG, grid, st);
+                const int jrc = jit_launch_flat(ch, p, agg == FO_CELL_NO_AGG, grid, st, may_compile);
                 if (jrc == FO_OK) return FO_OK;
                 if (jrc != kJitUnavailable) return jrc;
             }
@@ -531,23 +533,23 @@ static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
 // be asked for, once per device, with that device current.
 void *static_ws_address()
 {
-    static void *cached[64] = {nullptr};
+    static std::atomic<void *> cached[64];       // zero-initialised; a slot is only ever set to one value
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess || dev < 0 || dev >= 64) {
         cuda_fail(e != cudaSuccess ? e : cudaErrorInvalidDevice);
         return nullptr;
     }
-    if (!cached[dev]) {
-        void *ptr = nullptr;
+    void *ptr = cached[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         e = cudaGetSymbolAddress((void **)&ptr, g_static_ws);
         if (e != cudaSuccess) {
             cuda_fail(e);
             return nullptr;
         }
-        cached[dev] = ptr;
+        cached[dev].store(ptr, std::memory_order_release);
     }
-    return cached[dev];
+    return ptr;
 }
 
 }  // namespace
@@ -566,8 +568,10 @@ int fused_cell_static(const fo_chain *chain, const fo_mat *X, const fo_side *sid
     if (need > fo::kStaticWsBytes) return FO_ERR_STATIC_LIMIT;
     void *ws = fo::static_ws_address();
     if (!ws) return FO_ERR_CUDA;
+    // never compiles or loads a kernel: a chain specialised earlier is reused, any other
+    // one runs through the built-in code
     return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, false, out, ws,
-                        fo::kStaticWsBytes, stream);
+                        fo::kStaticWsBytes, stream, false);
 }
 
 size_t fused_cell_static_limit_bytes(void) { return fo::kStaticWsBytes; }
@@ -600,7 +604,7 @@ int fused_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int
                size_t ws_bytes, void *stream)
 {
     return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, false, out, ws,
-                        ws_bytes, stream);
+                        ws_bytes, stream, true);
 }
 
 int fused_magg(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
@@ -608,7 +612,7 @@ int fused_magg(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int
                void *stream)
 {
     return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, FO_CELL_FULL_AGG, true, out,
-                        ws, ws_bytes, stream);
+                        ws, ws_bytes, stream, true);
 }
 
 }  // extern "C"

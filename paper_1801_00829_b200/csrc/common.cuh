@@ -10,6 +10,7 @@
 #include <string.h>
 
 #include "../../include/fusedops.h"
+#include "../../include/fusedops_tools.h"
 #endif
 
 namespace fo {

@@ -9,6 +9,7 @@
 #include <dlfcn.h>
 #include <stdio.h>
 
+#include <atomic>
 #include <mutex>
 #include <string>
 #include <unordered_map>
@@ -40,6 +41,8 @@ typedef int (*cuModuleLoadData_t)(CUmodule *, const void *);
 typedef int (*cuModuleGetFunction_t)(CUfunction *, CUmodule, const char *);
 typedef int (*cuLaunchKernel_t)(CUfunction, unsigned, unsigned, unsigned, unsigned, unsigned, unsigned,
                                 unsigned, void *, void **, void **);
+typedef struct CUctx_st *CUcontext;
+typedef int (*cuCtxGetCurrent_t)(CUcontext *);
 
 struct Api {
     bool nvrtc_ok = false, driver_ok = false;
@@ -51,6 +54,7 @@ struct Api {
     cuModuleLoadData_t load = nullptr;
     cuModuleGetFunction_t getfn = nullptr;
     cuLaunchKernel_t launch = nullptr;
+    cuCtxGetCurrent_t ctx = nullptr;
 };
 
 void *open_first(const char *const *names)
@@ -84,16 +88,21 @@ Api &api()
             a.load = (cuModuleLoadData_t)dlsym(h, "cuModuleLoadData");
             a.getfn = (cuModuleGetFunction_t)dlsym(h, "cuModuleGetFunction");
             a.launch = (cuLaunchKernel_t)dlsym(h, "cuLaunchKernel");
-            a.driver_ok = a.load && a.getfn && a.launch;
+            a.ctx = (cuCtxGetCurrent_t)dlsym(h, "cuCtxGetCurrent");
+            a.driver_ok = a.load && a.getfn && a.launch && a.ctx;
         }
     });
     return a;
 }
 
 std::mutex g_mutex;
-std::unordered_map<std::string, CUfunction> g_cache;      // key: device + translated program
-bool g_enabled = true;
+// key: context + translated program.  A function handle belongs to the context it
+// was loaded in, so a new context (after a device reset, say) starts empty.
+std::unordered_map<std::string, CUfunction> g_cache;
+std::unordered_map<std::string, int> g_load_failures;     // module loads that failed, per key
+std::atomic<int> g_mode{1};                               // 0 off, 1 compile at first use, 2 prepared kernels only
 int g_compiled = 0, g_launches = 0, g_failures = 0;
+constexpr int kLoadRetries = 3;                           // a failed load (out of memory, say) is tried again this often
 std::string g_last_log;
 
 // ---- source generation
@@ -185,10 +194,10 @@ std::string generate_source(const DevChain &ch, bool store)
     return s;
 }
 
-std::string cache_key(const DevChain &ch, bool store, int dev)
+std::string cache_key(const DevChain &ch, bool store, CUcontext ctx)
 {
     std::string k;
-    k.append((const char *)&dev, sizeof(dev));
+    k.append((const char *)&ctx, sizeof(ctx));
     k.push_back(store ? 1 : 0);
     k.append((const char *)&ch.n_ops, sizeof(int32_t));
     k.append((const char *)&ch.n_out, sizeof(int32_t));
@@ -230,55 +239,110 @@ std::vector<char> compile(const std::string &src, const std::string &arch)
 
 }  // namespace
 
-bool jit_enabled() { return g_enabled; }
+bool jit_enabled() { return g_mode.load() != 0; }
 
-int jit_launch_flat(const DevChain &ch, const CellParams &p, bool store, int grid, cudaStream_t st)
+namespace {
+
+// The cached kernel of (ch, store) in the current context; compiles and loads it
+// first if `may_compile` and it is not there yet.  nullptr if there is none.
+// *status (optional): FO_OK, FO_ERR_UNSUPPORTED (no compiler / driver library /
+// context) or FO_ERR_CHAIN (the compilation or the load failed).
+CUfunction find_kernel(const DevChain &ch, bool store, bool may_compile, std::string *key_out, int *status)
 {
     Api &a = api();
-    if (!g_enabled || !a.nvrtc_ok || !a.driver_ok) return kJitUnavailable;
+    if (status) *status = FO_ERR_UNSUPPORTED;
+    if (!a.nvrtc_ok || !a.driver_ok) return nullptr;
     int dev = 0, major = 0, minor = 0;
+    // the runtime calls make sure the primary context exists and is current
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess)
-        return kJitUnavailable;
-    CUfunction fn = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        const std::string key = cache_key(ch, store, dev);
-        auto it = g_cache.find(key);
-        if (it != g_cache.end()) {
-            fn = it->second;
-        } else {
-            char arch[32];
-            snprintf(arch, sizeof(arch), "sm_%d%d%s", major, minor, major >= 9 ? "a" : "");
-            const std::vector<char> cubin = compile(generate_source(ch, store), arch);
-            CUmodule mod = nullptr;
-            if (!cubin.empty() && a.load(&mod, cubin.data()) == 0 && a.getfn(&fn, mod, "fo_jit_flat") == 0) {
-                ++g_compiled;
-            } else {
-                fn = nullptr;
-                ++g_failures;
-            }
-            g_cache.emplace(key, fn);         // a failed chain is not compiled again
-        }
-        if (fn) ++g_launches;
+        return nullptr;
+    CUcontext ctx = nullptr;
+    if (a.ctx(&ctx) != 0 || !ctx) {
+        if (!may_compile || cudaFree(nullptr) != cudaSuccess || a.ctx(&ctx) != 0 || !ctx) return nullptr;
     }
+    CUfunction fn = nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const std::string key = cache_key(ch, store, ctx);
+    if (key_out) *key_out = key;
+    auto it = g_cache.find(key);
+    if (it != g_cache.end()) {
+        if (status) *status = it->second ? FO_OK : FO_ERR_CHAIN;
+        return it->second;
+    }
+    if (!may_compile) return nullptr;
+    if (status) *status = FO_ERR_CHAIN;
+    auto lf = g_load_failures.find(key);
+    if (lf != g_load_failures.end() && lf->second >= kLoadRetries) return nullptr;
+    char arch[32];
+    snprintf(arch, sizeof(arch), "sm_%d%d%s", major, minor, major >= 9 ? "a" : "");
+    const std::vector<char> cubin = compile(generate_source(ch, store), arch);
+    if (cubin.empty()) {
+        ++g_failures;
+        g_cache.emplace(key, nullptr);        // the same source fails the same way: not compiled again
+        return nullptr;
+    }
+    CUmodule mod = nullptr;
+    if (a.load(&mod, cubin.data()) != 0 || a.getfn(&fn, mod, "fo_jit_flat") != 0) {
+        ++g_failures;
+        ++g_load_failures[key];               // may be transient: tried again a few times, then given up
+        return nullptr;
+    }
+    ++g_compiled;
+    g_cache.emplace(key, fn);
+    if (status) *status = FO_OK;
+    return fn;
+}
+
+}  // namespace
+
+int jit_launch_flat(const DevChain &ch, const CellParams &p, bool store, int grid, cudaStream_t st,
+                    bool may_compile)
+{
+    const int mode = g_mode.load();
+    if (mode == 0) return kJitUnavailable;
+    std::string key;
+    CUfunction fn = find_kernel(ch, store, may_compile && mode == 1, &key, nullptr);
     if (!fn) return kJitUnavailable;
     void *args[2] = {(void *)&ch, (void *)&p};
-    const int rc = a.launch(fn, (unsigned)grid, 1, 1, kThreads, 1, 1, 0, (void *)st, args, nullptr);
-    return rc == 0 ? FO_OK : cuda_fail(cudaErrorLaunchFailure);
+    const int rc = api().launch(fn, (unsigned)grid, 1, 1, kThreads, 1, 1, 0, (void *)st, args, nullptr);
+    if (rc == 0) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ++g_launches;
+        return FO_OK;
+    }
+    // CUDA_ERROR_INVALID_CONTEXT (201), CUDA_ERROR_INVALID_HANDLE (400), CUDA_ERROR_NOT_FOUND (500):
+    // the handle no longer belongs to a live context - forget it and let the caller interpret
+    if (rc == 201 || rc == 400 || rc == 500) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        g_cache.erase(key);
+        return kJitUnavailable;
+    }
+    return cuda_fail((cudaError_t)rc);        // driver and runtime share their error numbers
 }
 
 }  // namespace fo
 
 extern "C" {
 
-int fo_set_jit(int on)
+int fo_set_jit(int mode)
 {
-    std::lock_guard<std::mutex> lock(fo::g_mutex);
-    const int prev = fo::g_enabled ? 1 : 0;
-    fo::g_enabled = on != 0;
-    return prev;
+    if (mode < 0 || mode > 2) mode = 1;
+    return fo::g_mode.exchange(mode);
+}
+
+int fo_jit_prepare(const fo_chain *chain, int n_sides, int n_scalars, int store)
+{
+    using namespace fo;
+    double scalars[FO_MAX_SCALARS] = {0};
+    DevChain ch;
+    const int rc = translate_chain(chain, kUseCell, n_sides, scalars, n_scalars, 1, FO_MAX_OUT, &ch);
+    if (rc != FO_OK) return rc;
+    if (store && ch.n_out != 1) return FO_ERR_CHAIN;
+    int status = FO_ERR_UNSUPPORTED;
+    find_kernel(ch, store != 0, true, nullptr, &status);
+    return status;
 }
 
 int fo_jit_stats(int *compiled, int *launches, int *failures)

@@ -9,10 +9,14 @@ constexpr int kJitUnavailable = 1;     // not an error: the caller uses the inte
 
 bool jit_enabled();
 
-// Launches the flat streaming kernel specialised for `ch` (compiling and caching it
-// on first use).  Returns FO_OK if launched, kJitUnavailable if there is no
-// specialised kernel (NVRTC or the driver library missing, switched off, or the
-// compilation failed), FO_ERR_CUDA if the launch itself failed.
-int jit_launch_flat(const DevChain &ch, const CellParams &p, bool store, int grid, cudaStream_t st);
+// Launches the flat streaming kernel specialised for `ch`.  With `may_compile` (and
+// the process-wide mode "compile at first use") a chain seen for the first time is
+// compiled, loaded and cached; otherwise only an already cached kernel is used and
+// nothing is compiled, loaded or allocated.  Returns FO_OK if launched,
+// kJitUnavailable if there is no specialised kernel (not cached and compiling not
+// allowed, NVRTC or the driver library missing, switched off, or the compilation
+// failed), FO_ERR_CUDA if the launch itself failed.
+int jit_launch_flat(const DevChain &ch, const CellParams &p, bool store, int grid, cudaStream_t st,
+                    bool may_compile);
 
 }  // namespace fo

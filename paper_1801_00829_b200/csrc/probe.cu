@@ -7,7 +7,7 @@
 #include <stdint.h>
 
 #include "common.cuh"
-#include "fusedops.h"
+#include "fusedops_tools.h"
 
 namespace fo {
 namespace {

@@ -1,8 +1,9 @@
 """Host-side checks of the C ABI that need no GPU: the library builds, loads and
-exports every function include/fusedops.h declares; workspace sizes are plain
+exports every function the headers under include/ declare; workspace sizes are plain
 arithmetic; invalid arguments are refused with the documented status before
 anything touches the device."""
 import ctypes as C
+import glob
 import os
 import re
 
@@ -19,9 +20,11 @@ def lib():
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "fusedops.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"^(?:int|size_t|const char \*)\s*(\w+)\s*\(", text, flags=re.M)
+    names = []
+    for header in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))):
+        text = open(header).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names += re.findall(r"^(?:int|size_t|const char \*)\s*(\w+)\s*\(", text, flags=re.M)
     return names
 
 

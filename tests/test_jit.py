@@ -101,3 +101,30 @@ def test_jit_kernel_is_reused_for_other_constants_and_can_be_switched_off():
     finally:
         fo.set_jit(True)
     assert fo.jit_stats()[2] == launches and c == b                  # interpreter, same bits
+
+
+@pytest.mark.gpu
+def test_prepared_mode_never_compiles_inside_a_call():
+    rows, cols = 257, 130
+    X = datagen.normal(63, 0, rows * cols).reshape(rows, cols)
+    Xd = to_dev(X)
+    if not fo.jit_stats()[0]:
+        pytest.skip("NVRTC or the driver library is not usable here")
+    fresh = [("mul", "t0", "a", 1.5), ("max", "t1", "t0", "a"), ("sub", "t2", "t1", 0.125)]
+    ref = oracle.cell(fresh, "t2", X)
+    scale = np.abs(X).sum() * 1.5 + 0.125 * X.size
+    old = fo.set_jit(fo.binding.JIT_PREPARED)
+    try:
+        compiled, launches = fo.jit_stats()[1:3]
+        a = fo.fused_cell(fresh, "t2", Xd).item()                    # not prepared: the interpreter runs
+        assert fo.jit_stats()[1:3] == (compiled, launches)
+        fo.jit_prepare(fresh, "t2")
+        assert fo.jit_stats()[1] == compiled + 1
+        fo.jit_prepare(fresh, "t2")                                  # cached: nothing compiled again
+        assert fo.jit_stats()[1] == compiled + 1
+        b = fo.fused_cell(fresh, "t2", Xd).item()                    # the prepared kernel is picked up
+        assert fo.jit_stats()[1:3] == (compiled + 1, launches + 1)
+    finally:
+        fo.set_jit(old)
+    assert a == b
+    assert_close([a], [ref], absscale=scale)

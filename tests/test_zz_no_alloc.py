@@ -6,9 +6,11 @@ that share that one array, whether this file runs alone or after every other tes
 """
 import ctypes as C
 
+import numpy as np
 import pytest
 
 import datagen
+import oracle
 from util import assert_close, to_dev
 
 XYZ = [("mul", "t0", "a", "side0"), ("mul", "t1", "t0", "side1")]
@@ -26,6 +28,8 @@ def test_static_scratch_matches_workspace_entry_point(agg, chain, output):
     w = datagen.cell_workload(rows, cols, seed=51)
     X, sides = to_dev(w["X"]), [("cell", to_dev(w["Y"])), ("cell", to_dev(w["Z"]))]
     ref = fo.fused_cell(chain, output, X, sides, agg=agg).cpu().numpy()
+    assert_close(ref, oracle.cell(chain, output, w["X"], [("cell", w["Y"]), ("cell", w["Z"])], agg=agg),
+                 what="workspace entry point %s" % agg)
     out = torch.empty(ref.shape, dtype=torch.float64, device="cuda")   # the caller owns the output
     for call in range(2):                                      # two calls in a row share the scratch
         out.fill_(float("nan"))
@@ -41,6 +45,48 @@ def test_static_scratch_matches_workspace_entry_point(agg, chain, output):
     assert g2.tobytes() == r2.tobytes()
     fo.fused_cell_static(chain, output, X, sides, agg=agg, out=out)
     assert out.cpu().numpy().tobytes() == ref.tobytes()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("agg", ["full", "none"])
+def test_static_entry_point_first_with_a_fresh_chain_compiles_and_allocates_nothing(agg):
+    """The no-allocation promise, checked where it is hardest to keep: a chain that
+    nothing has specialised yet, over contiguous inputs, is the case in which
+    fused_cell would compile and load a kernel.  The static entry point must not:
+    the compile counter and the free device memory stay as they were, and the
+    result is the checker's."""
+    import torch
+    import paper_1801_00829_b200 as fo
+    fo.load_library()
+    rows, cols = 1029, 515
+    w = datagen.cell_workload(rows, cols, seed=53)
+    X, sides = to_dev(w["X"]), [("cell", to_dev(w["Y"])), ("cell", to_dev(w["Z"]))]
+    # constants differ per variant so that each run meets a program nobody compiled
+    k = {"full": 0.375, "none": 0.625}[agg]
+    fresh = [("add", "t0", "a", "side1"), ("min", "t1", "t0", "side0"), ("mul", "t2", "t1", k),
+             ("sub", "t3", "t2", "a")] + ([("neg", "t3", "t3")] if agg == "none" else [])
+    shape = () if agg == "full" else (rows, cols)
+    out = torch.empty(shape, dtype=torch.float64, device="cuda")
+    fo.fused_cell_static([("sq", "t0", "a")], "t0", X, agg="full")   # the one-time address lookup
+    torch.cuda.synchronize()
+    compiled = fo.jit_stats()[1]
+    free0 = torch.cuda.mem_get_info()[0]
+    fo.fused_cell_static(fresh, "t3", X, sides, agg=agg, out=out)
+    torch.cuda.synchronize()
+    assert fo.jit_stats()[1] == compiled, "the static entry point compiled a kernel"
+    assert torch.cuda.mem_get_info()[0] == free0, "device memory was allocated"
+    sides_h = [("cell", w["Y"]), ("cell", w["Z"])]
+    ref = oracle.cell(fresh, "t3", w["X"], sides_h, agg=agg)
+    if agg == "full":
+        scale = np.abs(w["X"]).sum() * 2 + np.abs(w["Y"]).sum() + np.abs(w["Z"]).sum()
+        assert_close([out.item()], [ref], absscale=scale, what="static, fresh chain")
+    else:
+        assert_close(out.cpu().numpy(), ref, what="static, fresh chain")
+    # after fused_cell has specialised the chain the static call reuses that kernel: same bits
+    first = out.cpu().numpy().copy()
+    again = fo.fused_cell(fresh, "t3", X, sides, agg=agg).cpu().numpy()
+    fo.fused_cell_static(fresh, "t3", X, sides, agg=agg, out=out)
+    assert out.cpu().numpy().tobytes() == again.tobytes() == first.tobytes()
 
 
 @pytest.mark.gpu
