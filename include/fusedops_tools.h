@@ -22,6 +22,26 @@ extern "C" {
  * (process-wide; for tests and measurements).  Returns the previous setting. */
 int fo_set_force_interpreter(int on);
 
+/* Measurement knobs (process-wide).  The library picks kernel shapes and
+ * schedules from the inputs; a knob overrides one such choice so that tests can
+ * reach every compiled kernel and measurements can compare them.  Results stay
+ * within the documented tolerance whatever the knobs say; only speed, and the
+ * order of partial sums, change.  value == NULL clears a knob.  Returns FO_OK,
+ * FO_ERR_UNSUPPORTED for an unknown name, FO_ERR_SHAPE for a value of 48 or
+ * more characters.  Names:
+ *   cell.ctas_per_sm  1..8   CTAs per SM of the streaming Cell / MAgg kernel
+ *   row.dense_shape   "c,w,r" chunks per lane, warps per group, rows per stage of the dense Row kernel
+ *   row.narrow        0      dense rows of at most 32 columns through the warp-per-row kernel
+ *   b1.mma            0 | 1  fused_row_b1: multiply-add kernel / tensor-core kernel
+ *   b1.shape, b1.mma_shape   compiled shapes of those two kernels ("p,r,kl" / "w,kb")
+ *   b1.narrow         0      fused_row_b1 without the thread-per-row kernel
+ *   outer.kernel      "bulk" | "pipe" | "direct" | "dense"   schedule of fused_outer
+ *   outer.depth, outer.warps   ring depth and warps per CTA of the bulk-copy Outer kernel
+ *   outer.hints       0 | 1  L2 eviction hints on the Outer kernel's copies
+ *   csr.variant       variant number of the CSR Row kernel
+ *   cell.stamps       1      Cell kernel records time stamps in its workspace tail */
+int fo_tune(const char *name, const char *value);
+
 /* Generates and compiles (for sm_100a, without loading or launching: no GPU
  * needed) the run-time specialised kernel of a Cell chain; FO_OK, a chain error,
  * FO_ERR_UNSUPPORTED without NVRTC; the compiler log is copied to `log`. */

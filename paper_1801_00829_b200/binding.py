@@ -83,7 +83,7 @@ EXPORTS = [
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
     "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_compile_check",
-    "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_fp64_fma", "fo_chain_describe",
+    "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_fp64_fma", "fo_chain_describe", "fo_tune",
 ]
 
 _lib = None
@@ -135,6 +135,8 @@ def load_library(path=None):
         ip = C.POINTER(C.c_int)
         lib.fo_jit_stats.argtypes = [ip, ip, ip]
         lib.fo_jit_stats.restype = C.c_int
+        lib.fo_tune.argtypes = [C.c_char_p, C.c_char_p]
+        lib.fo_tune.restype = C.c_int
         lib.fo_jit_prepare.argtypes = [chain_p, i32, i32, i32]
         lib.fo_jit_prepare.restype = C.c_int
         lib.fo_jit_compile_check.argtypes = [chain_p, i32, i32, i32, C.c_char_p, sz]
@@ -351,6 +353,11 @@ def force_interpreter(on):
     """Route every Cell / MAgg chain through the interpreter (True) or let known
     chains use their compile-time specialisation (False).  Returns the old setting."""
     return bool(load_library().fo_set_force_interpreter(1 if on else 0))
+
+
+def tune(name, value=None):
+    """Sets (or with value None clears) a measurement knob of the library; see fo_tune."""
+    _check(load_library().fo_tune(name.encode(), None if value is None else str(value).encode()), "fo_tune")
 
 
 JIT_OFF, JIT_FIRST_USE, JIT_PREPARED = 0, 1, 2

@@ -1,8 +1,12 @@
 // Host side of the operator chain: validation and translation of the ABI's
 // fo_chain into the flat register program the kernels run, plus small host
 // utilities shared by the entry points.
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
 #include <string>
 
 #include "common.cuh"
@@ -232,9 +236,65 @@ int sm_count()
     return cached[dev];
 }
 
+// ---- measurement knobs (fo_tune): a small table of named strings.  Kernels read
+// a knob at launch; a knob that was never set costs one relaxed atomic load.
+namespace {
+struct Knob {
+    const char *name;
+    char value[48];
+    bool set;
+};
+Knob g_knobs[] = {
+    {"cell.ctas_per_sm", "", false}, {"row.dense_shape", "", false}, {"row.narrow", "", false},
+    {"b1.shape", "", false},         {"b1.mma_shape", "", false},    {"b1.narrow", "", false},
+    {"b1.mma", "", false},           {"outer.kernel", "", false},    {"outer.depth", "", false},
+    {"outer.warps", "", false},      {"outer.hints", "", false},     {"outer.dense", "", false},
+    {"csr.variant", "", false},      {"cell.stamps", "", false},
+};
+std::mutex g_knob_mutex;
+std::atomic<int> g_knobs_set{0};
+}  // namespace
+
+bool tune_get(const char *name, char *value, size_t cap)
+{
+    if (g_knobs_set.load(std::memory_order_relaxed) == 0) return false;
+    std::lock_guard<std::mutex> lock(g_knob_mutex);
+    for (Knob &k : g_knobs)
+        if (k.set && strcmp(k.name, name) == 0) {
+            snprintf(value, cap, "%s", k.value);
+            return true;
+        }
+    return false;
+}
+
+int tune_int(const char *name, int fallback)
+{
+    char v[48];
+    if (!tune_get(name, v, sizeof(v))) return fallback;
+    char *end = nullptr;
+    const long x = strtol(v, &end, 10);
+    return end != v ? (int)x : fallback;
+}
+
 }  // namespace fo
 
 extern "C" {
+
+int fo_tune(const char *name, const char *value)
+{
+    if (!name) return FO_ERR_NULL;
+    std::lock_guard<std::mutex> lock(fo::g_knob_mutex);
+    for (fo::Knob &k : fo::g_knobs)
+        if (strcmp(k.name, name) == 0) {
+            if (value && strlen(value) >= sizeof(k.value)) return FO_ERR_SHAPE;
+            const bool was = k.set;
+            k.set = value != nullptr;
+            if (value) snprintf(k.value, sizeof(k.value), "%s", value);
+            fo::g_knobs_set.fetch_add((k.set ? 1 : 0) - (was ? 1 : 0));
+            return FO_OK;
+        }
+    return FO_ERR_UNSUPPORTED;
+}
 
 const char *fo_status_string(int status)
 {

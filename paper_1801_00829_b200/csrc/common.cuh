@@ -92,6 +92,10 @@ int chain_expression(const DevChain &ch, int k, char *text, size_t cap);
 // the general interpreter (cell.cu).
 bool force_interpreter();
 
+// Measurement knobs set through fo_tune (fusedops_tools.h): false / `fallback` unless set.
+bool tune_get(const char *name, char *value, size_t cap);
+int tune_int(const char *name, int fallback);
+
 int check_workspace(const void *ws, size_t ws_bytes, size_t need);
 int cuda_fail(cudaError_t e);
 int sm_count();

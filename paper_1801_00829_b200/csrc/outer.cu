@@ -10,6 +10,8 @@
 #include <stdio.h>
 #include <stdlib.h>
 
+#include <atomic>
+
 #include "chain.cuh"
 
 namespace fo {
@@ -52,6 +54,19 @@ __device__ __forceinline__ double2 ld_pair_cached(const double *row, int col, in
     return make_double2(0.0, 0.0);
 }
 
+// A chain without an inline form runs through the interpreter, out of line: its
+// register file would otherwise be counted against every kernel's main loop.
+__device__ __noinline__ double outer_chain_generic(const DevChain &ch, double a, double d)
+{
+    RegFile<kRegs, 1> f;
+    f.r[0][0] = a;
+    f.r[1][0] = d;
+    run_chain<kRegs, 1>(ch, f);
+    double o[1];
+    operand<kRegs, 1>(ch, f, ch.out[0], o);
+    return o[0];
+}
+
 __device__ __forceinline__ double outer_chain(const DevChain &ch, int kind, int kc, double a, double d)
 {
     if (kind == kOuterWsloss) {
@@ -62,22 +77,27 @@ __device__ __forceinline__ double outer_chain(const DevChain &ch, int kind, int 
     }
     if (kind == kOuterXlogd) return a * slow_log(d + ch.consts[kc]);
     if (kind == kOuterMaskDot) return (a != 0.0 ? 1.0 : 0.0) * d;      // (X != 0) * (U V^T), Eq. 1
-    RegFile<kRegs, 1> f;
-    f.r[0][0] = a;
-    f.r[1][0] = d;
-    run_chain<kRegs, 1>(ch, f);
-    double o[1];
-    operand<kRegs, 1>(ch, f, ch.out[0], o);
-    return o[0];
+    return outer_chain_generic(ch, a, d);
 }
 
-// First row r in [0, rows] with rowptr[r] >= target.
-__device__ __forceinline__ long long lower_row(const int *rowptr, long long rows, long long target)
+// First row r in [0, rows] with rowptr[r] >= target, found by the 32 lanes of a
+// warp together: 32 probes a round.
+__device__ __forceinline__ long long lower_row_warp(const int *rowptr, long long rows, long long target,
+                                                    int lane)
 {
     long long lo = 0, hi = rows;
     while (lo < hi) {
-        const long long mid = (lo + hi) >> 1;
-        if (__ldg(rowptr + mid) < target) lo = mid + 1; else hi = mid;
+        const long long step = (hi - lo + 31) / 32;
+        const long long idx = lo + step * lane;
+        const bool below = idx < hi && __ldg(rowptr + idx) < target;     // true for a prefix of the lanes
+        const int c = __popc(__ballot_sync(0xffffffffu, below));
+        if (c == 0) {
+            hi = lo;
+        } else {
+            const long long nhi = lo + step * c;
+            lo = lo + step * (c - 1) + 1;
+            if (nhi < hi) hi = nhi;
+        }
     }
     return lo;
 }
@@ -98,10 +118,11 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
     __shared__ unsigned int s_flag;
     __shared__ long long s_rows[2];
 
-    if (threadIdx.x == 0) {
-        const long long G = gridDim.x, b = blockIdx.x;
-        s_rows[0] = (b == 0) ? 0 : lower_row(p.rowptr, p.rows, (p.nnz * b) / G);
-        s_rows[1] = (b == G - 1) ? p.rows : lower_row(p.rowptr, p.rows, (p.nnz * (b + 1)) / G);
+    if (threadIdx.x < 64) {       // warps 0 and 1 find the CTA's first and last row, 32 probes a round
+        const long long G = gridDim.x, b = blockIdx.x + (threadIdx.x >> 5);
+        const long long r = (b == 0) ? 0 : (b == G) ? p.rows
+                            : lower_row_warp(p.rowptr, p.rows, (p.nnz * b) / G, threadIdx.x & 31);
+        if ((threadIdx.x & 31) == 0) s_rows[threadIdx.x >> 5] = r;
     }
     __syncthreads();
     const long long row_lo = s_rows[0], row_hi = s_rows[1];
@@ -229,163 +250,12 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
     }
 }
 
-// ------------------------------------------------------------------ staged
-// The same work with the V rows landing in shared memory first.  A warp owns a
-// buffer of 16 rows; for half a chunk (16 stored cells) it issues all the 16-byte
-// asynchronous copies of the 16 V rows at once, waits for them, and only then
-// forms the dot products from shared memory.  The copies need no registers, so a
-// warp keeps 16 rows (12.8 KB at rank 100) in flight instead of 8, and the right_mm
-// variant reuses the staged rows instead of gathering them twice.
-// Needs 16-byte aligned factor rows and an even rank (a row piece is one 16-byte copy).
 constexpr int kStageRows = 16;
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 {
     const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
-}
-
-template <int NK2, int AGG>
-__global__ void __launch_bounds__(kThreads, 2)
-outer_staged_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
-{
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    __shared__ double s_red[32];
-    __shared__ unsigned int s_flag;
-    __shared__ long long s_rows[2];
-
-    if (threadIdx.x == 0) {
-        const long long G = gridDim.x, b = blockIdx.x;
-        s_rows[0] = (b == 0) ? 0 : lower_row(p.rowptr, p.rows, (p.nnz * b) / G);
-        s_rows[1] = (b == G - 1) ? p.rows : lower_row(p.rowptr, p.rows, (p.nnz * (b + 1)) / G);
-    }
-    __syncthreads();
-    const long long row_lo = s_rows[0], row_hi = s_rows[1];
-
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int l8 = lane & 7, grp = lane >> 3;
-    const unsigned full = 0xffffffffu;
-    const int rank = p.rank;                       // even
-    double *buf = reinterpret_cast<double *>(smem_raw) + (size_t)warp * kStageRows * rank;
-    double acc = 0.0;
-
-    for (long long row = row_lo + warp; row < row_hi; row += kThreads / 32) {
-        const int beg = __ldg(p.rowptr + row), end = __ldg(p.rowptr + row + 1);
-        double2 u[NK2], racc[NK2];
-        const double *urow = p.U + row * p.ldu;
-#pragma unroll
-        for (int c = 0; c < NK2; ++c) {
-            const int col = 16 * c + 2 * l8;
-            u[c] = (beg < end && col < rank) ? __ldg(reinterpret_cast<const double2 *>(urow + col))
-                                             : make_double2(0.0, 0.0);
-            racc[c] = make_double2(0.0, 0.0);
-        }
-        for (int c0 = beg; c0 < end; c0 += 32) {
-            const int cnt = (end - c0 < 32) ? end - c0 : 32;
-            const bool valid = lane < cnt;
-            const int jmine = valid ? __ldg(p.colidx + c0 + lane) : 0;
-            const double amine = valid ? __ldg(p.vals + c0 + lane) : 0.0;
-            double dmine = 0.0, wmine = 0.0;
-            for (int h = 0; h < 2 && 16 * h < cnt; ++h) {
-                // land the V rows of cells 16h .. 16h+15: group grp takes cells 16h + 4i + grp
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int sidx = 16 * h + 4 * i + grp;
-                    const int j = __shfl_sync(full, jmine, sidx);
-                    if (sidx < cnt) {
-                        const double *vj = p.V + (long long)j * p.ldv;
-                        double *dst = buf + (4 * i + grp) * rank;
-#pragma unroll
-                        for (int c = 0; c < NK2; ++c) {
-                            const int col = 16 * c + 2 * l8;
-                            if (col < rank) cp_async16(dst + col, vj + col);
-                        }
-                    }
-                }
-                asm volatile("cp.async.commit_group;" ::: "memory");
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int sidx = 16 * h + 4 * i + grp;
-                    const double *src = buf + (4 * i + grp) * rank;
-                    double d = 0.0;
-                    if (sidx < cnt) {
-#pragma unroll
-                        for (int c = 0; c < NK2; ++c) {
-                            const int col = 16 * c + 2 * l8;
-                            if (col < rank) {
-                                const double2 x = *reinterpret_cast<const double2 *>(src + col);
-                                d = fma(u[c].x, x.x, d);
-                                d = fma(u[c].y, x.y, d);
-                            }
-                        }
-                    }
-                    d += __shfl_xor_sync(full, d, 4);
-                    d += __shfl_xor_sync(full, d, 2);
-                    d += __shfl_xor_sync(full, d, 1);
-                    // cell s of the chunk was handled by group (s & 3) in trip (s >> 2)
-                    const double all = __shfl_sync(full, d, (lane & 3) * 8);
-                    if ((lane >> 2) == 4 * h + i) dmine = all;
-                }
-                if (AGG == kOutRight) {
-                    // the chain's values for this half, then O_i += w * V_j from the staged rows
-                    const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
-                    if ((lane >> 4) == h) wmine = w;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int sidx = 16 * h + 4 * i + grp;
-                        const double ww = __shfl_sync(full, w, sidx);
-                        const double *src = buf + (4 * i + grp) * rank;
-                        if (sidx < cnt) {
-#pragma unroll
-                            for (int c = 0; c < NK2; ++c) {
-                                const int col = 16 * c + 2 * l8;
-                                if (col < rank) {
-                                    const double2 x = *reinterpret_cast<const double2 *>(src + col);
-                                    racc[c].x = fma(ww, x.x, racc[c].x);
-                                    racc[c].y = fma(ww, x.y, racc[c].y);
-                                }
-                            }
-                        }
-                    }
-                }
-                __syncwarp();          // the buffer is overwritten by the next half
-            }
-            if (AGG != kOutRight) {
-                const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
-                if (AGG == kOutFull) {
-                    if (valid) acc += w;
-                } else {
-                    if (valid) p.out[c0 + lane] = w;
-                }
-            }
-            (void)wmine;
-        }
-        if (AGG == kOutRight) {
-            // the four groups hold partial rows: add them in a fixed order
-#pragma unroll
-            for (int c = 0; c < NK2; ++c) {
-                racc[c].x += __shfl_xor_sync(full, racc[c].x, 8);
-                racc[c].y += __shfl_xor_sync(full, racc[c].y, 8);
-                racc[c].x += __shfl_xor_sync(full, racc[c].x, 16);
-                racc[c].y += __shfl_xor_sync(full, racc[c].y, 16);
-                const int col = 16 * c + 2 * l8;
-                if (grp == 0) {
-                    if (col < rank) p.out[row * rank + col] = racc[c].x;
-                    if (col + 1 < rank) p.out[row * rank + col + 1] = racc[c].y;
-                }
-            }
-        }
-    }
-
-    if (AGG == kOutFull) {
-        double v1[1] = {acc};
-        block_sum<1>(v1, s_red);
-        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
-        if (publish_and_is_last(p.head, &s_flag))
-            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
-    }
 }
 
 // ---------------------------------------------------------------- pipelined
@@ -406,10 +276,11 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
     __shared__ unsigned int s_flag;
     __shared__ long long s_rows[2];
 
-    if (threadIdx.x == 0) {
-        const long long G = gridDim.x, b = blockIdx.x;
-        s_rows[0] = (b == 0) ? 0 : lower_row(p.rowptr, p.rows, (p.nnz * b) / G);
-        s_rows[1] = (b == G - 1) ? p.rows : lower_row(p.rowptr, p.rows, (p.nnz * (b + 1)) / G);
+    if (threadIdx.x < 64) {       // warps 0 and 1 find the CTA's first and last row, 32 probes a round
+        const long long G = gridDim.x, b = blockIdx.x + (threadIdx.x >> 5);
+        const long long r = (b == 0) ? 0 : (b == G) ? p.rows
+                            : lower_row_warp(p.rowptr, p.rows, (p.nnz * b) / G, threadIdx.x & 31);
+        if ((threadIdx.x & 31) == 0) s_rows[threadIdx.x >> 5] = r;
     }
     __syncthreads();
     const long long row_lo = s_rows[0], row_hi = s_rows[1];
@@ -551,6 +422,183 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
     }
 }
 
+// -------------------------------------------------------------------- dense
+// full_agg / no_agg for a main input that stores a large share of its cells
+// (Section 5.2, "Outer-Product Operations": the dense end of the sparsity sweep).
+// Gathering a factor row per stored cell then costs more than forming U V^T
+// outright, so this schedule forms it, tile by tile, and never writes it out:
+// a CTA takes a block of 64 rows (U rows in shared memory) and sweeps 32-column
+// tiles of V; the 64 x 32 tile of dot products comes from the fp64 tensor-core
+// instruction (mma.sync m8n8k4, 8 warps of 16 x 16), goes to shared memory, and
+// the stored cells of the tile - a contiguous piece of each row of the CSR
+// matrix, found with a per-row cursor - pick their dot product there and run the
+// chain.  The next V tile is copied in while the cells are evaluated, and two
+// CTAs share an SM, so one's cell phase (waiting on the X stream) runs under the
+// other's tensor-core phase.  Work items are (row block, column range) pairs
+// dealt round-robin to the resident CTAs.
+constexpr int kDenseBM = 64, kDenseBN = 32;
+
+__host__ __device__ inline int dense_ld(int rank)
+{
+    int ld = (rank + 3) & ~3;            // whole steps of 4
+    while ((ld & 7) != 4) ld += 4;       // 4 (mod 8): the 8 x 4 fragment reads touch every bank once
+    return ld;
+}
+__host__ __device__ inline size_t dense_smem_bytes(int rank)
+{
+    return (size_t)((kDenseBM + kDenseBN) * dense_ld(rank) + kDenseBM * (kDenseBN + 2)) * sizeof(double) +
+           2 * kDenseBM * sizeof(int);
+}
+
+__device__ __forceinline__ void dmma_8x8x4(double &c0, double &c1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
+
+struct DenseSplit {
+    int row_blocks, col_splits, tiles_per_split, pad;
+};
+
+template <int AGG>
+__global__ void __launch_bounds__(kThreads, 2)
+outer_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p,
+                   const __grid_constant__ DenseSplit sp)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ double s_red[32];
+    __shared__ unsigned int s_flag;
+
+    const int rank = p.rank, ld = dense_ld(rank);
+    constexpr int PLD = kDenseBN + 2;
+    double *Us = reinterpret_cast<double *>(smem_raw);            // 64 x ld
+    double *Vs = Us + kDenseBM * ld;                              // 32 x ld
+    double *Ps = Vs + kDenseBN * ld;                              // 64 x 34
+    int *cur = reinterpret_cast<int *>(Ps + kDenseBM * PLD);
+    int *rend = cur + kDenseBM;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;                        // fragment coordinates
+    const int wm = warp >> 1, wn = warp & 1;                      // warp tile: rows 16 wm .., columns 16 wn ..
+    const unsigned full = 0xffffffffu;
+    const int pieces = rank >> 1;                                 // 16-byte pieces of a factor row
+
+    // columns rank .. ld - 1 of both operand buffers stay zero for good
+    for (int i = threadIdx.x; i < (kDenseBM + kDenseBN) * (ld - rank); i += kThreads) {
+        const int r = i / (ld - rank), c = rank + i % (ld - rank);
+        Us[(size_t)r * ld + c] = 0.0;            // r runs over the rows of Us and then of Vs
+    }
+
+    auto copy_rows = [&](double *dst, int nrows, const double *src, long long ldsrc, long long first,
+                         long long limit) {
+        // rows first .. first + nrows - 1 of a factor (those below `limit`) into dst
+        for (int i = threadIdx.x; i < nrows * pieces; i += kThreads) {
+            const int r = i / pieces, c = i % pieces;
+            if (first + r < limit) cp_async16(dst + (size_t)r * ld + 2 * c, src + (first + r) * ldsrc + 2 * c);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+
+    double acc = 0.0;
+    const long long items = (long long)sp.row_blocks * sp.col_splits;
+    const long long ntiles = (p.cols + kDenseBN - 1) / kDenseBN;
+    for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+        const long long row0 = (item / sp.col_splits) * kDenseBM;
+        const long long tile_lo = (item % sp.col_splits) * sp.tiles_per_split;
+        const long long tile_hi = tile_lo + sp.tiles_per_split < ntiles ? tile_lo + sp.tiles_per_split : ntiles;
+        __syncthreads();                                          // the buffers' last readers are done
+        copy_rows(Us, kDenseBM, p.U, p.ldu, row0, p.rows);
+        copy_rows(Vs, kDenseBN, p.V, p.ldv, tile_lo * kDenseBN, p.cols);
+        // per-row cursors: the first stored cell at or right of the column range's start
+        if (threadIdx.x < kDenseBM) {
+            const long long row = row0 + threadIdx.x;
+            int lo = 0, e = 0;
+            if (row < p.rows) {
+                lo = __ldg(p.rowptr + row);
+                e = __ldg(p.rowptr + row + 1);
+                const int want = (int)(tile_lo * kDenseBN);
+                int hi = e;
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (__ldg(p.colidx + mid) < want) lo = mid + 1; else hi = mid;
+                }
+            }
+            cur[threadIdx.x] = lo;
+            rend[threadIdx.x] = e;
+        }
+        for (long long tile = tile_lo; tile < tile_hi; ++tile) {
+            const int n0 = (int)(tile * kDenseBN);
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();                                      // U block and this V tile have landed
+            // ---- P = U_blk V_tile^T: warp tile 16 x 16 = 2 x 2 instruction tiles
+            double c[2][2][2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int j = 0; j < 2; ++j) c[i][j][0] = c[i][j][1] = 0.0;
+            const double *ua = Us + (size_t)(16 * wm + g) * ld + t;
+            const double *vb = Vs + (size_t)(16 * wn + g) * ld + t;
+#pragma unroll 4
+            for (int k = 0; k < ld; k += 4) {
+                double a[2], b[2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) a[i] = ua[(size_t)(8 * i) * ld + k];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) b[j] = vb[(size_t)(8 * j) * ld + k];
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) dmma_8x8x4(c[i][j][0], c[i][j][1], a[i], b[j]);
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    *reinterpret_cast<double2 *>(Ps + (size_t)(16 * wm + 8 * i + g) * PLD + 16 * wn + 8 * j + 2 * t) =
+                        make_double2(c[i][j][0], c[i][j][1]);
+            __syncthreads();                                      // P is complete; Vs is free
+            if (tile + 1 < tile_hi) copy_rows(Vs, kDenseBN, p.V, p.ldv, (tile + 1) * kDenseBN, p.cols);
+            // ---- the stored cells of this tile: warp w takes rows 8 w .. 8 w + 7 of the block, a lane
+            // the cell at its offset from the row's cursor; all loads first, then the chains
+            const int nhi = n0 + kDenseBN;
+            int jj[8];
+            double aa[8];
+#pragma unroll
+            for (int rr = 0; rr < 8; ++rr) {
+                const int pp = cur[8 * warp + rr] + lane;
+                jj[rr] = 0x7fffffff;
+                aa[rr] = 0.0;
+                if (pp < rend[8 * warp + rr]) {
+                    jj[rr] = __ldg(p.colidx + pp);
+                    aa[rr] = __ldg(p.vals + pp);
+                }
+            }
+#pragma unroll
+            for (int rr = 0; rr < 8; ++rr) {
+                const int r = 8 * warp + rr;
+                const bool in = jj[rr] < nhi;
+                if (in) {
+                    const double w = outer_chain(ch, p.chain_kind, p.kconst, aa[rr], Ps[(size_t)r * PLD + (jj[rr] - n0)]);
+                    if (AGG == kOutFull) acc += w;
+                    else p.out[cur[r] + lane] = w;
+                }
+                const int taken = __popc(__ballot_sync(full, in));
+                __syncwarp();
+                if (lane == 0) cur[r] += taken;
+            }
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+
+    if (AGG == kOutFull) {
+        double v1[1] = {acc};
+        block_sum<1>(v1, s_red);
+        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
+    }
+}
+
 __global__ void outer_fill_zero_kernel(double *out, long long n)
 {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -577,36 +625,65 @@ cudaError_t launch_outer(const DevChain &ch, const OuterParams &p, int agg, bool
     return cudaGetLastError();
 }
 
-template <int NK2>
-cudaError_t launch_outer_staged(const DevChain &ch, const OuterParams &p, int agg, int grid,
-                                cudaStream_t st)
+// full_agg / no_agg / right_mm through the pipelined kernel; NK2 is exactly ceil(rank / 16).
+template <int NK2, int AGG>
+cudaError_t launch_outer_pipe_one(const DevChain &ch, const OuterParams &p, int grid, cudaStream_t st)
 {
     const size_t smem = (size_t)(kThreads / 32) * kStageRows * p.rank * sizeof(double);
-    auto go = [&](auto kern) -> cudaError_t {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // the attribute sticks to the function: raise it when a call needs more than any before
+    static std::atomic<size_t> granted[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || granted[dev].load(std::memory_order_relaxed) < smem) {
+        e = cudaFuncSetAttribute(outer_pipe_kernel<NK2, AGG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kern<<<grid, kThreads, smem, st>>>(ch, p);
-        return cudaGetLastError();
-    };
-    if (agg == FO_OUTER_FULL_AGG) return go(outer_staged_kernel<NK2, kOutFull>);
-    if (agg == FO_OUTER_NO_AGG) return go(outer_staged_kernel<NK2, kOutNone>);
-    return go(outer_staged_kernel<NK2, kOutRight>);
+        if (dev >= 0 && dev < 64) granted[dev].store(smem, std::memory_order_relaxed);
+    }
+    outer_pipe_kernel<NK2, AGG><<<grid, kThreads, smem, st>>>(ch, p);
+    return cudaGetLastError();
 }
 
-// full_agg / no_agg / right_mm through the pipelined kernel; NK2 is exactly ceil(rank / 16).
 template <int NK2>
 cudaError_t launch_outer_pipe(const DevChain &ch, const OuterParams &p, int agg, int grid, cudaStream_t st)
 {
-    const size_t smem = (size_t)(kThreads / 32) * kStageRows * p.rank * sizeof(double);
-    auto go = [&](auto kern) -> cudaError_t {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (agg == FO_OUTER_FULL_AGG) return launch_outer_pipe_one<NK2, kOutFull>(ch, p, grid, st);
+    if (agg == FO_OUTER_NO_AGG) return launch_outer_pipe_one<NK2, kOutNone>(ch, p, grid, st);
+    return launch_outer_pipe_one<NK2, kOutRight>(ch, p, grid, st);
+}
+
+// full_agg / no_agg through the tiled schedule for densely stored inputs.
+template <int AGG>
+cudaError_t launch_outer_dense_one(const DevChain &ch, const OuterParams &p, int sms, cudaStream_t st)
+{
+    const size_t smem = dense_smem_bytes(p.rank);
+    static std::atomic<size_t> granted[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || granted[dev].load(std::memory_order_relaxed) < smem) {
+        e = cudaFuncSetAttribute(outer_dense_kernel<AGG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kern<<<grid, kThreads, smem, st>>>(ch, p);
-        return cudaGetLastError();
-    };
-    if (agg == FO_OUTER_FULL_AGG) return go(outer_pipe_kernel<NK2, kOutFull>);
-    if (agg == FO_OUTER_NO_AGG) return go(outer_pipe_kernel<NK2, kOutNone>);
-    return go(outer_pipe_kernel<NK2, kOutRight>);
+        if (dev >= 0 && dev < 64) granted[dev].store(smem, std::memory_order_relaxed);
+    }
+    DenseSplit sp;
+    const long long ntiles = (p.cols + kDenseBN - 1) / kDenseBN;
+    const long long rb = (p.rows + kDenseBM - 1) / kDenseBM;
+    // column ranges: enough work items for a few rounds over the SMs, so the last round is a small share
+    long long splits = (8ll * sms + rb - 1) / rb;
+    if (splits < 1) splits = 1;
+    if (splits > ntiles) splits = ntiles;
+    const long long per = (ntiles + splits - 1) / splits;
+    splits = (ntiles + per - 1) / per;
+    if (rb > 0x7fffffffll / splits) return cudaErrorInvalidValue;
+    sp.row_blocks = (int)rb;
+    sp.col_splits = (int)splits;
+    sp.tiles_per_split = (int)per;
+    sp.pad = 0;
+    long long grid = rb * splits;
+    if (grid > 2ll * sms) grid = 2ll * sms;
+    outer_dense_kernel<AGG><<<(unsigned)grid, kThreads, smem, st>>>(ch, p, sp);
+    return cudaGetLastError();
 }
 
 // Recognises the chains that outer_chain() evaluates inline by the text of the
@@ -711,30 +788,33 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
 
     cudaError_t e;
     const int nk2 = (rank + 15) / 16;
-    // factor rows that are 16-byte aligned pieces go through the staged kernel
-    const bool staged = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && agg != FO_OUTER_LEFT_MM &&
-                        !getenv("FUSEDOPS_OUTER_DIRECT");
-    if (staged) {
-        // FUSEDOPS_OUTER_PIPE=0 keeps the batch-at-a-time kernel (a measuring knob)
-        const char *pe = getenv("FUSEDOPS_OUTER_PIPE");
-        const bool pipe = !(pe && pe[0] == '0');
-        if (pipe) {
-            switch (nk2) {
-                case 1: e = launch_outer_pipe<1>(ch, p, agg, (int)grid, st); break;
-                case 2: e = launch_outer_pipe<2>(ch, p, agg, (int)grid, st); break;
-                case 3: e = launch_outer_pipe<3>(ch, p, agg, (int)grid, st); break;
-                case 4: e = launch_outer_pipe<4>(ch, p, agg, (int)grid, st); break;
-                case 5: e = launch_outer_pipe<5>(ch, p, agg, (int)grid, st); break;
-                case 6: e = launch_outer_pipe<6>(ch, p, agg, (int)grid, st); break;
-                case 7: e = launch_outer_pipe<7>(ch, p, agg, (int)grid, st); break;
-                default: e = launch_outer_pipe<8>(ch, p, agg, (int)grid, st); break;
-            }
-        } else
-        if (nk2 <= 1) e = launch_outer_staged<1>(ch, p, agg, (int)grid, st);
-        else if (nk2 <= 2) e = launch_outer_staged<2>(ch, p, agg, (int)grid, st);
-        else if (nk2 <= 4) e = launch_outer_staged<4>(ch, p, agg, (int)grid, st);
-        else if (nk2 <= 7) e = launch_outer_staged<7>(ch, p, agg, (int)grid, st);
-        else e = launch_outer_staged<8>(ch, p, agg, (int)grid, st);
+    // factor rows that are whole 16-byte pieces can be copied asynchronously into shared memory
+    const bool copyable = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && agg != FO_OUTER_LEFT_MM;
+    char which[48] = "";
+    tune_get("outer.kernel", which, sizeof(which));
+    const bool want_direct = strcmp(which, "direct") == 0;
+    // densely stored inputs: forming the tiles of U V^T beats a gathered row per stored cell
+    // once about one cell in seven is stored (measured crossover on this part)
+    const bool want_dense = strcmp(which, "dense") == 0;
+    const bool dense_ok = copyable && agg != FO_OUTER_RIGHT_MM && rank >= 8 &&
+                          dense_smem_bytes(rank) <= 200u * 1024u;
+    const double stored_share = (double)X->nnz / ((double)X->rows * (double)X->cols);
+    if (dense_ok && (want_dense || (which[0] == 0 && stored_share >= 0.15 && X->rows >= 64 && X->cols >= 64))) {
+        e = agg == FO_OUTER_FULL_AGG ? launch_outer_dense_one<kOutFull>(ch, p, sms, st)
+                                     : launch_outer_dense_one<kOutNone>(ch, p, sms, st);
+        return e == cudaSuccess ? FO_OK : cuda_fail(e);
+    }
+    if (copyable && !want_direct) {
+        switch (nk2) {
+            case 1: e = launch_outer_pipe<1>(ch, p, agg, (int)grid, st); break;
+            case 2: e = launch_outer_pipe<2>(ch, p, agg, (int)grid, st); break;
+            case 3: e = launch_outer_pipe<3>(ch, p, agg, (int)grid, st); break;
+            case 4: e = launch_outer_pipe<4>(ch, p, agg, (int)grid, st); break;
+            case 5: e = launch_outer_pipe<5>(ch, p, agg, (int)grid, st); break;
+            case 6: e = launch_outer_pipe<6>(ch, p, agg, (int)grid, st); break;
+            case 7: e = launch_outer_pipe<7>(ch, p, agg, (int)grid, st); break;
+            default: e = launch_outer_pipe<8>(ch, p, agg, (int)grid, st); break;
+        }
         return e == cudaSuccess ? FO_OK : cuda_fail(e);
     }
     if (nk2 <= 1) e = launch_outer<1>(ch, p, agg, aligned, (int)grid, st);

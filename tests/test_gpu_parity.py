@@ -463,6 +463,58 @@ def test_outer_log_chain(fo):
     assert_close(got.cpu().numpy(), [ref])
 
 
+@pytest.fixture
+def outer_schedule(fo):
+    """Sets the schedule knob of fused_outer for one test and clears it afterwards."""
+    def choose(name):
+        fo.tune("outer.kernel", name)
+    yield choose
+    fo.tune("outer.kernel", None)
+
+
+@pytest.mark.parametrize("rows,cols,rank,density", [
+    (64, 64, 8, 1.0), (200, 300, 100, 1.0), (129, 257, 100, 0.3), (130, 70, 128, 0.5), (1000, 90, 34, 0.2),
+    (65, 1000, 10, 0.9)])
+@pytest.mark.parametrize("agg", ["full", "none"])
+def test_outer_dense_schedule(fo, rows, cols, rank, density, agg):
+    """Densely stored main inputs run the tiled schedule (every tile of U V^T formed on
+    the tensor cores, stored cells sample it): against the dense-mode checker, which
+    forms U V^T outright, and against the per-cell schedule on the same input."""
+    w, Xh = outer_case(rows, cols, rank, density, seed=44)
+    w["vals"][::5] = 0.0                  # stored zeros are visited like any stored cell
+    Xh = host_csr(w)
+    Xd, Ud, Vd = csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"])
+    ref = oracle.outer(WSLOSS, "t3", Xh, w["U"], w["V"], agg=agg, mode="dense")
+    got = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()        # picks the tiled schedule itself
+    assert_close(got, ref, what="outer tiled %s" % agg)
+    try:
+        fo.tune("outer.kernel", "dense")
+        forced = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()
+        fo.tune("outer.kernel", "pipe")
+        per_cell = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()
+    finally:
+        fo.tune("outer.kernel", None)
+    assert forced.tobytes() == got.tobytes()
+    assert_close(per_cell, ref, what="outer per cell %s" % agg)
+    # a generic chain (interpreted) through the same schedule
+    gen = [("sub", "t1", "a", "d"), ("abs", "t2", "t1"), ("add", "t3", "t2", 0.25)]
+    assert_close(fo.fused_outer(gen, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy(),
+                 oracle.outer(gen, "t3", Xh, w["U"], w["V"], agg=agg, mode="dense"), what="outer tiled generic")
+
+
+@pytest.mark.parametrize("schedule", ["pipe", "direct", "dense"])
+def test_outer_every_schedule_on_a_sparse_input(fo, outer_schedule, schedule):
+    w, Xh = outer_case(700, 900, 100, 0.02, seed=15)
+    Xd, Ud, Vd = csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"])
+    outer_schedule(schedule)
+    for agg in ("full", "none"):
+        ref = oracle.outer(WSLOSS, "t3", Xh, w["U"], w["V"], agg=agg, mode="masked")
+        got = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()
+        assert_close(got, ref, what="outer %s %s" % (schedule, agg))
+        again = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()
+        assert again.tobytes() == got.tobytes()
+
+
 # ------------------------------------------------------------------ specialised vs interpreted chains
 @pytest.mark.parametrize("name,chain,outs,nsides", [
     ("mul2", [("mul", "t0", "a", "side0")], ["t0"], 1),
