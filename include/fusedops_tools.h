@@ -75,12 +75,22 @@ int fo_chain_describe(const fo_chain *chain, int use, int n_sides,
  *                         of the dense matrix V, 8 lanes per row, 16-byte loads:
  *                         n * V.cols * 8 bytes move.  V.cols and V.ld even, V.data
  *                         16-byte aligned, else FO_ERR_UNSUPPORTED.
+ *   fo_probe_bulk_gather() the same rows through the bulk-copy engine: 8 warps per SM, each
+ *                         with two slots of 16 rows in flight in shared memory, one bulk
+ *                         copy per row (a differently shaped measurement of the same
+ *                         rate: nothing of its access pattern is shared with
+ *                         fo_probe_l2_gather or the Outer kernels).  Same conditions on V;
+ *                         the doubles of a row pair must fit 220 KB / 256 per row.  `out`
+ *                         needs fo_probe_out_len() doubles here too (the kernel writes
+ *                         fewer and keeps one word behind them as the flag of its bounded
+ *                         waits: non-zero if one ran out).
  *   fo_probe_fp64_fma()   every one of the fo_probe_out_len() threads runs
  *                         8 * iters dependent-chain-of-8 multiply-adds from
  *                         registers: 16 * iters * fo_probe_out_len() flop.
  * Asynchronous; allocate nothing; errors as for the other calls. */
 size_t fo_probe_out_len(void);
 int fo_probe_l2_gather(const fo_dense *V, const int *idx, long long n, double *out, void *stream);
+int fo_probe_bulk_gather(const fo_dense *V, const int *idx, long long n, double *out, void *stream);
 int fo_probe_fp64_fma(long long iters, double *out, void *stream);
 
 #ifdef __cplusplus

@@ -83,7 +83,7 @@ EXPORTS = [
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
     "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_compile_check",
-    "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_fp64_fma", "fo_chain_describe", "fo_tune",
+    "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_bulk_gather", "fo_probe_fp64_fma", "fo_chain_describe", "fo_tune",
 ]
 
 _lib = None
@@ -149,6 +149,8 @@ def load_library(path=None):
         lib.fo_probe_out_len.restype = C.c_size_t
         lib.fo_probe_l2_gather.argtypes = [C.POINTER(fo_dense), vp, C.c_longlong, dp, vp]
         lib.fo_probe_l2_gather.restype = C.c_int
+        lib.fo_probe_bulk_gather.argtypes = [C.POINTER(fo_dense), vp, C.c_longlong, dp, vp]
+        lib.fo_probe_bulk_gather.restype = C.c_int
         lib.fo_probe_fp64_fma.argtypes = [C.c_longlong, dp, vp]
         lib.fo_probe_fp64_fma.restype = C.c_int
         if path is None:
@@ -414,6 +416,23 @@ def probe_l2_gather(V, idx, out=None):
     _check(lib.fo_probe_l2_gather(C.byref(vs), C.c_void_p(idx.data_ptr()), idx.numel(),
                                   C.c_void_p(out.data_ptr()), _stream(V.device)), "fo_probe_l2_gather")
     return idx.numel() * V.shape[1] * 8
+
+
+def probe_bulk_gather(V, idx, out=None):
+    """The same gather through the bulk-copy engine; returns the bytes moved.  After a
+    synchronise, out[probe_bulk_flag_index(V.device)] is 0.0 unless a bounded wait ran out."""
+    lib = load_library()
+    assert V.dtype == torch.float64 and V.dim() == 2 and idx.dtype == torch.int32 and idx.is_contiguous()
+    if out is None:
+        out = torch.empty(lib.fo_probe_out_len(), dtype=torch.float64, device=V.device)
+    vs = _dense_struct(V)
+    _check(lib.fo_probe_bulk_gather(C.byref(vs), C.c_void_p(idx.data_ptr()), idx.numel(),
+                                    C.c_void_p(out.data_ptr()), _stream(V.device)), "fo_probe_bulk_gather")
+    return idx.numel() * V.shape[1] * 8
+
+
+def probe_bulk_flag_index():
+    return int(load_library().fo_probe_out_len()) // 8
 
 
 def probe_fp64_fma(iters, out):
