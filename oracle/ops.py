@@ -111,6 +111,13 @@ def col_sums(t):
     return np.sum(t, axis=0, dtype=LD).astype(np.float64)
 
 
+def count_nonzero(values):
+    """Number of entries of an elementwise result that are not zero (the nnz a sparse
+    output would store; -0.0 counts as zero, NaN as non-zero): the comparison
+    `values != 0`, then a count."""
+    return int(np.count_nonzero(np.asarray(values, dtype=np.float64) != 0.0))
+
+
 def csr_row_ids(rows, rowptr):
     """Row index of every stored cell of a CSR matrix."""
     return np.repeat(np.arange(rows, dtype=np.int64), np.diff(np.asarray(rowptr, dtype=np.int64)))
@@ -376,8 +383,12 @@ def mlogreg_inner(X, V, P):
 # --------------------------------------------------------------------------
 # Outer template
 # --------------------------------------------------------------------------
-def outer(chain, output, X, U, V, scalars=(), agg="full", mode="masked"):
+def outer(chain, output, X, U, V, scalars=(), agg="full", mode="masked", sides=()):
     """Outer template over the stored cells of the CSR matrix X.
+
+    Side inputs (Table 1 binds dense side inputs to the Outer template too):
+    ("cell", m x n array) read at (i, j), ("row", m-vector) read at i, ("col",
+    n-vector) read at j; the chain names them "side0", "side1", ...
 
     mode "dense":  P = U V^T as a dense m x n array; the chain runs on every
                    cell (a = dense X, d = P); the result is kept only where X
@@ -395,13 +406,27 @@ def outer(chain, output, X, U, V, scalars=(), agg="full", mode="masked"):
     rid = csr_row_ids(m, X["rowptr"])
     cid = np.asarray(X["colidx"], dtype=np.int64)
     senv = {"s%d" % k: np.float64(s) for k, s in enumerate(scalars)}
+    dense_sides, cell_sides = {}, {}
+    for k, (access, arr) in enumerate(sides):
+        arr = np.asarray(arr, dtype=np.float64)
+        if access == "cell":
+            assert arr.shape == (m, n)
+            dense_sides["side%d" % k], cell_sides["side%d" % k] = arr, arr[rid, cid]
+        elif access == "row":
+            assert arr.shape == (m,)
+            dense_sides["side%d" % k], cell_sides["side%d" % k] = arr.reshape(m, 1), arr[rid]
+        elif access == "col":
+            assert arr.shape == (n,)
+            dense_sides["side%d" % k], cell_sides["side%d" % k] = arr.reshape(1, n), arr[cid]
+        else:
+            raise ValueError(access)
     if mode == "dense":
         Xd = np.zeros((m, n), dtype=np.float64)
         Xd[rid, cid] = X["vals"]
         pattern = np.zeros((m, n), dtype=np.float64)
         pattern[rid, cid] = 1.0
         P = U @ V.T
-        (T,) = eval_chain(chain, [output], dict(senv, a=Xd, d=P), (m, n))
+        (T,) = eval_chain(chain, [output], dict(senv, a=Xd, d=P, **dense_sides), (m, n))
         Wd = np.where(pattern != 0.0, T, 0.0)
         if agg == "full":
             return full_sum(Wd)
@@ -417,8 +442,8 @@ def outer(chain, output, X, U, V, scalars=(), agg="full", mode="masked"):
         Vg = V[cid]                      # nnz x k
         prod = Ug * Vg
         d = np.sum(prod, axis=1, dtype=LD).astype(np.float64) if prod.size else np.zeros(0)
-        (t,) = eval_chain(chain, [output], dict(senv, a=np.asarray(X["vals"], dtype=np.float64), d=d),
-                          d.shape)
+        (t,) = eval_chain(chain, [output], dict(senv, a=np.asarray(X["vals"], dtype=np.float64), d=d,
+                                                **cell_sides), d.shape)
         if agg == "full":
             return full_sum(t)
         if agg == "none":

@@ -601,3 +601,41 @@ def test_outer_empty():
     assert oracle.outer_wsloss_masked(X, U, V) == 0.0
     assert oracle.outer_wsloss_dense(X, U, V) == 0.0
     assert oracle.outer(WSLOSS, "t3", X, U, V, mode="masked") == 0.0
+
+
+def test_outer_side_inputs_bruteforce_and_mode_agreement():
+    """Outer with dense side inputs (Table 1): every stored cell reads a cell-shaped side
+    at (i, j), a row-vector side at j and a column-vector side at i; exact rationals."""
+    X, U, V = small_outer(10, 9, 4, 0.4, seed=21)
+    m, n = X["rows"], X["cols"]
+    S = datagen.uniform(21, 5, m * n, -1.0, 1.0).reshape(m, n)
+    r = datagen.uniform(21, 6, m, 0.5, 2.0)
+    c = datagen.uniform(21, 7, n, -2.0, 2.0)
+    chain = [("sub", "t0", "a", "d"), ("mul", "t1", "t0", "side0"), ("add", "t2", "t1", "side2"),
+             ("mul", "t3", "t2", "side1")]                         # ((a - d) * S_ij + c_j) * r_i
+    sides = [("cell", S), ("row", r), ("col", c)]
+    rid = oracle.csr_row_ids(m, X["rowptr"])
+    want = []
+    for p in range(len(X["vals"])):
+        i, j = int(rid[p]), int(X["colidx"][p])
+        d = sum((F(float(U[i, q])) * F(float(V[j, q])) for q in range(U.shape[1])), F(0))
+        want.append(float(((F(float(X["vals"][p])) - d) * F(float(S[i, j])) + F(float(c[j]))) * F(float(r[i]))))
+    for mode in ("dense", "masked"):
+        got = oracle.outer(chain, "t3", X, U, V, agg="none", mode=mode, sides=sides)
+        assert np.allclose(got, want, rtol=1e-12, atol=1e-14)
+        assert close(oracle.outer(chain, "t3", X, U, V, mode=mode, sides=sides), fsum_exact(want), 1e-12)
+    # a side of ones changes nothing; a constant row vector is a scalar
+    ones = [("cell", np.ones((m, n)))]
+    plain = oracle.outer(WSLOSS, "t3", X, U, V)
+    assert oracle.outer(WSLOSS + [("mul", "t4", "t3", "side0")], "t4", X, U, V, sides=ones) == plain
+    assert oracle.outer([("mul", "t0", "d", "side0")], "t0", X, U, V, sides=[("row", np.full(m, 3.0))]) == \
+        oracle.outer([("mul", "t0", "d", "s0")], "t0", X, U, V, [3.0])
+
+
+def test_count_nonzero_known_values():
+    assert oracle.count_nonzero([]) == 0
+    assert oracle.count_nonzero([0.0, -0.0, 1.0, -2.5, 5e-324, float("nan"), float("inf")]) == 5
+    assert oracle.count_nonzero(np.zeros((3, 4))) == 0
+    a = np.arange(-3, 4, dtype=np.float64)
+    assert oracle.count_nonzero(a) == 6
+    assert oracle.count_nonzero(np.outer(a, a)) == 36
