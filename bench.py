@@ -385,6 +385,16 @@ def machine_probes(fo, step, shapes):
         res[label + "_rows"] = nrows
     res["l2_gather"] = ("%d random rows of %d doubles from the first rows of V (%.0f MB resident set, resp. "
                         "all of V)" % (n, V.shape[1], 40_000 * V.shape[1] * 8 / 1e6))
+    # the same rows through the bulk-copy engine (a differently shaped measurement of the same rate)
+    idx = torch.randint(0, V.shape[0], (n,), generator=g, device=dev, dtype=torch.int32)
+    moved = [0]
+
+    def run_bulk(idx=idx):
+        moved[0] = fo.probe_bulk_gather(V, idx, out)
+    ms = min(_event_times(run_bulk, 5))
+    res["bulk_gather_all_rows_gbs"] = moved[0] / (ms * 1e-3) / 1e9
+    res["bulk_gather_wait_ran_out"] = bool(out[fo.probe_bulk_flag_index()].item() != 0.0)
+    res["sm_count"] = torch.cuda.get_device_properties(dev).multi_processor_count
     flops = [0]
 
     def fma():
@@ -445,13 +455,18 @@ def _device_csr(fo, rows, cols, density, g, device, lo=0.0, hi=1.0, chunk_rows=N
     return fo.CSR(rows, cols, rowptr, colidx, vals)
 
 
-def paper_suite(fo, device, reps=5):
+def paper_suite(fo, device, reps=5, peak_gbs=6650.0, fp64_tflops=37.0, l2_gather_gbs=18500.0):
     """The operator micro-benchmarks of Section 5.2 at the paper's own sizes (inputs made on the
     device from a seeded torch generator; parity of every kernel used here is covered by the tests):
     Cell sum(X*Y*Z), MAgg (sum(X*Y), sum(X*Z)), Row t(X)(Xv) and t(X)(XV) over x * 10^3 inputs,
     x = 10^3 .. 10^6, dense and at sparsity 0.1; Outer sum(X * log(U t(V) + 1e-15)) over
     2*10^4 x 2*10^4 at rank 100, sparsity 1 .. 10^-4.  Cold L2 (a 512 MB buffer is rewritten
-    before every run); times are the minimum of `reps` runs."""
+    before every run); times are the minimum of `reps` runs.  Every entry carries its roofline:
+    the bytes the operator must read once over the copy bandwidth (`*_frac`: ideal / measured
+    time); the Outer entries the slowest of three terms - compulsory bytes over the copy
+    bandwidth, gathered factor rows over the L2 gather rate (per-cell schedule) or the tile
+    products over the fp64 rate (tiled schedule, densely stored X), and the stored cells'
+    logarithms over a measured log rate."""
     import torch
     g = torch.Generator(device=device)
     g.manual_seed(12)
@@ -487,16 +502,44 @@ def paper_suite(fo, device, reps=5):
         e["row_xtxv_dense_us"] = t_us(lambda: fo.fused_row([], "d", X, v, out=qv))
         e["row_xtxv_sparse_us"] = t_us(lambda: fo.fused_row([], "d", Xs, v, out=qv))
         e["row_xtxV2_dense_us"] = t_us(lambda: fo.fused_row_b1(None, None, [], "d", X, V2, out=qm))
+        # rooflines: bytes each operator must read once (sparse: 12 per stored cell + row offsets; a dense
+        # side read at a stored cell costs its 8 bytes, a sparse side its own 12 per stored cell)
+        dense3, csr = 3 * 8 * rows * cols, 12 * Xs.nnz + 4 * (rows + 1)
+        algo = {"cell_dense": dense3, "magg_dense": dense3, "cell_sparse": csr + 16 * Xs.nnz,
+                "magg_sparse": csr + 16 * Xs.nnz, "cell_all_sparse": 3 * csr, "magg_all_sparse": 3 * csr,
+                "row_xtxv_dense": 8 * rows * cols + 16 * cols, "row_xtxv_sparse": csr + 16 * cols,
+                "row_xtxV2_dense": 8 * rows * cols + 4 * 8 * cols}
+        for name, nb in algo.items():
+            us = e[name + "_us"]
+            e[name + "_gbs"] = nb / (us * 1e-6) / 1e9
+            e[name + "_frac"] = nb / (peak_gbs * 1e9) / (us * 1e-6)
         out["cell_magg_row"].append(e)
         del X, Y, Z, Xs, sides
     m = 20_000
     U = torch.rand((m, 100), generator=g, dtype=torch.float64, device=device) + 0.1
     Vf = torch.rand((m, 100), generator=g, dtype=torch.float64, device=device) + 0.1
     xlog = [("add", "t0", "d", 1e-15), ("log", "t1", "t0"), ("mul", "t2", "a", "t1")]
+    # the rate of the chain's logarithm alone: log over a streamed array (the Cell kernel), cells per second
+    L = torch.rand(20_000_000, generator=g, dtype=torch.float64, device=device) + 0.5
+    log_us = t_us(lambda: fo.fused_cell([("log", "t0", "a")], "t0", L.view(20_000, 1000), out=one))
+    log_rate = L.numel() / (log_us * 1e-6)
+    del L
+    out["log_cells_per_s"] = log_rate
     for sp in (1.0, 0.1, 0.01, 0.001, 0.0001):
         Xs = _device_csr(fo, m, m, sp, g, device, chunk_rows=2000)
         us = t_us(lambda: fo.fused_outer(xlog, "t2", Xs, U, Vf, out=one))
-        out["outer"].append({"sparsity": sp, "nnz": Xs.nnz, "us": us, "nnz_per_s": Xs.nnz / (us * 1e-6)})
+        tiled = Xs.nnz >= 0.15 * m * m            # the schedule the library picks (stored share of X)
+        terms = {"hbm": (12 * Xs.nnz + 4 * (m + 1) + 2 * 8 * m * 100) / (peak_gbs * 1e9) * 1e6,
+                 "log": Xs.nnz / log_rate * 1e6}
+        if tiled:
+            terms["fp64_tiles"] = 2.0 * m * m * 100 / (fp64_tflops * 1e12) * 1e6
+        else:
+            terms["l2_gather"] = Xs.nnz * 800 / (l2_gather_gbs * 1e9) * 1e6
+        binding = max(terms, key=terms.get)
+        out["outer"].append({"sparsity": sp, "nnz": Xs.nnz, "us": us, "nnz_per_s": Xs.nnz / (us * 1e-6),
+                             "schedule": "tiled" if tiled else "per stored cell",
+                             "bound_terms_us": terms, "binding_term": binding,
+                             "frac_of_binding_term": terms[binding] / us})
         del Xs
     return out
 
@@ -620,6 +663,69 @@ def oracle_single_thread(np_inputs, shapes):
         if limit is not None:
             limit.restore_original_limits()
     return t
+
+
+REL_TOL = 1e-10           # spec tolerance for fp64 aggregates
+ABS_FLOOR = 1e-15         # times the sum of the magnitudes of a sum's terms (sums that cancel)
+
+
+def abs_scales(h, shapes, panel=100_000):
+    """Sum of the magnitudes of the terms of every result of the five operators (plain numpy, row
+    panels): the denominator of a sum's condition number."""
+    import oracle
+    sc = {"cell": np.array([np.sum(np.abs(h["cell.X"] * h["cell.Y"] * h["cell.Z"]))])}
+    X, Y, Z = h["magg.X"], h["magg.Y"], h["magg.Z"]
+    acc = np.zeros(3)
+    for r0 in range(0, X.shape[0], panel):
+        x, y, z = X[r0:r0 + panel], Y[r0:r0 + panel], Z[r0:r0 + panel]
+        acc += [np.abs(x * y).sum(), np.abs(x * z).sum(), (x * x).sum()]
+    sc["magg"] = acc
+    X, v, w = h["row_dense.X"], np.abs(h["row_dense.v"]), h["row_dense.w"]
+    acc = np.zeros(X.shape[1])
+    for r0 in range(0, X.shape[0], panel):
+        ax = np.abs(X[r0:r0 + panel])
+        acc += ax.T @ (np.abs(w[r0:r0 + panel]) * (ax @ v))
+    sc["row_dense"] = acc
+    s4 = shapes["row_csr"]
+    X4 = dict(rows=s4["rows"], cols=s4["cols"], rowptr=h["row_csr.rowptr"], colidx=h["row_csr.colidx"],
+              vals=np.abs(h["row_csr.vals"]))
+    sc["row_csr"] = np.asarray(oracle.row_chain_csr(X4, np.abs(h["row_csr.v"]), np.abs(h["row_csr.w"])))
+    sc["outer"] = None            # every term (a - d)^2 is non-negative: the sum is its own scale
+    return sc
+
+
+def parity_report(results, refs, scales):
+    """GPU results against the checker's, per operator: largest relative error, condition number
+    of the worst-conditioned element, and how many elements met the tolerance only through the
+    floor for cancelling sums.  ok: every element within REL_TOL, or within the floor."""
+    rep, ok_all = {}, True
+    for k in OPS:
+        if k not in refs or k not in results:
+            continue
+        g = np.asarray(results[k], dtype=np.float64).reshape(-1)
+        r = np.asarray(refs[k], dtype=np.float64).reshape(-1)
+        err = np.abs(g - r)
+        rel = err / np.maximum(np.abs(r), 1e-300)
+        sc = np.abs(r) if scales.get(k) is None else np.asarray(scales[k], dtype=np.float64).reshape(-1)
+        strict = err <= REL_TOL * np.abs(r)
+        floor = err <= ABS_FLOOR * sc
+        ok = bool(np.all(strict | floor))
+        rep[k] = {"max_rel_err": float(rel.max()), "cond_max": float(np.max(sc / np.maximum(np.abs(r), 1e-300))),
+                  "floor_used": int(np.count_nonzero(~strict & floor)), "elements": int(r.size), "ok": ok}
+        ok_all = ok_all and ok
+    rep["tolerance"] = "|gpu - ref| <= %g |ref|, or <= %g x sum of |terms| for sums that cancel" % (REL_TOL, ABS_FLOOR)
+    rep["ok"] = ok_all
+    return rep
+
+
+def cpu_model():
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.startswith("model name"):
+                return ln.split(":", 1)[1].strip()
+    except Exception:
+        pass
+    return "unknown"
 
 
 def host_threads():
@@ -874,14 +980,24 @@ def run_ours(args):
         line["probes"] = probes
         for n in roofline_per_op:
             roofline_per_op[n]["frac_of_stream_sum"] = per_op[n]["gbs"] / probes["stream_sum_gbs"]
-        # Outer: the slowest of compulsory bytes / HBM, gathered V rows / L2 gather rate, FMAs / fp64 rate
+        # Outer: the slowest of compulsory bytes / HBM, gathered V rows / L2 gather rate, FMAs / fp64 rate.
+        # The gather rate is quoted three ways: the per-lane-load probe, the bulk-copy probe (another
+        # access shape), and what the hardware's L2-to-SM path carries at most (64 bytes per clock and SM)
         rank5 = shapes["outer"]["rank"]
+        sm_mhz = float(peaks.get("sm_max_mhz", 1965.0))
+        probes["l2_to_sm_port_gbs"] = probes["sm_count"] * 64 * sm_mhz * 1e6 / 1e9
+        probes["l2_to_sm_port"] = "%d SMs x 64 B per clock x %.0f MHz" % (probes["sm_count"], sm_mhz)
+        gather_bytes = nnz5 * rank5 * 8
         terms = {"hbm": nbytes["outer"] / (peak_gbs * 1e9) * 1e3,
-                 "l2_gather": nnz5 * rank5 * 8 / (probes["l2_gather_gbs"] * 1e9) * 1e3,
+                 "l2_gather": gather_bytes / (probes["l2_gather_gbs"] * 1e9) * 1e3,
                  "fp64_fma": 2.0 * nnz5 * rank5 / (probes["fp64_fma_tflops"] * 1e12) * 1e3}
         binding = max(terms, key=terms.get)
-        roofline_per_op["outer"].update({"bound_terms_ms": terms, "binding_term": binding,
-                                         "frac_of_binding_term": terms[binding] / per_op["outer"]["ms"]})
+        roofline_per_op["outer"].update({
+            "bound_terms_ms": terms, "binding_term": binding,
+            "frac_of_binding_term": terms[binding] / per_op["outer"]["ms"],
+            "l2_gather_ms_by_bulk_copy_probe": gather_bytes / (probes["bulk_gather_all_rows_gbs"] * 1e9) * 1e3,
+            "l2_gather_ms_at_port_limit": gather_bytes / (probes["l2_to_sm_port_gbs"] * 1e9) * 1e3,
+            "frac_of_port_limit": gather_bytes / (probes["l2_to_sm_port_gbs"] * 1e9) * 1e3 / per_op["outer"]["ms"]})
         # the paper's cost model (Section 4.3: write time + max(read time, compute time)) fed with
         # this machine's measured rates: predicted time of each fused operator and of the plan of
         # basic operators it replaces, next to the measured time
@@ -902,20 +1018,29 @@ def run_ours(args):
         if args.frac == 1.0 and world == 1:
             line["size_sweep"] = size_sweep(fo, device)
         if args.paper_suite and world == 1:
-            line["paper_suite"] = paper_suite(fo, device)
+            line["paper_suite"] = paper_suite(fo, device, peak_gbs=peak_gbs, fp64_tflops=probes["fp64_fma_tflops"],
+                                              l2_gather_gbs=probes["l2_gather_gbs"])
 
-    # ---- CPU baseline: the checker on a bounded sample, rank 0 at N = 1 only
+    # ---- CPU baseline: the checker on a bounded sample, rank 0 at N = 1 only; at full size its
+    # results are also what the GPU results of the timed steps are checked against
+    parity_ok = True
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         chost, cshapes = row_sample(host, shapes, args.cpu_frac)
         cbytes = algorithmic_bytes(cshapes, chost)
-        t0 = time.perf_counter()
-        ct, _ = oracle_step(numpy_inputs(chost), cshapes)
-        cdt = time.perf_counter() - t0
+        cnp = numpy_inputs(chost)
+        runs = []
+        for _ in range(max(1, args.cpu_runs)):
+            t0 = time.perf_counter()
+            ct, cres = oracle_step(cnp, cshapes)
+            runs.append((time.perf_counter() - t0, ct))
+        cdt, ct = min(runs, key=lambda x: x[0])
         line["cpu_baseline"] = {
             "value": sum(cbytes.values()) / cdt / 1e9, "unit": UNIT, "cores": host_threads(),
             "kind": "oracle", "sample": "first %g of the rows of the bench inputs: %s" % (
                 args.cpu_frac, sample_description(cshapes)),
-            "seconds": cdt, "per_op_gbs": {k: cbytes[k] / ct[k] / 1e9 for k in OPS},
+            "seconds": cdt, "runs": len(runs), "seconds_all_runs": [r[0] for r in runs],
+            "per_op_gbs": {k: cbytes[k] / ct[k] / 1e9 for k in OPS},
+            "cpu_model": cpu_model(), "nproc": os.cpu_count(),
         }
         # one thread, configs 1 and 5 (Outer on a sixteenth of the sample's rows)
         shost, sshapes = row_sample(chost, cshapes, 1.0 / 16)
@@ -924,11 +1049,17 @@ def run_ours(args):
         line["cpu_baseline"]["single_thread_gbs"] = {k: sbytes[k] / st[k] / 1e9 for k in st}
         line["cpu_baseline"]["single_thread_sample"] = "cell full size; outer %d rows x %d" % (
             sshapes["outer"]["rows"], sshapes["outer"]["cols"])
+        if args.cpu_frac == 1.0 and step.enabled == set(OPS):
+            line["parity"] = parity_report(results, cres, abs_scales(cnp, cshapes))
+        else:       # only the Cell workload is whole in a sample
+            line["parity"] = parity_report({"cell": results["cell"]}, {"cell": cres["cell"]}, {"cell": None})
+            line["parity"]["note"] = "sampled CPU run: only the Cell workload is compared"
+        parity_ok = line["parity"]["ok"]
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
-    return 0
+    return 0 if parity_ok else 3
 
 
 def main():
@@ -940,6 +1071,7 @@ def main():
     ap.add_argument("--frac", type=float, default=1.0, help="scale the row counts (debugging)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-frac", type=float, default=1.0, help="sample of the workloads the CPU baseline runs")
+    ap.add_argument("--cpu-runs", type=int, default=2, help="runs of the CPU baseline (the best one is reported)")
     ap.add_argument("--ref-frac", type=float, default=0.01, help="sample per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the untimed-step variant measurements")

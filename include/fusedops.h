@@ -229,13 +229,21 @@ int fo_jit_stats(int *compiled, int *launches, int *failures);
  * Determinism: FO_CELL_COL_AGG over a CSR X adds into `out` with global atomics on
  * a zeroed result, so the order of its additions is not fixed; everything else
  * is bit-reproducible.
+ * out_nnz (device, one int64, or NULL): with FO_CELL_NO_AGG the number of written
+ * values that are not zero - what a sparse result would store (-0.0 counts as
+ * zero, NaN as non-zero).  It costs one more pass over `out`.  Not NULL with
+ * another variant: FO_ERR_UNSUPPORTED.  A CSR result keeps X's index arrays
+ * (values on X's pattern), so rowptr / colidx of the result are X's own.
  * Errors: FO_ERR_CHAIN if the chain uses FO_DOT; FO_ERR_SHAPE if a side does
  * not match X under its access kind; empty X (no cells) writes zeros.
+ * Aggregation is by sum; the paper's templates show sums only, and MIN / MAX
+ * aggregation is not built.
  */
 int fused_cell(const fo_chain *chain, const fo_mat *X,
                const fo_side *sides, int n_sides,
                const double *scalars, int n_scalars,
-               int agg, double *out, void *ws, size_t ws_bytes, void *stream);
+               int agg, double *out, long long *out_nnz,
+               void *ws, size_t ws_bytes, void *stream);
 
 /* ------------------------------------------------------- Cell, built-in scratch
  * (No counterpart in the paper: a deployment variant of fused_cell.)
@@ -248,7 +256,8 @@ int fused_cell(const fo_chain *chain, const fo_mat *X,
  * point takes no workspace: the scratch is a 1 MiB array that lives inside the
  * library image on every GPU that loads it, from load until the process exits.
  *
- * Same arguments, results and bits as fused_cell (dense X; all four variants).
+ * Same arguments (without the non-zero count), results and bits as fused_cell
+ * (dense X; all four variants).
  * It calls no cudaMalloc / cudaFree and no allocating library routine.  In
  * particular it never compiles or loads a run-time specialised kernel: a chain
  * that fused_cell or fo_jit_prepare specialised earlier is reused (a lookup),
@@ -299,6 +308,11 @@ int fused_magg(const fo_chain *chain, const fo_mat *X,
  *                     CSR X: out[p] = t_i * vals[p] for stored cell p of row i
  *                     (nnz doubles, X's pattern)
  * With the chain  t = side0 * d  this is  t(X) %*% (w * (X %*% v)).
+ * The row-wise operator is this fixed skeleton - a product with a side vector (or,
+ * in fused_row_b1, a side matrix), a scalar chain on it, and one of the Table 1
+ * aggregations - not a free program over the paper's vector primitives
+ * (vectMult, vectMinus, vectSum, vectMultAdd composed at will): that general
+ * form is not built.
  * X wider than 8192 columns returns FO_ERR_UNSUPPORTED (the single-pass
  * kernels keep a row, respectively v and the output vector, on chip).
  * Determinism: bit-reproducible except FO_ROW_COL_T_AGG / FO_ROW_COL_AGG over
@@ -349,7 +363,7 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
  * Table 1, Outer template; Fig. 1(d), Eq. 1 and the outer-product listing of
  * Section 2.2.  For every stored cell (i, j) of the CSR matrix X:
  *     a = X_ij,  d = U_i . V_j  (U: rows x rank, V: cols x rank, dense),
- *     w_ij = chain(a, d, scalars)
+ *     w_ij = chain(a, d, sides read at (i, j), scalars)
  *   FO_OUTER_FULL_AGG: out[0] = sum w_ij
  *   FO_OUTER_NO_AGG  : out[p] = w of stored cell p          (nnz doubles)
  *   FO_OUTER_RIGHT_MM: out[i * rank + c] = sum_j w_ij V_jc  (rows x rank, packed)
@@ -359,13 +373,29 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
  * other variants are bit-reproducible.
  * U V^T is never formed; cells that are not stored cost nothing.  Stored
  * zeros ARE visited (a chain tests a != 0 itself, as the listing does).
- * rank <= 256.  Errors: FO_ERR_SHAPE if U.rows != X.rows, V.rows != X.cols or
- * U.cols != V.cols.
+ * Side inputs (Table 1 binds dense side inputs to the Outer template as well): at
+ * most 3, dense; FO_AT_CELL sides are rows x cols and read at (i, j), FO_AT_ROW
+ * sides rows x 1 read at i, FO_AT_COL sides 1 x cols read at j.  A chain that
+ * reads a side runs through the general per-cell kernel (no staging of factor
+ * rows, no tiled schedule): correct for every variant, slower than a chain over
+ * a and d alone.
+ * out_nnz (device, one int64, or NULL): with FO_OUTER_NO_AGG the number of
+ * written values that are not zero, as for fused_cell; with another variant
+ * FO_ERR_UNSUPPORTED.
+ * Schedules: per stored cell (factor rows of V staged in shared memory), or -
+ * when about one cell in seven or more is stored - tile by tile, forming each
+ * 64 x 32 tile of U V^T on the fp64 tensor cores and sampling it at the stored
+ * cells (full_agg / no_agg).  The library chooses; results agree within the
+ * documented tolerance.
+ * rank <= 256.  Errors: FO_ERR_SHAPE if U.rows != X.rows, V.rows != X.cols,
+ * U.cols != V.cols or a side does not match X under its access kind.
  */
 int fused_outer(const fo_chain *chain, const fo_csr *X,
                 const fo_dense *U, const fo_dense *V,
+                const fo_side *sides, int n_sides,
                 const double *scalars, int n_scalars,
-                int agg, double *out, void *ws, size_t ws_bytes, void *stream);
+                int agg, double *out, long long *out_nnz,
+                void *ws, size_t ws_bytes, void *stream);
 
 #ifdef __cplusplus
 }

@@ -30,17 +30,24 @@ int fo_set_force_interpreter(int on);
  * FO_ERR_UNSUPPORTED for an unknown name, FO_ERR_SHAPE for a value of 48 or
  * more characters.  Names:
  *   cell.ctas_per_sm  1..8   CTAs per SM of the streaming Cell / MAgg kernel
- *   row.dense_shape   "c,w,r" chunks per lane, warps per group, rows per stage of the dense Row kernel
  *   row.narrow        0      dense rows of at most 32 columns through the warp-per-row kernel
  *   b1.mma            0 | 1  fused_row_b1: multiply-add kernel / tensor-core kernel
  *   b1.shape, b1.mma_shape   compiled shapes of those two kernels ("p,r,kl" / "w,kb")
  *   b1.narrow         0      fused_row_b1 without the thread-per-row kernel
- *   outer.kernel      "bulk" | "pipe" | "direct" | "dense"   schedule of fused_outer
- *   outer.depth, outer.warps   ring depth and warps per CTA of the bulk-copy Outer kernel
- *   outer.hints       0 | 1  L2 eviction hints on the Outer kernel's copies
- *   csr.variant       variant number of the CSR Row kernel
- *   cell.stamps       1      Cell kernel records time stamps in its workspace tail */
+ *   outer.kernel      "pipe" | "direct" | "dense"   schedule of fused_outer (per stored cell with
+ *                     staged factor rows / with plain gathers, or tile by tile for densely
+ *                     stored inputs); by default the library chooses from layout and stored share
+ *   cell.stamps       1      the streaming Cell / MAgg kernel records phase times (fo_cell_stamps) */
 int fo_tune(const char *name, const char *value);
+
+/* Phase times of the streaming Cell / MAgg kernel (full_agg), for measurements of small
+ * inputs where launch, first-load latency and the last stage are a large share.  With
+ * the knob cell.stamps set to 1 the kernel records, in nanoseconds of the GPU's global
+ * timer, ns[0] the earliest CTA start, ns[1] the latest end of a CTA's scan, ns[2] the
+ * latest publication of a partial sum, ns[3] the moment the result was written, in the
+ * control words of the workspace.  This call synchronises `stream`, returns the four
+ * stamps of the last such call and clears them. */
+int fo_cell_stamps(void *ws, void *stream, unsigned long long *ns);
 
 /* Generates and compiles (for sm_100a, without loading or launching: no GPU
  * needed) the run-time specialised kernel of a Cell chain; FO_OK, a chain error,

@@ -83,7 +83,7 @@ EXPORTS = [
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
     "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_compile_check",
-    "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_bulk_gather", "fo_probe_fp64_fma", "fo_chain_describe", "fo_tune",
+    "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_bulk_gather", "fo_probe_fp64_fma", "fo_chain_describe", "fo_tune", "fo_cell_stamps",
 ]
 
 _lib = None
@@ -100,11 +100,11 @@ def load_library(path=None):
         vp, dp, i32, sz = C.c_void_p, C.c_void_p, C.c_int, C.c_size_t
         chain_p, mat_p, side_p = C.POINTER(fo_chain), C.POINTER(fo_mat), C.POINTER(fo_side)
         scal_p = C.POINTER(C.c_double)
-        lib.fused_cell.argtypes = [chain_p, mat_p, side_p, i32, scal_p, i32, i32, dp, vp, sz, vp]
+        lib.fused_cell.argtypes = [chain_p, mat_p, side_p, i32, scal_p, i32, i32, dp, vp, vp, sz, vp]
         lib.fused_magg.argtypes = [chain_p, mat_p, side_p, i32, scal_p, i32, dp, vp, sz, vp]
         lib.fused_row.argtypes = [chain_p, mat_p, dp, side_p, i32, scal_p, i32, i32, dp, vp, sz, vp]
         lib.fused_outer.argtypes = [chain_p, C.POINTER(fo_csr), C.POINTER(fo_dense),
-                                    C.POINTER(fo_dense), scal_p, i32, i32, dp, vp, sz, vp]
+                                    C.POINTER(fo_dense), side_p, i32, scal_p, i32, i32, dp, vp, vp, sz, vp]
         lib.fused_row_b1.argtypes = [chain_p, chain_p, mat_p, C.POINTER(fo_dense), side_p, i32, scal_p, i32,
                                      i32, dp, vp, sz, vp]
         for f in (lib.fused_cell, lib.fused_magg, lib.fused_row, lib.fused_outer, lib.fused_row_b1):
@@ -135,6 +135,8 @@ def load_library(path=None):
         ip = C.POINTER(C.c_int)
         lib.fo_jit_stats.argtypes = [ip, ip, ip]
         lib.fo_jit_stats.restype = C.c_int
+        lib.fo_cell_stamps.argtypes = [vp, vp, C.POINTER(C.c_ulonglong)]
+        lib.fo_cell_stamps.restype = C.c_int
         lib.fo_tune.argtypes = [C.c_char_p, C.c_char_p]
         lib.fo_tune.restype = C.c_int
         lib.fo_jit_prepare.argtypes = [chain_p, i32, i32, i32]
@@ -362,6 +364,16 @@ def tune(name, value=None):
     _check(load_library().fo_tune(name.encode(), None if value is None else str(value).encode()), "fo_tune")
 
 
+def cell_stamps(device=None):
+    """(start, scan done, partials published, result written) of the last streaming Cell /
+    MAgg call made with the knob cell.stamps = 1, in ns of the GPU's global timer."""
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    buf = workspace(device, 16384)
+    ns = (C.c_ulonglong * 4)()
+    _check(load_library().fo_cell_stamps(C.c_void_p(buf.data_ptr()), _stream(device), ns), "fo_cell_stamps")
+    return tuple(int(x) for x in ns)
+
+
 JIT_OFF, JIT_FIRST_USE, JIT_PREPARED = 0, 1, 2
 
 
@@ -458,8 +470,10 @@ def device_status(device=None):
 
 
 # ------------------------------------------------------------------ the four calls
-def fused_cell(steps, output, X, sides=(), scalars=(), agg="full", out=None):
-    """Cell template.  Returns a tensor: scalar (1,), (rows,), (cols,) or (rows, cols)."""
+def fused_cell(steps, output, X, sides=(), scalars=(), agg="full", out=None, out_nnz=None):
+    """Cell template.  Returns a tensor: scalar (1,), (rows,), (cols,) or (rows, cols).
+    out_nnz: an int64 tensor of one element that receives the number of non-zero values
+    of a no_agg result."""
     lib = load_library()
     sides = list(sides)
     ch, keep = make_chain(steps, output)
@@ -474,9 +488,11 @@ def fused_cell(steps, output, X, sides=(), scalars=(), agg="full", out=None):
     need = lib.fused_cell_workspace_bytes(C.byref(m), a)
     ws = workspace(dev, max(need, 16384))
     sarr, sc = _sides(sides, rows, cols), _scalars(scalars)
+    if out_nnz is not None:
+        assert out_nnz.dtype == torch.int64 and out_nnz.numel() == 1 and out_nnz.device == dev
     _check(lib.fused_cell(C.byref(ch), C.byref(m), sarr, len(sides), sc, len(scalars), a,
-                          C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
-                          _stream(dev)), "fused_cell")
+                          C.c_void_p(out.data_ptr()), C.c_void_p(out_nnz.data_ptr()) if out_nnz is not None else None,
+                          C.c_void_p(ws.data_ptr()), ws.numel(), _stream(dev)), "fused_cell")
     return out
 
 
@@ -575,8 +591,9 @@ def fused_row_b1(pre, pre_out, post, post_out, X, B, sides=(), scalars=(), agg="
     return out
 
 
-def fused_outer(steps, output, X, U, V, scalars=(), agg="full", out=None):
-    """Outer template over the stored cells of the CSR matrix X."""
+def fused_outer(steps, output, X, U, V, scalars=(), agg="full", out=None, sides=(), out_nnz=None):
+    """Outer template over the stored cells of the CSR matrix X.  sides: dense side inputs
+    [("cell" | "row" | "col", tensor), ...] read at the stored cell; out_nnz as in fused_cell."""
     lib = load_library()
     ch, keep = make_chain(steps, output)
     xs = X.as_struct()
@@ -590,7 +607,12 @@ def fused_outer(steps, output, X, U, V, scalars=(), agg="full", out=None):
     need = lib.fused_outer_workspace_bytes(C.byref(xs), rank, a)
     ws = workspace(dev, max(need, 16384))
     sc = _scalars(scalars)
-    _check(lib.fused_outer(C.byref(ch), C.byref(xs), C.byref(us), C.byref(vs), sc, len(scalars), a,
-                           C.c_void_p(out.data_ptr()), C.c_void_p(ws.data_ptr()), ws.numel(),
-                           _stream(dev)), "fused_outer")
+    sides = list(sides)
+    sarr = _sides(sides, X.rows, X.cols)
+    if out_nnz is not None:
+        assert out_nnz.dtype == torch.int64 and out_nnz.numel() == 1 and out_nnz.device == dev
+    _check(lib.fused_outer(C.byref(ch), C.byref(xs), C.byref(us), C.byref(vs), sarr, len(sides), sc,
+                           len(scalars), a, C.c_void_p(out.data_ptr()),
+                           C.c_void_p(out_nnz.data_ptr()) if out_nnz is not None else None,
+                           C.c_void_p(ws.data_ptr()), ws.numel(), _stream(dev)), "fused_outer")
     return out

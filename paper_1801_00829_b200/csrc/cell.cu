@@ -250,6 +250,23 @@ cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ Ce
     }
 }
 
+// Non-zero entries of an elementwise result: integer counts, so the total does not
+// depend on the order in which the CTAs add theirs.
+__global__ void __launch_bounds__(kThreads)
+count_nonzero_kernel(const double *__restrict__ values, long long n, unsigned long long *out_nnz)
+{
+    __shared__ unsigned int s_count;
+    if (threadIdx.x == 0) s_count = 0u;
+    __syncthreads();
+    unsigned int mine = 0;
+    for (long long i = blockIdx.x * (long long)kThreads + threadIdx.x; i < n; i += (long long)gridDim.x * kThreads)
+        mine += __ldcg(values + i) != 0.0 ? 1u : 0u;
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&s_count, mine);
+    __syncthreads();
+    if (threadIdx.x == 0 && s_count) atomicAdd(out_nnz, (unsigned long long)s_count);
+}
+
 __global__ void fill_zero_kernel(double *out, long long n)
 {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n;
@@ -260,22 +277,12 @@ __global__ void fill_zero_kernel(double *out, long long n)
 // ------------------------------------------------------------------ host
 bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
-// CTAs per SM of the streaming kernels.  FUSEDOPS_CELL_CTAS_PER_SM (1..8, read once)
-// overrides the default; it is a tuning knob, results do not depend on it beyond
-// the order of the per-CTA partial sums.
+// CTAs per SM of the streaming kernels (the knob cell.ctas_per_sm, 1..8, overrides the
+// default; results do not depend on it beyond the order of the per-CTA partial sums).
 int cell_ctas_per_sm()
 {
-    static int cached = 0;
-    if (cached == 0) {
-        int v = 3;        // measured: 2-3 is best for 10-100 MB inputs, larger inputs do not care
-        const char *e = getenv("FUSEDOPS_CELL_CTAS_PER_SM");
-        if (e) {
-            const int x = atoi(e);
-            if (x >= 1 && x <= 8) v = x;
-        }
-        cached = v;
-    }
-    return cached;
+    const int v = tune_int("cell.ctas_per_sm", 3);    // measured: 2-3 is best for 10-100 MB inputs, larger inputs do not care
+    return (v >= 1 && v <= 8) ? v : 3;
 }
 
 // Grid of a streaming kernel: every CTA gets work, at most `cap` CTAs.
@@ -399,12 +406,22 @@ bool g_force_interpreter = false;
 
 // Common body of fused_cell and fused_magg.
 int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
-             const double *scalars, int n_scalars, int agg, bool magg, double *out, void *ws,
-             size_t ws_bytes, void *stream, bool may_compile)
+             const double *scalars, int n_scalars, int agg, bool magg, double *out, long long *out_nnz,
+             void *ws, size_t ws_bytes, void *stream, bool may_compile)
 {
     if (!chain || !X || !out) return FO_ERR_NULL;
     if (n_sides > 0 && !sides) return FO_ERR_NULL;
     if (agg < FO_CELL_NO_AGG || agg > FO_CELL_FULL_AGG) return FO_ERR_UNSUPPORTED;
+    if (out_nnz && agg != FO_CELL_NO_AGG) return FO_ERR_UNSUPPORTED;      // a count needs an elementwise result
+    if (out_nnz) {
+        // the elementwise result first, then one more pass over it for the count
+        const int rc = run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, magg, out, nullptr, ws,
+                                ws_bytes, stream, may_compile);
+        if (rc != FO_OK) return rc;
+        const long long n = X->kind == FO_CSR ? X->csr.nnz : X->dense.rows * X->dense.cols;
+        const cudaError_t e = launch_count_nonzero(out, n, out_nnz, (cudaStream_t)stream);
+        return e == cudaSuccess ? FO_OK : cuda_fail(e);
+    }
     if (X->kind == FO_CSR)
         return run_cell_csr(chain, X->csr, sides, n_sides, scalars, n_scalars, agg, magg, out, ws, ws_bytes,
                             stream);
@@ -459,6 +476,7 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     p.head = (WsHead *)ws;
     p.partials = (double *)((char *)ws + sizeof(WsHead));
     p.out = out;
+    p.stamps = tune_int("cell.stamps", 0) ? reinterpret_cast<unsigned long long *>(&p.head->pad[0]) : nullptr;
 
     cudaStream_t st = (cudaStream_t)stream;
     const long long ncells = xd.rows * xd.cols;
@@ -517,6 +535,17 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
 
 bool force_interpreter() { return g_force_interpreter; }
 
+cudaError_t launch_count_nonzero(const double *values, long long n, long long *out_nnz, cudaStream_t st)
+{
+    cudaError_t e = cudaMemsetAsync(out_nnz, 0, sizeof(long long), st);
+    if (e != cudaSuccess || n <= 0) return e;
+    long long grid = (n + 4 * kThreads - 1) / (4 * kThreads);
+    const long long cap = (long long)(sm_count() > 0 ? sm_count() : 148) * 8;
+    if (grid > cap) grid = cap;
+    count_nonzero_kernel<<<(unsigned)grid, kThreads, 0, st>>>(values, n, (unsigned long long *)out_nnz);
+    return cudaGetLastError();
+}
+
 }  // namespace fo
 
 namespace fo {
@@ -570,11 +599,27 @@ int fused_cell_static(const fo_chain *chain, const fo_mat *X, const fo_side *sid
     if (!ws) return FO_ERR_CUDA;
     // never compiles or loads a kernel: a chain specialised earlier is reused, any other
     // one runs through the built-in code
-    return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, false, out, ws,
+    return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, false, out, nullptr, ws,
                         fo::kStaticWsBytes, stream, false);
 }
 
 size_t fused_cell_static_limit_bytes(void) { return fo::kStaticWsBytes; }
+
+int fo_cell_stamps(void *ws, void *stream, unsigned long long *ns)
+{
+    if (!ws || !ns) return FO_ERR_NULL;
+    fo::WsHead *head = (fo::WsHead *)ws;
+    unsigned long long raw[4];
+    cudaError_t e = cudaMemcpyAsync(raw, &head->pad[0], sizeof(raw), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(&head->pad[0], 0, sizeof(raw), (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return fo::cuda_fail(e);
+    ns[0] = ~raw[0];
+    ns[1] = raw[1];
+    ns[2] = raw[2];
+    ns[3] = raw[3];
+    return FO_OK;
+}
 
 int fo_set_force_interpreter(int on)
 {
@@ -600,10 +645,10 @@ size_t fused_magg_workspace_bytes(const fo_mat *X, int n_out)
 }
 
 int fused_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
-               const double *scalars, int n_scalars, int agg, double *out, void *ws,
+               const double *scalars, int n_scalars, int agg, double *out, long long *out_nnz, void *ws,
                size_t ws_bytes, void *stream)
 {
-    return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, false, out, ws,
+    return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, agg, false, out, out_nnz, ws,
                         ws_bytes, stream, true);
 }
 
@@ -612,7 +657,7 @@ int fused_magg(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int
                void *stream)
 {
     return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, FO_CELL_FULL_AGG, true, out,
-                        ws, ws_bytes, stream, true);
+                        nullptr, ws, ws_bytes, stream, true);
 }
 
 }  // extern "C"

@@ -19,7 +19,19 @@ struct CellParams {
     double *out;
     int panels;           // cell_cols_kernel: number of row panels
     int cx;               // cell_cols_kernel: column pairs per CTA
+    unsigned long long *stamps;   // flat kernel: where to record phase times (measurement), or NULL
 };
+
+// Time stamps of the flat kernel's phases, in nanoseconds of the GPU's global timer,
+// kept in the workspace head when a measurement asks for them: [0] the complement of
+// the earliest CTA start, [1] the latest end of a CTA's scan, [2] the latest
+// publication of a partial sum, [3] the final result written.
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 
 constexpr int kV = 4;     // cells per thread per chain evaluation
 
@@ -57,8 +69,41 @@ __device__ __forceinline__ void cell_flat_body(const DevChain &ch, const CellPar
     const long long ncells = p.rows * p.cols;
     const long long ntiles = ncells >> 10;          // full tiles of 1024 cells
     const int t = threadIdx.x;
+    if (p.stamps && t == 0) atomicMax(&p.stamps[0], ~global_ns());
 
-    for (long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    // two tiles a trip while they last: twice the loads in flight per thread, which is what
+    // a small input (a few tiles per CTA in all) has to hide the memory latency with
+    // (straight-line chains only: the interpreter's register file does not fit twice)
+    long long tile = blockIdx.x;
+    for (; !EVAL::kInterp && tile + gridDim.x < ntiles; tile += 2ll * gridDim.x) {
+        const long long a0 = (tile << 10) + 2 * t, a1 = a0 + 512;
+        const long long b0 = ((tile + gridDim.x) << 10) + 2 * t, b1 = b0 + 512;
+        double in[kIn][kV], in2[kIn][kV];
+        put4(in[0], ld_stream2(p.X + a0), ld_stream2(p.X + a1));
+        put4(in2[0], ld_stream2(p.X + b0), ld_stream2(p.X + b1));
+#pragma unroll
+        for (int k = 0; k < FO_MAX_SIDES; ++k) {
+            if (EVAL::uses_side(ch, k)) {
+                const double *sp = p.sides.s[k].data;
+                put4(in[1 + k], ld_stream2(sp + a0), ld_stream2(sp + a1));
+                put4(in2[1 + k], ld_stream2(sp + b0), ld_stream2(sp + b1));
+            }
+        }
+        double o[NOUT][kV], o2[NOUT][kV];
+        EVAL::template run<kV, NOUT>(ch, in, o);
+        EVAL::template run<kV, NOUT>(ch, in2, o2);
+        if (STORE) {
+            *reinterpret_cast<double2 *>(p.out + a0) = make_double2(o[0][0], o[0][1]);
+            *reinterpret_cast<double2 *>(p.out + a1) = make_double2(o[0][2], o[0][3]);
+            *reinterpret_cast<double2 *>(p.out + b0) = make_double2(o2[0][0], o2[0][1]);
+            *reinterpret_cast<double2 *>(p.out + b1) = make_double2(o2[0][2], o2[0][3]);
+        } else {
+            const bool valid[kV] = {true, true, true, true};
+            add_outputs<NOUT>(o, valid, acc);
+            add_outputs<NOUT>(o2, valid, acc);
+        }
+    }
+    for (; tile < ntiles; tile += gridDim.x) {
         const long long o0 = (tile << 10) + 2 * t, o1 = o0 + 512;
         double in[kIn][kV];
         put4(in[0], ld_stream2(p.X + o0), ld_stream2(p.X + o1));
@@ -112,14 +157,19 @@ __device__ __forceinline__ void cell_flat_body(const DevChain &ch, const CellPar
     }
 
     if (!STORE) {
+        if (p.stamps && t == 0) atomicMax(&p.stamps[1], global_ns());
         block_sum<NOUT>(acc, s_red);
         if (t == 0) {
 #pragma unroll
             for (int k = 0; k < NOUT; ++k)
                 if (k < ch.n_out) p.partials[(size_t)blockIdx.x * ch.n_out + k] = acc[k];
         }
-        if (publish_and_is_last(p.head, &s_flag))
+        const bool last = publish_and_is_last(p.head, &s_flag);
+        if (p.stamps && t == 0) atomicMax(&p.stamps[2], global_ns());
+        if (last) {
             final_sum_small(p.partials, gridDim.x, ch.n_out, p.out, s_red);
+            if (p.stamps && t == 0) p.stamps[3] = global_ns();
+        }
     }
 }
 

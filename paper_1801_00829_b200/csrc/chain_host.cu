@@ -60,7 +60,7 @@ int locate(uint8_t o, Alloc &al, int imm_slot)
     const int cls = o >> 6, idx = o & 0x3f;
     switch (cls) {
         case 0: return al.reg_tmp[idx] >= 0 ? al.reg_tmp[idx] : kBad;
-        case 1: al.side_used |= 1u << idx; return 1 + idx;
+        case 1: al.side_used |= 1u << idx; return (al.use == kUseOuter ? 2 : 1) + idx;
         case 2: return 0x80 | idx;
         default:
             if (o == FO_MAIN) return 0;
@@ -83,7 +83,7 @@ int translate_chain(const fo_chain *chain, ChainUse use, int n_sides,
     if (n_sides < 0 || n_sides > FO_MAX_SIDES) return FO_ERR_UNSUPPORTED;
     if (n_scalars < 0 || n_scalars > FO_MAX_SCALARS) return FO_ERR_UNSUPPORTED;
     if (n_scalars > 0 && !scalars) return FO_ERR_NULL;
-    if (use == kUseOuter && n_sides != 0) return FO_ERR_UNSUPPORTED;
+    if (use == kUseOuter && n_sides > kOuterMaxSides) return FO_ERR_UNSUPPORTED;
 
     memset(out, 0, sizeof(*out));
     Alloc al;
@@ -91,7 +91,7 @@ int translate_chain(const fo_chain *chain, ChainUse use, int n_sides,
     al.use = use;
     al.n_sides = n_sides;
     al.n_scalars = n_scalars;
-    al.base = (use == kUseOuter) ? 2 : 1 + n_sides;
+    al.base = (use == kUseOuter) ? 2 + n_sides : 1 + n_sides;
     al.high = al.base;
     for (int k = 0; k < FO_MAX_TMPS; ++k) { al.reg_tmp[k] = -1; al.def_tmp[k] = -1; }
 
@@ -245,11 +245,10 @@ struct Knob {
     bool set;
 };
 Knob g_knobs[] = {
-    {"cell.ctas_per_sm", "", false}, {"row.dense_shape", "", false}, {"row.narrow", "", false},
+    {"cell.ctas_per_sm", "", false}, {"row.narrow", "", false},
     {"b1.shape", "", false},         {"b1.mma_shape", "", false},    {"b1.narrow", "", false},
-    {"b1.mma", "", false},           {"outer.kernel", "", false},    {"outer.depth", "", false},
-    {"outer.warps", "", false},      {"outer.hints", "", false},     {"outer.dense", "", false},
-    {"csr.variant", "", false},      {"cell.stamps", "", false},
+    {"b1.mma", "", false},           {"outer.kernel", "", false},
+    {"cell.stamps", "", false},
 };
 std::mutex g_knob_mutex;
 std::atomic<int> g_knobs_set{0};

@@ -39,8 +39,9 @@ constexpr int kThreads = 256;        // CTA size of the reduction kernels
 // a run-time index; temporaries follow, packed by live range):
 //   Cell / MAgg : R0 = a,  R(1+k) = side k
 //   Row         : R0 = d,  R(1+k) = side k
-//   Outer       : R0 = a,  R1 = d
+//   Outer       : R0 = a,  R1 = d,  R(2+k) = side k  (at most kOuterMaxSides sides)
 constexpr int kRegs = 13;            // 1 + FO_MAX_SIDES + FO_MAX_TMPS
+constexpr int kOuterMaxSides = 3;    // 2 + sides + FO_MAX_TMPS registers must fit kRegs
 constexpr int kConsts = 40;          // FO_MAX_SCALARS + FO_MAX_OPS
 
 struct DevOp {
@@ -97,6 +98,10 @@ bool tune_get(const char *name, char *value, size_t cap);
 int tune_int(const char *name, int fallback);
 
 int check_workspace(const void *ws, size_t ws_bytes, size_t need);
+
+// *out_nnz (device) = number of values[0..n) that are not zero: one more pass over an
+// elementwise result, asynchronous on `st` (cell.cu).
+cudaError_t launch_count_nonzero(const double *values, long long n, long long *out_nnz, cudaStream_t st);
 int cuda_fail(cudaError_t e);
 int sm_count();
 #endif

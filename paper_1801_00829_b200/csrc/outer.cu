@@ -34,6 +34,7 @@ struct OuterParams {
     double *out;
     int kconst;                  // constant-table index an inline chain reads
     int pad;
+    DevSides sides;              // dense side inputs read at the stored cell (outer_kernel only)
 };
 
 enum { kOutFull = 0, kOutNone = 1, kOutRight = 2, kOutLeft = 3 };
@@ -54,19 +55,30 @@ __device__ __forceinline__ double2 ld_pair_cached(const double *row, int col, in
     return make_double2(0.0, 0.0);
 }
 
-// A chain without an inline form runs through the interpreter, out of line: its
-// register file would otherwise be counted against every kernel's main loop.
-__device__ __noinline__ double outer_chain_generic(const DevChain &ch, double a, double d)
+// The interpreter for a chain without an inline form: R0 = a, R1 = d, R(2 + k) = side k.
+__device__ __forceinline__ double outer_chain_interp(const DevChain &ch, double a, double d,
+                                                     const double (&sv)[kOuterMaxSides])
 {
     RegFile<kRegs, 1> f;
     f.r[0][0] = a;
     f.r[1][0] = d;
+#pragma unroll
+    for (int k = 0; k < kOuterMaxSides; ++k) f.r[2 + k][0] = sv[k];
     run_chain<kRegs, 1>(ch, f);
     double o[1];
     operand<kRegs, 1>(ch, f, ch.out[0], o);
     return o[0];
 }
 
+// The same, out of line: for a kernel whose main loop should not carry the
+// interpreter's register file.
+__device__ __noinline__ double outer_chain_interp_call(const DevChain &ch, double a, double d)
+{
+    const double none[kOuterMaxSides] = {0.0, 0.0, 0.0};
+    return outer_chain_interp(ch, a, d, none);
+}
+
+template <bool OUT_OF_LINE = false>
 __device__ __forceinline__ double outer_chain(const DevChain &ch, int kind, int kc, double a, double d)
 {
     if (kind == kOuterWsloss) {
@@ -77,7 +89,9 @@ __device__ __forceinline__ double outer_chain(const DevChain &ch, int kind, int 
     }
     if (kind == kOuterXlogd) return a * slow_log(d + ch.consts[kc]);
     if (kind == kOuterMaskDot) return (a != 0.0 ? 1.0 : 0.0) * d;      // (X != 0) * (U V^T), Eq. 1
-    return outer_chain_generic(ch, a, d);
+    if (OUT_OF_LINE) return outer_chain_interp_call(ch, a, d);
+    const double none[kOuterMaxSides] = {0.0, 0.0, 0.0};
+    return outer_chain_interp(ch, a, d, none);
 }
 
 // First row r in [0, rows] with rowptr[r] >= target, found by the 32 lanes of a
@@ -183,7 +197,25 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
                 if ((lane >> 2) == it) dmine = allA;
                 if ((lane >> 2) == it + 1) dmine = allB;
             }
-            const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
+            double w;
+            if (ch.side_used) {
+                // side inputs at this lane's cell (i, j): a matrix at (i, j), a column vector at i,
+                // a row vector at j
+                double sv[kOuterMaxSides];
+#pragma unroll
+                for (int k = 0; k < kOuterMaxSides; ++k) {
+                    sv[k] = 0.0;
+                    if (valid && ((ch.side_used >> k) & 1u)) {
+                        const DevSide sd = p.sides.s[k];
+                        sv[k] = sd.access == FO_AT_ROW ? __ldg(sd.data + row * sd.ld)
+                              : sd.access == FO_AT_COL ? __ldg(sd.data + jmine)
+                                                       : __ldg(sd.data + row * sd.ld + jmine);
+                    }
+                }
+                w = outer_chain_interp(ch, amine, dmine, sv);
+            } else {
+                w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
+            }
             if (AGG == kOutFull) {
                 if (valid) acc += w;
             } else if (AGG == kOutNone) {
@@ -578,7 +610,7 @@ outer_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ 
                 const int r = 8 * warp + rr;
                 const bool in = jj[rr] < nhi;
                 if (in) {
-                    const double w = outer_chain(ch, p.chain_kind, p.kconst, aa[rr], Ps[(size_t)r * PLD + (jj[rr] - n0)]);
+                    const double w = outer_chain<true>(ch, p.chain_kind, p.kconst, aa[rr], Ps[(size_t)r * PLD + (jj[rr] - n0)]);
                     if (AGG == kOutFull) acc += w;
                     else p.out[cur[r] + lane] = w;
                 }
@@ -727,14 +759,16 @@ size_t fused_outer_workspace_bytes(const fo_csr *X, int rank, int agg)
 }
 
 int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const fo_dense *V,
-                const double *scalars, int n_scalars, int agg, double *out, void *ws,
-                size_t ws_bytes, void *stream)
+                const fo_side *sides, int n_sides, const double *scalars, int n_scalars, int agg, double *out,
+                long long *out_nnz, void *ws, size_t ws_bytes, void *stream)
 {
     using namespace fo;
     if (!chain || !X || !U || !V || !out) return FO_ERR_NULL;
+    if (n_sides > 0 && !sides) return FO_ERR_NULL;
     if (agg != FO_OUTER_FULL_AGG && agg != FO_OUTER_NO_AGG && agg != FO_OUTER_RIGHT_MM &&
         agg != FO_OUTER_LEFT_MM)
         return FO_ERR_UNSUPPORTED;
+    if (out_nnz && agg != FO_OUTER_NO_AGG) return FO_ERR_UNSUPPORTED;     // a count needs an elementwise result
     if (X->rows < 0 || X->cols < 0 || X->nnz < 0) return FO_ERR_SHAPE;
     if (X->nnz >= (1ll << 31)) return FO_ERR_UNSUPPORTED;
     if (U->rows != X->rows || V->rows != X->cols || U->cols != V->cols) return FO_ERR_SHAPE;
@@ -744,15 +778,37 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     if (!X->rowptr) return FO_ERR_NULL;
     if (X->nnz > 0 && (!X->colidx || !X->vals)) return FO_ERR_NULL;
     if (rank > 0 && ((X->rows > 0 && !U->data) || (X->cols > 0 && !V->data))) return FO_ERR_NULL;
+    if (out_nnz) {
+        // the elementwise result first, then one more pass over it for the count
+        const int rc0 = fused_outer(chain, X, U, V, sides, n_sides, scalars, n_scalars, agg, out, nullptr, ws,
+                                    ws_bytes, stream);
+        if (rc0 != FO_OK) return rc0;
+        const cudaError_t ce = launch_count_nonzero(out, X->nnz, out_nnz, (cudaStream_t)stream);
+        return ce == cudaSuccess ? FO_OK : cuda_fail(ce);
+    }
 
     DevChain ch;
-    int rc = translate_chain(chain, kUseOuter, 0, scalars, n_scalars, 1, 1, &ch);
+    int rc = translate_chain(chain, kUseOuter, n_sides, scalars, n_scalars, 1, 1, &ch);
     if (rc != FO_OK) return rc;
     rc = check_workspace(ws, ws_bytes, fused_outer_workspace_bytes(X, rank, agg));
     if (rc != FO_OK) return rc;
 
     OuterParams p;
     memset(&p, 0, sizeof(p));
+    p.sides.n = n_sides;
+    for (int k = 0; k < n_sides; ++k) {
+        const fo_side &sd = sides[k];
+        if (sd.sparse) return FO_ERR_UNSUPPORTED;            // dense side inputs only
+        if (sd.m.rows < 0 || sd.m.cols < 0 || sd.m.ld < sd.m.cols) return FO_ERR_SHAPE;
+        const bool fits = sd.access == FO_AT_CELL ? (sd.m.rows == X->rows && sd.m.cols == X->cols)
+                        : sd.access == FO_AT_ROW ? (sd.m.rows == X->rows && sd.m.cols == 1)
+                        : sd.access == FO_AT_COL ? (sd.m.rows == 1 && sd.m.cols == X->cols) : false;
+        if (!fits) return FO_ERR_SHAPE;
+        if (sd.m.rows > 0 && sd.m.cols > 0 && !sd.m.data) return FO_ERR_NULL;
+        p.sides.s[k].data = sd.m.data;
+        p.sides.s[k].ld = sd.m.ld;
+        p.sides.s[k].access = sd.access;
+    }
     p.rowptr = X->rowptr; p.colidx = X->colidx; p.vals = X->vals;
     p.rows = X->rows; p.cols = X->cols; p.nnz = X->nnz; p.rank = rank;
     p.U = U->data; p.ldu = U->ld; p.V = V->data; p.ldv = V->ld;
@@ -789,7 +845,10 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     cudaError_t e;
     const int nk2 = (rank + 15) / 16;
     // factor rows that are whole 16-byte pieces can be copied asynchronously into shared memory
-    const bool copyable = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && agg != FO_OUTER_LEFT_MM;
+    // (a chain that reads side inputs runs through the kernel that gathers into registers:
+    // it is the one that knows every cell's row and column where the chain is evaluated)
+    const bool copyable = aligned && rank % 2 == 0 && rank >= 2 && nk2 <= 8 && agg != FO_OUTER_LEFT_MM &&
+                          ch.side_used == 0;
     char which[48] = "";
     tune_get("outer.kernel", which, sizeof(which));
     const bool want_direct = strcmp(which, "direct") == 0;

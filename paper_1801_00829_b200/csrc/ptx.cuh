@@ -38,10 +38,11 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned 
         : "memory");
     return ok != 0;
 }
-// Bounded wait: returns false (and the caller records it) if the phase never completes.
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity)
+// Bounded wait: returns false (and the caller records it) if the phase has not completed
+// after `limit` polls.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, unsigned limit = kWaitLimit)
 {
-    for (unsigned i = 0; i < kWaitLimit; ++i)
+    for (unsigned i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

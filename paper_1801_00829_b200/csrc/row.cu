@@ -728,20 +728,9 @@ struct DenseShape {
     int nch, w, r;
 };
 
-// Shapes that are compiled.  FUSEDOPS_DENSE_SHAPE="nch,w,r" (read per call; a
-// tuning knob) picks one of them if it covers the column count.
-const DenseShape kDenseShapes[] = {{1, 1, 4}, {1, 2, 4}, {1, 4, 8}, {1, 8, 8}, {1, 16, 8}, {2, 16, 4},
-                                   {4, 16, 2}, {8, 16, 1}, {2, 8, 4}, {4, 4, 2}, {8, 2, 1}, {4, 4, 1}, {2, 8, 2}, {2, 4, 4}, {4, 8, 2}, {1, 1, 8}, {1, 2, 8}};
-
+// The shapes below are the ones compiled.
 DenseShape dense_shape(long long n)
 {
-    const char *e = getenv("FUSEDOPS_DENSE_SHAPE");
-    if (e) {
-        int a = 0, b = 0, c = 0;
-        if (sscanf(e, "%d,%d,%d", &a, &b, &c) == 3)
-            for (const DenseShape &k : kDenseShapes)
-                if (k.nch == a && k.w == b && k.r == c && (long long)64 * a * b >= n) return k;
-    }
     // measured on B200: several small independent groups beat one large group
     // (1000 columns: {4,4,2} 6.6 TB/s, {2,8,4} 6.4, {1,16,8} 5.1)
     // (512: {1,8,8} 6.2 vs {2,4,4} 5.9; 2048: {2,16,4} 6.0 vs {4,8,2} 5.1)
@@ -762,9 +751,8 @@ cudaError_t launch_dense(const DevChain &ch, const RowParams &p, int agg, int gr
     const DenseShape k = dense_shape(p.cols);
 #define FO_SHAPE(A, B, C) \
     if (k.nch == A && k.w == B && k.r == C) return launch_dense_agg<A, B, C, STAGED>(ch, p, agg, grid, smem, st);
-    FO_SHAPE(1, 1, 4) FO_SHAPE(1, 2, 4) FO_SHAPE(1, 4, 8) FO_SHAPE(1, 8, 8) FO_SHAPE(1, 16, 8)
-    FO_SHAPE(2, 16, 4) FO_SHAPE(4, 16, 2) FO_SHAPE(8, 16, 1) FO_SHAPE(2, 8, 4) FO_SHAPE(4, 4, 2)
-    FO_SHAPE(8, 2, 1) FO_SHAPE(4, 4, 1) FO_SHAPE(2, 8, 2) FO_SHAPE(2, 4, 4) FO_SHAPE(4, 8, 2) FO_SHAPE(1, 1, 8) FO_SHAPE(1, 2, 8)
+    FO_SHAPE(1, 1, 8) FO_SHAPE(1, 2, 8) FO_SHAPE(1, 4, 8) FO_SHAPE(1, 8, 8) FO_SHAPE(4, 4, 2)
+    FO_SHAPE(2, 16, 4) FO_SHAPE(4, 16, 2) FO_SHAPE(8, 16, 1)
 #undef FO_SHAPE
     return cudaErrorInvalidValue;
 }
@@ -908,9 +896,8 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
         p.X = X->dense.data; p.ldx = X->dense.ld;
         p.out_vec = (aligned16(out) && cols % 2 == 0) ? 1 : 0;
         if (cols <= kNarrowMax) {
-            // a thread per row; FUSEDOPS_ROW_NARROW=0 keeps the warp-per-row-slice kernel (a measuring knob)
-            const char *ne = getenv("FUSEDOPS_ROW_NARROW");
-            if (!(ne && ne[0] == '0')) {
+            // a thread per row; the knob row.narrow = 0 keeps the warp-per-row-slice kernel
+            if (tune_int("row.narrow", 1) != 0) {
                 const bool vec = aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0);
                 long long grid = (rows + kThreads - 1) / kThreads;
                 const long long cap = (long long)sms * 4 < row_grid_cap() ? (long long)sms * 4 : row_grid_cap();

@@ -937,9 +937,9 @@ bool b1_complete(B1Shape &s, long long n, int k)
 
 bool b1_shape(long long n, int k, B1Shape *out)
 {
-    // FUSEDOPS_B1_SHAPE="nch,r,kl" (read per call; a tuning knob) picks a compiled shape
-    const char *e = getenv("FUSEDOPS_B1_SHAPE");
-    if (e) {
+    // the knob b1.shape = "nch,r,kl" picks a compiled shape
+    char e[48];
+    if (tune_get("b1.shape", e, sizeof(e))) {
         int a = 0, b = 0, c = 0;
         if (sscanf(e, "%d,%d,%d", &a, &b, &c) == 3)
             for (const auto &t : kB1Compiled)
@@ -1007,9 +1007,9 @@ bool b1_mma_shape(long long n, int k, int nw, MmaShape *out)
 {
     const int kb = pow2_at_least((k + 7) / 8);
     if (kb > nw || n < 2) return false;
-    // FUSEDOPS_B1_MMA_SHAPE="ncb,w" (read per call; a tuning knob)
-    const char *e = getenv("FUSEDOPS_B1_MMA_SHAPE");
-    if (e) {
+    // the knob b1.mma_shape = "ncb,w"
+    char e[48];
+    if (tune_get("b1.mma_shape", e, sizeof(e))) {
         int a = 0, b = 0;
         if (sscanf(e, "%d,%d", &a, &b) == 2 && (a == 8 || a == 14 || a == 16 || a == 20) && b >= 1 &&
             (b & (b - 1)) == 0 && b * kb <= nw && (long long)8 * a * b >= n) {
@@ -1203,11 +1203,10 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
         return e2 == cudaSuccess ? FO_OK : cuda_fail(e2);
     }
     const bool staged = b1_aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0) && cols >= 2;
-    // narrow rows: a thread per row (FUSEDOPS_B1_NARROW=0 switches it off; a measuring knob)
+    // narrow rows: a thread per row (the knob b1.narrow = 0 switches it off)
     {
-        const char *ne = getenv("FUSEDOPS_B1_NARROW");
         const int nc = cols <= 8 ? 8 : 16, kc = k <= 2 ? 2 : k <= 4 ? 4 : 8;
-        if (!(ne && ne[0] == '0') && cols <= 16 && k <= 8 && nc * kc <= 64) {
+        if (tune_int("b1.narrow", 1) != 0 && cols <= 16 && k <= 8 && nc * kc <= 64) {
             const bool vec = b1_aligned16(p.X) && (p.ldx % 2 == 0) && (cols % 2 == 0);
             long long grid = (rows + kB1NarrowThreads - 1) / kB1NarrowThreads;
             const long long cap = (long long)sms * 2 < b1_grid_cap() ? (long long)sms * 2 : b1_grid_cap();
@@ -1234,11 +1233,11 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
             return en == cudaSuccess ? FO_OK : cuda_fail(en);
         }
     }
-    // tensor-core variant where its layout fits (FUSEDOPS_B1_MMA=0 / 1 forces the choice)
+    // tensor-core variant where its layout fits (the knob b1.mma = 0 / 1 forces the choice)
     {
         MmaShape ms;
-        const char *env = getenv("FUSEDOPS_B1_MMA");
-        const bool want = env ? env[0] != '0' : (k > 2 || cols <= 160);
+        const int forced = tune_int("b1.mma", -1);
+        const bool want = forced >= 0 ? forced != 0 : (k > 2 || cols <= 160);
         // 8 warps (two per scheduler, up to 255 registers each) measured faster than 16
         // warps of 128 registers in every layout tried: 0.81 against 1.06 ms at best for
         // 5 000 000 x 100, k = 8

@@ -82,7 +82,7 @@ def call_cell(lib, steps, output, m, sides=(), n_scalars=0, agg=3, ws=0x10000, w
     sarr = (B.fo_side * max(1, len(sides)))(*sides)
     sc = (C.c_double * 8)()
     return lib.fused_cell(C.byref(ch), C.byref(m), sarr, len(sides), sc, n_scalars, agg,
-                          C.c_void_p(out), C.c_void_p(ws), ws_bytes, None)
+                          C.c_void_p(out), None, C.c_void_p(ws), ws_bytes, None)
 
 
 def side(rows, cols, access, ptr=0x3000):
@@ -123,14 +123,14 @@ def test_sparse_side_is_refused_outside_the_sparse_driver_kernels(lib):
     ch, keep = B.make_chain([("mul", "t0", "a", "side0")], "t0")
     sc = (C.c_double * 8)()
     m = dense_mat(10, 10)
-    assert lib.fused_cell(C.byref(ch), C.byref(m), sd, 1, sc, 0, 3, C.c_void_p(0x2000),
+    assert lib.fused_cell(C.byref(ch), C.byref(m), sd, 1, sc, 0, 3, C.c_void_p(0x2000), None,
                           C.c_void_p(0x10000), 1 << 24, None) == -4
     # over a CSR main input: the side must have the main input's shape and be read at the cell
     x = B.fo_mat()
     x.kind = 1
     x.csr.rows, x.csr.cols, x.csr.nnz = 10, 12, 5
     x.csr.rowptr, x.csr.colidx, x.csr.vals = 0x5000, 0x6000, 0x7000
-    assert lib.fused_cell(C.byref(ch), C.byref(x), sd, 1, sc, 0, 3, C.c_void_p(0x2000),
+    assert lib.fused_cell(C.byref(ch), C.byref(x), sd, 1, sc, 0, 3, C.c_void_p(0x2000), None,
                           C.c_void_p(0x10000), 1 << 24, None) == -2
 
 
@@ -145,8 +145,12 @@ def test_chain_limits(lib):
     keep[0].opcode = 200
     sarr = (B.fo_side * 1)()
     sc = (C.c_double * 8)()
-    assert lib.fused_cell(C.byref(ch), C.byref(m), sarr, 0, sc, 0, 3, C.c_void_p(0x2000),
+    assert lib.fused_cell(C.byref(ch), C.byref(m), sarr, 0, sc, 0, 3, C.c_void_p(0x2000), None,
                           C.c_void_p(0x10000), 1 << 24, None) == -3
+    # a count of non-zero results needs an elementwise result
+    ok, keep_ok = B.make_chain([("mov", "t0", "a")], "t0")
+    assert lib.fused_cell(C.byref(ok), C.byref(m), sarr, 0, sc, 0, 3, C.c_void_p(0x2000), C.c_void_p(0x4000),
+                          C.c_void_p(0x10000), 1 << 24, None) == -4
 
 
 def test_row_and_outer_argument_errors(lib):
@@ -176,9 +180,11 @@ def test_row_and_outer_argument_errors(lib):
     v.rows, v.cols, v.ld, v.data = 12, 4, 4, 0x9000
     ch3, keep3 = B.make_chain([("sub", "t0", "a", "d")], "t0")
 
-    def outer(xx=x, uu=u, vv=v, agg=3):
-        return lib.fused_outer(C.byref(ch3), C.byref(xx), C.byref(uu), C.byref(vv), sc, 0, agg,
-                               C.c_void_p(0x2000), C.c_void_p(0x10000), 1 << 24, None)
+    no_sides = (B.fo_side * 1)()
+
+    def outer(xx=x, uu=u, vv=v, agg=3, chain=ch3, sides=no_sides, ns=0, nnz=None):
+        return lib.fused_outer(C.byref(chain), C.byref(xx), C.byref(uu), C.byref(vv), sides, ns, sc, 0, agg,
+                               C.c_void_p(0x2000), nnz, C.c_void_p(0x10000), 1 << 24, None)
 
     v2 = B.fo_dense()
     v2.rows, v2.cols, v2.ld, v2.data = 12, 5, 5, 0x9000
@@ -191,6 +197,14 @@ def test_row_and_outer_argument_errors(lib):
     x2.rows, x2.cols, x2.nnz = 10, 12, 1 << 31
     x2.rowptr, x2.colidx, x2.vals = 0x5000, 0x6000, 0x7000
     assert outer(xx=x2) == -4
+    # side inputs of the Outer template: dense, at most three, shaped like X under their access kind
+    ch4, keep4 = B.make_chain([("mul", "t0", "d", "side0")], "t0")
+    assert outer(chain=ch4) == -3                          # the chain names a side that is not passed
+    assert outer(chain=ch4, sides=(B.fo_side * 1)(side(10, 1, 1)), ns=1, agg=7) == -4
+    assert outer(chain=ch4, sides=(B.fo_side * 1)(side(10, 12, 1)), ns=1) == -2     # a column vector is rows x 1
+    assert outer(chain=ch4, sides=(B.fo_side * 1)(side(1, 10, 2)), ns=1) == -2      # a row vector is 1 x cols
+    assert outer(chain=ch4, sides=(B.fo_side * 4)(*[side(10, 1, 1)] * 4), ns=4) == -4
+    assert outer(nnz=C.c_void_p(0x4000)) == -4             # a count needs the no_agg variant
 
 
 def test_row_b1_argument_errors(lib):

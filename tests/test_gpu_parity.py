@@ -515,6 +515,77 @@ def test_outer_every_schedule_on_a_sparse_input(fo, outer_schedule, schedule):
         assert again.tobytes() == got.tobytes()
 
 
+@pytest.mark.parametrize("agg", ["full", "none", "right", "left"])
+@pytest.mark.parametrize("rank", [10, 100])
+def test_outer_side_inputs(fo, agg, rank):
+    """Dense side inputs of the Outer template (Table 1): a matrix read at (i, j), a column
+    vector at i, a row vector at j, in one chain; against the checker's masked and dense modes."""
+    w, Xh = outer_case(300, 260, rank, 0.05, seed=54)
+    m, n = w["rows"], w["cols"]
+    S = datagen.uniform(54, 5, m * n, -1.0, 1.0).reshape(m, n)
+    r = datagen.uniform(54, 6, m, 0.5, 2.0)
+    c = datagen.uniform(54, 7, n, -2.0, 2.0)
+    chain = [("sub", "t0", "a", "d"), ("mul", "t1", "t0", "side0"), ("add", "t2", "t1", "side2"),
+             ("mul", "t3", "t2", "side1")]                         # ((a - d) * S_ij + c_j) * r_i
+    sides_h = [("cell", S), ("row", r), ("col", c)]
+    sides_d = [("cell", to_dev(S)), ("row", to_dev(r)), ("col", to_dev(c))]
+    ref = oracle.outer(chain, "t3", Xh, w["U"], w["V"], agg=agg, mode="masked", sides=sides_h)
+    got = fo.fused_outer(chain, "t3", csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"]), agg=agg,
+                         sides=sides_d).cpu().numpy()
+    absch = [("sub", "t0", "a", "d"), ("abs", "t0", "t0"), ("mul", "t1", "t0", "side0"), ("add", "t2", "t1", "side2"),
+             ("mul", "t3", "t2", "side1")]
+    scale = oracle.outer(absch, "t3", Xh, np.abs(w["U"]), np.abs(w["V"]), agg=agg, mode="masked",
+                         sides=[("cell", np.abs(S)), ("row", r), ("col", np.abs(c))])
+    assert_close(got, ref, absscale=np.abs(scale) + 1e-300, what="outer sides %s" % agg)
+    if agg in ("full", "none"):
+        assert_close(got, oracle.outer(chain, "t3", Xh, w["U"], w["V"], agg=agg, mode="dense", sides=sides_h),
+                     absscale=np.abs(scale) + 1e-300, what="outer sides, dense mode")
+    # a side the chain does not read changes nothing: the staged schedule runs, same bits as without sides
+    if agg != "left":
+        plain = fo.fused_outer(WSLOSS, "t3", csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"]), agg=agg).cpu().numpy()
+        unused = fo.fused_outer(WSLOSS, "t3", csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"]), agg=agg,
+                                sides=sides_d[:1]).cpu().numpy()
+        assert plain.tobytes() == unused.tobytes()
+
+
+def test_nonzero_count_of_elementwise_results(fo):
+    """out_nnz: the number of non-zero values of a no_agg result - the nnz a sparse output
+    would store - equals the checker's count exactly (Cell over dense and CSR, Outer)."""
+    import torch
+    nnz = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    # Cell over CSR: the chain zeroes about half the stored cells, and X stores zeros of its own
+    w, Xh = outer_case(900, 700, 4, 0.05, seed=64)
+    w["vals"][::7] = 0.0
+    Xh = host_csr(w)
+    Y = datagen.normal(64, 9, w["rows"] * w["cols"]).reshape(w["rows"], w["cols"])
+    chain = [("gt", "t0", "side0", 0.0), ("mul", "t1", "a", "t0")]                 # a * (Y > 0)
+    ref = oracle.cell(chain, "t1", Xh, [("cell", Y)], agg="none")
+    got = fo.fused_cell(chain, "t1", csr_to_dev(w), [("cell", to_dev(Y))], agg="none", out_nnz=nnz).cpu().numpy()
+    assert_close(got, ref, what="cell csr none")
+    assert nnz.item() == oracle.count_nonzero(ref) and 0 < nnz.item() < len(ref)
+    # Cell over a dense input, ragged size
+    Xd = datagen.normal(64, 10, 501 * 333).reshape(501, 333)
+    chain = [("max", "t0", "a", 0.0)]                                              # relu: about half are zero
+    ref = oracle.cell(chain, "t0", Xd, agg="none")
+    got = fo.fused_cell(chain, "t0", to_dev(Xd), agg="none", out_nnz=nnz).cpu().numpy()
+    assert got.tobytes() == ref.tobytes()
+    assert nnz.item() == oracle.count_nonzero(ref)
+    # Outer no_agg: (a != 0) * d keeps the stored zeros of X at zero
+    chain = [("ne", "t0", "a", 0.0), ("mul", "t1", "t0", "d")]
+    ref = oracle.outer(chain, "t1", Xh, w["U"], w["V"], agg="none", mode="masked")
+    got = fo.fused_outer(chain, "t1", csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"]), agg="none",
+                         out_nnz=nnz).cpu().numpy()
+    assert_close(got, ref, what="outer none")
+    assert nnz.item() == oracle.count_nonzero(ref) == np.count_nonzero(w["vals"])
+    # an empty result counts zero; an aggregating variant refuses the count
+    empty = dict(rows=5, cols=6, rowptr=np.zeros(6, np.int32), colidx=np.zeros(0, np.int32), vals=np.zeros(0))
+    fo.fused_cell([("mov", "t0", "a")], "t0", csr_to_dev(empty), agg="none", out_nnz=nnz,
+                  out=torch.zeros(1, dtype=torch.float64, device="cuda"))       # (nothing is written to it)
+    assert nnz.item() == 0
+    with pytest.raises(fo.FusedOpsError):
+        fo.fused_cell(chain[:1], "t0", to_dev(Xd), agg="full", out_nnz=nnz)
+
+
 # ------------------------------------------------------------------ specialised vs interpreted chains
 @pytest.mark.parametrize("name,chain,outs,nsides", [
     ("mul2", [("mul", "t0", "a", "side0")], ["t0"], 1),

@@ -31,13 +31,10 @@ def fo():
 def path(request):
     """Runs a test once on the multiply-add kernels and once with the tensor-core
     kernels preferred (they take over wherever their layout fits)."""
-    old = os.environ.get("FUSEDOPS_B1_MMA")
-    os.environ["FUSEDOPS_B1_MMA"] = "0" if request.param == "fma" else "1"
+    import paper_1801_00829_b200 as fo_
+    fo_.tune("b1.mma", "0" if request.param == "fma" else "1")
     yield request.param
-    if old is None:
-        del os.environ["FUSEDOPS_B1_MMA"]
-    else:
-        os.environ["FUSEDOPS_B1_MMA"] = old
+    fo_.tune("b1.mma", None)
 
 
 def mm_scale(X, V):
@@ -132,10 +129,8 @@ def test_b1_every_compiled_shape(fo, shape):
     k = kl if kl > 2 else 2
     rows, cols = 3000 + r - 1, 200
     w = datagen.row_b1_workload(rows, cols, k, seed=9)
-    old = os.environ.get("FUSEDOPS_B1_SHAPE")
-    old_mma = os.environ.get("FUSEDOPS_B1_MMA")
-    os.environ["FUSEDOPS_B1_SHAPE"] = shape
-    os.environ["FUSEDOPS_B1_MMA"] = "0"
+    fo.tune("b1.shape", shape)
+    fo.tune("b1.mma", "0")
     try:
         for kk in (k, 2 * k):
             ww = w if kk == k else datagen.row_b1_workload(rows, cols, kk, seed=9)
@@ -144,11 +139,8 @@ def test_b1_every_compiled_shape(fo, shape):
             got = fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", to_dev(X), to_dev(V), [("cell", to_dev(P))])
             assert_close(got.cpu().numpy(), ref, absscale=mlr_scale(X, V, P), what="shape %s k=%d" % (shape, kk))
     finally:
-        for name, val in (("FUSEDOPS_B1_SHAPE", old), ("FUSEDOPS_B1_MMA", old_mma)):
-            if val is None:
-                del os.environ[name]
-            else:
-                os.environ[name] = val
+        fo.tune("b1.shape", None)
+        fo.tune("b1.mma", None)
     assert fo.device_status() == 0
 
 
@@ -252,14 +244,10 @@ def test_b1_narrow_rows_strided_unaligned(fo, cols, k):
             tabs = Q + P * Q.sum(axis=1, keepdims=True)
             assert_close(got.cpu().numpy(), ref, absscale=tabs if agg == "none" else np.abs(Xh).T @ tabs,
                          what="b1 narrow %dx%d off=%d %s" % (cols, k, off, agg))
-    old = os.environ.get("FUSEDOPS_B1_NARROW")
-    os.environ["FUSEDOPS_B1_NARROW"] = "0"
+    fo.tune("b1.narrow", "0")
     try:
         wide = fo.fused_row_b1(MLR_PRE, "t0", MLR_POST, "t2", Xd, to_dev(V), [("cell", to_dev(P))]).cpu().numpy()
     finally:
-        if old is None:
-            del os.environ["FUSEDOPS_B1_NARROW"]
-        else:
-            os.environ["FUSEDOPS_B1_NARROW"] = old
+        fo.tune("b1.narrow", None)
     assert_close(wide, oracle.mlogreg_inner(Xh, V, P), absscale=mlr_scale(Xh, V, P))
     assert fo.device_status() == 0
