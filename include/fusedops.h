@@ -199,17 +199,25 @@ int fo_last_cuda_error(void);
  *                     FO_JIT_PREPARED: the calls only look kernels up; a chain that
  *                     was not prepared runs through the interpreter, and no call
  *                     ever compiles, loads or allocates.  Returns the old mode.
- *   fo_jit_prepare()  compiles, loads and caches the kernel of a chain now, for the
- *                     current device (n_sides / n_scalars as in the later calls;
- *                     store != 0: the no_agg form, else the aggregating form).
+ *   fo_jit_prepare()  compiles, loads and caches the flat-stream kernel of a chain now,
+ *                     for the current device (n_sides / n_scalars as in the later
+ *                     calls; store != 0: the no_agg form, else the aggregating form).
  *                     FO_OK (also when it was cached already), a chain error,
  *                     FO_ERR_UNSUPPORTED without NVRTC / the driver library,
  *                     FO_ERR_CHAIN if the compilation or the load failed.
+ *   fo_jit_prepare_call()  the same for exactly the kernel a later fused_cell (magg = 0)
+ *                     or fused_magg (magg != 0) call with these arguments would run:
+ *                     X and the sides are looked at for shapes, leading dimensions
+ *                     and alignment only (no device access).  FO_OK also when the
+ *                     chain has a built-in form; FO_ERR_UNSUPPORTED for a CSR X (its
+ *                     kernel is compiled at first use, or never in FO_JIT_PREPARED).
  *   fo_jit_stats()    kernels compiled, specialised launches, failed compilations so
  *                     far; returns 1 if NVRTC and the driver library are usable. */
 enum { FO_JIT_OFF = 0, FO_JIT_FIRST_USE = 1, FO_JIT_PREPARED = 2 };
 int fo_set_jit(int mode);
 int fo_jit_prepare(const fo_chain *chain, int n_sides, int n_scalars, int store);
+int fo_jit_prepare_call(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
+                        int n_scalars, int agg, int magg);
 int fo_jit_stats(int *compiled, int *launches, int *failures);
 
 /* ------------------------------------------------------------------ Cell

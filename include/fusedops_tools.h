@@ -50,8 +50,11 @@ int fo_tune(const char *name, const char *value);
 int fo_cell_stamps(void *ws, void *stream, unsigned long long *ns);
 
 /* Generates and compiles (for sm_100a, without loading or launching: no GPU
- * needed) the run-time specialised kernel of a Cell chain; FO_OK, a chain error,
- * FO_ERR_UNSUPPORTED without NVRTC; the compiler log is copied to `log`. */
+ * needed) a run-time specialised kernel of a Cell chain; FO_OK, a chain error,
+ * FO_ERR_UNSUPPORTED without NVRTC; the compiler log is copied to `log`.
+ * `store` picks the skeleton: 0 flat stream (aggregating), 1 flat stream (no_agg),
+ * 2 / 3 / 4 row-wise kernel (row_agg / no_agg / full_agg), 5 column kernel, 6 / 7 / 8
+ * CSR main input with 2 / 8 / 32 lanes per row. */
 int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int store,
                          char *log, size_t log_bytes);
 

@@ -82,7 +82,7 @@ EXPORTS = [
     "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
-    "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_compile_check",
+    "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_prepare_call", "fo_jit_compile_check",
     "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_bulk_gather", "fo_probe_fp64_fma", "fo_chain_describe", "fo_tune", "fo_cell_stamps",
 ]
 
@@ -139,6 +139,8 @@ def load_library(path=None):
         lib.fo_cell_stamps.restype = C.c_int
         lib.fo_tune.argtypes = [C.c_char_p, C.c_char_p]
         lib.fo_tune.restype = C.c_int
+        lib.fo_jit_prepare_call.argtypes = [chain_p, mat_p, side_p, i32, i32, i32, i32]
+        lib.fo_jit_prepare_call.restype = C.c_int
         lib.fo_jit_prepare.argtypes = [chain_p, i32, i32, i32]
         lib.fo_jit_prepare.restype = C.c_int
         lib.fo_jit_compile_check.argtypes = [chain_p, i32, i32, i32, C.c_char_p, sz]
@@ -364,6 +366,17 @@ def tune(name, value=None):
     _check(load_library().fo_tune(name.encode(), None if value is None else str(value).encode()), "fo_tune")
 
 
+def jit_prepare_call(steps, outputs, X, sides=(), n_scalars=0, agg="full", magg=False):
+    """Compiles and caches exactly the kernel that fused_cell / fused_magg would run for
+    these arguments (dense X)."""
+    ch, keep = make_chain(steps, outputs)
+    sides = list(sides)
+    m = _mat(X)
+    sarr = _sides(sides, X.shape[0], X.shape[1])
+    _check(load_library().fo_jit_prepare_call(C.byref(ch), C.byref(m), sarr, len(sides), n_scalars,
+                                              CELL_AGG[agg], 1 if magg else 0), "fo_jit_prepare_call")
+
+
 def cell_stamps(device=None):
     """(start, scan done, partials published, result written) of the last streaming Cell /
     MAgg call made with the knob cell.stamps = 1, in ns of the GPU's global timer."""
@@ -399,11 +412,12 @@ def jit_stats():
 
 
 def jit_compile_check(steps, outputs, n_sides=0, n_scalars=0, store=False):
-    """Generates and compiles the specialised kernel of a Cell chain without running
-    it (no GPU needed).  Returns (status, compiler log)."""
+    """Generates and compiles a specialised kernel of a Cell chain without running it (no GPU
+    needed).  store: False / True the flat stream (aggregating / no_agg), 2 .. 8 the other
+    skeletons (see fo_jit_compile_check).  Returns (status, compiler log)."""
     ch, keep = make_chain(steps, outputs)
     log = C.create_string_buffer(1 << 16)
-    rc = load_library().fo_jit_compile_check(C.byref(ch), n_sides, n_scalars, 1 if store else 0, log, len(log))
+    rc = load_library().fo_jit_compile_check(C.byref(ch), n_sides, n_scalars, int(store), log, len(log))
     return rc, log.value.decode(errors="replace")
 
 

@@ -66,7 +66,7 @@ def _compile_one(src: str, verbose: bool) -> str:
     return obj
 
 
-JIT_HEADERS = ["common.cuh", "cell_flat.cuh"]      # what a run-time specialised kernel is made of
+JIT_HEADERS = ["common.cuh", "cell_flat.cuh", "cell_tiles.cuh", "cell_csr.cuh"]      # what a run-time specialised kernel is made of
 
 
 def _write_jit_source() -> None:

@@ -15,7 +15,7 @@
 
 #include <atomic>
 
-#include "cell_flat.cuh"
+#include "cell_tiles.cuh"
 #include "jit.h"
 #include "cell_csr.h"
 #include "spec.cuh"
@@ -23,232 +23,6 @@
 namespace fo {
 
 namespace {
-
-// ------------------------------------------------------------------ rows
-// Loads the pair (col, col+1) of a row; elements at or beyond `cols` read as 0.
-template <bool ALIGNED>
-__device__ __forceinline__ double2 load_pair(const double *row, long long col, long long cols)
-{
-    if (col + 1 < cols) {
-        if (ALIGNED) return ld_stream2(row + col);
-        return make_double2(ld_stream1(row + col), ld_stream1(row + col + 1));
-    }
-    if (col < cols) return make_double2(ld_stream1(row + col), 0.0);
-    return make_double2(0.0, 0.0);
-}
-
-__device__ __forceinline__ double2 load_pair_cached(const double *row, long long col, long long cols)
-{
-    return make_double2(col < cols ? __ldg(row + col) : 0.0, col + 1 < cols ? __ldg(row + col + 1) : 0.0);
-}
-
-// Inputs of the cells (rowa, ca), (rowa, ca+1), (rowb, cb), (rowb, cb+1).
-template <class EVAL, bool ALIGNED>
-__device__ __forceinline__ void load_inputs_2d(const DevChain &ch, const CellParams &p,
-                                               long long rowa, long long ca, long long rowb,
-                                               long long cb, bool have_b, double (&in)[kIn][kV])
-{
-    put4(in[0], load_pair<ALIGNED>(p.X + rowa * p.ldx, ca, p.cols),
-         have_b ? load_pair<ALIGNED>(p.X + rowb * p.ldx, cb, p.cols) : make_double2(0.0, 0.0));
-#pragma unroll
-    for (int k = 0; k < FO_MAX_SIDES; ++k) {
-        if (EVAL::uses_side(ch, k)) {
-            const DevSide sd = p.sides.s[k];
-            if (sd.access == FO_AT_ROW) {
-                const double va = __ldg(sd.data + rowa * sd.ld);
-                const double vb = have_b ? __ldg(sd.data + rowb * sd.ld) : 0.0;
-                put4(in[1 + k], make_double2(va, va), make_double2(vb, vb));
-            } else if (sd.access == FO_AT_CELL) {
-                put4(in[1 + k], load_pair<ALIGNED>(sd.data + rowa * sd.ld, ca, p.cols),
-                     have_b ? load_pair<ALIGNED>(sd.data + rowb * sd.ld, cb, p.cols)
-                            : make_double2(0.0, 0.0));
-            } else {              // row vector, reused by every row: keep it cached
-                put4(in[1 + k], load_pair_cached(sd.data, ca, p.cols),
-                     have_b ? load_pair_cached(sd.data, cb, p.cols) : make_double2(0.0, 0.0));
-            }
-        }
-    }
-}
-
-template <class EVAL, int NOUT, int AGG, bool ALIGNED>
-__global__ void __launch_bounds__(kThreads)
-cell_rows_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ CellParams p)
-{
-    __shared__ double s_red[NOUT * 32];
-    __shared__ unsigned int s_flag;
-    double acc[NOUT];
-#pragma unroll
-    for (int k = 0; k < NOUT; ++k) acc[k] = 0.0;
-
-    const int lane = threadIdx.x & 31;
-    const long long warp0 = (long long)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-    const long long nwarps = (long long)gridDim.x * (kThreads / 32);
-
-    // Rows of at most 64 columns: a warp takes several rows at a time instead of leaving most
-    // lanes without a column.  LPR lanes (a power of two >= cols / 2) share a row, 32 / LPR rows
-    // go into the first pair of values of a lane and as many into the second.
-    if (p.cols <= 64) {
-        int lpr = 1;
-        while (2 * lpr < p.cols) lpr <<= 1;
-        const int rw = 32 / lpr, sub = lane % lpr, rsel = lane / lpr;
-        const long long ca = 2 * sub;
-        for (long long r0 = warp0 * (2 * rw); r0 < p.rows; r0 += nwarps * (2 * rw)) {
-            const long long rowa = r0 + rsel, rowb = r0 + rw + rsel;
-            const bool have_a = rowa < p.rows, have_b = rowb < p.rows;
-            const long long ra = have_a ? rowa : p.rows - 1;        // loads stay inside the matrix
-            double in[kIn][kV];
-            load_inputs_2d<EVAL, ALIGNED>(ch, p, ra, ca, rowb, ca, have_b, in);
-            double o[NOUT][kV];
-            EVAL::template run<kV, NOUT>(ch, in, o);
-            const bool valid[kV] = {have_a && ca < p.cols, have_a && ca + 1 < p.cols,
-                                    have_b && ca < p.cols, have_b && ca + 1 < p.cols};
-            if (AGG == kAggNone) {
-                double *oa = p.out + rowa * p.cols, *ob = p.out + rowb * p.cols;
-                if (valid[0]) oa[ca] = o[0][0];
-                if (valid[1]) oa[ca + 1] = o[0][1];
-                if (valid[2]) ob[ca] = o[0][2];
-                if (valid[3]) ob[ca + 1] = o[0][3];
-            } else if (AGG == kAggRow) {
-                double sa = (valid[0] ? o[0][0] : 0.0) + (valid[1] ? o[0][1] : 0.0);
-                double sb = (valid[2] ? o[0][2] : 0.0) + (valid[3] ? o[0][3] : 0.0);
-                for (int off = lpr >> 1; off >= 1; off >>= 1) {
-                    sa += __shfl_xor_sync(0xffffffffu, sa, off);
-                    sb += __shfl_xor_sync(0xffffffffu, sb, off);
-                }
-                if (sub == 0 && have_a) p.out[rowa] = sa;
-                if (sub == 0 && have_b) p.out[rowb] = sb;
-            } else {
-                add_outputs<NOUT>(o, valid, acc);
-            }
-        }
-    } else
-    for (long long row = warp0; row < p.rows; row += nwarps) {
-        double rowacc[NOUT];
-#pragma unroll
-        for (int k = 0; k < NOUT; ++k) rowacc[k] = 0.0;
-        for (long long c0 = 0; c0 < p.cols; c0 += 128) {
-            const long long ca = c0 + 2 * lane, cb = ca + 64;
-            double in[kIn][kV];
-            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, ca, row, cb, true, in);
-            double o[NOUT][kV];
-            EVAL::template run<kV, NOUT>(ch, in, o);
-            const bool valid[kV] = {ca < p.cols, ca + 1 < p.cols, cb < p.cols, cb + 1 < p.cols};
-            if (AGG == kAggNone) {
-                double *orow = p.out + row * p.cols;
-                if (valid[0]) orow[ca] = o[0][0];
-                if (valid[1]) orow[ca + 1] = o[0][1];
-                if (valid[2]) orow[cb] = o[0][2];
-                if (valid[3]) orow[cb + 1] = o[0][3];
-            } else if (AGG == kAggRow) {
-                add_outputs<NOUT>(o, valid, rowacc);
-            } else {
-                add_outputs<NOUT>(o, valid, acc);
-            }
-        }
-        if (AGG == kAggRow) {
-            const double s = warp_sum(rowacc[0]);
-            if (lane == 0) p.out[row] = s;
-        }
-    }
-
-    if (AGG == kAggFull) {
-        block_sum<NOUT>(acc, s_red);
-        if (threadIdx.x == 0) {
-#pragma unroll
-            for (int k = 0; k < NOUT; ++k)
-                if (k < ch.n_out) p.partials[(size_t)blockIdx.x * ch.n_out + k] = acc[k];
-        }
-        if (publish_and_is_last(p.head, &s_flag))
-            final_sum_small(p.partials, gridDim.x, ch.n_out, p.out, s_red);
-    }
-}
-
-// ------------------------------------------------------------------ cols
-// grid.x: tiles of 2 * cx columns; grid.y: row panels.  The 256 threads of a CTA
-// form cx column pairs by 256 / cx row lanes (cx = p.cx <= 256, chosen so that the
-// column tiles are equal and narrow matrices still fill the CTA); a thread owns a column pair
-// and walks every (256 / cx)-th row of its panel, two rows per chain evaluation;
-// the row lanes are then added in order through shared memory.
-template <class EVAL, bool ALIGNED>
-__global__ void __launch_bounds__(kThreads)
-cell_cols_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ CellParams p)
-{
-    __shared__ unsigned int s_flag;
-    __shared__ double2 s_lane[kThreads];
-    const int cx = p.cx, ry = kThreads / cx;          // threads beyond cx * ry idle
-    const int tx = threadIdx.x % cx, ty = threadIdx.x / cx;
-    const long long col = ((long long)blockIdx.x * cx + tx) * 2;
-    const long long per = (p.rows + p.panels - 1) / p.panels;
-    const long long r0 = (long long)blockIdx.y * per;
-    const long long r1 = (r0 + per < p.rows) ? r0 + per : p.rows;
-    double a0 = 0.0, a1 = 0.0;
-
-    if (col < p.cols && ty < ry) {
-        long long row = r0 + ty;
-        // four rows per turn while they last: twice the loads in flight per thread
-        for (; row + 3 * ry < r1; row += 4 * ry) {
-            double in[kIn][kV], in2[kIn][kV];
-            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, col, row + ry, col, true, in);
-            load_inputs_2d<EVAL, ALIGNED>(ch, p, row + 2 * ry, col, row + 3 * ry, col, true, in2);
-            double o[1][kV], o2[1][kV];
-            EVAL::template run<kV, 1>(ch, in, o);
-            EVAL::template run<kV, 1>(ch, in2, o2);
-            a0 += o[0][0];
-            a1 += o[0][1];
-            a0 += o[0][2];
-            a1 += o[0][3];
-            a0 += o2[0][0];
-            a1 += o2[0][1];
-            a0 += o2[0][2];
-            a1 += o2[0][3];
-        }
-        for (; row < r1; row += 2 * ry) {
-            const bool two = row + ry < r1;
-            double in[kIn][kV];
-            load_inputs_2d<EVAL, ALIGNED>(ch, p, row, col, row + ry, col, two, in);
-            double o[1][kV];
-            EVAL::template run<kV, 1>(ch, in, o);
-            a0 += o[0][0];
-            a1 += o[0][1];
-            if (two) {
-                a0 += o[0][2];
-                a1 += o[0][3];
-            }
-        }
-    }
-    if (ry > 1) {
-        s_lane[threadIdx.x] = make_double2(a0, a1);
-        __syncthreads();
-        if (ty == 0) {
-            for (int k = 1; k < ry; ++k) {
-                a0 += s_lane[k * cx + tx].x;
-                a1 += s_lane[k * cx + tx].y;
-            }
-        }
-    }
-    if (col < p.cols && ty == 0) {
-        if (p.panels == 1) {
-            p.out[col] = a0;
-            if (col + 1 < p.cols) p.out[col + 1] = a1;
-        } else {
-            double *pp = p.partials + (size_t)blockIdx.y * p.cols;
-            pp[col] = a0;
-            if (col + 1 < p.cols) pp[col + 1] = a1;
-        }
-    }
-    if (p.panels == 1) return;
-    // the last panel of this column tile to finish adds the tile's partials, panel 0 first
-    if (take_ticket(&p.head->group[blockIdx.x], (unsigned)p.panels, &s_flag) && col < p.cols && ty == 0) {
-        double s0 = 0.0, s1 = 0.0;
-        const bool two = col + 1 < p.cols;
-        for (int g = 0; g < p.panels; ++g) {
-            s0 += __ldcg(p.partials + (size_t)g * p.cols + col);
-            if (two) s1 += __ldcg(p.partials + (size_t)g * p.cols + col + 1);
-        }
-        p.out[col] = s0;
-        if (two) p.out[col + 1] = s1;
-    }
-}
 
 // Non-zero entries of an elementwise result: integer counts, so the total does not
 // depend on the order in which the CTAs add theirs.
@@ -401,15 +175,46 @@ cudaError_t launch_cell_spec(const DevChain &ch, const CellParams &p, int agg, b
     return launch_cell<EvalSpec<ID>, SpecFn<ID>::kOut>(ch, p, agg, flat, aligned, grid, st);
 }
 
+// The run-time specialised kernel of a chain without a built-in form: the same three
+// skeletons (flat stream, rows, columns) with the chain written out as straight-line
+// code.  FO_OK if launched (launch = false: made ready), kJitUnavailable if the caller
+// should interpret instead.
+int launch_cell_jit(const DevChain &ch, const CellParams &p, int agg, bool flat, bool aligned, int grid,
+                    cudaStream_t st, bool may_compile, bool launch)
+{
+    if (agg == FO_CELL_COL_AGG) {
+        if (ch.n_out != 1) return kJitUnavailable;
+        const JitSpec sp = {kJitCols, aligned ? 1 : 0, 0, 0};
+        const int rc = jit_launch(sp, ch, &p, 1, 1, st, may_compile, false);
+        if (rc != FO_OK || !launch) return rc;
+        // row panels as for the ahead-of-time kernels: one full wave of resident CTAs
+        const long long tiles = (p.cols + 2 * p.cx - 1) / (2 * p.cx);
+        CellParams q = p;
+        const int nb = jit_occupancy(sp, ch), sms = sm_count();
+        if (nb > 0 && sms > 0) {
+            long long want = ((long long)sms * nb) / tiles;
+            if (want < 1) want = 1;
+            if (want < q.panels) q.panels = (int)want;
+        }
+        return jit_launch(sp, ch, &q, (unsigned)tiles, (unsigned)q.panels, st, false, true);
+    }
+    JitSpec sp;
+    if (flat) sp = JitSpec{kJitFlat, agg == FO_CELL_NO_AGG ? 1 : 0, 0, 0};
+    else sp = JitSpec{kJitRows, agg == FO_CELL_FULL_AGG ? kAggFull : agg == FO_CELL_ROW_AGG ? kAggRow : kAggNone,
+                      aligned ? 1 : 0, 0};
+    if (sp.kind == kJitRows && agg != FO_CELL_FULL_AGG && ch.n_out != 1) return kJitUnavailable;
+    return jit_launch(sp, ch, &p, (unsigned)grid, 1, st, may_compile, launch);
+}
+
 // Test / benchmark switch: run every chain through the interpreter.
 bool g_force_interpreter = false;
 
 // Common body of fused_cell and fused_magg.
 int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides,
              const double *scalars, int n_scalars, int agg, bool magg, double *out, long long *out_nnz,
-             void *ws, size_t ws_bytes, void *stream, bool may_compile)
+             void *ws, size_t ws_bytes, void *stream, bool may_compile, bool prepare_only = false)
 {
-    if (!chain || !X || !out) return FO_ERR_NULL;
+    if (!chain || !X || (!out && !prepare_only)) return FO_ERR_NULL;
     if (n_sides > 0 && !sides) return FO_ERR_NULL;
     if (agg < FO_CELL_NO_AGG || agg > FO_CELL_FULL_AGG) return FO_ERR_UNSUPPORTED;
     if (out_nnz && agg != FO_CELL_NO_AGG) return FO_ERR_UNSUPPORTED;      // a count needs an elementwise result
@@ -424,7 +229,7 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     }
     if (X->kind == FO_CSR)
         return run_cell_csr(chain, X->csr, sides, n_sides, scalars, n_scalars, agg, magg, out, ws, ws_bytes,
-                            stream);
+                            stream, may_compile);
     if (X->kind != FO_DENSE) return FO_ERR_SHAPE;
     const fo_dense &xd = X->dense;
     int rc = check_dense(xd);
@@ -471,7 +276,7 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     if (agg == FO_CELL_ROW_AGG || agg == FO_CELL_COL_AGG) flat = false;
 
     const size_t need = cell_ws_bytes(xd.rows, xd.cols, agg, ch.n_out);
-    rc = check_workspace(ws, ws_bytes, need);
+    rc = prepare_only ? FO_OK : check_workspace(ws, ws_bytes, need);
     if (rc != FO_OK) return rc;
     p.head = (WsHead *)ws;
     p.partials = (double *)((char *)ws + sizeof(WsHead));
@@ -480,6 +285,7 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
 
     cudaStream_t st = (cudaStream_t)stream;
     const long long ncells = xd.rows * xd.cols;
+    if (ncells == 0 && prepare_only) return FO_OK;
     if (ncells == 0) {      // nothing to scan: the aggregates are empty sums
         const long long nout = agg == FO_CELL_FULL_AGG ? ch.n_out
                              : agg == FO_CELL_ROW_AGG ? xd.rows
@@ -504,7 +310,9 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
     }
 
     cudaError_t e;
-    switch (g_force_interpreter ? kSpecNone : match_cell_spec(ch)) {
+    const int spec = g_force_interpreter ? kSpecNone : match_cell_spec(ch);
+    if (prepare_only && spec != kSpecNone) return FO_OK;       // built-in straight-line code: nothing to make ready
+    switch (spec) {
         case kSpecMul2: e = launch_cell_spec<kSpecMul2>(ch, p, agg, flat, aligned, grid, st); break;
         case kSpecMul3: e = launch_cell_spec<kSpecMul3>(ch, p, agg, flat, aligned, grid, st); break;
         case kSpecSq: e = launch_cell_spec<kSpecSq>(ch, p, agg, flat, aligned, grid, st); break;
@@ -517,13 +325,14 @@ int run_cell(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n
             break;
         }
         default:
-            // no built-in specialisation: a kernel compiled for this chain at run time
-            // (flat streaming case), else the interpreter
-            if (!g_force_interpreter && flat && (agg == FO_CELL_FULL_AGG || agg == FO_CELL_NO_AGG)) {
-                const int jrc = jit_launch_flat(ch, p, agg == FO_CELL_NO_AGG, grid, st, may_compile);
+            // no built-in specialisation: a kernel compiled for this chain at run time, else the interpreter
+            if (!g_force_interpreter) {
+                const bool compile_ok = prepare_only || (may_compile && jit_first_use());
+                const int jrc = launch_cell_jit(ch, p, agg, flat, aligned, grid, st, compile_ok, !prepare_only);
                 if (jrc == FO_OK) return FO_OK;
                 if (jrc != kJitUnavailable) return jrc;
             }
+            if (prepare_only) return jit_enabled() ? FO_ERR_CHAIN : FO_ERR_UNSUPPORTED;
             if (ch.n_regs <= 4) e = launch_cell_interp<4>(ch, p, agg, flat, aligned, grid, st);
             else if (ch.n_regs <= 8) e = launch_cell_interp<8>(ch, p, agg, flat, aligned, grid, st);
             else e = launch_cell_interp<kRegs>(ch, p, agg, flat, aligned, grid, st);
@@ -604,6 +413,16 @@ int fused_cell_static(const fo_chain *chain, const fo_mat *X, const fo_side *sid
 }
 
 size_t fused_cell_static_limit_bytes(void) { return fo::kStaticWsBytes; }
+
+int fo_jit_prepare_call(const fo_chain *chain, const fo_mat *X, const fo_side *sides, int n_sides, int n_scalars,
+                        int agg, int magg)
+{
+    if (n_scalars < 0 || n_scalars > FO_MAX_SCALARS) return FO_ERR_UNSUPPORTED;
+    const double scalars[FO_MAX_SCALARS] = {0};
+    if (X && X->kind == FO_CSR) return FO_ERR_UNSUPPORTED;     // chains over a CSR main input are interpreted
+    return fo::run_cell(chain, X, sides, n_sides, scalars, n_scalars, magg ? FO_CELL_FULL_AGG : agg, magg != 0,
+                        nullptr, nullptr, nullptr, 0, nullptr, true, true);
+}
 
 int fo_cell_stamps(void *ws, void *stream, unsigned long long *ns)
 {

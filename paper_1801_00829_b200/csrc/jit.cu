@@ -43,6 +43,7 @@ typedef int (*cuLaunchKernel_t)(CUfunction, unsigned, unsigned, unsigned, unsign
                                 unsigned, void *, void **, void **);
 typedef struct CUctx_st *CUcontext;
 typedef int (*cuCtxGetCurrent_t)(CUcontext *);
+typedef int (*cuOccupancy_t)(int *, CUfunction, int, size_t);
 
 struct Api {
     bool nvrtc_ok = false, driver_ok = false;
@@ -55,6 +56,7 @@ struct Api {
     cuModuleGetFunction_t getfn = nullptr;
     cuLaunchKernel_t launch = nullptr;
     cuCtxGetCurrent_t ctx = nullptr;
+    cuOccupancy_t occupancy = nullptr;
 };
 
 void *open_first(const char *const *names)
@@ -89,6 +91,7 @@ Api &api()
             a.getfn = (cuModuleGetFunction_t)dlsym(h, "cuModuleGetFunction");
             a.launch = (cuLaunchKernel_t)dlsym(h, "cuLaunchKernel");
             a.ctx = (cuCtxGetCurrent_t)dlsym(h, "cuCtxGetCurrent");
+            a.occupancy = (cuOccupancy_t)dlsym(h, "cuOccupancyMaxActiveBlocksPerMultiprocessor");
             a.driver_ok = a.load && a.getfn && a.launch && a.ctx;
         }
     });
@@ -144,7 +147,30 @@ std::string op_text(const DevOp &op)
     }
 }
 
-std::string generate_source(const DevChain &ch, bool store)
+// The wrapper kernel of one kernel instance: which skeleton, with which template arguments.
+std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
+{
+    char buf[512];
+    const char *tf[2] = {"false", "true"};
+    switch (sp.kind) {
+        case kJitFlat:          // a = STORE
+            snprintf(buf, sizeof(buf), "fo::cell_flat_body<fo::EvalFn<JitFn>, %d, %s>(ch, p);", ch.n_out, tf[sp.a & 1]);
+            break;
+        case kJitRows:          // a = AGG, b = ALIGNED
+            snprintf(buf, sizeof(buf), "fo::cell_rows_body<fo::EvalFn<JitFn>, %d, %d, %s>(ch, p);", ch.n_out, sp.a,
+                     tf[sp.b & 1]);
+            break;
+        case kJitCols:          // a = ALIGNED
+            snprintf(buf, sizeof(buf), "fo::cell_cols_body<fo::EvalFn<JitFn>, %s>(ch, p);", tf[sp.a & 1]);
+            break;
+        default:                // kJitCsr: a = lanes per row
+            snprintf(buf, sizeof(buf), "fo::cell_csr_body<fo::EvalFn<JitFn>, %d, %d>(ch, p);", ch.n_out, sp.a);
+            break;
+    }
+    return buf;
+}
+
+std::string generate_source(const DevChain &ch, const JitSpec &sp)
 {
     char buf[512];
     std::string s;
@@ -152,14 +178,18 @@ std::string generate_source(const DevChain &ch, bool store)
     snprintf(buf, sizeof(buf),
              "typedef unsigned char uint8_t;\ntypedef int int32_t;\ntypedef unsigned int uint32_t;\n"
              "#define FO_MAX_OPS %d\n#define FO_MAX_TMPS %d\n#define FO_MAX_SIDES %d\n"
-             "#define FO_MAX_SCALARS %d\n#define FO_MAX_OUT %d\n",
-             FO_MAX_OPS, FO_MAX_TMPS, FO_MAX_SIDES, FO_MAX_SCALARS, FO_MAX_OUT);
+             "#define FO_MAX_SCALARS %d\n#define FO_MAX_OUT %d\n"
+             "enum { FO_AT_CELL = %d, FO_AT_ROW = %d, FO_AT_COL = %d };\n"
+             "enum { FO_CELL_NO_AGG = %d, FO_CELL_ROW_AGG = %d, FO_CELL_COL_AGG = %d, FO_CELL_FULL_AGG = %d };\n",
+             FO_MAX_OPS, FO_MAX_TMPS, FO_MAX_SIDES, FO_MAX_SCALARS, FO_MAX_OUT, (int)FO_AT_CELL, (int)FO_AT_ROW,
+             (int)FO_AT_COL, (int)FO_CELL_NO_AGG, (int)FO_CELL_ROW_AGG, (int)FO_CELL_COL_AGG, (int)FO_CELL_FULL_AGG);
     s += buf;
     s += kSkeleton;
     snprintf(buf, sizeof(buf),
              "static_assert(sizeof(fo::DevChain) == %zu, \"chain layout\");\n"
-             "static_assert(sizeof(fo::CellParams) == %zu, \"parameter layout\");\n",
-             sizeof(DevChain), sizeof(CellParams));
+             "static_assert(sizeof(fo::CellParams) == %zu, \"parameter layout\");\n"
+             "static_assert(sizeof(fo::CsrCellParams) == %zu, \"parameter layout\");\n",
+             sizeof(DevChain), sizeof(CellParams), sizeof(CsrCellParams));
     s += buf;
     s += "struct JitFn {\n";
     snprintf(buf, sizeof(buf), "    static constexpr unsigned kSideMask = %uu;\n    static constexpr int kOut = %d;\n",
@@ -187,18 +217,18 @@ std::string generate_source(const DevChain &ch, bool store)
     s += "        (void)c; (void)in;\n    }\n};\n";
     snprintf(buf, sizeof(buf),
              "extern \"C\" __global__ void __launch_bounds__(%d)\n"
-             "fo_jit_flat(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::CellParams p)\n"
-             "{\n    fo::cell_flat_body<fo::EvalFn<JitFn>, %d, %s>(ch, p);\n}\n",
-             kThreads, ch.n_out, store ? "true" : "false");
+             "fo_jit_kernel(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::%s p)\n"
+             "{\n    ", kThreads, sp.kind == kJitCsr ? "CsrCellParams" : "CellParams");
     s += buf;
+    s += wrapper_text(ch, sp) + "\n}\n";
     return s;
 }
 
-std::string cache_key(const DevChain &ch, bool store, CUcontext ctx)
+std::string cache_key(const DevChain &ch, const JitSpec &sp, CUcontext ctx)
 {
     std::string k;
     k.append((const char *)&ctx, sizeof(ctx));
-    k.push_back(store ? 1 : 0);
+    k.append((const char *)&sp, sizeof(sp));
     k.append((const char *)&ch.n_ops, sizeof(int32_t));
     k.append((const char *)&ch.n_out, sizeof(int32_t));
     k.append((const char *)&ch.n_regs, sizeof(int32_t));
@@ -240,6 +270,7 @@ std::vector<char> compile(const std::string &src, const std::string &arch)
 }  // namespace
 
 bool jit_enabled() { return g_mode.load() != 0; }
+bool jit_first_use() { return g_mode.load() == 1; }
 
 namespace {
 
@@ -247,7 +278,7 @@ namespace {
 // first if `may_compile` and it is not there yet.  nullptr if there is none.
 // *status (optional): FO_OK, FO_ERR_UNSUPPORTED (no compiler / driver library /
 // context) or FO_ERR_CHAIN (the compilation or the load failed).
-CUfunction find_kernel(const DevChain &ch, bool store, bool may_compile, std::string *key_out, int *status)
+CUfunction find_kernel(const DevChain &ch, const JitSpec &sp, bool may_compile, std::string *key_out, int *status)
 {
     Api &a = api();
     if (status) *status = FO_ERR_UNSUPPORTED;
@@ -264,7 +295,7 @@ CUfunction find_kernel(const DevChain &ch, bool store, bool may_compile, std::st
     }
     CUfunction fn = nullptr;
     std::lock_guard<std::mutex> lock(g_mutex);
-    const std::string key = cache_key(ch, store, ctx);
+    const std::string key = cache_key(ch, sp, ctx);
     if (key_out) *key_out = key;
     auto it = g_cache.find(key);
     if (it != g_cache.end()) {
@@ -277,14 +308,14 @@ CUfunction find_kernel(const DevChain &ch, bool store, bool may_compile, std::st
     if (lf != g_load_failures.end() && lf->second >= kLoadRetries) return nullptr;
     char arch[32];
     snprintf(arch, sizeof(arch), "sm_%d%d%s", major, minor, major >= 9 ? "a" : "");
-    const std::vector<char> cubin = compile(generate_source(ch, store), arch);
+    const std::vector<char> cubin = compile(generate_source(ch, sp), arch);
     if (cubin.empty()) {
         ++g_failures;
         g_cache.emplace(key, nullptr);        // the same source fails the same way: not compiled again
         return nullptr;
     }
     CUmodule mod = nullptr;
-    if (a.load(&mod, cubin.data()) != 0 || a.getfn(&fn, mod, "fo_jit_flat") != 0) {
+    if (a.load(&mod, cubin.data()) != 0 || a.getfn(&fn, mod, "fo_jit_kernel") != 0) {
         ++g_failures;
         ++g_load_failures[key];               // may be transient: tried again a few times, then given up
         return nullptr;
@@ -297,16 +328,17 @@ CUfunction find_kernel(const DevChain &ch, bool store, bool may_compile, std::st
 
 }  // namespace
 
-int jit_launch_flat(const DevChain &ch, const CellParams &p, bool store, int grid, cudaStream_t st,
-                    bool may_compile)
+int jit_launch(const JitSpec &sp, const DevChain &ch, const void *params, unsigned grid_x, unsigned grid_y,
+               cudaStream_t st, bool may_compile, bool launch)
 {
     const int mode = g_mode.load();
     if (mode == 0) return kJitUnavailable;
     std::string key;
-    CUfunction fn = find_kernel(ch, store, may_compile && mode == 1, &key, nullptr);
+    CUfunction fn = find_kernel(ch, sp, may_compile, &key, nullptr);
     if (!fn) return kJitUnavailable;
-    void *args[2] = {(void *)&ch, (void *)&p};
-    const int rc = api().launch(fn, (unsigned)grid, 1, 1, kThreads, 1, 1, 0, (void *)st, args, nullptr);
+    if (!launch) return FO_OK;
+    void *args[2] = {(void *)&ch, (void *)params};
+    const int rc = api().launch(fn, grid_x, grid_y, 1, kThreads, 1, 1, 0, (void *)st, args, nullptr);
     if (rc == 0) {
         std::lock_guard<std::mutex> lock(g_mutex);
         ++g_launches;
@@ -320,6 +352,16 @@ int jit_launch_flat(const DevChain &ch, const CellParams &p, bool store, int gri
         return kJitUnavailable;
     }
     return cuda_fail((cudaError_t)rc);        // driver and runtime share their error numbers
+}
+
+int jit_occupancy(const JitSpec &sp, const DevChain &ch)
+{
+    Api &a = api();
+    if (g_mode.load() == 0 || !a.occupancy) return 0;
+    CUfunction fn = find_kernel(ch, sp, false, nullptr, nullptr);
+    int nb = 0;
+    if (!fn || a.occupancy(&nb, fn, kThreads, 0) != 0) return 0;
+    return nb;
 }
 
 }  // namespace fo
@@ -341,7 +383,8 @@ int fo_jit_prepare(const fo_chain *chain, int n_sides, int n_scalars, int store)
     if (rc != FO_OK) return rc;
     if (store && ch.n_out != 1) return FO_ERR_CHAIN;
     int status = FO_ERR_UNSUPPORTED;
-    find_kernel(ch, store != 0, true, nullptr, &status);
+    const JitSpec sp = {kJitFlat, store != 0 ? 1 : 0, 0, 0};
+    find_kernel(ch, sp, true, nullptr, &status);
     return status;
 }
 
@@ -365,7 +408,16 @@ int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int 
     if (rc != FO_OK) return rc;
     if (!api().nvrtc_ok) return FO_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lock(g_mutex);
-    const std::vector<char> cubin = compile(generate_source(ch, store != 0), "sm_100a");
+    JitSpec sp = {kJitFlat, store != 0 ? 1 : 0, 0, 0};
+    if (store >= 2 && store <= 5) {     // the other skeletons over a dense input
+        sp.kind = store == 5 ? kJitCols : kJitRows;
+        sp.a = store == 5 ? 1 : store == 2 ? kAggRow : store == 3 ? kAggNone : kAggFull;
+        sp.b = 1;
+    } else if (store >= 6) {            // over a CSR input: 2, 8 or 32 lanes per row
+        sp.kind = kJitCsr;
+        sp.a = store == 6 ? 2 : store == 7 ? 8 : 32;
+    }
+    const std::vector<char> cubin = compile(generate_source(ch, sp), "sm_100a");
     if (log && log_bytes) snprintf(log, log_bytes, "%s", g_last_log.c_str());
     return cubin.empty() ? FO_ERR_CHAIN : FO_OK;
 }

@@ -128,3 +128,98 @@ def test_prepared_mode_never_compiles_inside_a_call():
         fo.set_jit(old)
     assert a == b
     assert_close([a], [ref], absscale=scale)
+
+
+@pytest.mark.parametrize("skeleton", [2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("name", ["abs-fma", "scalars", "math"])
+def test_every_kernel_skeleton_compiles_without_a_gpu(name, skeleton):
+    """The row-wise, column and CSR kernels of the Cell template with a generated chain
+    (2 - 4 rows: row_agg, no_agg, full_agg; 5 columns; 6 - 8 CSR with 2, 8, 32 lanes per row)."""
+    steps, outs, n_sides, n_scalars = CHAINS[name]
+    rc, log = fo.jit_compile_check(steps, outs, n_sides, n_scalars, skeleton)
+    if rc == -4:
+        pytest.skip("NVRTC not available here")
+    assert rc == 0, log
+    assert "error" not in log
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", ["abs-fma", "scalars", "cmp-sel"])
+def test_jit_in_the_row_column_and_csr_kernels_equals_interpreter_bitwise_and_checker(name):
+    """Layouts that do not take the flat stream: a padded leading dimension, a column-vector
+    side, row and column aggregation, and a CSR main input.  Each runs a kernel compiled
+    for the chain; the bits are the interpreter's, the values the checker's."""
+    import torch
+    steps, outs, n_sides, n_scalars = CHAINS[name]
+    if not fo.jit_stats()[0]:
+        pytest.skip("NVRTC or the driver library is not usable here")
+    rows, cols = 517, 131
+    X = datagen.uniform(71, 0, rows * cols, -1.0, 2.0).reshape(rows, cols)
+    S = [datagen.uniform(71, 2 + k, rows * cols, -1.0, 2.0).reshape(rows, cols) for k in range(n_sides)]
+    scalars = [1.25, -0.5][:n_scalars]
+    pad = torch.zeros((rows, cols + 3), dtype=torch.float64, device="cuda")
+    pad[:, :cols] = to_dev(X)
+    Xd = pad[:, :cols]                                             # leading dimension cols + 3
+    sides_d = [("cell", to_dev(s)) for s in S]
+    sides_h = [("cell", s) for s in S]
+    for agg in ("full", "row", "col", "none"):
+        launches = fo.jit_stats()[2]
+        got = fo.fused_cell(steps, outs[0], Xd, sides_d, scalars, agg=agg).cpu().numpy()
+        assert fo.jit_stats()[2] == launches + 1, "the %s kernel was not specialised" % agg
+        try:
+            fo.force_interpreter(True)
+            slow = fo.fused_cell(steps, outs[0], Xd, sides_d, scalars, agg=agg).cpu().numpy()
+        finally:
+            fo.force_interpreter(False)
+        assert got.tobytes() == slow.tobytes()
+        ref = oracle.cell(steps, outs[0], X, sides_h, scalars, agg=agg)
+        absref = oracle.cell(steps + [("abs", "t7", outs[0])], "t7", X, sides_h, scalars, agg=agg)
+        assert_close(got, ref, absscale=np.asarray(absref) + 1.0, what="%s %s" % (name, agg))
+    # a CSR main input: stored cells only
+    w = datagen.outer_workload(rows, cols, 2, 0.1, seed=72)
+    Xh = {k: w[k] for k in ("rows", "cols", "rowptr", "colidx", "vals")}
+    Xc = fo.CSR(rows, cols, to_dev(w["rowptr"]), to_dev(w["colidx"]), to_dev(w["vals"]))
+    for agg in ("full", "row", "col", "none"):
+        launches = fo.jit_stats()[2]
+        got = fo.fused_cell(steps, outs[0], Xc, sides_d, scalars, agg=agg).cpu().numpy()
+        assert fo.jit_stats()[2] == launches + 1
+        try:
+            fo.force_interpreter(True)
+            slow = fo.fused_cell(steps, outs[0], Xc, sides_d, scalars, agg=agg).cpu().numpy()
+        finally:
+            fo.force_interpreter(False)
+        if agg != "col":                                           # (col_agg over CSR adds through atomics)
+            assert got.tobytes() == slow.tobytes()
+        ref = oracle.cell(steps, outs[0], Xh, sides_h, scalars, agg=agg)
+        absref = oracle.cell(steps + [("abs", "t7", outs[0])], "t7", Xh, sides_h, scalars, agg=agg)
+        assert_close(got, ref, absscale=np.asarray(absref) + 1.0, what="%s csr %s" % (name, agg))
+
+
+@pytest.mark.gpu
+def test_prepare_call_makes_the_kernel_of_a_call_ready():
+    import torch
+    if not fo.jit_stats()[0]:
+        pytest.skip("NVRTC or the driver library is not usable here")
+    rows, cols = 300, 77
+    X = datagen.normal(73, 0, rows * cols).reshape(rows, cols)
+    r = datagen.uniform(73, 1, rows, 0.5, 1.5)
+    Xd, rd = to_dev(X), to_dev(r)
+    fresh = [("mul", "t0", "a", "side0"), ("min", "t1", "t0", 0.625), ("add", "t2", "t1", "a")]
+    old = fo.set_jit(fo.binding.JIT_PREPARED)
+    try:
+        compiled, launches = fo.jit_stats()[1:3]
+        fo.jit_prepare_call(fresh, "t2", Xd, [("row", rd)], agg="row")       # a column-vector side: the row-wise kernel
+        assert fo.jit_stats()[1] == compiled + 1
+        got = fo.fused_cell(fresh, "t2", Xd, [("row", rd)], agg="row").cpu().numpy()
+        assert fo.jit_stats()[1:3] == (compiled + 1, launches + 1)
+        other = fo.fused_cell(fresh, "t2", Xd, [("row", rd)], agg="col").cpu().numpy()   # not prepared: interpreted
+        assert fo.jit_stats()[1:3] == (compiled + 1, launches + 1)
+    finally:
+        fo.set_jit(old)
+    assert_close(got, oracle.cell(fresh, "t2", X, [("row", r)], agg="row"),
+                 absscale=np.abs(X).sum(axis=1) * 3 + cols, what="prepared row_agg")
+    assert_close(other, oracle.cell(fresh, "t2", X, [("row", r)], agg="col"),
+                 absscale=np.abs(X).sum(axis=0) * 3 + rows, what="interpreted col_agg")
+    # a chain with a built-in form needs nothing
+    fo.jit_prepare_call([("mul", "t0", "a", "side0")], "t0", Xd, [("cell", Xd)], agg="full")
+    assert fo.jit_stats()[1] == compiled + 1
