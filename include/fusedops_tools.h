@@ -57,6 +57,11 @@ int fo_cell_stamps(void *ws, void *stream, unsigned long long *ns);
  * CSR main input with 2 / 8 / 32 lanes per row. */
 int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int store,
                          char *log, size_t log_bytes);
+/* The same for a chain of the Outer template.  `kernel`: 0 / 1 the per-cell kernel with
+ * plain gathers (full_agg at rank <= 112, left_mm at rank <= 256), 2 / 3 the kernel that
+ * stages factor rows (full_agg, right_mm), 4 / 5 the tiled kernel (full_agg, no_agg). */
+int fo_jit_compile_check_outer(const fo_chain *chain, int n_sides, int n_scalars, int kernel,
+                               char *log, size_t log_bytes);
 
 /* The k-th result of a chain written out as an expression over the inputs,
  * after validation and translation for a template (`use`: 0 Cell / MAgg,

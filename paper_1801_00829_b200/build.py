@@ -66,26 +66,29 @@ def _compile_one(src: str, verbose: bool) -> str:
     return obj
 
 
-JIT_HEADERS = ["common.cuh", "cell_flat.cuh", "cell_tiles.cuh", "cell_csr.cuh"]      # what a run-time specialised kernel is made of
+# what the run-time specialised kernels are made of: Cell / MAgg, and Outer
+JIT_HEADERS = {"jit_source.inc": ["common.cuh", "cell_flat.cuh", "cell_tiles.cuh", "cell_csr.cuh"],
+               "jit_source_outer.inc": ["common.cuh", "outer_kernels.cuh"]}
 
 
 def _write_jit_source() -> None:
-    """Embeds the headers the run-time compiled kernels consist of as a C++ string
-    literal (_build/jit_source.inc), without their #include / #pragma once lines."""
-    chunks = []
-    for name in JIT_HEADERS:
-        with open(os.path.join(CSRC, name)) as fh:
-            lines = [l for l in fh.read().splitlines()
-                     if not l.lstrip().startswith("#include") and not l.lstrip().startswith("#pragma once")]
-        chunks.append("// ---- %s\n" % name + "\n".join(lines) + "\n")
-    text = "".join(chunks)
-    assert ')FOJIT"' not in text
-    out = []
-    step = 8000                                   # keep each literal well below compiler limits
-    for i in range(0, len(text), step):
-        out.append('R"FOJIT(' + text[i:i + step] + ')FOJIT"\n')
-    with open(os.path.join(OBJ_DIR, "jit_source.inc"), "w") as fh:
-        fh.write("".join(out))
+    """Embeds the headers the run-time compiled kernels consist of as C++ string
+    literals (_build/jit_source*.inc), without their #include / #pragma once lines."""
+    for target, names in JIT_HEADERS.items():
+        chunks = []
+        for name in names:
+            with open(os.path.join(CSRC, name)) as fh:
+                lines = [l for l in fh.read().splitlines()
+                         if not l.lstrip().startswith("#include") and not l.lstrip().startswith("#pragma once")]
+            chunks.append("// ---- %s\n" % name + "\n".join(lines) + "\n")
+        text = "".join(chunks)
+        assert ')FOJIT"' not in text
+        out = []
+        step = 8000                                   # keep each literal well below compiler limits
+        for i in range(0, len(text), step):
+            out.append('R"FOJIT(' + text[i:i + step] + ')FOJIT"\n')
+        with open(os.path.join(OBJ_DIR, target), "w") as fh:
+            fh.write("".join(out))
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:

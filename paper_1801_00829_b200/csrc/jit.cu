@@ -15,8 +15,8 @@
 #include <unordered_map>
 #include <vector>
 
-#include "cell_flat.cuh"
 #include "jit.h"
+#include "outer_kernels.cuh"
 
 namespace fo {
 
@@ -24,6 +24,9 @@ namespace {
 
 const char kSkeleton[] =
 #include "jit_source.inc"
+    ;
+const char kSkeletonOuter[] =
+#include "jit_source_outer.inc"
     ;
 
 // ---- the few NVRTC / driver entry points used, declared here so that neither
@@ -44,6 +47,7 @@ typedef int (*cuLaunchKernel_t)(CUfunction, unsigned, unsigned, unsigned, unsign
 typedef struct CUctx_st *CUcontext;
 typedef int (*cuCtxGetCurrent_t)(CUcontext *);
 typedef int (*cuOccupancy_t)(int *, CUfunction, int, size_t);
+typedef int (*cuFuncSetAttribute_t)(CUfunction, int, int);
 
 struct Api {
     bool nvrtc_ok = false, driver_ok = false;
@@ -57,6 +61,7 @@ struct Api {
     cuLaunchKernel_t launch = nullptr;
     cuCtxGetCurrent_t ctx = nullptr;
     cuOccupancy_t occupancy = nullptr;
+    cuFuncSetAttribute_t setattr = nullptr;
 };
 
 void *open_first(const char *const *names)
@@ -92,6 +97,7 @@ Api &api()
             a.launch = (cuLaunchKernel_t)dlsym(h, "cuLaunchKernel");
             a.ctx = (cuCtxGetCurrent_t)dlsym(h, "cuCtxGetCurrent");
             a.occupancy = (cuOccupancy_t)dlsym(h, "cuOccupancyMaxActiveBlocksPerMultiprocessor");
+            a.setattr = (cuFuncSetAttribute_t)dlsym(h, "cuFuncSetAttribute");
             a.driver_ok = a.load && a.getfn && a.launch && a.ctx;
         }
     });
@@ -163,35 +169,30 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
         case kJitCols:          // a = ALIGNED
             snprintf(buf, sizeof(buf), "fo::cell_cols_body<fo::EvalFn<JitFn>, %s>(ch, p);", tf[sp.a & 1]);
             break;
-        default:                // kJitCsr: a = lanes per row
+        case kJitCsr:           // a = lanes per row
             snprintf(buf, sizeof(buf), "fo::cell_csr_body<fo::EvalFn<JitFn>, %d, %d>(ch, p);", ch.n_out, sp.a);
+            break;
+        case kJitOuterDirect:   // a = NK2, b = AGG, c = ALIGNED
+            snprintf(buf, sizeof(buf), "fo::outer_body<%d, %d, %s>(ch, p);", sp.a, sp.b, tf[sp.c & 1]);
+            break;
+        case kJitOuterPipe:     // a = NK2, b = AGG
+            snprintf(buf, sizeof(buf), "fo::outer_pipe_body<%d, %d>(ch, p);", sp.a, sp.b);
+            break;
+        default:                // kJitOuterDense: a = AGG
+            snprintf(buf, sizeof(buf), "fo::outer_dense_body<%d>(ch, p, sp);", sp.a);
             break;
     }
     return buf;
 }
 
-std::string generate_source(const DevChain &ch, const JitSpec &sp)
+bool is_outer(const JitSpec &sp) { return sp.kind >= kJitOuterDirect; }
+
+// The chain as a straight-line functor: in[] holds the input registers (Cell: a, sides;
+// Outer: a, d, sides), c the constant table, o the results.
+std::string functor_text(const DevChain &ch)
 {
     char buf[512];
-    std::string s;
-    // what the system headers and fusedops.h provide in the ahead-of-time build
-    snprintf(buf, sizeof(buf),
-             "typedef unsigned char uint8_t;\ntypedef int int32_t;\ntypedef unsigned int uint32_t;\n"
-             "#define FO_MAX_OPS %d\n#define FO_MAX_TMPS %d\n#define FO_MAX_SIDES %d\n"
-             "#define FO_MAX_SCALARS %d\n#define FO_MAX_OUT %d\n"
-             "enum { FO_AT_CELL = %d, FO_AT_ROW = %d, FO_AT_COL = %d };\n"
-             "enum { FO_CELL_NO_AGG = %d, FO_CELL_ROW_AGG = %d, FO_CELL_COL_AGG = %d, FO_CELL_FULL_AGG = %d };\n",
-             FO_MAX_OPS, FO_MAX_TMPS, FO_MAX_SIDES, FO_MAX_SCALARS, FO_MAX_OUT, (int)FO_AT_CELL, (int)FO_AT_ROW,
-             (int)FO_AT_COL, (int)FO_CELL_NO_AGG, (int)FO_CELL_ROW_AGG, (int)FO_CELL_COL_AGG, (int)FO_CELL_FULL_AGG);
-    s += buf;
-    s += kSkeleton;
-    snprintf(buf, sizeof(buf),
-             "static_assert(sizeof(fo::DevChain) == %zu, \"chain layout\");\n"
-             "static_assert(sizeof(fo::CellParams) == %zu, \"parameter layout\");\n"
-             "static_assert(sizeof(fo::CsrCellParams) == %zu, \"parameter layout\");\n",
-             sizeof(DevChain), sizeof(CellParams), sizeof(CsrCellParams));
-    s += buf;
-    s += "struct JitFn {\n";
+    std::string s = "struct JitFn {\n";
     snprintf(buf, sizeof(buf), "    static constexpr unsigned kSideMask = %uu;\n    static constexpr int kOut = %d;\n",
              ch.side_used, ch.n_out);
     s += buf;
@@ -215,6 +216,51 @@ std::string generate_source(const DevChain &ch, const JitSpec &sp)
         s += operand_text(ch.out[k]) + ";\n";
     }
     s += "        (void)c; (void)in;\n    }\n};\n";
+    return s;
+}
+
+std::string generate_source(const DevChain &ch, const JitSpec &sp)
+{
+    char buf[1024];
+    std::string s;
+    // what the system headers and fusedops.h provide in the ahead-of-time build
+    snprintf(buf, sizeof(buf),
+             "typedef unsigned char uint8_t;\ntypedef int int32_t;\ntypedef unsigned int uint32_t;\n"
+             "#define FO_MAX_OPS %d\n#define FO_MAX_TMPS %d\n#define FO_MAX_SIDES %d\n"
+             "#define FO_MAX_SCALARS %d\n#define FO_MAX_OUT %d\n"
+             "enum { FO_AT_CELL = %d, FO_AT_ROW = %d, FO_AT_COL = %d };\n"
+             "enum { FO_CELL_NO_AGG = %d, FO_CELL_ROW_AGG = %d, FO_CELL_COL_AGG = %d, FO_CELL_FULL_AGG = %d };\n",
+             FO_MAX_OPS, FO_MAX_TMPS, FO_MAX_SIDES, FO_MAX_SCALARS, FO_MAX_OUT, (int)FO_AT_CELL, (int)FO_AT_ROW,
+             (int)FO_AT_COL, (int)FO_CELL_NO_AGG, (int)FO_CELL_ROW_AGG, (int)FO_CELL_COL_AGG, (int)FO_CELL_FULL_AGG);
+    s += buf;
+    if (is_outer(sp)) {
+        // the Outer kernels call the functor from inside: it comes first
+        s += "#define FO_JIT_OUTER 1\n";
+        s += functor_text(ch);
+        s += kSkeletonOuter;
+        snprintf(buf, sizeof(buf),
+                 "static_assert(sizeof(fo::DevChain) == %zu, \"chain layout\");\n"
+                 "static_assert(sizeof(fo::OuterParams) == %zu, \"parameter layout\");\n"
+                 "static_assert(sizeof(fo::DenseSplit) == %zu, \"parameter layout\");\n",
+                 sizeof(DevChain), sizeof(OuterParams), sizeof(DenseSplit));
+        s += buf;
+        snprintf(buf, sizeof(buf),
+                 "extern \"C\" __global__ void __launch_bounds__(%d, %d)\n"
+                 "fo_jit_kernel(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::OuterParams p%s)\n"
+                 "{\n    ", kThreads, (sp.kind == kJitOuterDirect && sp.a > 8) ? 1 : 2,
+                 sp.kind == kJitOuterDense ? ", const __grid_constant__ fo::DenseSplit sp" : "");
+        s += buf;
+        s += wrapper_text(ch, sp) + "\n}\n";
+        return s;
+    }
+    s += kSkeleton;
+    snprintf(buf, sizeof(buf),
+             "static_assert(sizeof(fo::DevChain) == %zu, \"chain layout\");\n"
+             "static_assert(sizeof(fo::CellParams) == %zu, \"parameter layout\");\n"
+             "static_assert(sizeof(fo::CsrCellParams) == %zu, \"parameter layout\");\n",
+             sizeof(DevChain), sizeof(CellParams), sizeof(CsrCellParams));
+    s += buf;
+    s += functor_text(ch);
     snprintf(buf, sizeof(buf),
              "extern \"C\" __global__ void __launch_bounds__(%d)\n"
              "fo_jit_kernel(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::%s p)\n"
@@ -329,7 +375,7 @@ CUfunction find_kernel(const DevChain &ch, const JitSpec &sp, bool may_compile, 
 }  // namespace
 
 int jit_launch(const JitSpec &sp, const DevChain &ch, const void *params, unsigned grid_x, unsigned grid_y,
-               cudaStream_t st, bool may_compile, bool launch)
+               cudaStream_t st, bool may_compile, bool launch, size_t smem, const void *params2)
 {
     const int mode = g_mode.load();
     if (mode == 0) return kJitUnavailable;
@@ -337,8 +383,13 @@ int jit_launch(const JitSpec &sp, const DevChain &ch, const void *params, unsign
     CUfunction fn = find_kernel(ch, sp, may_compile, &key, nullptr);
     if (!fn) return kJitUnavailable;
     if (!launch) return FO_OK;
-    void *args[2] = {(void *)&ch, (void *)params};
-    const int rc = api().launch(fn, grid_x, grid_y, 1, kThreads, 1, 1, 0, (void *)st, args, nullptr);
+    if (smem > 48u * 1024u) {
+        // CU_FUNC_ATTRIBUTE_MAX_DYNAMIC_SHARED_SIZE_BYTES
+        const int arc = api().setattr ? api().setattr(fn, 8, (int)smem) : 1;
+        if (arc != 0) return kJitUnavailable;
+    }
+    void *args[3] = {(void *)&ch, (void *)params, (void *)params2};
+    const int rc = api().launch(fn, grid_x, grid_y, 1, kThreads, 1, 1, (unsigned)smem, (void *)st, args, nullptr);
     if (rc == 0) {
         std::lock_guard<std::mutex> lock(g_mutex);
         ++g_launches;
@@ -413,10 +464,36 @@ int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int 
         sp.kind = store == 5 ? kJitCols : kJitRows;
         sp.a = store == 5 ? 1 : store == 2 ? kAggRow : store == 3 ? kAggNone : kAggFull;
         sp.b = 1;
-    } else if (store >= 6) {            // over a CSR input: 2, 8 or 32 lanes per row
+    } else if (store >= 6 && store <= 8) {     // over a CSR input: 2, 8 or 32 lanes per row
         sp.kind = kJitCsr;
         sp.a = store == 6 ? 2 : store == 7 ? 8 : 32;
     }
+    const std::vector<char> cubin = compile(generate_source(ch, sp), "sm_100a");
+    if (log && log_bytes) snprintf(log, log_bytes, "%s", g_last_log.c_str());
+    return cubin.empty() ? FO_ERR_CHAIN : FO_OK;
+}
+
+int fo_jit_compile_check_outer(const fo_chain *chain, int n_sides, int n_scalars, int kernel, char *log,
+                                size_t log_bytes)
+{
+    using namespace fo;
+    if (log && log_bytes) log[0] = 0;
+    double scalars[FO_MAX_SCALARS] = {0};
+    DevChain ch;
+    const int rc = translate_chain(chain, kUseOuter, n_sides, scalars, n_scalars, 1, 1, &ch);
+    if (rc != FO_OK) return rc;
+    if (!api().nvrtc_ok) return FO_ERR_UNSUPPORTED;
+    JitSpec sp;
+    switch (kernel) {
+        case 0: sp = JitSpec{kJitOuterDirect, 7, kOutFull, 1}; break;
+        case 1: sp = JitSpec{kJitOuterDirect, 16, kOutLeft, 0}; break;
+        case 2: sp = JitSpec{kJitOuterPipe, 7, kOutFull, 0}; break;
+        case 3: sp = JitSpec{kJitOuterPipe, 2, kOutRight, 0}; break;
+        case 4: sp = JitSpec{kJitOuterDense, kOutFull, 0, 0}; break;
+        case 5: sp = JitSpec{kJitOuterDense, kOutNone, 0, 0}; break;
+        default: return FO_ERR_UNSUPPORTED;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
     const std::vector<char> cubin = compile(generate_source(ch, sp), "sm_100a");
     if (log && log_bytes) snprintf(log, log_bytes, "%s", g_last_log.c_str());
     return cubin.empty() ? FO_ERR_CHAIN : FO_OK;

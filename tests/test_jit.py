@@ -223,3 +223,52 @@ def test_prepare_call_makes_the_kernel_of_a_call_ready():
     # a chain with a built-in form needs nothing
     fo.jit_prepare_call([("mul", "t0", "a", "side0")], "t0", Xd, [("cell", Xd)], agg="full")
     assert fo.jit_stats()[1] == compiled + 1
+
+
+OUTER_GENERIC = [("sub", "t1", "a", "d"), ("abs", "t2", "t1"), ("add", "t3", "t2", 0.25)]
+
+
+@pytest.mark.parametrize("kernel", range(6))
+def test_outer_kernels_compile_with_a_generated_chain_without_a_gpu(kernel):
+    rc, log = fo.jit_compile_check_outer(OUTER_GENERIC, "t3", 0, 0, kernel)
+    if rc == -4:
+        pytest.skip("NVRTC not available here")
+    assert rc == 0, log
+    assert "error" not in log
+    sides_chain = [("sub", "t0", "a", "d"), ("mul", "t1", "t0", "side0"), ("add", "t2", "t1", "side1")]
+    rc, log = fo.jit_compile_check_outer(sides_chain, "t2", 2, 0, kernel)
+    assert rc == 0, log
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("schedule", ["pipe", "direct", "dense"])
+def test_outer_chain_compiled_at_run_time_equals_interpreter_bitwise_and_checker(schedule):
+    if not fo.jit_stats()[0]:
+        pytest.skip("NVRTC or the driver library is not usable here")
+    w = datagen.outer_workload(300, 257, 20, 0.3 if schedule == "dense" else 0.05, seed=77)
+    Xh = {k: w[k] for k in ("rows", "cols", "rowptr", "colidx", "vals")}
+    X = fo.CSR(w["rows"], w["cols"], to_dev(w["rowptr"]), to_dev(w["colidx"]), to_dev(w["vals"]))
+    Ud, Vd = to_dev(w["U"]), to_dev(w["V"])
+    fo.tune("outer.kernel", schedule)
+    try:
+        for agg in ("full", "none") + (() if schedule == "dense" else ("right",)) + (("left",) if schedule == "direct" else ()):
+            launches = fo.jit_stats()[2]
+            fast = fo.fused_outer(OUTER_GENERIC, "t3", X, Ud, Vd, agg=agg).cpu().numpy()
+            assert fo.jit_stats()[2] == launches + 1, "%s %s was not specialised" % (schedule, agg)
+            try:
+                fo.force_interpreter(True)
+                slow = fo.fused_outer(OUTER_GENERIC, "t3", X, Ud, Vd, agg=agg).cpu().numpy()
+            finally:
+                fo.force_interpreter(False)
+            if agg != "left":                                      # (left_mm adds through atomics)
+                assert fast.tobytes() == slow.tobytes()
+            ref = oracle.outer(OUTER_GENERIC, "t3", Xh, w["U"], w["V"], agg=agg, mode="masked")
+            assert_close(fast, ref, absscale=np.abs(ref) + 1.0, what="outer jit %s %s" % (schedule, agg))
+    finally:
+        fo.tune("outer.kernel", None)
+    # side inputs through a compiled chain (the per-cell kernel with plain gathers)
+    r = datagen.uniform(77, 9, w["rows"], 0.5, 2.0)
+    chain = [("sub", "t0", "a", "d"), ("mul", "t1", "t0", "side0")]
+    got = fo.fused_outer(chain, "t1", X, Ud, Vd, agg="none", sides=[("row", to_dev(r))]).cpu().numpy()
+    assert_close(got, oracle.outer(chain, "t1", Xh, w["U"], w["V"], agg="none", sides=[("row", r)]),
+                 what="outer jit sides")
