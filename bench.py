@@ -6,7 +6,7 @@ Row dense, Row CSR, Outer) each run once on their full-size seeded workload.
 The reported value is effective input bandwidth: the bytes the five operators
 must read once, divided by the time of a step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-paper-suite]
 
 `--impl reference` times the CPU checker (oracle/) on bounded samples of the same
 workloads; it runs on host cores only.
@@ -222,6 +222,8 @@ def time_variants(fo, step, shapes, reps=10):
     ocol = shapes["outer"]["cols"]
     o_left = torch.empty((ocol, rank), dtype=torch.float64, device=dev)
     generic = [("sub", "t0", "a", "side0"), ("abs", "t1", "t0"), ("fma", "t2", "t1", "side1", 0.5)]
+    outer_generic = [("sub", "t1", "a", "d"), ("abs", "t2", "t1"), ("add", "t3", "t2", 0.25)]
+    o_rc = torch.empty(rc, dtype=torch.float64, device=dev)
 
     def interpreted(fn):
         fo.force_interpreter(True)
@@ -245,6 +247,14 @@ def time_variants(fo, step, shapes, reps=10):
          lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="full", out=o_one), in3 + 8),
         ("cell_full_agg_interpreted_chain", lambda: interpreted(
             lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="full", out=o_one)), in3 + 8),
+        # the same chain in the row-wise and column kernels (compiled at run time too), against the
+        # built-in product chain of cell_row_agg / cell_col_agg above
+        ("cell_row_agg_runtime_compiled_chain",
+         lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="row", out=o_row), in3 + 8 * mr),
+        ("cell_col_agg_runtime_compiled_chain",
+         lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="col", out=o_col), in3 + 8 * mc),
+        ("cell_row_agg_interpreted_chain", lambda: interpreted(
+            lambda: fo.fused_cell(generic, "t2", d["magg.X"], sides, agg="row", out=o_row)), in3 + 8 * mr),
         ("row_dense_row_agg", lambda: fo.fused_row(WD, "t0", d["row_dense.X"], d["row_dense.v"],
                                                    [("row", d["row_dense.w"])], agg="row", out=o_rr),
          8 * rr * rc + 16 * rr + 8 * rc),
@@ -267,6 +277,18 @@ def time_variants(fo, step, shapes, reps=10):
             d["outer.U"], d["outer.V"], [10.0], agg="full", out=o_one), outer_in + 8),
         ("outer_left_mm", lambda: fo.fused_outer(WSLOSS, "t3", step.csr5, d["outer.U"], d["outer.V"],
                                                  agg="left", out=o_left), outer_in + 8 * ocol * rank),
+        # a chain without an inline form (|a - d| + 0.25): compiled at run time, and interpreted
+        ("outer_full_agg_runtime_compiled_chain", lambda: fo.fused_outer(
+            outer_generic, "t3", step.csr5, d["outer.U"], d["outer.V"], out=o_one), outer_in + 8),
+        ("outer_right_mm_runtime_compiled_chain", lambda: fo.fused_outer(
+            outer_generic, "t3", step.csr5, d["outer.U"], d["outer.V"], agg="right", out=o_right),
+         outer_in + 8 * orow * rank),
+        ("outer_full_agg_interpreted_chain", lambda: interpreted(lambda: fo.fused_outer(
+            outer_generic, "t3", step.csr5, d["outer.U"], d["outer.V"], out=o_one)), outer_in + 8),
+        # the Row chain |w * d| - 0.5, interpreted once per row (the Row template's chains are not compiled)
+        ("row_dense_col_t_agg_interpreted_chain", lambda: fo.fused_row(
+            [("mul", "t0", "side0", "d"), ("abs", "t1", "t0"), ("sub", "t2", "t1", 0.5)], "t2", d["row_dense.X"],
+            d["row_dense.v"], [("row", d["row_dense.w"])], out=o_rc), 8 * rr * rc + 8 * rr + 16 * rc),
     ]
     # sparse-safe Cell / MAgg (Section 5.2's sparse variants): X at density 0.1 as the CSR driver,
     # dense Y and Z read at the stored cells
@@ -1077,8 +1099,9 @@ def main():
     ap.add_argument("--no-variants", action="store_true", help="skip the untimed-step variant measurements")
     ap.add_argument("--full-outer", action="store_true", help="keep the Outer workload at full size under --frac")
     ap.add_argument("--ops", default="", help="comma-separated subset of the five operators (profiling)")
-    ap.add_argument("--paper-suite", action="store_true",
-                    help="also time the paper's operator micro-benchmarks at their own sizes (adds about a minute)")
+    ap.add_argument("--paper-suite", action="store_true", default=True,
+                    help="time the paper's operator micro-benchmarks at their own sizes too (the default; about a minute)")
+    ap.add_argument("--no-paper-suite", dest="paper_suite", action="store_false")
     ap.add_argument("--interp", action="store_true", help="run Cell / MAgg chains through the interpreter")
     args = ap.parse_args()
     if args.impl == "reference":
