@@ -223,6 +223,7 @@ def time_variants(fo, step, shapes, reps=10):
     o_left = torch.empty((ocol, rank), dtype=torch.float64, device=dev)
     generic = [("sub", "t0", "a", "side0"), ("abs", "t1", "t0"), ("fma", "t2", "t1", "side1", 0.5)]
     outer_generic = [("sub", "t1", "a", "d"), ("abs", "t2", "t1"), ("add", "t3", "t2", 0.25)]
+    row_generic = [("mul", "t0", "side0", "d"), ("abs", "t1", "t0"), ("sub", "t2", "t1", 0.5)]
     o_rc = torch.empty(rc, dtype=torch.float64, device=dev)
 
     def interpreted(fn):
@@ -285,10 +286,13 @@ def time_variants(fo, step, shapes, reps=10):
          outer_in + 8 * orow * rank),
         ("outer_full_agg_interpreted_chain", lambda: interpreted(lambda: fo.fused_outer(
             outer_generic, "t3", step.csr5, d["outer.U"], d["outer.V"], out=o_one)), outer_in + 8),
-        # the Row chain |w * d| - 0.5, interpreted once per row (the Row template's chains are not compiled)
-        ("row_dense_col_t_agg_interpreted_chain", lambda: fo.fused_row(
-            [("mul", "t0", "side0", "d"), ("abs", "t1", "t0"), ("sub", "t2", "t1", 0.5)], "t2", d["row_dense.X"],
-            d["row_dense.v"], [("row", d["row_dense.w"])], out=o_rc), 8 * rr * rc + 8 * rr + 16 * rc),
+        # the Row chain |w * d| - 0.5: compiled at run time, and interpreted (once per row, warp-wide)
+        ("row_dense_col_t_agg_runtime_compiled_chain", lambda: fo.fused_row(
+            row_generic, "t2", d["row_dense.X"], d["row_dense.v"], [("row", d["row_dense.w"])], out=o_rc),
+         8 * rr * rc + 8 * rr + 16 * rc),
+        ("row_dense_col_t_agg_interpreted_chain", lambda: interpreted(lambda: fo.fused_row(
+            row_generic, "t2", d["row_dense.X"], d["row_dense.v"], [("row", d["row_dense.w"])], out=o_rc)),
+         8 * rr * rc + 8 * rr + 16 * rc),
     ]
     # sparse-safe Cell / MAgg (Section 5.2's sparse variants): X at density 0.1 as the CSR driver,
     # dense Y and Z read at the stored cells
@@ -449,6 +453,38 @@ def size_sweep(fo, device, cols=1000, rows_list=(1_000, 10_000, 100_000, 1_000_0
                            "gbs_at_median": nbytes / (statistics.median(ms) * 1e-3) / 1e9}
         res.append(entry)
         del X, Y, Z
+    return res
+
+
+def cell_phases(fo, device, rows=1000, cols=1000, reps=8):
+    """Where the small Cell workload (config 1: 24 MB) spends its time: the streaming kernel's own
+    phase stamps (GPU global timer, ns; cold L2) for 1 .. 8 CTAs per SM, and CUDA events around the call."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(13)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+    one = torch.empty(1, dtype=torch.float64, device=device)
+    X, Y, Z = (torch.rand((rows, cols), generator=g, dtype=torch.float64, device=device) for _ in range(3))
+    sides = [("cell", Y), ("cell", Z)]
+    res = {}
+    try:
+        for cps in (1, 2, 3, 4, 6, 8):
+            fo.tune("cell.ctas_per_sm", cps)
+            fo.tune("cell.stamps", 0)
+            ev = _event_times(lambda: fo.fused_cell(XYZ, "t1", X, sides, out=one), reps, before=flush.zero_)
+            fo.tune("cell.stamps", 1)
+            ph = []
+            for _ in range(reps):
+                flush.zero_()
+                fo.fused_cell(XYZ, "t1", X, sides, out=one)
+                st = fo.cell_stamps(device)
+                ph.append((st[1] - st[0], st[2] - st[1], st[3] - st[2], st[3] - st[0]))
+            med = [int(statistics.median(p[i] for p in ph[2:])) for i in range(4)]
+            res["ctas_per_sm_%d" % cps] = {"scan_ns": med[0], "publish_ns": med[1], "final_ns": med[2],
+                                           "kernel_ns": med[3], "events_us_min": min(ev) * 1e3}
+    finally:
+        fo.tune("cell.ctas_per_sm", None)
+        fo.tune("cell.stamps", None)
     return res
 
 
@@ -1039,6 +1075,7 @@ def run_ours(args):
         line["cost_model"] = cm
         if args.frac == 1.0 and world == 1:
             line["size_sweep"] = size_sweep(fo, device)
+            line["cell_phases"] = cell_phases(fo, device)
         if args.paper_suite and world == 1:
             line["paper_suite"] = paper_suite(fo, device, peak_gbs=peak_gbs, fp64_tflops=probes["fp64_fma_tflops"],
                                               l2_gather_gbs=probes["l2_gather_gbs"])

@@ -62,6 +62,11 @@ int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int 
  * stages factor rows (full_agg, right_mm), 4 / 5 the tiled kernel (full_agg, no_agg). */
 int fo_jit_compile_check_outer(const fo_chain *chain, int n_sides, int n_scalars, int kernel,
                                char *log, size_t log_bytes);
+/* The same for a chain of the Row template.  `kernel`: 0 / 1 / 2 the dense kernel (1000-column
+ * shape col_t_agg, 8192-column shape no_agg unstaged, 64-column shape row_agg), 3 the
+ * thread-per-row kernel, 4 the CSR column-scatter kernel, 5 the CSR register kernel. */
+int fo_jit_compile_check_row(const fo_chain *chain, int n_sides, int n_scalars, int kernel,
+                             char *log, size_t log_bytes);
 
 /* The k-th result of a chain written out as an expression over the inputs,
  * after validation and translation for a template (`use`: 0 Cell / MAgg,

@@ -82,7 +82,7 @@ EXPORTS = [
     "fused_outer_workspace_bytes", "fo_workspace_init", "fo_query_device_status",
     "fo_status_string", "fo_last_cuda_error", "fo_set_force_interpreter",
     "fused_cell_static", "fused_cell_static_limit_bytes",
-    "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_prepare_call", "fo_jit_compile_check", "fo_jit_compile_check_outer",
+    "fo_set_jit", "fo_jit_stats", "fo_jit_prepare", "fo_jit_prepare_call", "fo_jit_compile_check", "fo_jit_compile_check_outer", "fo_jit_compile_check_row",
     "fo_probe_out_len", "fo_probe_l2_gather", "fo_probe_bulk_gather", "fo_probe_fp64_fma", "fo_chain_describe", "fo_tune", "fo_cell_stamps",
 ]
 
@@ -147,6 +147,8 @@ def load_library(path=None):
         lib.fo_jit_compile_check.restype = C.c_int
         lib.fo_jit_compile_check_outer.argtypes = [chain_p, i32, i32, i32, C.c_char_p, sz]
         lib.fo_jit_compile_check_outer.restype = C.c_int
+        lib.fo_jit_compile_check_row.argtypes = [chain_p, i32, i32, i32, C.c_char_p, sz]
+        lib.fo_jit_compile_check_row.restype = C.c_int
         lib.fo_set_force_interpreter.argtypes = [C.c_int]
         lib.fo_set_force_interpreter.restype = C.c_int
         lib.fo_chain_describe.argtypes = [chain_p, i32, i32, scal_p, i32, i32, C.c_char_p, sz]
@@ -429,6 +431,15 @@ def jit_compile_check_outer(steps, output, n_sides=0, n_scalars=0, kernel=0):
     ch, keep = make_chain(steps, output)
     log = C.create_string_buffer(1 << 16)
     rc = load_library().fo_jit_compile_check_outer(C.byref(ch), n_sides, n_scalars, int(kernel), log, len(log))
+    return rc, log.value.decode(errors="replace")
+
+
+def jit_compile_check_row(steps, output, n_sides=0, n_scalars=0, kernel=0):
+    """Generates and compiles a specialised Row kernel for a chain (no GPU needed).
+    Returns (status, compiler log)."""
+    ch, keep = make_chain(steps, output)
+    log = C.create_string_buffer(1 << 16)
+    rc = load_library().fo_jit_compile_check_row(C.byref(ch), n_sides, n_scalars, int(kernel), log, len(log))
     return rc, log.value.decode(errors="replace")
 
 

@@ -17,6 +17,7 @@
 
 #include "jit.h"
 #include "outer_kernels.cuh"
+#include "row_kernels.cuh"
 
 namespace fo {
 
@@ -27,6 +28,9 @@ const char kSkeleton[] =
     ;
 const char kSkeletonOuter[] =
 #include "jit_source_outer.inc"
+    ;
+const char kSkeletonRow[] =
+#include "jit_source_row.inc"
     ;
 
 // ---- the few NVRTC / driver entry points used, declared here so that neither
@@ -178,14 +182,28 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
         case kJitOuterPipe:     // a = NK2, b = AGG
             snprintf(buf, sizeof(buf), "fo::outer_pipe_body<%d, %d>(ch, p);", sp.a, sp.b);
             break;
-        default:                // kJitOuterDense: a = AGG
+        case kJitOuterDense:    // a = AGG
             snprintf(buf, sizeof(buf), "fo::outer_dense_body<%d>(ch, p, sp);", sp.a);
+            break;
+        case kJitRowDense:      // a = NCH, b = W, c = R, d = AGG, e = STAGED
+            snprintf(buf, sizeof(buf), "fo::row_dense_body<%d, %d, %d, %d, %s>(ch, p);", sp.a, sp.b, sp.c, sp.d,
+                     tf[sp.e & 1]);
+            break;
+        case kJitRowNarrow:     // a = NC, b = AGG, c = VEC
+            snprintf(buf, sizeof(buf), "fo::row_narrow_body<%d, %d, %s>(ch, p);", sp.a, sp.b, tf[sp.c & 1]);
+            break;
+        case kJitRowCsr:        // a = G
+            snprintf(buf, sizeof(buf), "fo::row_csr_body<%d>(ch, p);", sp.a);
+            break;
+        default:                // kJitRowCsrReg: a = AGG, b = G
+            snprintf(buf, sizeof(buf), "fo::row_csr_reg_body<%d, %d>(ch, p);", sp.a, sp.b);
             break;
     }
     return buf;
 }
 
-bool is_outer(const JitSpec &sp) { return sp.kind >= kJitOuterDirect; }
+bool is_outer(const JitSpec &sp) { return sp.kind >= kJitOuterDirect && sp.kind <= kJitOuterDense; }
+bool is_row(const JitSpec &sp) { return sp.kind >= kJitRowDense; }
 
 // The chain as a straight-line functor: in[] holds the input registers (Cell: a, sides;
 // Outer: a, d, sides), c the constant table, o the results.
@@ -250,6 +268,27 @@ std::string generate_source(const DevChain &ch, const JitSpec &sp)
                  "{\n    ", kThreads, (sp.kind == kJitOuterDirect && sp.a > 8) ? 1 : 2,
                  sp.kind == kJitOuterDense ? ", const __grid_constant__ fo::DenseSplit sp" : "");
         s += buf;
+        s += wrapper_text(ch, sp) + "\n}\n";
+        return s;
+    }
+    if (is_row(sp)) {
+        // the Row kernels call the functor from inside as well
+        s += "#define FO_JIT_ROW 1\n";
+        s += functor_text(ch);
+        s += kSkeletonRow;
+        snprintf(buf, sizeof(buf),
+                 "static_assert(sizeof(fo::DevChain) == %zu, \"chain layout\");\n"
+                 "static_assert(sizeof(fo::RowParams) == %zu, \"parameter layout\");\n",
+                 sizeof(DevChain), sizeof(RowParams));
+        s += buf;
+        if (sp.kind == kJitRowDense)
+            snprintf(buf, sizeof(buf), "extern \"C\" __global__ void __launch_bounds__(%d, 1)\n", kDenseBlock);
+        else if (sp.kind == kJitRowNarrow)
+            snprintf(buf, sizeof(buf), "extern \"C\" __global__ void __launch_bounds__(%d)\n", kThreads);
+        else
+            snprintf(buf, sizeof(buf), "extern \"C\" __global__ void __launch_bounds__(%d, 3)\n", kThreads);
+        s += buf;
+        s += "fo_jit_kernel(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::RowParams p)\n{\n    ";
         s += wrapper_text(ch, sp) + "\n}\n";
         return s;
     }
@@ -375,7 +414,7 @@ CUfunction find_kernel(const DevChain &ch, const JitSpec &sp, bool may_compile, 
 }  // namespace
 
 int jit_launch(const JitSpec &sp, const DevChain &ch, const void *params, unsigned grid_x, unsigned grid_y,
-               cudaStream_t st, bool may_compile, bool launch, size_t smem, const void *params2)
+               cudaStream_t st, bool may_compile, bool launch, size_t smem, const void *params2, unsigned block)
 {
     const int mode = g_mode.load();
     if (mode == 0) return kJitUnavailable;
@@ -389,7 +428,7 @@ int jit_launch(const JitSpec &sp, const DevChain &ch, const void *params, unsign
         if (arc != 0) return kJitUnavailable;
     }
     void *args[3] = {(void *)&ch, (void *)params, (void *)params2};
-    const int rc = api().launch(fn, grid_x, grid_y, 1, kThreads, 1, 1, (unsigned)smem, (void *)st, args, nullptr);
+    const int rc = api().launch(fn, grid_x, grid_y, 1, block, 1, 1, (unsigned)smem, (void *)st, args, nullptr);
     if (rc == 0) {
         std::lock_guard<std::mutex> lock(g_mutex);
         ++g_launches;
@@ -491,6 +530,32 @@ int fo_jit_compile_check_outer(const fo_chain *chain, int n_sides, int n_scalars
         case 3: sp = JitSpec{kJitOuterPipe, 2, kOutRight, 0}; break;
         case 4: sp = JitSpec{kJitOuterDense, kOutFull, 0, 0}; break;
         case 5: sp = JitSpec{kJitOuterDense, kOutNone, 0, 0}; break;
+        default: return FO_ERR_UNSUPPORTED;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const std::vector<char> cubin = compile(generate_source(ch, sp), "sm_100a");
+    if (log && log_bytes) snprintf(log, log_bytes, "%s", g_last_log.c_str());
+    return cubin.empty() ? FO_ERR_CHAIN : FO_OK;
+}
+
+int fo_jit_compile_check_row(const fo_chain *chain, int n_sides, int n_scalars, int kernel, char *log,
+                              size_t log_bytes)
+{
+    using namespace fo;
+    if (log && log_bytes) log[0] = 0;
+    double scalars[FO_MAX_SCALARS] = {0};
+    DevChain ch;
+    const int rc = translate_chain(chain, kUseRow, n_sides, scalars, n_scalars, 1, 1, &ch);
+    if (rc != FO_OK) return rc;
+    if (!api().nvrtc_ok) return FO_ERR_UNSUPPORTED;
+    JitSpec sp;
+    switch (kernel) {
+        case 0: sp = JitSpec{kJitRowDense, 4, 4, 2, kRowColT, 1}; break;
+        case 1: sp = JitSpec{kJitRowDense, 8, 16, 1, kRowNone, 0}; break;
+        case 2: sp = JitSpec{kJitRowDense, 1, 1, 8, kRowRow, 1}; break;
+        case 3: sp = JitSpec{kJitRowNarrow, 16, kRowColT, 1, 0, 0}; break;
+        case 4: sp = JitSpec{kJitRowCsr, 2, 0, 0, 0, 0}; break;
+        case 5: sp = JitSpec{kJitRowCsrReg, kRowFull, 8, 0, 0, 0}; break;
         default: return FO_ERR_UNSUPPORTED;
     }
     std::lock_guard<std::mutex> lock(g_mutex);

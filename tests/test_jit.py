@@ -272,3 +272,50 @@ def test_outer_chain_compiled_at_run_time_equals_interpreter_bitwise_and_checker
     got = fo.fused_outer(chain, "t1", X, Ud, Vd, agg="none", sides=[("row", to_dev(r))]).cpu().numpy()
     assert_close(got, oracle.outer(chain, "t1", Xh, w["U"], w["V"], agg="none", sides=[("row", r)]),
                  what="outer jit sides")
+
+
+ROW_GENERIC = [("mul", "t0", "side0", "d"), ("abs", "t1", "t0"), ("sub", "t2", "t1", 0.5)]
+
+
+@pytest.mark.parametrize("kernel", range(6))
+def test_row_kernels_compile_with_a_generated_chain_without_a_gpu(kernel):
+    rc, log = fo.jit_compile_check_row(ROW_GENERIC, "t2", 1, 0, kernel)
+    if rc == -4:
+        pytest.skip("NVRTC not available here")
+    assert rc == 0, log
+    assert "error" not in log
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("layout", ["dense-1000", "dense-100", "narrow-10", "csr"])
+def test_row_chain_compiled_at_run_time_equals_interpreter_bitwise_and_checker(layout):
+    if not fo.jit_stats()[0]:
+        pytest.skip("NVRTC or the driver library is not usable here")
+    rows = 3001
+    if layout == "csr":
+        c = datagen.row_csr_workload(rows, 500, 0.02, seed=91)
+        Xh = {k: c[k] for k in ("rows", "cols", "rowptr", "colidx", "vals")}
+        X = fo.CSR(rows, 500, to_dev(c["rowptr"]), to_dev(c["colidx"]), to_dev(c["vals"]))
+        v, w = c["v"], c["w"]
+        Xabs = dict(Xh, vals=np.abs(c["vals"]))
+    else:
+        cols = int(layout.split("-")[1])
+        r = datagen.row_dense_workload(rows, cols, seed=91)
+        Xh, v, w = r["X"], r["v"], r["w"]
+        X = to_dev(Xh)
+        Xabs = np.abs(Xh)
+    for agg in ("col_t", "row", "full", "none"):
+        launches = fo.jit_stats()[2]
+        fast = fo.fused_row(ROW_GENERIC, "t2", X, to_dev(v), [("row", to_dev(w))], agg=agg).cpu().numpy()
+        assert fo.jit_stats()[2] == launches + 1, "%s %s was not specialised" % (layout, agg)
+        try:
+            fo.force_interpreter(True)
+            slow = fo.fused_row(ROW_GENERIC, "t2", X, to_dev(v), [("row", to_dev(w))], agg=agg).cpu().numpy()
+        finally:
+            fo.force_interpreter(False)
+        if not (layout == "csr" and agg == "col_t"):               # (the CSR column scatter adds through atomics)
+            assert fast.tobytes() == slow.tobytes()
+        ref = oracle.row(ROW_GENERIC, "t2", Xh, v, [("row", w)], agg=agg)
+        scale = oracle.row([("mul", "t0", "side0", "d"), ("add", "t2", "t0", 0.5)], "t2", Xabs, np.abs(v),
+                           [("row", w)], agg=agg)
+        assert_close(fast, ref, absscale=np.abs(scale) + 1e-300, what="row jit %s %s" % (layout, agg))
