@@ -19,10 +19,10 @@
  *     are HOST memory; they are copied at launch and may be freed on return.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
  *     the default stream).  No call allocates, frees or synchronises, with one
- *     documented exception: the first use of a Cell / MAgg chain that the library
+ *     documented exception: the first use of a chain that the library
  *     specialises at run time (see fo_set_jit) compiles and loads a kernel inside
- *     fused_cell / fused_magg unless the chain was prepared with fo_jit_prepare or
- *     the mode forbids it.  fused_cell_static never does.
+ *     the fused_* call unless the chain was prepared (fo_jit_prepare,
+ *     fo_jit_prepare_call) or the mode forbids it.  fused_cell_static never does.
  *   - Inputs are never written.  `out` is fully overwritten.
  *   - `ws` is scratch of at least fused_*_workspace_bytes() bytes, 256-byte
  *     aligned, prepared once with fo_workspace_init(); every call leaves it
@@ -183,17 +183,19 @@ const char *fo_status_string(int status);
 int fo_last_cuda_error(void);
 
 /* Run-time specialisation (the paper's template expansion to source, compilation
- * and plan cache, Section 2.1 "Codegen Architecture").  A Cell / MAgg chain over
- * contiguous inputs (full_agg, MAgg, no_agg) that has no built-in specialisation
- * is written out as straight-line code inside the library's streaming kernel,
- * compiled for the current GPU with NVRTC (a few hundred ms) and cached under its
- * translated program, per CUDA context, for the life of the process; calls with
- * the same chain - whatever the values of its scalars and immediates - reuse it.
+ * and plan cache, Section 2.1 "Codegen Architecture").  A chain that has no
+ * built-in straight-line form - in any call: fused_cell / fused_magg over dense or
+ * CSR inputs, fused_row, fused_outer - is written out as straight-line code inside
+ * the kernel the call would otherwise interpret it in, compiled for the current
+ * GPU with NVRTC (a few hundred ms to a second) and cached under kernel and
+ * translated program, per CUDA context, for the life of the process; calls with the
+ * same chain - whatever the values of its scalars and immediates - reuse it.  (The
+ * pre / post chains of fused_row_b1 are interpreted.)
  * Results are bit-identical to the interpreter's.  NVRTC and the driver library
  * are loaded on demand; if they are missing or a compilation fails the
  * interpreter runs instead, so results never depend on them.
  *   fo_set_jit(mode)  FO_JIT_OFF: never specialise.  FO_JIT_FIRST_USE (default):
- *                     fused_cell / fused_magg compile a chain the first time they
+ *                     the fused_* calls compile a chain the first time they
  *                     see it - that one call compiles, loads a module (which
  *                     allocates) and may synchronise; do it outside stream capture.
  *                     FO_JIT_PREPARED: the calls only look kernels up; a chain that
