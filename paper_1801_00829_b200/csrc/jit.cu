@@ -180,7 +180,7 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
             snprintf(buf, sizeof(buf), "fo::outer_body<%d, %d, %s>(ch, p);", sp.a, sp.b, tf[sp.c & 1]);
             break;
         case kJitOuterPipe:     // a = NK2, b = AGG
-            snprintf(buf, sizeof(buf), "fo::outer_pipe_body<%d, %d>(ch, p);", sp.a, sp.b);
+            snprintf(buf, sizeof(buf), "fo::outer_pipe_body<%d, %d, true>(ch, p);", sp.a, sp.b);
             break;
         case kJitOuterDense:    // a = AGG
             snprintf(buf, sizeof(buf), "fo::outer_dense_body<%d>(ch, p, sp);", sp.a);
@@ -193,7 +193,7 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
             snprintf(buf, sizeof(buf), "fo::row_narrow_body<%d, %d, %s>(ch, p);", sp.a, sp.b, tf[sp.c & 1]);
             break;
         case kJitRowCsr:        // a = G
-            snprintf(buf, sizeof(buf), "fo::row_csr_body<%d>(ch, p);", sp.a);
+            snprintf(buf, sizeof(buf), "fo::row_csr_body<%d, true>(ch, p);", sp.a);
             break;
         default:                // kJitRowCsrReg: a = AGG, b = G
             snprintf(buf, sizeof(buf), "fo::row_csr_reg_body<%d, %d>(ch, p);", sp.a, sp.b);

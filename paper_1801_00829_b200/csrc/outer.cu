@@ -46,8 +46,8 @@ cudaError_t launch_outer(const DevChain &ch, const OuterParams &p, int agg, bool
 }
 
 // full_agg / no_agg / right_mm through the pipelined kernel; NK2 is exactly ceil(rank / 16).
-template <int NK2, int AGG>
-cudaError_t launch_outer_pipe_one(const DevChain &ch, const OuterParams &p, int grid, cudaStream_t st)
+template <int NK2, int AGG, bool GENERIC>
+cudaError_t launch_outer_pipe_gen(const DevChain &ch, const OuterParams &p, int grid, cudaStream_t st)
 {
     const size_t smem = (size_t)(kThreads / 32) * kStageRows * p.rank * sizeof(double);
     // the attribute sticks to the function: raise it when a call needs more than any before
@@ -56,12 +56,20 @@ cudaError_t launch_outer_pipe_one(const DevChain &ch, const OuterParams &p, int 
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || granted[dev].load(std::memory_order_relaxed) < smem) {
-        e = cudaFuncSetAttribute(outer_pipe_kernel<NK2, AGG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = cudaFuncSetAttribute(outer_pipe_kernel<NK2, AGG, GENERIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) granted[dev].store(smem, std::memory_order_relaxed);
     }
-    outer_pipe_kernel<NK2, AGG><<<grid, kThreads, smem, st>>>(ch, p);
+    outer_pipe_kernel<NK2, AGG, GENERIC><<<grid, kThreads, smem, st>>>(ch, p);
     return cudaGetLastError();
+}
+
+// an instance with the interpreter for chains without an inline form, one without it for the rest
+template <int NK2, int AGG>
+cudaError_t launch_outer_pipe_one(const DevChain &ch, const OuterParams &p, int grid, cudaStream_t st)
+{
+    return p.chain_kind == kOuterGeneric ? launch_outer_pipe_gen<NK2, AGG, true>(ch, p, grid, st)
+                                         : launch_outer_pipe_gen<NK2, AGG, false>(ch, p, grid, st);
 }
 
 template <int NK2>

@@ -57,6 +57,11 @@ __device__ __forceinline__ double outer_chain(const DevChain &ch, int, int, doub
     JitFn::eval(in, ch.consts, o);
     return o[0];
 }
+template <bool GENERIC>
+__device__ __forceinline__ double outer_chain_split(const DevChain &ch, int kind, int kc, double a, double d)
+{
+    return outer_chain(ch, kind, kc, a, d);
+}
 __device__ __forceinline__ double outer_chain_sides(const DevChain &ch, double a, double d,
                                                     const double (&sv)[kOuterMaxSides])
 {
@@ -103,6 +108,24 @@ __device__ __forceinline__ double outer_chain(const DevChain &ch, int kind, int 
     if (OUT_OF_LINE) return outer_chain_interp_call(ch, a, d);
     const double none[kOuterMaxSides] = {0.0, 0.0, 0.0};
     return outer_chain_sides(ch, a, d, none);
+}
+
+// The same with the choice made at compile time: a kernel instance either carries the
+// interpreter (GENERIC) or the inline forms, not both - the inline forms' instance then
+// needs fewer registers.
+template <bool GENERIC>
+__device__ __forceinline__ double outer_chain_split(const DevChain &ch, int kind, int kc, double a, double d)
+{
+    if (GENERIC) {
+        const double none[kOuterMaxSides] = {0.0, 0.0, 0.0};
+        return outer_chain_sides(ch, a, d, none);
+    }
+    if (kind == kOuterXlogd) return a * slow_log(d + ch.consts[kc]);
+    if (kind == kOuterMaskDot) return (a != 0.0 ? 1.0 : 0.0) * d;
+    const double t0 = a != 0.0 ? 1.0 : 0.0;       // kOuterWsloss
+    const double t1 = a - d;
+    const double t2 = t1 * t1;
+    return t0 * t2;
 }
 #endif
 
@@ -310,7 +333,7 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 // every step (an empty group at the tail) so that "all but the newest" always
 // names the step about to be used.
 // NK2 = ceil(rank / 16) exactly: only the last 16-column piece of a row needs a bounds check.
-template <int NK2, int AGG>
+template <int NK2, int AGG, bool GENERIC>
 __device__ __forceinline__ void outer_pipe_body(const DevChain &ch, const OuterParams &p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -405,7 +428,7 @@ __device__ __forceinline__ void outer_pipe_body(const DevChain &ch, const OuterP
                     // the second), then O_i += w * V_j from the rows still in the buffer
                     const int sidx = 8 * s + 4 * ((lane >> 2) & 1) + grp;
                     const double a = __shfl_sync(full, amine, sidx & 31);
-                    double w = outer_chain(ch, p.chain_kind, p.kconst, a, v);
+                    double w = outer_chain_split<GENERIC>(ch, p.chain_kind, p.kconst, a, v);
                     if (sidx >= cnt) w = 0.0;         // a row fetched again at a ragged end adds nothing
                     const double w0 = __shfl_sync(full, w, grp * 8), w1 = __shfl_sync(full, w, grp * 8 + 4);
 #pragma unroll
@@ -430,7 +453,7 @@ __device__ __forceinline__ void outer_pipe_body(const DevChain &ch, const OuterP
             }
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             if (AGG != kOutRight) {
-                const double w = outer_chain(ch, p.chain_kind, p.kconst, amine, dmine);
+                const double w = outer_chain_split<GENERIC>(ch, p.chain_kind, p.kconst, amine, dmine);
                 if (AGG == kOutFull) {
                     if (valid) acc += w;
                 } else {
@@ -646,11 +669,11 @@ outer_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterP
     outer_body<NK2, AGG, ALIGNED>(ch, p);
 }
 
-template <int NK2, int AGG>
+template <int NK2, int AGG, bool GENERIC>
 __global__ void __launch_bounds__(kThreads, 2)
 outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
 {
-    outer_pipe_body<NK2, AGG>(ch, p);
+    outer_pipe_body<NK2, AGG, GENERIC>(ch, p);
 }
 
 template <int AGG>

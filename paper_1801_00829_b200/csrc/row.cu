@@ -234,7 +234,9 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
                 if (jrc == FO_OK) return cudaSuccess;
                 if (jrc != kJitUnavailable) return cudaErrorLaunchFailure;
             }
-            if (agg == FO_ROW_COL_T_AGG) return go(row_csr_kernel<G>, smem);
+            if (agg == FO_ROW_COL_T_AGG)
+                return p.chain_kind == kChainGeneric ? go(row_csr_kernel<G, true>, smem)
+                                                     : go(row_csr_kernel<G, false>, smem);
             if (agg == FO_ROW_NO_AGG) return go(row_csr_reg_kernel<kRowNone, G>, smem_reg);
             if (agg == FO_ROW_ROW_AGG) return go(row_csr_reg_kernel<kRowRow, G>, smem_reg);
             return go(row_csr_reg_kernel<kRowFull, G>, smem_reg);

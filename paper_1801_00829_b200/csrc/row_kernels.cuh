@@ -459,7 +459,7 @@ __device__ __forceinline__ void row_narrow_body(const DevChain &ch, const RowPar
 // the scatter uses shared-memory atomics (their order is not fixed).
 constexpr int kCsrStage = 512;            // stored cells a warp can stage per block of rows
 
-template <int G>
+template <int G, bool GENERIC>
 __device__ __forceinline__ void row_csr_body(const DevChain &ch, const RowParams &p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -538,7 +538,9 @@ __device__ __forceinline__ void row_csr_body(const DevChain &ch, const RowParams
             const double dall = __shfl_sync(0xffffffffu, d, (lane & (32 / G - 1)) * G);
             if (lane / (32 / G) == it) dmine = dall;
         }
-        const double t = lane_chain(ch, p.chain_kind, dmine, sv);
+        // (an instance either carries the interpreter or the two inline forms)
+        const double t = GENERIC ? lane_chain(ch, kChainGeneric, dmine, sv)
+                                 : (p.chain_kind == kChainDot ? dmine : sv[0] * dmine);
 #pragma unroll 1
         for (int it = 0; it < nit; ++it) {
             const int rr = it * (32 / G) + grp;
@@ -698,11 +700,11 @@ row_narrow_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ R
     row_narrow_body<NC, AGG, VEC>(ch, p);
 }
 
-template <int G>
+template <int G, bool GENERIC>
 __global__ void __launch_bounds__(kThreads, 3)
 row_csr_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ RowParams p)
 {
-    row_csr_body<G>(ch, p);
+    row_csr_body<G, GENERIC>(ch, p);
 }
 
 template <int AGG, int G>
