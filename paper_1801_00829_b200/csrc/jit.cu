@@ -196,7 +196,7 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
             snprintf(buf, sizeof(buf), "fo::row_csr_body<%d, true>(ch, p);", sp.a);
             break;
         default:                // kJitRowCsrReg: a = AGG, b = G
-            snprintf(buf, sizeof(buf), "fo::row_csr_reg_body<%d, %d>(ch, p);", sp.a, sp.b);
+            snprintf(buf, sizeof(buf), "fo::row_csr_reg_body<%d, %d, true>(ch, p);", sp.a, sp.b);
             break;
     }
     return buf;

@@ -237,9 +237,15 @@ int fused_row(const fo_chain *chain, const fo_mat *X, const double *v, const fo_
             if (agg == FO_ROW_COL_T_AGG)
                 return p.chain_kind == kChainGeneric ? go(row_csr_kernel<G, true>, smem)
                                                      : go(row_csr_kernel<G, false>, smem);
-            if (agg == FO_ROW_NO_AGG) return go(row_csr_reg_kernel<kRowNone, G>, smem_reg);
-            if (agg == FO_ROW_ROW_AGG) return go(row_csr_reg_kernel<kRowRow, G>, smem_reg);
-            return go(row_csr_reg_kernel<kRowFull, G>, smem_reg);
+            const bool gen = p.chain_kind == kChainGeneric;
+            if (agg == FO_ROW_NO_AGG)
+                return gen ? go(row_csr_reg_kernel<kRowNone, G, true>, smem_reg)
+                           : go(row_csr_reg_kernel<kRowNone, G, false>, smem_reg);
+            if (agg == FO_ROW_ROW_AGG)
+                return gen ? go(row_csr_reg_kernel<kRowRow, G, true>, smem_reg)
+                           : go(row_csr_reg_kernel<kRowRow, G, false>, smem_reg);
+            return gen ? go(row_csr_reg_kernel<kRowFull, G, true>, smem_reg)
+                       : go(row_csr_reg_kernel<kRowFull, G, false>, smem_reg);
         };
         if (mean_len <= 12.0) e = by_agg(std::integral_constant<int, 2>());
         else if (mean_len <= 24.0) e = by_agg(std::integral_constant<int, 4>());
