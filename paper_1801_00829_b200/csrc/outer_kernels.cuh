@@ -368,14 +368,39 @@ __device__ __forceinline__ void outer_pipe_body(const DevChain &ch, const OuterP
             u[c] = (beg < end && col < rank) ? __ldg(reinterpret_cast<const double2 *>(urow + col))
                                              : make_double2(0.0, 0.0);
         }
+        // X and U stream from HBM once: ask the L2 now for what this warp's next row will read first
+        // (its U row, and the head of its cells), so that those loads find it there
+        {
+            const long long nrow = row + kThreads / 32;
+            if (nrow < row_hi) {
+                const int nb = __ldg(p.rowptr + nrow);
+                const char *pu = reinterpret_cast<const char *>(p.U + nrow * p.ldu);
+                const char *pc = reinterpret_cast<const char *>(p.colidx + nb);
+                const char *pv = reinterpret_cast<const char *>(p.vals + nb);
+                const char *what = lane < 8 ? pu + 128 * lane : lane < 12 ? pc + 128 * (lane - 8) : pv + 128 * (lane - 12);
+                const bool ok = lane < 8 ? 128 * lane < rank * 8 : lane < 12 ? nb + 32 * (lane - 8) < p.nnz
+                                                                 : lane < 20 && nb + 16 * (lane - 12) < p.nnz;
+                if (ok) asm volatile("prefetch.global.L2 [%0];" ::"l"(what));
+            }
+        }
         double2 racc[AGG == kOutRight ? NK2 : 1];      // right_mm: this group's share of O_i
 #pragma unroll
         for (int c = 0; c < (AGG == kOutRight ? NK2 : 1); ++c) racc[c] = make_double2(0.0, 0.0);
+        // the cells of a chunk arrive a chunk ahead
+        int jnext = (beg + lane < end) ? __ldg(p.colidx + beg + lane) : 0;
+        double anext = (beg + lane < end) ? __ldg(p.vals + beg + lane) : 0.0;
         for (int c0 = beg; c0 < end; c0 += 32) {
             const int cnt = (end - c0 < 32) ? end - c0 : 32;
             const bool valid = lane < cnt;
-            const int jmine = valid ? __ldg(p.colidx + c0 + lane) : 0;
-            const double amine = valid ? __ldg(p.vals + c0 + lane) : 0.0;
+            const int jmine = jnext;
+            const double amine = anext;
+            if (c0 + 32 + lane < end) {
+                jnext = __ldg(p.colidx + c0 + 32 + lane);
+                anext = __ldg(p.vals + c0 + 32 + lane);
+            } else {
+                jnext = 0;
+                anext = 0.0;
+            }
             const int nsteps = (cnt + 7) >> 3;
             double dmine = 0.0;
 
