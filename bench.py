@@ -42,9 +42,9 @@ WSLOSS = [("ne", "t0", "a", 0.0), ("sub", "t1", "a", "d"), ("mul", "t2", "t1", "
 NCU_DRAM_BYTES_PER_UNIT = {
     "cell": 24.014e6 / 1e6,                      # per cell (3 inputs)
     "magg": (480.018e6 + 3.727e6) / 2e7,         # per cell (3 inputs; 200 000 x 100 capture)
-    "row_dense": (1601.768e6 + 7.483e6) / 2e5,   # per row of 1000 columns (200 000 x 1000 capture)
-    "row_csr": (264.970e6 + 5.619e6) / 19998162, # per stored cell (2 000 000 x 1000 @ 0.01 capture)
-    "outer": (1365.918e6 + 3.832e6) / 9996322,   # per stored cell (full-size capture, outer_pipe_kernel)
+    "row_dense": (1601.696e6 + 7.937e6) / 2e5,   # per row of 1000 columns (200 000 x 1000 capture)
+    "row_csr": (264.047e6 + 3.881e6) / 19998162, # per stored cell (2 000 000 x 1000 @ 0.01 capture)
+    "outer": (1582.646e6 + 3.686e6) / 9996322,   # per stored cell (full-size capture, outer_pipe_kernel)
 }
 
 FULL = {
