@@ -723,7 +723,7 @@ def oracle_single_thread(np_inputs, shapes):
     return t
 
 
-REL_TOL = 1e-10           # spec tolerance for fp64 aggregates
+REL_TOL = 1e-10           # relative tolerance for fp64 aggregates and elementwise outputs
 ABS_FLOOR = 1e-15         # times the sum of the magnitudes of a sum's terms (sums that cancel)
 
 
