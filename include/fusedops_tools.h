@@ -34,9 +34,10 @@ int fo_set_force_interpreter(int on);
  *   b1.mma            0 | 1  fused_row_b1: multiply-add kernel / tensor-core kernel
  *   b1.shape, b1.mma_shape   compiled shapes of those two kernels ("p,r,kl" / "w,kb")
  *   b1.narrow         0      fused_row_b1 without the thread-per-row kernel
- *   outer.kernel      "pipe" | "direct" | "dense"   schedule of fused_outer (per stored cell with
- *                     staged factor rows / with plain gathers, or tile by tile for densely
- *                     stored inputs); by default the library chooses from layout and stored share
+ *   outer.kernel      "bulk" | "pipe" | "direct" | "dense"   schedule of fused_outer (per stored cell with
+ *                     factor rows staged by bulk copies / by 16-byte copies / with plain gathers,
+ *                     or tile by tile for densely stored inputs); by default the library chooses
+ *                     from layout, rank and stored share
  *   cell.stamps       1      the streaming Cell / MAgg kernel records phase times (fo_cell_stamps) */
 int fo_tune(const char *name, const char *value);
 
@@ -59,7 +60,8 @@ int fo_jit_compile_check(const fo_chain *chain, int n_sides, int n_scalars, int 
                          char *log, size_t log_bytes);
 /* The same for a chain of the Outer template.  `kernel`: 0 / 1 the per-cell kernel with
  * plain gathers (full_agg at rank <= 112, left_mm at rank <= 256), 2 / 3 the kernel that
- * stages factor rows (full_agg, right_mm), 4 / 5 the tiled kernel (full_agg, no_agg). */
+ * stages factor rows with 16-byte copies (full_agg, right_mm), 4 / 5 the tiled kernel (full_agg,
+ * no_agg), 6 / 7 the kernel that stages factor rows with bulk copies (full_agg, no_agg). */
 int fo_jit_compile_check_outer(const fo_chain *chain, int n_sides, int n_scalars, int kernel,
                                char *log, size_t log_bytes);
 /* The same for a chain of the Row template.  `kernel`: 0 / 1 / 2 the dense kernel (1000-column

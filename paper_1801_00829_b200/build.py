@@ -68,7 +68,7 @@ def _compile_one(src: str, verbose: bool) -> str:
 
 # what the run-time specialised kernels are made of: Cell / MAgg, and Outer
 JIT_HEADERS = {"jit_source.inc": ["common.cuh", "cell_flat.cuh", "cell_tiles.cuh", "cell_csr.cuh"],
-               "jit_source_outer.inc": ["common.cuh", "outer_kernels.cuh"],
+               "jit_source_outer.inc": ["common.cuh", "ptx.cuh", "outer_kernels.cuh"],
                "jit_source_row.inc": ["common.cuh", "ptx.cuh", "row_kernels.cuh"]}
 
 

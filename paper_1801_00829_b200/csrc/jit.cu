@@ -182,6 +182,9 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
         case kJitOuterPipe:     // a = NK2, b = AGG
             snprintf(buf, sizeof(buf), "fo::outer_pipe_body<%d, %d, true>(ch, p);", sp.a, sp.b);
             break;
+        case kJitOuterBulk:     // a = NK2, b = AGG
+            snprintf(buf, sizeof(buf), "fo::outer_bulk_body<%d, %d, true>(ch, p);", sp.a, sp.b);
+            break;
         case kJitOuterDense:    // a = AGG
             snprintf(buf, sizeof(buf), "fo::outer_dense_body<%d>(ch, p, sp);", sp.a);
             break;
@@ -202,8 +205,8 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
     return buf;
 }
 
-bool is_outer(const JitSpec &sp) { return sp.kind >= kJitOuterDirect && sp.kind <= kJitOuterDense; }
-bool is_row(const JitSpec &sp) { return sp.kind >= kJitRowDense; }
+bool is_outer(const JitSpec &sp) { return (sp.kind >= kJitOuterDirect && sp.kind <= kJitOuterDense) || sp.kind == kJitOuterBulk; }
+bool is_row(const JitSpec &sp) { return sp.kind >= kJitRowDense && sp.kind <= kJitRowCsrReg; }
 
 // The chain as a straight-line functor: in[] holds the input registers (Cell: a, sides;
 // Outer: a, d, sides), c the constant table, o the results.
@@ -265,7 +268,8 @@ std::string generate_source(const DevChain &ch, const JitSpec &sp)
         snprintf(buf, sizeof(buf),
                  "extern \"C\" __global__ void __launch_bounds__(%d, %d)\n"
                  "fo_jit_kernel(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::OuterParams p%s)\n"
-                 "{\n    ", kThreads, (sp.kind == kJitOuterDirect && sp.a > 8) ? 1 : 2,
+                 "{\n    ", sp.kind == kJitOuterBulk ? kBulkWarps * 32 : kThreads,
+                 (sp.kind == kJitOuterBulk || (sp.kind == kJitOuterDirect && sp.a > 8)) ? 1 : 2,
                  sp.kind == kJitOuterDense ? ", const __grid_constant__ fo::DenseSplit sp" : "");
         s += buf;
         s += wrapper_text(ch, sp) + "\n}\n";
@@ -530,6 +534,8 @@ int fo_jit_compile_check_outer(const fo_chain *chain, int n_sides, int n_scalars
         case 3: sp = JitSpec{kJitOuterPipe, 2, kOutRight, 0}; break;
         case 4: sp = JitSpec{kJitOuterDense, kOutFull, 0, 0}; break;
         case 5: sp = JitSpec{kJitOuterDense, kOutNone, 0, 0}; break;
+        case 6: sp = JitSpec{kJitOuterBulk, 7, kOutFull, 0}; break;
+        case 7: sp = JitSpec{kJitOuterBulk, 4, kOutNone, 0}; break;
         default: return FO_ERR_UNSUPPORTED;
     }
     std::lock_guard<std::mutex> lock(g_mutex);

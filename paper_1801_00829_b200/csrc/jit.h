@@ -14,7 +14,8 @@ bool jit_first_use();          // the mode in which an entry point may compile a
 // Which skeleton a run-time specialised kernel instantiates, and with which template
 // arguments (their meaning depends on the kind; see wrapper_text in jit.cu).
 enum JitKind { kJitFlat = 0, kJitRows = 1, kJitCols = 2, kJitCsr = 3, kJitOuterDirect = 4, kJitOuterPipe = 5,
-               kJitOuterDense = 6, kJitRowDense = 7, kJitRowNarrow = 8, kJitRowCsr = 9, kJitRowCsrReg = 10 };
+               kJitOuterDense = 6, kJitRowDense = 7, kJitRowNarrow = 8, kJitRowCsr = 9, kJitRowCsrReg = 10,
+               kJitOuterBulk = 11 };
 struct JitSpec {
     int kind, a, b, c, d, e;
 };

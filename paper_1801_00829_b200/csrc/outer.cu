@@ -80,6 +80,37 @@ cudaError_t launch_outer_pipe(const DevChain &ch, const OuterParams &p, int agg,
     return launch_outer_pipe_one<NK2, kOutRight>(ch, p, grid, st);
 }
 
+// full_agg / no_agg through the bulk-copy kernel; NK2 is exactly ceil(rank / 16) (at most 7 here).
+constexpr int kBulkMinRank = 96;    // below, a row is too short to be worth the ~54 cycles its copy holds the warp
+
+template <int NK2, int AGG, bool GENERIC>
+cudaError_t launch_outer_bulk_one(const DevChain &ch, const OuterParams &p, int grid, size_t smem, cudaStream_t st)
+{
+    static std::atomic<size_t> granted[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || granted[dev].load(std::memory_order_relaxed) < smem) {
+        e = cudaFuncSetAttribute(outer_bulk_kernel<NK2, AGG, GENERIC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) granted[dev].store(smem, std::memory_order_relaxed);
+    }
+    outer_bulk_kernel<NK2, AGG, GENERIC><<<grid, kBulkWarps * 32, smem, st>>>(ch, p);
+    return cudaGetLastError();
+}
+
+template <int NK2>
+cudaError_t launch_outer_bulk(const DevChain &ch, const OuterParams &p, int agg, int grid, size_t smem, cudaStream_t st)
+{
+    const bool gen = p.chain_kind == kOuterGeneric;
+    if (agg == FO_OUTER_FULL_AGG)
+        return gen ? launch_outer_bulk_one<NK2, kOutFull, true>(ch, p, grid, smem, st)
+                   : launch_outer_bulk_one<NK2, kOutFull, false>(ch, p, grid, smem, st);
+    return gen ? launch_outer_bulk_one<NK2, kOutNone, true>(ch, p, grid, smem, st)
+               : launch_outer_bulk_one<NK2, kOutNone, false>(ch, p, grid, smem, st);
+}
+
 // Work split of the tiled schedule: column ranges so that there are enough work items for a
 // few rounds over the SMs (the last round a small share), and the grid.
 bool dense_plan(const OuterParams &p, int sms, DenseSplit *sp, long long *grid)
@@ -280,6 +311,35 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
         }
         e = agg == FO_OUTER_FULL_AGG ? launch_outer_dense_one<kOutFull>(ch, p, sms, st)
                                      : launch_outer_dense_one<kOutNone>(ch, p, sms, st);
+        return e == cudaSuccess ? FO_OK : cuda_fail(e);
+    }
+    // full_agg / no_agg: factor rows landed by bulk copies where 16 warps with two slots of eight
+    // rows each fit in an SM's shared memory and a row is long enough to be worth a copy of its own
+    const bool want_bulk = strcmp(which, "bulk") == 0, want_pipe = strcmp(which, "pipe") == 0;
+    const bool bulk_fits = (size_t)kBulkWarps * bulk_warp_bytes(rank) <= 225u * 1024u;
+    if (copyable && !want_direct && !want_pipe && agg != FO_OUTER_RIGHT_MM && bulk_fits &&
+        (want_bulk || rank >= kBulkMinRank)) {
+        const size_t smem = (size_t)kBulkWarps * bulk_warp_bytes(rank);
+        long long g = sms;
+        const long long by_cells = (X->nnz + 8ll * kBulkWarps - 1) / (8ll * kBulkWarps);    // a stage per warp at least
+        if (g > by_cells) g = by_cells;
+        if (g < 1) g = 1;
+        if (try_jit) {
+            const JitSpec js = {kJitOuterBulk, nk2, kagg, 0};
+            const int jrc = jit_launch(js, ch, &p, (unsigned)g, 1, st, jit_first_use(), true, smem, nullptr,
+                                       kBulkWarps * 32);
+            if (jrc == FO_OK) return FO_OK;
+            if (jrc != kJitUnavailable) return jrc;
+        }
+        switch (nk2) {
+            case 1: e = launch_outer_bulk<1>(ch, p, agg, (int)g, smem, st); break;
+            case 2: e = launch_outer_bulk<2>(ch, p, agg, (int)g, smem, st); break;
+            case 3: e = launch_outer_bulk<3>(ch, p, agg, (int)g, smem, st); break;
+            case 4: e = launch_outer_bulk<4>(ch, p, agg, (int)g, smem, st); break;
+            case 5: e = launch_outer_bulk<5>(ch, p, agg, (int)g, smem, st); break;
+            case 6: e = launch_outer_bulk<6>(ch, p, agg, (int)g, smem, st); break;
+            default: e = launch_outer_bulk<7>(ch, p, agg, (int)g, smem, st); break;
+        }
         return e == cudaSuccess ? FO_OK : cuda_fail(e);
     }
     if (copyable && !want_direct) {

@@ -4,6 +4,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ptx.cuh"
 #ifndef FO_JIT_OUTER
 #include "chain.cuh"
 #endif
@@ -510,6 +511,217 @@ __device__ __forceinline__ void outer_pipe_body(const DevChain &ch, const OuterP
         if (publish_and_is_last(p.head, &s_flag))
             final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
     }
+}
+
+// --------------------------------------------------------------------- bulk
+// full_agg / no_agg with the factor rows landed by the bulk-copy engine.  Every warp
+// owns a contiguous range of rows holding an equal share of the stored cells and
+// works through it in stages of up to eight cells of one row.  A stage's V rows are
+// fetched by ONE bulk copy each (a lane per copy, so one instruction starts them all)
+// into a slot of the warp's private two-slot ring and counted on the slot's mbarrier;
+// the warp never waits for anyone but its own copies (every wait bounded).  Column
+// indices and values run ahead of the copies through a small ring in shared memory,
+// filled 32 cells at a time; U_i is read at a row's first stage, having been requested
+// from L2 when that stage's copies were started.
+// Starting a bulk copy holds the issuing warp for about 54 cycles per row, so this
+// schedule needs many warps: it is used where 16 of them fit (two slots of eight rows
+// each: factor rows of up to 108 doubles), and there it beats the 16-byte asynchronous
+// copies of outer_pipe_kernel (0.636 against 0.659 ms at rank 100).
+constexpr int kBulkWarps = 16;       // warps per CTA, one CTA per SM
+constexpr int kBulkDepth = 2;        // slots per ring
+constexpr int kBulkRing = 64;        // cells of (colidx, vals) kept per warp
+constexpr int kBulkCells = 8;        // cells per stage
+
+__host__ __device__ inline size_t bulk_warp_bytes(int rank)
+{
+    return (size_t)kBulkDepth * kBulkCells * rank * 8 + kBulkRing * 12 + kBulkDepth * 16;
+}
+
+template <int NK2, int AGG, bool GENERIC>
+__device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterParams &p)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ unsigned long long s_bar[kBulkWarps * kBulkDepth];
+    __shared__ double s_red[32];
+    __shared__ unsigned int s_flag;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int W = blockDim.x >> 5;
+    constexpr int D = kBulkDepth;
+    const int l8 = lane & 7, grp = lane >> 3;
+    const unsigned full = 0xffffffffu;
+    const int rank = p.rank;                           // even
+    const unsigned rowbytes = (unsigned)rank * 8u;
+    const int slot_doubles = kBulkCells * rank;        // a stage's V rows
+    unsigned char *base = smem_raw + (size_t)warp * bulk_warp_bytes(rank);
+    double *slots = reinterpret_cast<double *>(base);
+    double *aring = slots + (size_t)D * slot_doubles;
+    int *jring = reinterpret_cast<int *>(aring + kBulkRing);
+    int4 *meta = reinterpret_cast<int4 *>(jring + kBulkRing);
+    unsigned long long *bar = s_bar + warp * kBulkDepth;
+
+    if (lane == 0) {
+        for (int s = 0; s < D; ++s) mbar_init(&bar[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const long long GW = (long long)gridDim.x * W, gw = (long long)blockIdx.x * W + warp;
+    const long long row_lo = gw == 0 ? 0 : lower_row_warp(p.rowptr, p.rows, (p.nnz * gw) / GW, lane);
+    const long long row_hi = gw == GW - 1 ? p.rows : lower_row_warp(p.rowptr, p.rows, (p.nnz * (gw + 1)) / GW, lane);
+    const long long P0 = __ldg(p.rowptr + row_lo), P1 = __ldg(p.rowptr + row_hi);
+
+    // (colidx, vals) ring: cells [.., S) relative to P0 are in shared memory, the chunk
+    // [S, S + 32) is on its way in registers
+    int S = 0, jn = 0;
+    double an = 0.0;
+    auto load_chunk = [&]() {
+        const long long pp = P0 + S + lane;
+        if (pp < P1) {
+            jn = __ldg(p.colidx + pp);
+            an = __ldg(p.vals + pp);
+        }
+    };
+    auto store_chunk = [&]() {
+        jring[(S + lane) & (kBulkRing - 1)] = jn;
+        aring[(S + lane) & (kBulkRing - 1)] = an;
+        S += 32;
+    };
+    load_chunk();
+    store_chunk();
+    load_chunk();
+    __syncwarp();
+
+    long long irow = row_lo, ipos = P0, iend = P0;
+    bool ifirst = true;
+    auto next_row = [&]() {
+        while (irow < row_hi) {
+            iend = __ldg(p.rowptr + irow + 1);
+            if (iend > ipos) break;
+            ++irow;
+        }
+    };
+    next_row();
+    auto issue = [&](int slot) {
+        const int q = (int)(ipos - P0);
+        const int cnt = (iend - ipos < kBulkCells) ? (int)(iend - ipos) : kBulkCells;
+        if (q + cnt > S) {
+            store_chunk();
+            load_chunk();
+            __syncwarp();
+        }
+        const int j = lane < cnt ? jring[(q + lane) & (kBulkRing - 1)] : 0;
+        if (lane == 0) {
+            meta[slot] = make_int4(q, cnt | (ifirst ? 0x100 : 0), (int)(irow - row_lo), 0);
+            mbar_expect_tx(&bar[slot], (unsigned)cnt * rowbytes);
+        }
+        __syncwarp();
+        double *sl = slots + (size_t)slot * slot_doubles;
+        if (lane < cnt) bulk_g2s(sl + lane * rank, p.V + (long long)j * p.ldv, rowbytes, &bar[slot]);
+        else if (ifirst && lane >= 16 && 128 * (lane - 16) < rank * 8)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.U + irow * p.ldu) + 128 * (lane - 16)));
+        ipos += cnt;
+        ifirst = false;
+        if (ipos == iend) {
+            ++irow;
+            next_row();
+            ifirst = true;
+        }
+    };
+
+    int issued = 0;
+    while (issued < D && irow < row_hi) issue(issued++);
+
+    double2 u[NK2];
+#pragma unroll
+    for (int c = 0; c < NK2; ++c) u[c] = make_double2(0.0, 0.0);
+    double acc = 0.0;
+    bool timed_out = false;
+    const int t = grp + 4 * ((lane >> 2) & 1);        // the stage's cell whose total this lane ends up with
+    const bool holder = (lane & 3) == 0;
+
+    int cslot = 0, inflight = issued;
+    unsigned cphase = 0;
+    while (inflight > 0) {
+        const int4 m = meta[cslot];
+        const int q = m.x, cnt = m.y & 0xff;
+        const bool first = (m.y & 0x100) != 0;
+        const double a = aring[(q + t) & (kBulkRing - 1)];
+        if (!__all_sync(full, mbar_wait(&bar[cslot], cphase))) {      // the whole warp leaves together
+            timed_out = true;
+            break;
+        }
+        const double *sl = slots + (size_t)cslot * slot_doubles;
+        if (first) {
+            const double *us = p.U + (row_lo + m.z) * p.ldu;
+#pragma unroll
+            for (int c = 0; c < NK2; ++c)
+                if (c < NK2 - 1 || 16 * c + 2 * l8 < rank)
+                    u[c] = __ldg(reinterpret_cast<const double2 *>(us + 16 * c + 2 * l8));
+        }
+        double dx[2] = {0.0, 0.0}, dy[2] = {0.0, 0.0};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const double *src = sl + (grp + 4 * i) * rank + 2 * l8;
+#pragma unroll
+            for (int c = 0; c < NK2; ++c) {
+                if (c < NK2 - 1 || 16 * c + 2 * l8 < rank) {
+                    const double2 x = *reinterpret_cast<const double2 *>(src + 16 * c);
+                    dx[i] = fma(u[c].x, x.x, dx[i]);
+                    dy[i] = fma(u[c].y, x.y, dy[i]);
+                }
+            }
+        }
+        const double d0 = dx[0] + dy[0], d1 = dx[1] + dy[1];
+        const bool up = (lane & 4) != 0;
+        double v = (up ? d1 : d0) + __shfl_xor_sync(full, up ? d0 : d1, 4);
+        v += __shfl_xor_sync(full, v, 2);
+        v += __shfl_xor_sync(full, v, 1);
+        const double w = outer_chain_split<GENERIC>(ch, p.chain_kind, p.kconst, a, v);
+        if (AGG == kOutFull) {
+            if (holder && t < cnt) acc += w;
+        } else {
+            if (holder && t < cnt) p.out[P0 + q + t] = w;
+        }
+        __syncwarp();                  // everyone is done with the slot: refill it
+        --inflight;
+        if (irow < row_hi) {
+            issue(cslot);
+            ++inflight;
+        }
+        if (++cslot == D) {
+            cslot = 0;
+            cphase ^= 1u;
+        }
+    }
+    if (timed_out) {
+        // give the copies still in flight a (bounded) chance to land before the CTA's
+        // shared memory is given up
+        for (int k = 0; k < inflight; ++k) {
+            mbar_wait(&bar[cslot], cphase);
+            if (++cslot == D) {
+                cslot = 0;
+                cphase ^= 1u;
+            }
+        }
+        if (lane == 0) atomicExch(&p.head->status, 1u);
+    }
+
+    if (AGG == kOutFull) {
+        double v1[1] = {acc};
+        block_sum<1>(v1, s_red);
+        if (threadIdx.x == 0) p.partials[blockIdx.x] = v1[0];
+        if (publish_and_is_last(p.head, &s_flag))
+            final_sum_small(p.partials, gridDim.x, 1, p.out, s_red);
+    }
+}
+
+template <int NK2, int AGG, bool GENERIC>
+__global__ void __launch_bounds__(kBulkWarps * 32, 1)
+outer_bulk_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
+{
+    outer_bulk_body<NK2, AGG, GENERIC>(ch, p);
 }
 
 // -------------------------------------------------------------------- dense

@@ -502,17 +502,36 @@ def test_outer_dense_schedule(fo, rows, cols, rank, density, agg):
                  oracle.outer(gen, "t3", Xh, w["U"], w["V"], agg=agg, mode="dense"), what="outer tiled generic")
 
 
-@pytest.mark.parametrize("schedule", ["pipe", "direct", "dense"])
+@pytest.mark.parametrize("schedule", ["bulk", "pipe", "direct", "dense"])
 def test_outer_every_schedule_on_a_sparse_input(fo, outer_schedule, schedule):
     w, Xh = outer_case(700, 900, 100, 0.02, seed=15)
+    w["rowptr"] = w["rowptr"].copy()
     Xd, Ud, Vd = csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"])
     outer_schedule(schedule)
+    assert fo.device_status() == 0
     for agg in ("full", "none"):
         ref = oracle.outer(WSLOSS, "t3", Xh, w["U"], w["V"], agg=agg, mode="masked")
         got = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()
         assert_close(got, ref, what="outer %s %s" % (schedule, agg))
         again = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()
         assert again.tobytes() == got.tobytes()
+    assert fo.device_status() == 0               # no bounded wait ran out
+
+
+@pytest.mark.parametrize("rows,cols,rank,density", [
+    (257, 129, 34, 0.2), (100, 90, 2, 0.3), (64, 5000, 108, 0.01), (5000, 64, 100, 0.3), (3, 40, 64, 1.0),
+    (1, 1, 100, 1.0), (400, 300, 100, 0.0)])
+def test_outer_bulk_copy_schedule_shapes(fo, outer_schedule, rows, cols, rank, density):
+    """The schedule that lands factor rows with bulk copies: short rows, rows longer than a
+    stage, rows without cells, a single cell, ranks down to one 16-byte piece per row."""
+    w, Xh = outer_case(rows, cols, rank, density, seed=16)
+    Xd, Ud, Vd = csr_to_dev(w), to_dev(w["U"]), to_dev(w["V"])
+    outer_schedule("bulk")
+    for agg in ("full", "none") if len(w["vals"]) else ("full",):     # (no cells: nothing to write per cell)
+        ref = oracle.outer(WSLOSS, "t3", Xh, w["U"], w["V"], agg=agg, mode="masked")
+        got = fo.fused_outer(WSLOSS, "t3", Xd, Ud, Vd, agg=agg).cpu().numpy()
+        assert_close(got, ref, what="outer bulk %s rank %d" % (agg, rank))
+    assert fo.device_status() == 0
 
 
 @pytest.mark.parametrize("agg", ["full", "none", "right", "left"])

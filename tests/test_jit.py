@@ -228,7 +228,7 @@ def test_prepare_call_makes_the_kernel_of_a_call_ready():
 OUTER_GENERIC = [("sub", "t1", "a", "d"), ("abs", "t2", "t1"), ("add", "t3", "t2", 0.25)]
 
 
-@pytest.mark.parametrize("kernel", range(6))
+@pytest.mark.parametrize("kernel", range(8))
 def test_outer_kernels_compile_with_a_generated_chain_without_a_gpu(kernel):
     rc, log = fo.jit_compile_check_outer(OUTER_GENERIC, "t3", 0, 0, kernel)
     if rc == -4:
@@ -241,7 +241,7 @@ def test_outer_kernels_compile_with_a_generated_chain_without_a_gpu(kernel):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("schedule", ["pipe", "direct", "dense"])
+@pytest.mark.parametrize("schedule", ["bulk", "pipe", "direct", "dense"])
 def test_outer_chain_compiled_at_run_time_equals_interpreter_bitwise_and_checker(schedule):
     if not fo.jit_stats()[0]:
         pytest.skip("NVRTC or the driver library is not usable here")
@@ -251,7 +251,7 @@ def test_outer_chain_compiled_at_run_time_equals_interpreter_bitwise_and_checker
     Ud, Vd = to_dev(w["U"]), to_dev(w["V"])
     fo.tune("outer.kernel", schedule)
     try:
-        for agg in ("full", "none") + (() if schedule == "dense" else ("right",)) + (("left",) if schedule == "direct" else ()):
+        for agg in ("full", "none") + (() if schedule in ("dense", "bulk") else ("right",)) + (("left",) if schedule == "direct" else ()):
             launches = fo.jit_stats()[2]
             fast = fo.fused_outer(OUTER_GENERIC, "t3", X, Ud, Vd, agg=agg).cpu().numpy()
             assert fo.jit_stats()[2] == launches + 1, "%s %s was not specialised" % (schedule, agg)
