@@ -44,7 +44,7 @@ NCU_DRAM_BYTES_PER_UNIT = {
     "magg": (480.018e6 + 3.727e6) / 2e7,         # per cell (3 inputs; 200 000 x 100 capture)
     "row_dense": (1601.696e6 + 7.937e6) / 2e5,   # per row of 1000 columns (200 000 x 1000 capture)
     "row_csr": (264.047e6 + 3.881e6) / 19998162, # per stored cell (2 000 000 x 1000 @ 0.01 capture)
-    "outer": (1582.646e6 + 3.686e6) / 9996322,   # per stored cell (full-size capture, outer_pipe_kernel)
+    "outer": (1390.703e6 + 4.754e6) / 9996322,   # per stored cell (full-size capture, outer_bulk_kernel)
 }
 
 FULL = {

@@ -392,7 +392,8 @@ int fused_row_b1(const fo_chain *pre, const fo_chain *post, const fo_mat *X, con
  * out_nnz (device, one int64, or NULL): with FO_OUTER_NO_AGG the number of
  * written values that are not zero, as for fused_cell; with another variant
  * FO_ERR_UNSUPPORTED.
- * Schedules: per stored cell (factor rows of V staged in shared memory), or -
+ * Schedules: per stored cell (factor rows of V staged in shared memory, by bulk
+ * copies or 16-byte asynchronous copies depending on the rank), or -
  * when about one cell in seven or more is stored - tile by tile, forming each
  * 64 x 32 tile of U V^T on the fp64 tensor cores and sampling it at the stored
  * cells (full_agg / no_agg).  The library chooses; results agree within the
