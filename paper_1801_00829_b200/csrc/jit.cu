@@ -183,7 +183,7 @@ std::string wrapper_text(const DevChain &ch, const JitSpec &sp)
             snprintf(buf, sizeof(buf), "fo::outer_pipe_body<%d, %d, true>(ch, p);", sp.a, sp.b);
             break;
         case kJitOuterBulk:     // a = NK2, b = AGG
-            snprintf(buf, sizeof(buf), "fo::outer_bulk_body<%d, %d, true>(ch, p);", sp.a, sp.b);
+            snprintf(buf, sizeof(buf), "fo::outer_bulk_body<%d, %d, 0>(ch, p);", sp.a, sp.b);
             break;
         case kJitOuterDense:    // a = AGG
             snprintf(buf, sizeof(buf), "fo::outer_dense_body<%d>(ch, p, sp);", sp.a);

@@ -83,7 +83,7 @@ cudaError_t launch_outer_pipe(const DevChain &ch, const OuterParams &p, int agg,
 // full_agg / no_agg through the bulk-copy kernel; NK2 is exactly ceil(rank / 16) (at most 7 here).
 constexpr int kBulkMinRank = 96;    // below, a row is too short to be worth the ~54 cycles its copy holds the warp
 
-template <int NK2, int AGG, bool GENERIC>
+template <int NK2, int AGG, int KIND>
 cudaError_t launch_outer_bulk_one(const DevChain &ch, const OuterParams &p, int grid, size_t smem, cudaStream_t st)
 {
     static std::atomic<size_t> granted[64];
@@ -91,24 +91,32 @@ cudaError_t launch_outer_bulk_one(const DevChain &ch, const OuterParams &p, int 
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || granted[dev].load(std::memory_order_relaxed) < smem) {
-        e = cudaFuncSetAttribute(outer_bulk_kernel<NK2, AGG, GENERIC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(outer_bulk_kernel<NK2, AGG, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) granted[dev].store(smem, std::memory_order_relaxed);
     }
-    outer_bulk_kernel<NK2, AGG, GENERIC><<<grid, kBulkWarps * 32, smem, st>>>(ch, p);
+    outer_bulk_kernel<NK2, AGG, KIND><<<grid, kBulkWarps * 32, smem, st>>>(ch, p);
     return cudaGetLastError();
+}
+
+// three instances: the interpreter and the logarithm chain (evaluated once per four stages), and the
+// cheap inline forms (evaluated per stage)
+template <int NK2, int AGG>
+cudaError_t launch_outer_bulk_agg(const DevChain &ch, const OuterParams &p, int grid, size_t smem, cudaStream_t st)
+{
+    switch (p.chain_kind) {
+        case kOuterGeneric: return launch_outer_bulk_one<NK2, AGG, kOuterGeneric>(ch, p, grid, smem, st);
+        case kOuterXlogd: return launch_outer_bulk_one<NK2, AGG, kOuterXlogd>(ch, p, grid, smem, st);
+        default: return launch_outer_bulk_one<NK2, AGG, kOuterWsloss>(ch, p, grid, smem, st);   // the cheap inline forms
+    }
 }
 
 template <int NK2>
 cudaError_t launch_outer_bulk(const DevChain &ch, const OuterParams &p, int agg, int grid, size_t smem, cudaStream_t st)
 {
-    const bool gen = p.chain_kind == kOuterGeneric;
-    if (agg == FO_OUTER_FULL_AGG)
-        return gen ? launch_outer_bulk_one<NK2, kOutFull, true>(ch, p, grid, smem, st)
-                   : launch_outer_bulk_one<NK2, kOutFull, false>(ch, p, grid, smem, st);
-    return gen ? launch_outer_bulk_one<NK2, kOutNone, true>(ch, p, grid, smem, st)
-               : launch_outer_bulk_one<NK2, kOutNone, false>(ch, p, grid, smem, st);
+    if (agg == FO_OUTER_FULL_AGG) return launch_outer_bulk_agg<NK2, kOutFull>(ch, p, grid, smem, st);
+    return launch_outer_bulk_agg<NK2, kOutNone>(ch, p, grid, smem, st);
 }
 
 // Work split of the tiled schedule: column ranges so that there are enough work items for a

@@ -63,6 +63,11 @@ __device__ __forceinline__ double outer_chain_split(const DevChain &ch, int kind
 {
     return outer_chain(ch, kind, kc, a, d);
 }
+template <int KIND>
+__device__ __forceinline__ double outer_chain_fixed(const DevChain &ch, int kc, double a, double d)
+{
+    return outer_chain(ch, KIND, kc, a, d);
+}
 __device__ __forceinline__ double outer_chain_sides(const DevChain &ch, double a, double d,
                                                     const double (&sv)[kOuterMaxSides])
 {
@@ -123,6 +128,22 @@ __device__ __forceinline__ double outer_chain_split(const DevChain &ch, int kind
     }
     if (kind == kOuterXlogd) return a * slow_log(d + ch.consts[kc]);
     if (kind == kOuterMaskDot) return (a != 0.0 ? 1.0 : 0.0) * d;
+    const double t0 = a != 0.0 ? 1.0 : 0.0;       // kOuterWsloss
+    const double t1 = a - d;
+    const double t2 = t1 * t1;
+    return t0 * t2;
+}
+
+// The form of the chain fixed at compile time: the instance carries exactly one of them.
+template <int KIND>
+__device__ __forceinline__ double outer_chain_fixed(const DevChain &ch, int kc, double a, double d)
+{
+    if (KIND == kOuterGeneric) {
+        const double none[kOuterMaxSides] = {0.0, 0.0, 0.0};
+        return outer_chain_sides(ch, a, d, none);
+    }
+    if (KIND == kOuterXlogd) return a * slow_log(d + ch.consts[kc]);
+    if (KIND == kOuterMaskDot) return (a != 0.0 ? 1.0 : 0.0) * d;
     const double t0 = a != 0.0 ? 1.0 : 0.0;       // kOuterWsloss
     const double t1 = a - d;
     const double t2 = t1 * t1;
@@ -537,7 +558,7 @@ __host__ __device__ inline size_t bulk_warp_bytes(int rank)
     return (size_t)kBulkDepth * kBulkCells * rank * 8 + kBulkRing * 12 + kBulkDepth * 16;
 }
 
-template <int NK2, int AGG, bool GENERIC>
+template <int NK2, int AGG, int KIND>
 __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterParams &p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -638,16 +659,36 @@ __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterP
     for (int c = 0; c < NK2; ++c) u[c] = make_double2(0.0, 0.0);
     double acc = 0.0;
     bool timed_out = false;
-    const int t = grp + 4 * ((lane >> 2) & 1);        // the stage's cell whose total this lane ends up with
-    const bool holder = (lane & 3) == 0;
+    // A chain that costs more than a few instructions (the interpreter, a logarithm) runs once per
+    // four stages, a cell per lane: stage number sb of a batch leaves its cells' values and dot
+    // products with lanes 8 sb .. 8 sb + 7.  The cheap inline forms run per stage on the lanes that
+    // hold the totals (measured 2 % faster for them, 15 % slower for the logarithm).
+    constexpr bool BATCH = (KIND == kOuterGeneric || KIND == kOuterXlogd);
+    double pa = 0.0, pd = 0.0;
+    int ppos = -1;                                    // this lane's pending cell (position behind P0), or none
+    int sb = 0;
+    auto flush = [&]() {
+        const double w = outer_chain_fixed<KIND>(ch, p.kconst, pa, pd);
+        if (AGG == kOutFull) {
+            if (ppos >= 0) acc += w;
+        } else {
+            if (ppos >= 0) p.out[P0 + ppos] = w;
+        }
+        ppos = -1;
+        sb = 0;
+    };
 
+    const int tcell = grp + 4 * ((lane >> 2) & 1);    // the stage's cell whose total this lane ends up with
+    const bool holder = (lane & 3) == 0;
     int cslot = 0, inflight = issued;
     unsigned cphase = 0;
     while (inflight > 0) {
         const int4 m = meta[cslot];
         const int q = m.x, cnt = m.y & 0xff;
         const bool first = (m.y & 0x100) != 0;
-        const double a = aring[(q + t) & (kBulkRing - 1)];
+        // the value of the cell this lane will run the chain for: cell l8 of the stage if the chain is
+        // batched, else the cell whose total the lane ends up with
+        const double a = aring[(q + (BATCH ? l8 : tcell)) & (kBulkRing - 1)];
         if (!__all_sync(full, mbar_wait(&bar[cslot], cphase))) {      // the whole warp leaves together
             timed_out = true;
             break;
@@ -674,15 +715,28 @@ __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterP
             }
         }
         const double d0 = dx[0] + dy[0], d1 = dx[1] + dy[1];
+        // two values over the 8 lanes of a group: the lower four lanes end up with the total of
+        // cell grp, the upper four with that of cell grp + 4
         const bool up = (lane & 4) != 0;
         double v = (up ? d1 : d0) + __shfl_xor_sync(full, up ? d0 : d1, 4);
         v += __shfl_xor_sync(full, v, 2);
         v += __shfl_xor_sync(full, v, 1);
-        const double w = outer_chain_split<GENERIC>(ch, p.chain_kind, p.kconst, a, v);
-        if (AGG == kOutFull) {
-            if (holder && t < cnt) acc += w;
+        if (BATCH) {
+            // cell c of the stage goes to lane 8 sb + c: its total sits in group c & 3, half c >> 2
+            const double vv = __shfl_sync(full, v, 8 * (lane & 3) + 4 * ((lane >> 2) & 1));
+            if ((lane >> 3) == sb) {
+                pd = vv;
+                pa = a;
+                ppos = l8 < cnt ? q + l8 : -1;
+            }
+            if (++sb == 4) flush();
         } else {
-            if (holder && t < cnt) p.out[P0 + q + t] = w;
+            const double w = outer_chain_split<false>(ch, p.chain_kind, p.kconst, a, v);    // an inline form
+            if (AGG == kOutFull) {
+                if (holder && tcell < cnt) acc += w;
+            } else {
+                if (holder && tcell < cnt) p.out[P0 + q + tcell] = w;
+            }
         }
         __syncwarp();                  // everyone is done with the slot: refill it
         --inflight;
@@ -695,6 +749,7 @@ __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterP
             cphase ^= 1u;
         }
     }
+    if (!timed_out && sb > 0) flush();
     if (timed_out) {
         // give the copies still in flight a (bounded) chance to land before the CTA's
         // shared memory is given up
@@ -717,11 +772,11 @@ __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterP
     }
 }
 
-template <int NK2, int AGG, bool GENERIC>
+template <int NK2, int AGG, int KIND>
 __global__ void __launch_bounds__(kBulkWarps * 32, 1)
 outer_bulk_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p)
 {
-    outer_bulk_body<NK2, AGG, GENERIC>(ch, p);
+    outer_bulk_body<NK2, AGG, KIND>(ch, p);
 }
 
 // -------------------------------------------------------------------- dense
