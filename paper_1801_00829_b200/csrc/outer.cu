@@ -81,10 +81,10 @@ cudaError_t launch_outer_pipe(const DevChain &ch, const OuterParams &p, int agg,
 }
 
 // full_agg / no_agg through the bulk-copy kernel; NK2 is exactly ceil(rank / 16) (at most 7 here).
-constexpr int kBulkMinRank = 96;    // below, a row is too short to be worth the ~54 cycles its copy holds the warp
 
 template <int NK2, int AGG, int KIND>
-cudaError_t launch_outer_bulk_one(const DevChain &ch, const OuterParams &p, int grid, size_t smem, cudaStream_t st)
+cudaError_t launch_outer_bulk_one(const DevChain &ch, const OuterParams &p, int grid, int warps, size_t smem,
+                                  cudaStream_t st)
 {
     static std::atomic<size_t> granted[64];
     int dev = 0;
@@ -96,27 +96,29 @@ cudaError_t launch_outer_bulk_one(const DevChain &ch, const OuterParams &p, int 
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) granted[dev].store(smem, std::memory_order_relaxed);
     }
-    outer_bulk_kernel<NK2, AGG, KIND><<<grid, kBulkWarps * 32, smem, st>>>(ch, p);
+    outer_bulk_kernel<NK2, AGG, KIND><<<grid, warps * 32, smem, st>>>(ch, p);
     return cudaGetLastError();
 }
 
 // three instances: the interpreter and the logarithm chain (evaluated once per four stages), and the
 // cheap inline forms (evaluated per stage)
 template <int NK2, int AGG>
-cudaError_t launch_outer_bulk_agg(const DevChain &ch, const OuterParams &p, int grid, size_t smem, cudaStream_t st)
+cudaError_t launch_outer_bulk_agg(const DevChain &ch, const OuterParams &p, int grid, int warps, size_t smem,
+                                  cudaStream_t st)
 {
     switch (p.chain_kind) {
-        case kOuterGeneric: return launch_outer_bulk_one<NK2, AGG, kOuterGeneric>(ch, p, grid, smem, st);
-        case kOuterXlogd: return launch_outer_bulk_one<NK2, AGG, kOuterXlogd>(ch, p, grid, smem, st);
-        default: return launch_outer_bulk_one<NK2, AGG, kOuterWsloss>(ch, p, grid, smem, st);   // the cheap inline forms
+        case kOuterGeneric: return launch_outer_bulk_one<NK2, AGG, kOuterGeneric>(ch, p, grid, warps, smem, st);
+        case kOuterXlogd: return launch_outer_bulk_one<NK2, AGG, kOuterXlogd>(ch, p, grid, warps, smem, st);
+        default: return launch_outer_bulk_one<NK2, AGG, kOuterWsloss>(ch, p, grid, warps, smem, st);   // the cheap inline forms
     }
 }
 
 template <int NK2>
-cudaError_t launch_outer_bulk(const DevChain &ch, const OuterParams &p, int agg, int grid, size_t smem, cudaStream_t st)
+cudaError_t launch_outer_bulk(const DevChain &ch, const OuterParams &p, int agg, int grid, int warps, size_t smem,
+                              cudaStream_t st)
 {
-    if (agg == FO_OUTER_FULL_AGG) return launch_outer_bulk_agg<NK2, kOutFull>(ch, p, grid, smem, st);
-    return launch_outer_bulk_agg<NK2, kOutNone>(ch, p, grid, smem, st);
+    if (agg == FO_OUTER_FULL_AGG) return launch_outer_bulk_agg<NK2, kOutFull>(ch, p, grid, warps, smem, st);
+    return launch_outer_bulk_agg<NK2, kOutNone>(ch, p, grid, warps, smem, st);
 }
 
 // Work split of the tiled schedule: column ranges so that there are enough work items for a
@@ -321,32 +323,38 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
                                      : launch_outer_dense_one<kOutNone>(ch, p, sms, st);
         return e == cudaSuccess ? FO_OK : cuda_fail(e);
     }
-    // full_agg / no_agg: factor rows landed by bulk copies where 16 warps with two slots of eight
-    // rows each fit in an SM's shared memory and a row is long enough to be worth a copy of its own
+    // full_agg / no_agg: factor rows landed by bulk copies where that measured faster than 16-byte copies -
+    // long rows whose 16-byte pieces straddle 128-byte lines (rank 97 .. 112 with a leading dimension that is
+    // not a multiple of 16 doubles: 0.58 against 0.66 ms at rank 100), and rows so long that only one CTA of
+    // the 16-byte-copy kernel fits on an SM (rank above 112: 0.67 against 0.90 ms at rank 120).  Below rank 97
+    // a row is too short to be worth the ~54 cycles its copy holds the warp (rank 80: 0.58 against 0.43 ms).
     const bool want_bulk = strcmp(which, "bulk") == 0, want_pipe = strcmp(which, "pipe") == 0;
-    const bool bulk_fits = (size_t)kBulkWarps * bulk_warp_bytes(rank) <= 225u * 1024u;
-    if (copyable && !want_direct && !want_pipe && agg != FO_OUTER_RIGHT_MM && bulk_fits &&
-        (want_bulk || rank >= kBulkMinRank)) {
-        const size_t smem = (size_t)kBulkWarps * bulk_warp_bytes(rank);
+    int bulk_warps = (int)((225u * 1024u) / bulk_warp_bytes(rank));
+    if (bulk_warps > kBulkWarps) bulk_warps = kBulkWarps;
+    const bool bulk_pays = bulk_warps >= 12 && (rank > 112 || (rank > 96 && V->ld % 16 != 0));
+    if (copyable && !want_direct && !want_pipe && agg != FO_OUTER_RIGHT_MM && bulk_warps >= 8 &&
+        (want_bulk || bulk_pays)) {
+        const size_t smem = (size_t)bulk_warps * bulk_warp_bytes(rank);
         long long g = sms;
-        const long long by_cells = (X->nnz + 8ll * kBulkWarps - 1) / (8ll * kBulkWarps);    // a stage per warp at least
+        const long long by_cells = (X->nnz + 8ll * bulk_warps - 1) / (8ll * bulk_warps);    // a stage per warp at least
         if (g > by_cells) g = by_cells;
         if (g < 1) g = 1;
         if (try_jit) {
             const JitSpec js = {kJitOuterBulk, nk2, kagg, 0};
             const int jrc = jit_launch(js, ch, &p, (unsigned)g, 1, st, jit_first_use(), true, smem, nullptr,
-                                       kBulkWarps * 32);
+                                       bulk_warps * 32);
             if (jrc == FO_OK) return FO_OK;
             if (jrc != kJitUnavailable) return jrc;
         }
         switch (nk2) {
-            case 1: e = launch_outer_bulk<1>(ch, p, agg, (int)g, smem, st); break;
-            case 2: e = launch_outer_bulk<2>(ch, p, agg, (int)g, smem, st); break;
-            case 3: e = launch_outer_bulk<3>(ch, p, agg, (int)g, smem, st); break;
-            case 4: e = launch_outer_bulk<4>(ch, p, agg, (int)g, smem, st); break;
-            case 5: e = launch_outer_bulk<5>(ch, p, agg, (int)g, smem, st); break;
-            case 6: e = launch_outer_bulk<6>(ch, p, agg, (int)g, smem, st); break;
-            default: e = launch_outer_bulk<7>(ch, p, agg, (int)g, smem, st); break;
+            case 1: e = launch_outer_bulk<1>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
+            case 2: e = launch_outer_bulk<2>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
+            case 3: e = launch_outer_bulk<3>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
+            case 4: e = launch_outer_bulk<4>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
+            case 5: e = launch_outer_bulk<5>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
+            case 6: e = launch_outer_bulk<6>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
+            case 7: e = launch_outer_bulk<7>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
+            default: e = launch_outer_bulk<8>(ch, p, agg, (int)g, bulk_warps, smem, st); break;
         }
         return e == cudaSuccess ? FO_OK : cuda_fail(e);
     }

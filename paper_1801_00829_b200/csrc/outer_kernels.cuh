@@ -544,10 +544,10 @@ __device__ __forceinline__ void outer_pipe_body(const DevChain &ch, const OuterP
 // indices and values run ahead of the copies through a small ring in shared memory,
 // filled 32 cells at a time; U_i is read at a row's first stage, having been requested
 // from L2 when that stage's copies were started.
-// Starting a bulk copy holds the issuing warp for about 54 cycles per row, so this
-// schedule needs many warps: it is used where 16 of them fit (two slots of eight rows
-// each: factor rows of up to 108 doubles), and there it beats the 16-byte asynchronous
-// copies of outer_pipe_kernel (0.636 against 0.659 ms at rank 100).
+// Starting a bulk copy holds the issuing warp for about 54 cycles per row, whatever the
+// row's length, so this schedule needs many warps (16 fit with rows of up to 108
+// doubles, 13 at 128) and long rows; where it is chosen over the 16-byte asynchronous
+// copies of outer_pipe_kernel is decided, from measurements, by the host code.
 constexpr int kBulkWarps = 16;       // warps per CTA, one CTA per SM
 constexpr int kBulkDepth = 2;        // slots per ring
 constexpr int kBulkRing = 64;        // cells of (colidx, vals) kept per warp

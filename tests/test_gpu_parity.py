@@ -520,7 +520,7 @@ def test_outer_every_schedule_on_a_sparse_input(fo, outer_schedule, schedule):
 
 @pytest.mark.parametrize("rows,cols,rank,density", [
     (257, 129, 34, 0.2), (100, 90, 2, 0.3), (64, 5000, 108, 0.01), (5000, 64, 100, 0.3), (3, 40, 64, 1.0),
-    (1, 1, 100, 1.0), (400, 300, 100, 0.0)])
+    (1, 1, 100, 1.0), (400, 300, 100, 0.0), (300, 200, 128, 0.2), (150, 100, 120, 0.3)])
 def test_outer_bulk_copy_schedule_shapes(fo, outer_schedule, rows, cols, rank, density):
     """The schedule that lands factor rows with bulk copies: short rows, rows longer than a
     stage, rows without cells, a single cell, ranks down to one 16-byte piece per row."""
