@@ -689,7 +689,7 @@ __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterP
         // the value of the cell this lane will run the chain for: cell l8 of the stage if the chain is
         // batched, else the cell whose total the lane ends up with
         const double a = aring[(q + (BATCH ? l8 : tcell)) & (kBulkRing - 1)];
-        if (!__all_sync(full, mbar_wait(&bar[cslot], cphase))) {      // the whole warp leaves together
+        if (!__all_sync(full, mbar_wait_hint(&bar[cslot], cphase, 2000u))) {      // the whole warp leaves together
             timed_out = true;
             break;
         }

@@ -38,6 +38,28 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, unsigned 
         : "memory");
     return ok != 0;
 }
+// The same with a hint of how long (ns) the hardware may keep the thread suspended before the
+// instruction returns false: fewer polls while a copy is on its way.
+__device__ __forceinline__ bool mbar_try_wait_hint(unsigned long long *bar, unsigned parity, unsigned ns)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_hint(unsigned long long *bar, unsigned parity, unsigned ns,
+                                               unsigned limit = kWaitLimit)
+{
+    for (unsigned i = 0; i < limit; ++i)
+        if (mbar_try_wait_hint(bar, parity, ns)) return true;
+    return false;
+}
+
 // Bounded wait: returns false (and the caller records it) if the phase has not completed
 // after `limit` polls.
 __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, unsigned limit = kWaitLimit)
