@@ -640,8 +640,9 @@ __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterP
         __syncwarp();
         double *sl = slots + (size_t)slot * slot_doubles;
         if (lane < cnt) bulk_g2s(sl + lane * rank, p.V + (long long)j * p.ldv, rowbytes, &bar[slot]);
-        else if (ifirst && lane >= 16 && 128 * (lane - 16) < rank * 8)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.U + irow * p.ldu) + 128 * (lane - 16)));
+        else if (ifirst && lane >= 16 && 128 * (lane - 16) < rank * 8 && irow + 1 < row_hi)
+            // U streams from HBM once: ask the L2 for the NEXT row's U_i now, a row of stages ahead of its use
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.U + (irow + 1) * p.ldu) + 128 * (lane - 16)));
         ipos += cnt;
         ifirst = false;
         if (ipos == iend) {
@@ -651,6 +652,8 @@ __device__ __forceinline__ void outer_bulk_body(const DevChain &ch, const OuterP
         }
     };
 
+    if (irow < row_hi && 128 * lane < rank * 8)       // the first row's U_i
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.U + irow * p.ldu) + 128 * lane));
     int issued = 0;
     while (issued < D && irow < row_hi) issue(issued++);
 
