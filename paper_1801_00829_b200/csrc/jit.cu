@@ -268,8 +268,8 @@ std::string generate_source(const DevChain &ch, const JitSpec &sp)
         snprintf(buf, sizeof(buf),
                  "extern \"C\" __global__ void __launch_bounds__(%d, %d)\n"
                  "fo_jit_kernel(const __grid_constant__ fo::DevChain ch, const __grid_constant__ fo::OuterParams p%s)\n"
-                 "{\n    ", sp.kind == kJitOuterBulk ? kBulkWarps * 32 : kThreads,
-                 (sp.kind == kJitOuterBulk || (sp.kind == kJitOuterDirect && sp.a > 8)) ? 1 : 2,
+                 "{\n    ", sp.kind == kJitOuterBulk ? kBulkWarps * 32 : sp.kind == kJitOuterDense ? kDenseThreadsAll : kThreads,
+                 (sp.kind == kJitOuterBulk || sp.kind == kJitOuterDense || (sp.kind == kJitOuterDirect && sp.a > 8)) ? 1 : 2,
                  sp.kind == kJitOuterDense ? ", const __grid_constant__ fo::DenseSplit sp" : "");
         s += buf;
         s += wrapper_text(ch, sp) + "\n}\n";

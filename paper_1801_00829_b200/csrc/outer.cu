@@ -138,7 +138,7 @@ bool dense_plan(const OuterParams &p, int sms, DenseSplit *sp, long long *grid)
     sp->tiles_per_split = (int)per;
     sp->pad = 0;
     *grid = rb * splits;
-    if (*grid > 2ll * sms) *grid = 2ll * sms;
+    if (*grid > sms) *grid = sms;
     return true;
 }
 
@@ -159,7 +159,7 @@ cudaError_t launch_outer_dense_one(const DevChain &ch, const OuterParams &p, int
     DenseSplit sp;
     long long grid = 0;
     if (!dense_plan(p, sms, &sp, &grid)) return cudaErrorInvalidValue;
-    outer_dense_kernel<AGG><<<(unsigned)grid, kThreads, smem, st>>>(ch, p, sp);
+    outer_dense_kernel<AGG><<<(unsigned)grid, kDenseThreadsAll, smem, st>>>(ch, p, sp);
     return cudaGetLastError();
 }
 
@@ -301,7 +301,7 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
     // once about one cell in seven is stored (measured crossover on this part)
     const bool want_dense = strcmp(which, "dense") == 0;
     const bool dense_ok = copyable && agg != FO_OUTER_RIGHT_MM && rank >= 8 &&
-                          dense_smem_bytes(rank) <= 200u * 1024u;
+                          dense_smem_bytes(rank) <= 220u * 1024u;
     const double stored_share = (double)X->nnz / ((double)X->rows * (double)X->cols);
     // a chain without an inline form: the same kernels compiled for it at run time, else interpreted
     const bool try_jit = p.chain_kind == kOuterGeneric && !force_interpreter();
@@ -314,7 +314,7 @@ int fused_outer(const fo_chain *chain, const fo_csr *X, const fo_dense *U, const
             if (dense_plan(p, sms, &sp, &g)) {
                 const JitSpec js = {kJitOuterDense, kagg, 0, 0};
                 const int jrc = jit_launch(js, ch, &p, (unsigned)g, 1, st, jit_first_use(), true,
-                                           dense_smem_bytes(rank), &sp);
+                                           dense_smem_bytes(rank), &sp, kDenseThreadsAll);
                 if (jrc == FO_OK) return FO_OK;
                 if (jrc != kJitUnavailable) return jrc;
             }

@@ -788,15 +788,22 @@ outer_bulk_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
 // Gathering a factor row per stored cell then costs more than forming U V^T
 // outright, so this schedule forms it, tile by tile, and never writes it out:
 // a CTA takes a block of 64 rows (U rows in shared memory) and sweeps 32-column
-// tiles of V; the 64 x 32 tile of dot products comes from the fp64 tensor-core
-// instruction (mma.sync m8n8k4, 8 warps of 16 x 16), goes to shared memory, and
-// the stored cells of the tile - a contiguous piece of each row of the CSR
-// matrix, found with a per-row cursor - pick their dot product there and run the
-// chain.  The next V tile is copied in while the cells are evaluated, and two
-// CTAs share an SM, so one's cell phase (waiting on the X stream) runs under the
-// other's tensor-core phase.  Work items are (row block, column range) pairs
-// dealt round-robin to the resident CTAs.
+// tiles of V.  Its warps have two jobs.  Eight of them form the 64 x 32 tile of
+// dot products with the fp64 tensor-core instruction (mma.sync m8n8k4, a 16 x 16
+// piece per warp) and leave it in one of two tile buffers in shared memory; eight
+// others take the previous tile from the other buffer and evaluate its stored
+// cells - a contiguous piece of each row of the CSR matrix, found with a per-row
+// cursor: they pick their dot product from the buffer and run the chain.  So the
+// cell work, which mostly waits for X to stream in from HBM, runs under the
+// tensor-core work instead of between it.  The groups hand the buffers over with
+// named barriers (full / empty per buffer: arrive on one side, sync on the
+// other; both sides execute the same tile loop, so the counts always meet).  The
+// V tiles are double-buffered too: the copy of the next one runs under the
+// products of this one.  Work items are (row block, column range) pairs dealt
+// round-robin to one CTA per SM.
 constexpr int kDenseBM = 64, kDenseBN = 32;
+constexpr int kDenseMmaWarps = 8, kDenseCellWarps = 8;
+constexpr int kDenseThreadsAll = (kDenseMmaWarps + kDenseCellWarps) * 32;
 
 __host__ __device__ inline int dense_ld(int rank)
 {
@@ -806,14 +813,23 @@ __host__ __device__ inline int dense_ld(int rank)
 }
 __host__ __device__ inline size_t dense_smem_bytes(int rank)
 {
-    return (size_t)((kDenseBM + kDenseBN) * dense_ld(rank) + kDenseBM * (kDenseBN + 2)) * sizeof(double) +
-           2 * kDenseBM * sizeof(int);
+    return (size_t)((kDenseBM + 2 * kDenseBN) * dense_ld(rank) + 2 * kDenseBM * (kDenseBN + 2)) * sizeof(double);
 }
 
 __device__ __forceinline__ void dmma_8x8x4(double &c0, double &c1, double a, double b)
 {
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
                  : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
+
+// Named barriers of the tiled kernel (0 is __syncthreads).
+__device__ __forceinline__ void named_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void named_arrive(int id, int threads)
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 struct DenseSplit {
@@ -829,124 +845,157 @@ __device__ __forceinline__ void outer_dense_body(const DevChain &ch, const Outer
 
     const int rank = p.rank, ld = dense_ld(rank);
     constexpr int PLD = kDenseBN + 2;
+    constexpr int kMma = kDenseMmaWarps * 32;                     // threads that form the tiles
+    constexpr int kBarMma = 1, kBarFull = 2, kBarEmpty = 4;       // named barriers: + buffer number
     double *Us = reinterpret_cast<double *>(smem_raw);            // 64 x ld
-    double *Vs = Us + kDenseBM * ld;                              // 32 x ld
-    double *Ps = Vs + kDenseBN * ld;                              // 64 x 34
-    int *cur = reinterpret_cast<int *>(Ps + kDenseBM * PLD);
-    int *rend = cur + kDenseBM;
+    double *Vs = Us + kDenseBM * ld;                              // 2 x 32 x ld
+    double *Ps = Vs + 2 * kDenseBN * ld;                          // 2 x 64 x 34
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int g = lane >> 2, t = lane & 3;                        // fragment coordinates
-    const int wm = warp >> 1, wn = warp & 1;                      // warp tile: rows 16 wm .., columns 16 wn ..
+    const bool mma_warp = warp < kDenseMmaWarps;
     const unsigned full = 0xffffffffu;
     const int pieces = rank >> 1;                                 // 16-byte pieces of a factor row
 
-    // columns rank .. ld - 1 of both operand buffers stay zero for good
-    for (int i = threadIdx.x; i < (kDenseBM + kDenseBN) * (ld - rank); i += kThreads) {
+    // columns rank .. ld - 1 of the operand buffers stay zero for good
+    for (int i = threadIdx.x; i < (kDenseBM + 2 * kDenseBN) * (ld - rank); i += kDenseThreadsAll) {
         const int r = i / (ld - rank), c = rank + i % (ld - rank);
-        Us[(size_t)r * ld + c] = 0.0;            // r runs over the rows of Us and then of Vs
+        Us[(size_t)r * ld + c] = 0.0;            // r runs over the rows of Us and then of both Vs
     }
-
-    auto copy_rows = [&](double *dst, int nrows, const double *src, long long ldsrc, long long first,
-                         long long limit) {
-        // rows first .. first + nrows - 1 of a factor (those below `limit`) into dst
-        for (int i = threadIdx.x; i < nrows * pieces; i += kThreads) {
-            const int r = i / pieces, c = i % pieces;
-            if (first + r < limit) cp_async16(dst + (size_t)r * ld + 2 * c, src + (first + r) * ldsrc + 2 * c);
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    };
+    __syncthreads();
 
     double acc = 0.0;
     const long long items = (long long)sp.row_blocks * sp.col_splits;
     const long long ntiles = (p.cols + kDenseBN - 1) / kDenseBN;
-    for (long long item = blockIdx.x; item < items; item += gridDim.x) {
-        const long long row0 = (item / sp.col_splits) * kDenseBM;
-        const long long tile_lo = (item % sp.col_splits) * sp.tiles_per_split;
-        const long long tile_hi = tile_lo + sp.tiles_per_split < ntiles ? tile_lo + sp.tiles_per_split : ntiles;
-        __syncthreads();                                          // the buffers' last readers are done
-        copy_rows(Us, kDenseBM, p.U, p.ldu, row0, p.rows);
-        copy_rows(Vs, kDenseBN, p.V, p.ldv, tile_lo * kDenseBN, p.cols);
-        // per-row cursors: the first stored cell at or right of the column range's start
-        if (threadIdx.x < kDenseBM) {
-            const long long row = row0 + threadIdx.x;
-            int lo = 0, e = 0;
-            if (row < p.rows) {
-                lo = __ldg(p.rowptr + row);
-                e = __ldg(p.rowptr + row + 1);
-                const int want = (int)(tile_lo * kDenseBN);
-                int hi = e;
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    if (__ldg(p.colidx + mid) < want) lo = mid + 1; else hi = mid;
-                }
+    long long n = 0;                             // tiles this CTA has been through: buffer n & 1
+
+    if (mma_warp) {
+        const int g = lane >> 2, t = lane & 3;                    // fragment coordinates
+        const int wm = warp >> 1, wn = warp & 1;                  // warp tile: rows 16 wm .., columns 16 wn ..
+        auto copy_rows = [&](double *dst, int nrows, const double *src, long long ldsrc, long long first,
+                             long long limit) {
+            // rows first .. first + nrows - 1 of a factor (those below `limit`) into dst
+            for (int i = threadIdx.x; i < nrows * pieces; i += kMma) {
+                const int r = i / pieces, c = i % pieces;
+                if (first + r < limit) cp_async16(dst + (size_t)r * ld + 2 * c, src + (first + r) * ldsrc + 2 * c);
             }
-            cur[threadIdx.x] = lo;
-            rend[threadIdx.x] = e;
-        }
-        for (long long tile = tile_lo; tile < tile_hi; ++tile) {
-            const int n0 = (int)(tile * kDenseBN);
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            __syncthreads();                                      // U block and this V tile have landed
-            // ---- P = U_blk V_tile^T: warp tile 16 x 16 = 2 x 2 instruction tiles
-            double c[2][2][2];
-#pragma unroll
-            for (int i = 0; i < 2; ++i)
-#pragma unroll
-                for (int j = 0; j < 2; ++j) c[i][j][0] = c[i][j][1] = 0.0;
-            const double *ua = Us + (size_t)(16 * wm + g) * ld + t;
-            const double *vb = Vs + (size_t)(16 * wn + g) * ld + t;
-#pragma unroll 4
-            for (int k = 0; k < ld; k += 4) {
-                double a[2], b[2];
-#pragma unroll
-                for (int i = 0; i < 2; ++i) a[i] = ua[(size_t)(8 * i) * ld + k];
-#pragma unroll
-                for (int j = 0; j < 2; ++j) b[j] = vb[(size_t)(8 * j) * ld + k];
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+            const long long row0 = (item / sp.col_splits) * kDenseBM;
+            const long long tile_lo = (item % sp.col_splits) * sp.tiles_per_split;
+            const long long tile_hi = tile_lo + sp.tiles_per_split < ntiles ? tile_lo + sp.tiles_per_split : ntiles;
+            named_sync(kBarMma, kMma);                            // the last products on the old U block are done
+            copy_rows(Us, kDenseBM, p.U, p.ldu, row0, p.rows);
+            copy_rows(Vs + (size_t)(n & 1) * kDenseBN * ld, kDenseBN, p.V, p.ldv, tile_lo * kDenseBN, p.cols);
+            for (long long tile = tile_lo; tile < tile_hi; ++tile, ++n) {
+                const int b = (int)(n & 1);
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                named_sync(kBarMma, kMma);                        // this V tile (and U) landed; the other V buffer is free
+                if (tile + 1 < tile_hi)
+                    copy_rows(Vs + (size_t)(b ^ 1) * kDenseBN * ld, kDenseBN, p.V, p.ldv, (tile + 1) * kDenseBN, p.cols);
+                // ---- P = U_blk V_tile^T: warp tile 16 x 16 = 2 x 2 instruction tiles
+                double c[2][2][2];
 #pragma unroll
                 for (int i = 0; i < 2; ++i)
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) dmma_8x8x4(c[i][j][0], c[i][j][1], a[i], b[j]);
-            }
+                    for (int j = 0; j < 2; ++j) c[i][j][0] = c[i][j][1] = 0.0;
+                const double *ua = Us + (size_t)(16 * wm + g) * ld + t;
+                const double *vb = Vs + (size_t)b * kDenseBN * ld + (size_t)(16 * wn + g) * ld + t;
+#pragma unroll 4
+                for (int k = 0; k < ld; k += 4) {
+                    double a[2], bb[2];
 #pragma unroll
-            for (int i = 0; i < 2; ++i)
+                    for (int i = 0; i < 2; ++i) a[i] = ua[(size_t)(8 * i) * ld + k];
 #pragma unroll
-                for (int j = 0; j < 2; ++j)
-                    *reinterpret_cast<double2 *>(Ps + (size_t)(16 * wm + 8 * i + g) * PLD + 16 * wn + 8 * j + 2 * t) =
-                        make_double2(c[i][j][0], c[i][j][1]);
-            __syncthreads();                                      // P is complete; Vs is free
-            if (tile + 1 < tile_hi) copy_rows(Vs, kDenseBN, p.V, p.ldv, (tile + 1) * kDenseBN, p.cols);
-            // ---- the stored cells of this tile: warp w takes rows 8 w .. 8 w + 7 of the block, a lane
-            // the cell at its offset from the row's cursor; all loads first, then the chains
-            const int nhi = n0 + kDenseBN;
-            int jj[8];
-            double aa[8];
+                    for (int j = 0; j < 2; ++j) bb[j] = vb[(size_t)(8 * j) * ld + k];
 #pragma unroll
-            for (int rr = 0; rr < 8; ++rr) {
-                const int pp = cur[8 * warp + rr] + lane;
-                jj[rr] = 0x7fffffff;
-                aa[rr] = 0.0;
-                if (pp < rend[8 * warp + rr]) {
-                    jj[rr] = __ldg(p.colidx + pp);
-                    aa[rr] = __ldg(p.vals + pp);
+                    for (int i = 0; i < 2; ++i)
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) dmma_8x8x4(c[i][j][0], c[i][j][1], a[i], bb[j]);
                 }
-            }
+                if (n >= 2) named_sync(kBarEmpty + b, kDenseThreadsAll);   // the cells of tile n - 2 are done with this buffer
+                double *pb = Ps + (size_t)b * kDenseBM * PLD;
 #pragma unroll
-            for (int rr = 0; rr < 8; ++rr) {
-                const int r = 8 * warp + rr;
-                const bool in = jj[rr] < nhi;
-                if (in) {
-                    const double w = outer_chain<true>(ch, p.chain_kind, p.kconst, aa[rr], Ps[(size_t)r * PLD + (jj[rr] - n0)]);
-                    if (AGG == kOutFull) acc += w;
-                    else p.out[cur[r] + lane] = w;
-                }
-                const int taken = __popc(__ballot_sync(full, in));
-                __syncwarp();
-                if (lane == 0) cur[r] += taken;
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+                        *reinterpret_cast<double2 *>(pb + (size_t)(16 * wm + 8 * i + g) * PLD + 16 * wn + 8 * j + 2 * t) =
+                            make_double2(c[i][j][0], c[i][j][1]);
+                __threadfence_block();
+                named_arrive(kBarFull + b, kDenseThreadsAll);     // the tile is there
             }
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else {
+        const int cw = warp - kDenseMmaWarps;                     // cell warp 0 .. 7: rows 8 cw .. 8 cw + 7
+        for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+            const long long row0 = (item / sp.col_splits) * kDenseBM;
+            const long long tile_lo = (item % sp.col_splits) * sp.tiles_per_split;
+            const long long tile_hi = tile_lo + sp.tiles_per_split < ntiles ? tile_lo + sp.tiles_per_split : ntiles;
+            // per-row cursors of this warp's rows (lane r keeps row r's): the first stored cell at or
+            // right of the column range's start, and the row's end
+            int mycur = 0, myend = 0;
+            if (lane < 8) {
+                const long long row = row0 + 8 * cw + lane;
+                if (row < p.rows) {
+                    mycur = __ldg(p.rowptr + row);
+                    myend = __ldg(p.rowptr + row + 1);
+                    const int want = (int)(tile_lo * kDenseBN);
+                    int hi = myend;
+                    while (mycur < hi) {
+                        const int mid = (mycur + hi) >> 1;
+                        if (__ldg(p.colidx + mid) < want) mycur = mid + 1; else hi = mid;
+                    }
+                }
+            }
+            // the cells of a tile: a lane per cell at its offset from the row's cursor.  Their loads do
+            // not need the tile, and where the next tile's cells start is known as soon as this tile's
+            // column indices are: so the loads run a tile ahead of the chains.
+            int jj[8], jn[8], pos[8];
+            double aa[8], an[8];
+            auto load_cells = [&](int (&j8)[8], double (&a8)[8]) {
+#pragma unroll
+                for (int rr = 0; rr < 8; ++rr) {
+                    const int pp = __shfl_sync(full, mycur, rr) + lane;
+                    j8[rr] = 0x7fffffff;
+                    a8[rr] = 0.0;
+                    if (pp < __shfl_sync(full, myend, rr)) {
+                        j8[rr] = __ldg(p.colidx + pp);
+                        a8[rr] = __ldg(p.vals + pp);
+                    }
+                }
+            };
+            load_cells(jn, an);
+            for (long long tile = tile_lo; tile < tile_hi; ++tile, ++n) {
+                const int b = (int)(n & 1);
+                const int n0 = (int)(tile * kDenseBN), nhi = n0 + kDenseBN;
+#pragma unroll
+                for (int rr = 0; rr < 8; ++rr) {
+                    jj[rr] = jn[rr];
+                    aa[rr] = an[rr];
+                    pos[rr] = __shfl_sync(full, mycur, rr) + lane;
+                    // the row's cells in this tile are a prefix of what was loaded: move the cursor past them
+                    const int taken = __popc(__ballot_sync(full, jj[rr] < nhi));
+                    if (lane == rr) mycur += taken;
+                }
+                if (tile + 1 < tile_hi) load_cells(jn, an);       // the next tile's cells, under this tile's chains
+                named_sync(kBarFull + b, kDenseThreadsAll);       // tile n is in buffer b
+                const double *pb = Ps + (size_t)b * kDenseBM * PLD;
+#pragma unroll
+                for (int rr = 0; rr < 8; ++rr) {
+                    if (jj[rr] < nhi) {
+                        const double w = outer_chain<true>(ch, p.chain_kind, p.kconst, aa[rr],
+                                                           pb[(size_t)(8 * cw + rr) * PLD + (jj[rr] - n0)]);
+                        if (AGG == kOutFull) acc += w;
+                        else p.out[pos[rr]] = w;
+                    }
+                }
+                __syncwarp();
+                named_arrive(kBarEmpty + b, kDenseThreadsAll);    // done with the buffer
+            }
+        }
     }
+    __syncthreads();
 
     if (AGG == kOutFull) {
         double v1[1] = {acc};
@@ -972,7 +1021,7 @@ outer_pipe_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ O
 }
 
 template <int AGG>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kDenseThreadsAll, 1)
 outer_dense_kernel(const __grid_constant__ DevChain ch, const __grid_constant__ OuterParams p,
                    const __grid_constant__ DenseSplit sp)
 {
